@@ -1,0 +1,402 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+The paper prints no worked example of the SSD arithmetic, so every pin is a
+closed form, an invariant, a special case that reduces to a library routine,
+an error bound, or brute force on a tiny input.  Each test is chosen so that a
+plausible mistake in the oracle (dropped term, wrong sign or index, transposed
+operand, off-by-one chunk) fails it.
+"""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2608_21952_b200 import inputs
+from paper_2608_21952_b200.inputs import SSDConfig, CONFIGS
+from helpers import TINY, TWO_BLOCK, dequant, rms, group_of
+
+
+# --------------------------------------------------------------------------- exp32
+def test_exp32_matches_libm():
+    x = np.concatenate([np.linspace(-80, 0, 400001), -np.logspace(-8, 1.9, 2000), [0.0]]).astype(np.float32)
+    e = orc.exp32(x).astype(np.float64)
+    ref = np.exp(x.astype(np.float64))
+    assert np.max(np.abs(e - ref) / ref) < 2e-7
+
+
+def test_exp32_special_values():
+    e = orc.exp32(np.array([0.0, -0.0, -80.5, -1000.0, -np.inf], np.float32))
+    assert e[0] == 1.0 and e[1] == 1.0 and np.all(e[2:] == 0.0)
+    # monotone on a fine grid (a rounding decision must never see a decay that grows with distance)
+    x = np.linspace(-30, 0, 300001).astype(np.float32)
+    assert np.all(np.diff(orc.exp32(x)) >= 0)
+
+
+# --------------------------------------------------------------------------- Eq. 1 quantiser
+def test_quantizer_bounds_and_extremes():
+    rng = np.random.default_rng(0)
+    R, Ch, I = 37, 5, 3
+    v = (rng.standard_normal((R, Ch, I)) * rng.uniform(0.1, 30, (1, Ch, 1))).astype(np.float32)
+    q, s = orc.quantize(v, R, Ch, I, mode=1)
+    assert q.dtype == np.int8 and np.abs(q.astype(int)).max() <= 127
+    for ch in range(Ch):
+        am = np.abs(v[:, ch, :]).max()
+        assert s[ch] == np.float32(am) / np.float32(127.0)
+        idx = np.unravel_index(np.argmax(np.abs(v[:, ch, :])), (R, I))
+        assert abs(int(q[idx[0], ch, idx[1]])) == 127
+    err = np.abs(v.astype(np.float64) - q.astype(np.float64) * s.astype(np.float64)[None, :, None])
+    assert np.all(err <= 0.5 * s[None, :, None] * (1 + 1e-5))
+
+
+def test_quantizer_idempotent_and_static():
+    rng = np.random.default_rng(1)
+    v = rng.standard_normal((64, 4, 2)).astype(np.float32)
+    q, s = orc.quantize(v, 64, 4, 2, mode=1)
+    deq = (q.astype(np.float32) * s[None, :, None]).astype(np.float32)
+    q2, _ = orc.quantize(deq, 64, 4, 2, scale=s, mode=0)
+    assert np.array_equal(q, q2)
+
+
+def test_quantizer_ties_to_even_saturation_zero_channel():
+    v = np.array([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 1000.0, -1000.0, 127.5, 126.5, 0.0], np.float32)
+    q, _ = orc.quantize(v.reshape(-1, 1, 1), v.size, 1, 1, scale=np.ones(1, np.float32), mode=0)
+    assert q.ravel().tolist() == [0, 2, 2, 0, -2, -2, 4, 127, -127, 127, 126, 0]
+    z = np.zeros((8, 2, 1), np.float32)
+    z[:, 1, 0] = 3.0
+    q, s = orc.quantize(z, 8, 2, 1, mode=1)
+    assert s[0] == 1.0 and np.all(q[:, 0, 0] == 0) and np.all(q[:, 1, 0] == 127)
+
+
+def test_quantizer_observe_mode_keeps_running_max():
+    a = np.full((4, 1, 1), 2.0, np.float32)
+    b = np.full((4, 1, 1), 1.0, np.float32)
+    _, s = orc.quantize(a, 4, 1, 1, scale=np.zeros(1, np.float32), mode=2, want_out=False)
+    _, s = orc.quantize(b, 4, 1, 1, scale=s, mode=2, want_out=False)
+    assert s[0] == np.float32(2.0) / np.float32(127.0)
+
+
+def test_quantizer_brute_force_small_grid():
+    # every value of a fine grid against the definition written with Python floats
+    alpha = np.float32(0.37)
+    v = (np.arange(-20000, 20001) * 0.0031).astype(np.float32)
+    q, _ = orc.quantize(v.reshape(-1, 1, 1), v.size, 1, 1, scale=np.array([alpha]), mode=0)
+    quo = (v / alpha).astype(np.float32)  # binary32 division
+    expect = np.clip(np.rint(quo), -127, 127).astype(np.int8)  # rint: ties to even
+    assert np.array_equal(q.ravel(), expect)
+
+
+# --------------------------------------------------------------------------- L0 recurrence
+def test_recurrence_closed_form_geometric():
+    # x = 1, B = C = e_1, dt = delta, A = a:  h_t = r h_{t-1} + delta, y_t = h_t + D
+    cfg = SSDConfig("cf", 1, 40, 1, 2, 3, 1, 8, 0, 1, 0)
+    delta, a, Dv = 0.3, -1.7, 0.25
+    x = np.ones((1, 40, 1, 2))
+    B = np.zeros((1, 40, 1, 3)); B[..., 0] = 1
+    dt = np.full((1, 40, 1), delta)
+    y, fin = orc.ssd_recurrence(cfg, x, B, B.copy(), dt, np.array([a]), np.array([Dv]))
+    r = np.exp(delta * a)
+    t = np.arange(40)
+    expect = delta * (1 - r ** (t + 1)) / (1 - r) + Dv
+    assert np.allclose(y[0, :, 0, 0], expect, rtol=1e-13)
+    assert np.allclose(fin[0, 0, :, 0], expect[-1] - Dv, rtol=1e-13) and np.all(fin[0, 0, :, 1:] == 0)
+
+
+def test_recurrence_single_token():
+    cfg = SSDConfig("l1", 2, 1, 2, 3, 4, 1, 1, 0, 1, 0)
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((2, 1, 2, 3)); B = rng.standard_normal((2, 1, 1, 4)); C = rng.standard_normal((2, 1, 1, 4))
+    dt = rng.uniform(0.01, 0.2, (2, 1, 2)); A = -rng.uniform(1, 4, 2); D = rng.standard_normal(2)
+    y, _ = orc.ssd_recurrence(cfg, x, B, C, dt, A, D)
+    cb = np.einsum("bgn,bgn->b", C[:, 0], B[:, 0])
+    expect = dt[:, 0, :, None] * cb[:, None, None] * x[:, 0] + D[None, :, None] * x[:, 0]
+    assert np.allclose(y[:, 0], expect, rtol=1e-13)
+
+
+# --------------------------------------------------------------------------- L1 == L0 (duality, chunk invariance)
+@pytest.mark.parametrize("Q", [1, 2, 8, 32])
+def test_chunked_equals_recurrence_every_chunk_size(Q):
+    cfg = TINY.replace(chunk=Q)
+    t = inputs.make_prefill(cfg)
+    rng = np.random.default_rng(5)
+    corr = rng.standard_normal(cfg.channels)
+    init = rng.standard_normal((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate))
+    y0, f0 = orc.ssd_recurrence(cfg, t["x"], t["B"], t["C"], t["dt"], t["A"], t["D"], corr, init)
+    y1, f1 = orc.ssd_chunked(cfg, t["x"], t["B"], t["C"], t["dt"], t["A"], t["D"], corr, init)
+    assert np.abs(y1 - y0).max() <= 1e-11 * rms(y0)
+    assert np.abs(f1 - f0).max() <= 1e-11 * rms(f0)
+
+
+def test_chunked_equals_recurrence_cfg0_shapes():
+    cfg = CONFIGS["cfg0"]
+    t = inputs.make_prefill(cfg)
+    y0, f0 = orc.ssd_recurrence(cfg, t["x"], t["B"], t["C"], t["dt"], t["A"], t["D"])
+    for Q in (64, 512):
+        y1, f1 = orc.ssd_chunked(cfg.replace(chunk=Q), t["x"], t["B"], t["C"], t["dt"], t["A"], t["D"])
+        assert np.abs(y1 - y0).max() <= 1e-10 * rms(y0)
+        assert np.abs(f1 - f0).max() <= 1e-10 * rms(f0)
+
+
+def test_a_to_zero_is_masked_linear_attention():
+    cfg = TINY.replace(chunk=16)
+    t = inputs.make_prefill(cfg)
+    A = np.zeros(cfg.nheads)
+    y1, _ = orc.ssd_chunked(cfg, t["x"], t["B"], t["C"], t["dt"], A, t["D"])
+    x, B, C, dt = (t[k].astype(np.float64) for k in ("x", "B", "C", "dt"))
+    L = cfg.seqlen
+    for b in range(cfg.batch):
+        for h in range(cfg.nheads):
+            g = group_of(cfg, h)
+            W = np.tril(C[b, :, g] @ B[b, :, g].T) * dt[b, :, h][None, :]
+            expect = W @ x[b, :, h] + t["D"][h] * x[b, :, h]
+            assert np.allclose(y1[b, :, h], expect, rtol=1e-11, atol=1e-11)
+
+
+def test_dt_zero_gives_skip_connection_only():
+    cfg = TINY
+    t = inputs.make_prefill(cfg)
+    corr = np.linspace(-1, 1, cfg.channels)
+    for fn in (orc.ssd_recurrence, orc.ssd_chunked):
+        y, fin = fn(cfg, t["x"], t["B"], t["C"], np.zeros_like(t["dt"]), t["A"], t["D"], corr)
+        expect = t["D"].astype(np.float64)[None, None, :, None] * t["x"] + corr.reshape(cfg.nheads, cfg.headdim)
+        assert np.allclose(y, expect, rtol=1e-13, atol=1e-13) and np.all(fin == 0)
+
+
+# --------------------------------------------------------------------------- L2 stages
+def _l2(cfg, init=None, corr=None):
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t, init)
+    y, fin, taps = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                 q["A"], q["D"], corr, q["s_xs"], q["s_cb"], q["s_h"], init,
+                                 taps=tuple(orc.TAP_SPECS))
+    return t, q, y, fin, taps
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK, CONFIGS["cfg0"]], ids=lambda c: c.name)
+def test_l2_cumsum_and_decay(cfg):
+    t, q, y, fin, taps = _l2(cfg)
+    dA = t["dt"].astype(np.float64) * t["A"].astype(np.float64)[None, None, :]
+    ref = np.cumsum(dA.reshape(cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads), axis=2).transpose(0, 3, 1, 2)
+    assert np.abs(taps["cs"] - ref).max() <= 1e-6 * max(1.0, np.abs(ref).max())
+    assert np.all(np.diff(taps["cs"], axis=-1) <= 0)  # dt > 0, A < 0
+    gam = orc.chunk_decay(cfg, taps["cs"])
+    assert np.allclose(gam, np.exp(ref[..., -1]), rtol=1e-5)
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK, CONFIGS["cfg0"]], ids=lambda c: c.name)
+def test_l2_integer_gemms_against_numpy(cfg):
+    t, q, y, fin, taps = _l2(cfg)
+    b, c, Q, H, P, N, G = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads, cfg.headdim, cfg.dstate, cfg.ngroups
+    Cq = q["Cq"].astype(np.int64).reshape(b, c, Q, G, N)
+    Bq = q["Bq"].astype(np.int64).reshape(b, c, Q, G, N)
+    xq = q["xq"].astype(np.int64).reshape(b, c, Q, H, P)
+    hg = np.arange(H) // (H // G)
+    # ChunkBMM: CB[i,j] = sum_n C[i,n] B[j,n]
+    assert np.array_equal(taps["acc_cb"], np.einsum("bcign,bcjgn->bcgij", Cq, Bq))
+    # ChunkState: acc[p,n] = sum_i Xs_q[i,p] B[i,n]
+    Xs = taps["Xsq"].astype(np.int64).reshape(b, c, Q, H, P)
+    assert np.array_equal(taps["acc_st"], np.einsum("bcihp,bcihn->bchpn", Xs, Bq[:, :, :, hg]))
+    # ChunkScan1: acc[i,p] = sum_n C[i,n] hq[p,n]
+    hq = taps["hq"].astype(np.int64)
+    ao = np.einsum("bcihn,bchpn->bcihp", Cq[:, :, :, hg], hq).reshape(b, c * Q, H, P)
+    assert np.array_equal(taps["acc_off"], ao)
+    # ChunkScan2: acc[i,p] = sum_j Mq[i,j] x[j,p], Mq strictly lower-triangular + diagonal
+    Mq = taps["Mq"].astype(np.int64)
+    assert np.all(np.triu(Mq, 1) == 0)
+    ad = np.einsum("bchij,bcjhp->bcihp", Mq, xq).reshape(b, c * Q, H, P)
+    assert np.array_equal(taps["acc_diag"], ad)
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK, CONFIGS["cfg0"]], ids=lambda c: c.name)
+def test_l2_requantisation_error_bounds(cfg):
+    """Each internal int8 tensor reconstructs the real-valued tensor of Algorithm 2
+    (computed here in fp64 from the plain definitions) to within half a step."""
+    t, q, y, fin, taps = _l2(cfg)
+    b, c, Q, H, P, N, G = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads, cfg.headdim, cfg.dstate, cfg.ngroups
+    hg = np.arange(H) // (H // G)
+    cs = taps["cs"].astype(np.float64)                              # [b,H,c,Q]
+    dt = t["dt"].astype(np.float64).reshape(b, c, Q, H).transpose(0, 3, 1, 2)  # [b,H,c,Q]
+    s_x = q["s_x"].astype(np.float64).reshape(H, P); s_xs = q["s_xs"].astype(np.float64).reshape(H, P)
+    fuzz = 1 + 1e-5
+    # CBq: acc_cb s_C s_B / s_cb
+    real = taps["acc_cb"] * (q["s_C"].astype(np.float64) * q["s_B"] / q["s_cb"])[None, None, :, None, None]
+    tril = np.tril(np.ones((Q, Q), bool))
+    assert np.all(np.abs(taps["CBq"] - real)[..., tril] <= 0.5 * fuzz)
+    assert np.abs(taps["CBq"][..., tril].astype(int)).max() == 127        # calibrated on this tensor
+    # Xs_q: LUT_state (x) X, LUT_state = dt exp(cs_last - cs)
+    lut = dt * np.exp(cs[..., -1:] - cs)                                     # [b,H,c,Q]
+    xh = q["xq"].astype(np.float64).reshape(b, c, Q, H, P) * s_x
+    xs_real = xh * lut.transpose(0, 2, 3, 1)[..., None]
+    err = np.abs(taps["Xsq"].reshape(b, c, Q, H, P) * s_xs - xs_real)
+    assert np.all(err <= 0.5 * s_xs * fuzz + 1e-30)
+    # hq: prev / s_h
+    s_h = q["s_h"].astype(np.float64).reshape(H, P)[None, None, :, :, None]
+    assert np.all(np.abs(taps["hq"] * s_h - taps["prev"]) <= 0.5 * s_h * fuzz)
+    # Mq: CBq[i,j] dt_j exp(cs_i - cs_j) on j <= i, one step size rowmax/127 per output row
+    cbq = taps["CBq"].astype(np.float64)[:, :, hg]                           # [b,c,H,Q,Q]
+    csT = cs.transpose(0, 2, 1, 3)                                           # [b,c,H,Q]
+    decay = np.exp(np.minimum(csT[..., :, None] - csT[..., None, :], 0.0)) * tril
+    Mreal = cbq * decay * dt.transpose(0, 2, 1, 3)[..., None, :]
+    rowmax = taps["rowmax"].astype(np.float64).reshape(b, c, Q, H).transpose(0, 1, 3, 2)  # [b,c,H,Q]
+    assert np.allclose(rowmax, np.abs(Mreal).max(-1), rtol=2e-6, atol=1e-30)
+    step = rowmax[..., None] / 127.0
+    assert np.all(np.abs(taps["Mq"] * step - Mreal) <= 0.5 * step * (1 + 1e-4) + 1e-30)
+    assert np.all(np.abs(taps["Mq"].astype(int)).max(-1)[rowmax > 0] == 127)
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK], ids=lambda c: c.name)
+def test_l2_state_passing_against_numpy_loop(cfg):
+    rng = np.random.default_rng(9)
+    init = rng.standard_normal((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate)).astype(np.float32)
+    t, q, y, fin, taps = _l2(cfg, init=init)
+    gam = np.exp(taps["cs"][..., -1].astype(np.float64))                     # [b,H,c]
+    S = init.astype(np.float64)
+    for k in range(cfg.nchunks):
+        assert np.allclose(taps["prev"][:, k], S, rtol=1e-5, atol=1e-6 * rms(S))
+        S = taps["loc"][:, k].astype(np.float64) + gam[:, :, k, None, None] * S
+    assert np.allclose(fin, S, rtol=1e-5, atol=1e-6 * rms(S))
+    assert np.array_equal(taps["prev"][:, 0], init)
+
+
+def test_l2_chunk_state_exact_when_scales_are_trivial():
+    """A = 0 and dt = 1 make every decay exactly 1; with s_xs = s_x the
+    re-quantisation is the identity, so loc must equal s_x s_B sum_i xq B exactly."""
+    cfg = TINY
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    s_x = np.full(cfg.channels, 0.5, np.float32); s_B = np.full(cfg.ngroups, 0.25, np.float32)
+    dt = np.ones_like(t["dt"]); cs = orc.chunk_cumsum(cfg, dt, np.zeros(cfg.nheads, np.float32))
+    assert np.all(cs == 0)
+    xsq, acc, loc = orc.chunk_state(cfg, q["xq"], q["Bq"], s_x, s_x, s_B, dt, cs)
+    assert np.array_equal(xsq, q["xq"])
+    b, c, Q, H, P, N, G = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads, cfg.headdim, cfg.dstate, cfg.ngroups
+    hg = np.arange(H) // (H // G)
+    ref = np.einsum("bcihp,bcihn->bchpn", q["xq"].astype(np.int64).reshape(b, c, Q, H, P),
+                    q["Bq"].astype(np.int64).reshape(b, c, Q, G, N)[:, :, :, hg])
+    assert np.array_equal(loc, (ref * 0.125).astype(np.float32))
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK, CONFIGS["cfg0"]], ids=lambda c: c.name)
+def test_l2_close_to_unquantised_dual_form(cfg):
+    """SSDi8 output stays within the quantisation noise of Algorithm 2 on the same
+    dequantised inputs; a dropped term or wrong index would give an O(1) error."""
+    rng = np.random.default_rng(2)
+    corr = (0.01 * rng.standard_normal(cfg.channels)).astype(np.float32)
+    t, q, y, fin, taps = _l2(cfg, corr=corr)
+    xh, Bh, Ch = dequant(cfg, q)
+    y1, f1 = orc.ssd_chunked(cfg, xh, Bh, Ch, t["dt"], t["A"], t["D"], corr)
+    rel = np.sqrt(((y - y1) ** 2).sum() / (y1 ** 2).sum())
+    assert rel < 3e-2, rel
+    assert np.sqrt(((fin - f1) ** 2).sum() / (f1 ** 2).sum()) < 5e-2
+
+
+def test_l2_output_recombines_taps():
+    cfg = CONFIGS["cfg0"]
+    t, q, y, fin, taps = _l2(cfg)
+    b, c, Q, H, P = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads, cfg.headdim
+    hg = np.arange(H) // (H // cfg.ngroups)
+    s_x = q["s_x"].astype(np.float64).reshape(H, P); s_h = q["s_h"].astype(np.float64).reshape(H, P)
+    dec = np.exp(taps["cs"].astype(np.float64)).transpose(0, 2, 3, 1).reshape(b, c * Q, H)
+    y_off = dec[..., None] * q["s_C"].astype(np.float64)[hg][None, None, :, None] * s_h * taps["acc_off"]
+    s_m = q["s_cb"].astype(np.float64)[hg][None, None, :] * taps["rowmax"] / 127.0
+    y_diag = s_m[..., None] * s_x * taps["acc_diag"]
+    skip = t["D"].astype(np.float64)[None, None, :, None] * s_x * q["xq"]
+    assert np.allclose(y, y_off + y_diag + skip, rtol=1e-12, atol=1e-12 * rms(y))
+
+
+def test_x_scaled_is_sparse_after_quantisation():
+    # Section 4.2 / Fig. 3: Q(X_scaled) is highly sparse
+    t, q, y, fin, taps = _l2(CONFIGS["cfg0"])
+    assert (taps["Xsq"] == 0).mean() > 0.5
+
+
+def test_calibration_matches_plain_definitions():
+    cfg = TWO_BLOCK
+    t, q, y, fin, taps = _l2(cfg)
+    b, c, Q, H, P = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads, cfg.headdim
+    cs = taps["cs"].astype(np.float64)
+    dt = t["dt"].astype(np.float64).reshape(b, c, Q, H).transpose(0, 3, 1, 2)
+    lut = (dt * np.exp(cs[..., -1:] - cs)).transpose(0, 2, 3, 1)[..., None]
+    xs = np.abs(q["xq"].astype(np.float64).reshape(b, c, Q, H, P) * q["s_x"].astype(np.float64).reshape(H, P) * lut)
+    assert np.allclose(q["s_xs"].reshape(H, P), xs.max((0, 1, 2)) / 127, rtol=1e-5)
+    tril = np.tril(np.ones((Q, Q), bool))
+    m = np.abs(taps["acc_cb"])[..., tril].max()
+    assert np.allclose(q["s_cb"][0], m * float(q["s_C"][0]) * float(q["s_B"][0]) / 127, rtol=1e-5)
+    allS = np.concatenate([taps["prev"], fin[:, None]], 1)
+    assert np.allclose(q["s_h"].reshape(H, P), np.abs(allS).max((0, 1, 4)) / 127, rtol=1e-6)
+
+
+# --------------------------------------------------------------------------- L3 step
+def _quant_step(cfg, s, scales):
+    st = inputs.make_decode_step(cfg, s)
+    xq, _ = orc.quantize(st["x"], cfg.batch, cfg.channels, 1, scale=scales["s_x"], mode=0)
+    Bq, _ = orc.quantize(st["B"], cfg.batch, cfg.ngroups, cfg.dstate, scale=scales["s_B"], mode=0)
+    Cq, _ = orc.quantize(st["C"], cfg.batch, cfg.ngroups, cfg.dstate, scale=scales["s_C"], mode=0)
+    return xq, Bq, Cq, st["dt"]
+
+
+def test_step_iterated_equals_recurrence_and_handoff():
+    cfg = SSDConfig("dec", 2, 1, 4, 8, 16, 2, 8, 0.05, 20.0, 13, decode_steps=24)
+    prm = inputs.make_decode_params(cfg)
+    scales = dict(s_x=np.full(cfg.channels, 0.05, np.float32), s_B=np.full(cfg.ngroups, 0.03, np.float32),
+                  s_C=np.full(cfg.ngroups, 0.03, np.float32))
+    corr = np.linspace(-0.1, 0.1, cfg.channels).astype(np.float32)
+    T = cfg.decode_steps
+    state = np.zeros((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate))
+    ys, seq = [], []
+    for s in range(T):
+        xq, Bq, Cq, dt = _quant_step(cfg, s, scales)
+        seq.append((xq, Bq, Cq, dt))
+        ys.append(orc.ssd_step(cfg, xq, scales["s_x"], Bq, scales["s_B"], Cq, scales["s_C"], dt,
+                               prm["A"], prm["D"], corr, state))
+    ys = np.stack(ys, 1)
+    full = cfg.replace(seqlen=T)
+    xh = np.stack([s[0] for s in seq], 1) * scales["s_x"].astype(np.float64).reshape(cfg.nheads, cfg.headdim)
+    Bh = np.stack([s[1] for s in seq], 1) * np.float64(scales["s_B"][0])
+    Ch = np.stack([s[2] for s in seq], 1) * np.float64(scales["s_C"][0])
+    dts = np.stack([s[3] for s in seq], 1)
+    y0, f0 = orc.ssd_recurrence(full, xh, Bh, Ch, dts, prm["A"], prm["D"], corr)
+    assert np.abs(ys - y0).max() <= 1e-12 * rms(y0) and np.abs(state - f0).max() <= 1e-12 * rms(f0)
+    # hand-off: dual form over the first 16 tokens, then 8 single-token steps
+    pre = cfg.replace(seqlen=16, chunk=8)
+    y1, f1 = orc.ssd_chunked(pre, xh[:, :16], Bh[:, :16], Ch[:, :16], dts[:, :16], prm["A"], prm["D"], corr)
+    st = f1.copy()
+    for s in range(16, T):
+        xq, Bq, Cq, dt = seq[s]
+        ystep = orc.ssd_step(cfg, xq, scales["s_x"], Bq, scales["s_B"], Cq, scales["s_C"], dt,
+                             prm["A"], prm["D"], corr, st)
+        assert np.abs(ystep - y0[:, s]).max() <= 1e-11 * rms(y0)
+    assert np.abs(st - f0).max() <= 1e-11 * rms(f0)
+
+
+# --------------------------------------------------------------------------- Eq. 8 mean correction
+def test_mean_correction_is_least_squares_optimum_and_streaming_mean():
+    rng = np.random.default_rng(4)
+    Y = rng.standard_normal((200, 6)); Yq = Y + 0.1 * rng.standard_normal((200, 6)) + np.linspace(-1, 1, 6)
+    c = orc.mean_correction(Y, Yq, 1.0)
+    grad = -2 * (Y - Yq - c).sum(0)          # d/dc ||Y - (Yq + c)||_F^2
+    assert np.allclose(grad, 0, atol=1e-10)
+    for e in np.eye(6):
+        assert ((Y - Yq - c) ** 2).sum() < ((Y - Yq - c - 1e-3 * e) ** 2).sum()
+    assert np.allclose(orc.mean_correction(Y, Yq, 0.15), 0.15 * c)
+    # Algorithm 1's running update mu += (n_s / N)(m_s - mu) equals the global mean
+    mu, N = np.zeros(6), 0
+    for part in np.array_split(Yq, [30, 110, 150]):
+        N += len(part)
+        mu += len(part) / N * (part.mean(0) - mu)
+    assert np.allclose(mu, Yq.mean(0), atol=1e-12)
+    assert np.allclose(c, Y.mean(0) - mu, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- stored digests
+def test_oracle_reproduces_stored_digests():
+    import json, os, importlib.util
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec); spec.loader.exec_module(mg)
+    stored = json.load(open(os.path.join(here, "l2_digest.json")))
+    for name, cfg in (("cfg0", CONFIGS["cfg0"]), ("two_block", TWO_BLOCK)):
+        got = mg.digest(cfg)
+        for k, v in stored[name].items():
+            if isinstance(v, float):
+                assert abs(got[k] - v) <= 1e-9 * abs(v), (name, k)
+            else:
+                assert got[k] == v, (name, k)
