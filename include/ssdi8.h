@@ -1,0 +1,201 @@
+/* ssdi8.h -- C ABI of the B200 (sm_100a) INT8 State Space Duality layer.
+ *
+ * The library computes the forward pass of one quantised Mamba-2 SSD layer
+ * (SSDi8, Algorithm 2 with the INT8 path of Section 4.2) and its single-token
+ * recurrent step.  Symbols follow the paper: batch B (here `batch`), length L,
+ * heads H, head dimension P, state dimension N, groups G, chunk length l
+ * (here Q = `chunk`), c = L / Q chunks, D = H * P channels, g(h) = h / (H / G).
+ *
+ * Conventions for every entry point
+ *  - All pointers are DEVICE pointers unless the comment says "host".  The
+ *    caller owns every buffer; except where stated the library allocates no
+ *    device memory and keeps no mutable global state.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Calls are asynchronous on that stream.
+ *  - The return value reports everything that can be checked on the host
+ *    before launch (null pointers, unsupported shapes, alignment, short
+ *    workspace, wrong device architecture, launch failure).  Nothing throws
+ *    and nothing aborts.  A condition detected on the device (a bounded wait
+ *    that ran out) is written to the caller's `status` word, to be read after
+ *    synchronising the stream.
+ *  - Tensors are dense, row-major, last axis contiguous.
+ *  - Supported shapes: P = 64, N in {64, 128}, Q in {64, 128, 256}, L % Q = 0,
+ *    H % G = 0; otherwise SSDI8_ERR_SHAPE.
+ *  - Every int8 code the library produces lies in [-127, 127].
+ *  - Results are deterministic: no floating-point atomics in any result.
+ *
+ * Arithmetic that decides an integer code is carried out in IEEE binary32 with
+ * round-to-nearest-even, in the operation order written in each comment below
+ * (fmul, fsub, fdiv, fmaf are single correctly rounded operations; rne rounds
+ * half to even and the result is then saturated to [-127, 127]).  exp32 is the
+ * library's binary32 exponential: n = rint(x * 0x3FB8AA3B), r = fmaf(n,
+ * -0x3F317200, x), r = fmaf(n, -0x35BFBE8E, r), degree-7 Taylor polynomial in r
+ * by Horner with fmaf, result scaled by 2^n; 0 for x < -80.
+ */
+#ifndef SSDI8_H_
+#define SSDI8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t ssdi8_status_t;
+enum {
+  SSDI8_OK = 0,
+  SSDI8_ERR_NULL = -1,           /* a required pointer is NULL                        */
+  SSDI8_ERR_SHAPE = -2,          /* unsupported or inconsistent dimensions            */
+  SSDI8_ERR_ALIGN = -3,          /* a pointer is not 16-byte aligned                  */
+  SSDI8_ERR_WORKSPACE = -4,      /* workspace shorter than ssdi8_workspace_bytes()    */
+  SSDI8_ERR_ARCH = -5,           /* current device is not compute capability 10.0     */
+  SSDI8_ERR_CUDA = -6,           /* a CUDA runtime call or a launch failed            */
+  SSDI8_ERR_DEVICE_TIMEOUT = -7, /* written to *status by a kernel whose wait ran out */
+  SSDI8_ERR_UNSUPPORTED = -8     /* a flag or mode that is not implemented            */
+};
+
+typedef struct {
+  int32_t batch, seqlen, nheads, headdim, dstate, ngroups, chunk;
+} ssdi8_dims_t;
+
+/* module selection bits of ssdi8_chunk_scan_fwd's flags (Algorithm 2's modules) */
+enum {
+  SSDI8_PHASE_CUMSUM = 1u << 8,
+  SSDI8_PHASE_BMM = 1u << 9,
+  SSDI8_PHASE_CHUNK_STATE = 1u << 10,
+  SSDI8_PHASE_STATE_PASSING = 1u << 11,
+  SSDI8_PHASE_SCAN = 1u << 12,
+  SSDI8_PHASE_ALL = 0x1f00u
+};
+
+/* host, pure: static string for a status code */
+const char* ssdi8_status_string(ssdi8_status_t s);
+
+/* host, pure: bytes of scratch ssdi8_chunk_scan_fwd / ssdi8_calibrate need for
+ * these dimensions (0 if the dimensions are unsupported). */
+size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags);
+
+/* Activation quantiser (Eq. 1): uniform symmetric 8-bit, one step size per
+ * channel of the view in[R][Ch][I]  (x: R = B*L, Ch = D, I = 1;  B and C,
+ * quantised once on the group axis before any broadcast to heads, Section 4.2
+ * "Quantization of B,C": R = B*L, Ch = G, I = N).
+ *   alpha = fdiv(absmax, 127)  (1 if the channel is all zero)
+ *   q     = rne(fdiv(v, alpha)) saturated
+ * mode 0 static:    read scale[Ch], write out.
+ * mode 1 calibrate: write scale[Ch] from this tensor, then write out.
+ * mode 2 observe:   scale[Ch] = max(scale[Ch], alpha of this tensor); `out`
+ *                   may be NULL (nothing is quantised then).
+ * in, out: 16-byte aligned; I == 1 or I % 4 == 0; (Ch * I) % 4 == 0. */
+ssdi8_status_t ssdi8_quantize_act(const float* in, int64_t R, int64_t Ch, int64_t I,
+                                  float* scale, int32_t mode, int8_t* out, void* stream);
+
+typedef struct {
+  /* layer inputs */
+  const int8_t* xq;        /* [B,L,H,P]  per-channel codes of X                         */
+  const int8_t* Bq;        /* [B,L,G,N]  per-group codes of B                           */
+  const int8_t* Cq;        /* [B,L,G,N]  per-group codes of C                           */
+  const float* s_x;        /* [H*P] step sizes of xq                                    */
+  const float* s_B;        /* [G]                                                       */
+  const float* s_C;        /* [G]                                                       */
+  const float* dt;         /* [B,L,H] time step, already positive (after softplus)      */
+  const float* A;          /* [H] decay rate, negative                                  */
+  const float* D;          /* [H] skip weight, or NULL                                  */
+  const float* corr;       /* [H*P] per-channel mean correction (Eq. 8), or NULL        */
+  /* static step sizes of the internal int8 tensors (from ssdi8_calibrate) */
+  const float* s_xs;       /* [H*P] Q(X_scaled), Eq. 3                                  */
+  const float* s_cb;       /* [G]   Q(CB)                                               */
+  const float* s_h;        /* [H*P] Q(State), Eq. 4; one scale for all chunks           */
+  const float* init_state; /* [B,H,P,N] state before the first token, or NULL (zeros)   */
+  /* outputs */
+  float* y;                /* [B,L,H,P]                                                  */
+  float* final_state;      /* [B,H,P,N] state after the last token, or NULL             */
+  int32_t* status;         /* 1 word, or NULL: 0 or an SSDI8_ERR_* written by a kernel   */
+  /* optional taps of the intermediate tensors (tests); each may be NULL */
+  float* tap_cs;           /* [B,H,c,Q]   chunk-local cumulative sum of dt*A            */
+  int32_t* tap_acc_cb;     /* [B,c,G,Q,Q] INT32 C B^T, entries with j <= i              */
+  int8_t* tap_CBq;         /* [B,c,G,Q,Q] its int8 codes, entries with j <= i           */
+  int8_t* tap_Xsq;         /* [B,L,H,P]   Q(X_scaled)                                   */
+  int32_t* tap_acc_st;     /* [B,c,H,P,N] INT32 chunk state                             */
+  float* tap_loc;          /* [B,c,H,P,N] chunk-local state, fp32                       */
+  float* tap_prev;         /* [B,c,H,P,N] state entering chunk k                        */
+  int8_t* tap_hq;          /* [B,c,H,P,N] its int8 codes                                */
+  int32_t* tap_acc_off;    /* [B,L,H,P]   INT32 C h                                     */
+  float* tap_rowmax;       /* [B,L,H]     absmax of each row of the masked operand      */
+  int8_t* tap_Mq;          /* [B,c,H,Q,Q] int8 masked operand, zero above the diagonal  */
+  int32_t* tap_acc_diag;   /* [B,L,H,P]   INT32 Mq x                                    */
+} ssdi8_fwd_args_t;
+
+/* SSD layer forward (Algorithm 2) from int8 x, B, C to fp32 y and final state.
+ *  ChunkCumsum   cs[k,i] = (float) sum_{i'<=i} (double)dt * (double)A, in token order;
+ *                Gamma_k = exp32(cs[k,Q-1])                         (Decay_pass, Eq. 5)
+ *  ChunkBMM      acc_cb[i,j] = sum_n Cq[i,n] Bq[j,n]  per (b, chunk, group), INT32;
+ *                CBq = rne(fmul(float(acc_cb), fdiv(fmul(s_C, s_B), s_cb)))
+ *  ChunkState    sparse-aware reformulation, Eq. 3:
+ *                LUT_state[i] = fmul(dt_i, exp32(fsub(cs_last, cs_i)))
+ *                Xs_q[i,p] = rne(fmul(fmul(float(xq[i,p]), fdiv(s_x, s_xs)), LUT_state[i]))
+ *                acc_st[p,n] = sum_i Xs_q[i,p] Bq[i,n], INT32;
+ *                loc = fmul(float(acc_st), fmul(s_xs, s_B))          (Eq. 4 rescale)
+ *  StatePassing  S_k = fmaf(Gamma_k, S_{k-1}, loc_k), S_{-1} = init_state (Eq. 6), fp32;
+ *                hq[k] = rne(fmul(S_{k-1}, fdiv(1, s_h)))
+ *  ChunkScan1    acc_off[i,p] = sum_n Cq[i,n] hq[k][p,n], INT32;
+ *                y_off = exp(cs_i) s_C s_h acc_off   (decay only; no dt factor)
+ *  ChunkScan2    the masked operand CB o LUT_scan2 (LUT_scan2[i,j] = dt_j exp(cs_i - cs_j),
+ *                j <= i) is re-quantised per output row so that its product with int8 X is
+ *                an integer GEMM.  With sub-blocks of SB = min(64, Q) tokens and je the last
+ *                column of the sub-block of j:
+ *                  same sub-block : w = fmul(dt_j, exp32(fsub(cs_i, cs_j))),  f = 1
+ *                  earlier block  : w = fmul(dt_j, exp32(fsub(cs_je, cs_j))), f = exp32(fsub(cs_i, cs_je))
+ *                  t = fmul(float(CBq[i,j]), w)
+ *                  rowmax_i = max over sub-blocks of fmul(max_j |t|, f)
+ *                  inv_i = rowmax_i >= 1e-30 ? fdiv(127, rowmax_i) : 0
+ *                  Mq[i,j] = rne(fmul(t, fmul(f, inv_i)))
+ *                acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p], INT32;
+ *                y_diag = (s_cb rowmax_i / 127) s_x acc_diag
+ *  Output        y = y_off + y_diag + D s_x xq + corr
+ * flags: bit 0 is reserved for the paper's FP16 ChunkScan2 operand and must be 0.  Bits 8-12
+ * select modules (SSDI8_PHASE_*); 0 in those bits runs all five in order.  A partial run
+ * reads the intermediates a previous call left in the same workspace (per-module timing,
+ * tests); any other bit set gives SSDI8_ERR_UNSUPPORTED.
+ * workspace: at least ssdi8_workspace_bytes(dims, flags) bytes, 256-byte aligned; its
+ * contents are scratch.  All tensor pointers 16-byte aligned. */
+ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
+                                    uint32_t flags, void* workspace, size_t workspace_bytes,
+                                    void* stream);
+
+/* Static calibration of the internal step sizes (Eq. 1 applied once to the internal
+ * tensors of this input; the paper calibrates offline, Section 5 "Quantization Setup"):
+ *   s_xs[h,p] = absmax over (b,t) of |fmul(fmul(float(xq), s_x), LUT_state)| / 127
+ *   s_cb[g]   = absmax over the causal half of |acc_cb| * fmul(s_C, s_B) / 127
+ *   s_h[h,p]  = absmax over init_state and every S_k, all b and n, / 127
+ * (each 1 if its absmax is 0).  Reads xq, Bq, Cq, s_x, s_B, s_C, dt, A, init_state of `args`;
+ * ignores its other members.  Writes s_xs [H*P], s_cb [G], s_h [H*P]. */
+ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
+                               float* s_xs, float* s_cb, float* s_h, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+/* StatePassing alone (Eq. 5-6; Algorithm 2 module 3) on fp32 states.
+ *   S_k = fmaf(gamma[b,h,k], S_{k-1}, loc[b,k,h,p,n]),  S_{-1} = init_state or 0
+ *   prev[b,k] = S_{k-1} (may be NULL; may alias loc), final_state = S_{c-1} (may be NULL),
+ *   hq[b,k] = rne(fmul(S_{k-1}, fdiv(1, s_h[h,p]))) when hq and s_h are non-NULL.
+ * loc, prev [B,c,H,P,N]; gamma [B,H,c]; init_state, final_state [B,H,P,N]; hq [B,c,H,P,N]. */
+ssdi8_status_t ssdi8_state_passing(const ssdi8_dims_t* dims, const float* loc, const float* gamma,
+                                   const float* init_state, float* prev, float* final_state,
+                                   int8_t* hq, const float* s_h, void* stream);
+
+/* One recurrent-mode token for every sequence of the batch (the recurrence
+ * h_t = exp(dt A) h_{t-1} + dt B_t x_t^T, y_t = C_t h_t + D x_t that the dual form of
+ * Algorithm 2 unrolls; the paper gives no algorithm for this mode).  fp32 throughout:
+ *   a = exp(dt[b,h] A[h]);  S[p,n] = a S[p,n] + (dt s_x[h,p] s_B[g]) xq[p] Bq[n]
+ *   y[p] = s_C[g] sum_n Cq[n] S[p,n] + D[h] s_x[h,p] xq[p] + corr[h,p]   (updated state)
+ * xq [B,H,P]; Bq, Cq [B,G,N]; dt [B,H]; state [B,H,P,N] updated IN PLACE; y [B,H,P].
+ * dims.seqlen and dims.chunk are ignored.  D and corr may be NULL. */
+ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const float* s_x,
+                              const int8_t* Bq, const float* s_B, const int8_t* Cq,
+                              const float* s_C, const float* dt, const float* A, const float* D,
+                              const float* corr, float* state, float* y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSDI8_H_ */

@@ -7,13 +7,10 @@ of ssdi8_oracle.cpp; it contains no arithmetic of its own beyond dtype casts.
 from __future__ import annotations
 
 import ctypes as C
-import os
-import sys
 
 import numpy as np
 
-sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
-import build as _build  # noqa: E402  (oracle/build.py)
+from . import build as _build
 
 _lib = C.CDLL(_build.build())
 

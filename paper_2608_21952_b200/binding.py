@@ -1,0 +1,149 @@
+"""Thin ctypes binding of libssdi8 (argument marshalling only).
+
+The functions carry the names of the C entry points declared in include/ssdi8.h
+and take torch CUDA tensors; every step of the computation runs inside the
+library's kernels.  There is no fallback: if the library cannot be loaded the
+import raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+_LIB_PATH = _build.LIB
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2608_21952_b200.build` "
+        "(nvcc, sm_100a); there is no CPU or PyTorch fallback")
+_lib = C.CDLL(_LIB_PATH)
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = \
+    -1, -2, -3, -4, -5, -6, -7, -8
+
+PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1 << k for k in range(8, 13))
+
+EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
+           "ssdi8_chunk_scan_fwd", "ssdi8_calibrate", "ssdi8_state_passing", "ssdi8_ssd_step")
+
+
+class Dims(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in
+                ("batch", "seqlen", "nheads", "headdim", "dstate", "ngroups", "chunk")]
+
+
+_FWD_FIELDS = ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "corr", "s_xs", "s_cb", "s_h",
+               "init_state", "y", "final_state", "status",
+               "tap_cs", "tap_acc_cb", "tap_CBq", "tap_Xsq", "tap_acc_st", "tap_loc", "tap_prev",
+               "tap_hq", "tap_acc_off", "tap_rowmax", "tap_Mq", "tap_acc_diag")
+
+
+class FwdArgs(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in _FWD_FIELDS]
+
+
+_lib.ssdi8_status_string.restype = C.c_char_p
+_lib.ssdi8_status_string.argtypes = [C.c_int32]
+_lib.ssdi8_workspace_bytes.restype = C.c_size_t
+_lib.ssdi8_workspace_bytes.argtypes = [C.POINTER(Dims), C.c_uint32]
+_lib.ssdi8_quantize_act.restype = C.c_int32
+_lib.ssdi8_quantize_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                    C.c_int32, C.c_void_p, C.c_void_p]
+_lib.ssdi8_chunk_scan_fwd.restype = C.c_int32
+_lib.ssdi8_chunk_scan_fwd.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_uint32, C.c_void_p,
+                                      C.c_size_t, C.c_void_p]
+_lib.ssdi8_calibrate.restype = C.c_int32
+_lib.ssdi8_calibrate.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_void_p, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.ssdi8_state_passing.restype = C.c_int32
+_lib.ssdi8_state_passing.argtypes = [C.POINTER(Dims)] + [C.c_void_p] * 8
+_lib.ssdi8_ssd_step.restype = C.c_int32
+_lib.ssdi8_ssd_step.argtypes = [C.POINTER(Dims)] + [C.c_void_p] * 13
+
+
+class SSDi8Error(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {ssdi8_status_string(code)} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise SSDi8Error(code, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def dims_of(cfg) -> Dims:
+    return Dims(cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim, cfg.dstate, cfg.ngroups, cfg.chunk)
+
+
+def ssdi8_status_string(code: int) -> str:
+    return _lib.ssdi8_status_string(int(code)).decode()
+
+
+def ssdi8_workspace_bytes(dims: Dims, flags: int = 0) -> int:
+    return int(_lib.ssdi8_workspace_bytes(C.byref(dims), flags))
+
+
+def ssdi8_quantize_act(inp, R: int, Ch: int, I: int, scale, mode: int, out, stream=None) -> None:
+    _check(_lib.ssdi8_quantize_act(_ptr(inp), R, Ch, I, _ptr(scale), mode, _ptr(out), _stream(stream)),
+           "ssdi8_quantize_act")
+
+
+def make_fwd_args(**tensors) -> FwdArgs:
+    a = FwdArgs()
+    for k, v in tensors.items():
+        if k not in _FWD_FIELDS:
+            raise KeyError(k)
+        setattr(a, k, _ptr(v))
+    a._keepalive = dict(tensors)  # the struct holds raw pointers: keep the tensors alive with it
+    return a
+
+
+def ssdi8_chunk_scan_fwd(dims: Dims, args: FwdArgs, workspace, flags: int = 0, stream=None) -> None:
+    _check(_lib.ssdi8_chunk_scan_fwd(C.byref(dims), C.byref(args), flags, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "ssdi8_chunk_scan_fwd")
+
+
+def ssdi8_calibrate(dims: Dims, args: FwdArgs, s_xs, s_cb, s_h, workspace, stream=None) -> None:
+    _check(_lib.ssdi8_calibrate(C.byref(dims), C.byref(args), _ptr(s_xs), _ptr(s_cb), _ptr(s_h),
+                                _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                _stream(stream)), "ssdi8_calibrate")
+
+
+def ssdi8_state_passing(dims: Dims, loc, gamma, init_state, prev, final_state, hq, s_h,
+                        stream=None) -> None:
+    _check(_lib.ssdi8_state_passing(C.byref(dims), _ptr(loc), _ptr(gamma), _ptr(init_state), _ptr(prev),
+                                    _ptr(final_state), _ptr(hq), _ptr(s_h), _stream(stream)),
+           "ssdi8_state_passing")
+
+
+def ssdi8_ssd_step(dims: Dims, xq, s_x, Bq, s_B, Cq, s_C, dt, A, D, corr, state, y, stream=None) -> None:
+    _check(_lib.ssdi8_ssd_step(C.byref(dims), _ptr(xq), _ptr(s_x), _ptr(Bq), _ptr(s_B), _ptr(Cq),
+                               _ptr(s_C), _ptr(dt), _ptr(A), _ptr(D), _ptr(corr), _ptr(state), _ptr(y),
+                               _stream(stream)), "ssdi8_ssd_step")
+
+
+def alloc_workspace(dims: Dims, device="cuda"):
+    n = ssdi8_workspace_bytes(dims)
+    if n == 0:
+        raise SSDi8Error(ERR_SHAPE, "ssdi8_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)

@@ -1,0 +1,225 @@
+// C-ABI entry points of libssdi8: argument validation, workspace layout, kernel sequencing.
+#include <cstring>
+
+#include "kernels.h"
+
+using namespace ssdi8;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool dims_supported(const ssdi8_dims_t* d, bool need_chunks) {
+  if (!d) return false;
+  if (d->batch <= 0 || d->nheads <= 0 || d->ngroups <= 0) return false;
+  if (d->headdim != 64) return false;
+  if (d->dstate != 64 && d->dstate != 128) return false;
+  if (d->nheads % d->ngroups != 0) return false;
+  if (need_chunks) {
+    if (d->chunk != 64 && d->chunk != 128 && d->chunk != 256) return false;
+    if (d->seqlen <= 0 || d->seqlen % d->chunk != 0) return false;
+  }
+  return true;
+}
+
+// The kernels are built for sm_100a only (tensor-memory MMA does not exist elsewhere).
+ssdi8_status_t check_arch() {
+  static int ok_device[64];  // 0 unknown, 1 ok, -1 wrong
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SSDI8_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
+  if (ok_device[dev] == 0) {
+    int major = 0, minor = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess)
+      return SSDI8_ERR_CUDA;
+    ok_device[dev] = (major == 10 && minor == 0) ? 1 : -1;
+  }
+  return ok_device[dev] == 1 ? SSDI8_OK : SSDI8_ERR_ARCH;
+}
+
+struct Workspace {
+  size_t cs, gamma, cbq, loc, hq, total;
+};
+
+Workspace layout(const Dims& d) {
+  Workspace w;
+  size_t o = 0;
+  const size_t nst = (size_t)d.b * d.c * d.H * d.P * d.N;
+  w.cs = o;    o = align_up(o + sizeof(float) * (size_t)d.b * d.H * d.L, 256);
+  w.gamma = o; o = align_up(o + sizeof(float) * (size_t)d.b * d.H * d.c, 256);
+  w.cbq = o;   o = align_up(o + (size_t)d.b * d.c * d.G * d.Q * d.Q, 256);
+  w.loc = o;   o = align_up(o + sizeof(float) * nst, 256);
+  w.hq = o;    o = align_up(o + nst, 256);
+  w.total = o;
+  return w;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ssdi8_status_string(ssdi8_status_t s) {
+  switch (s) {
+    case SSDI8_OK: return "ok";
+    case SSDI8_ERR_NULL: return "a required pointer is NULL";
+    case SSDI8_ERR_SHAPE: return "unsupported or inconsistent dimensions";
+    case SSDI8_ERR_ALIGN: return "a pointer is not 16-byte aligned";
+    case SSDI8_ERR_WORKSPACE: return "workspace too small";
+    case SSDI8_ERR_ARCH: return "device is not compute capability 10.0 (sm_100a)";
+    case SSDI8_ERR_CUDA: return "CUDA runtime or launch failure";
+    case SSDI8_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case SSDI8_ERR_UNSUPPORTED: return "flag or mode not implemented";
+    default: return "unknown status";
+  }
+}
+
+size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
+  if ((flags & ~(uint32_t)SSDI8_PHASE_ALL) != 0 || !dims_supported(dims, true)) return 0;
+  return layout(make_dims(dims)).total;
+}
+
+ssdi8_status_t ssdi8_quantize_act(const float* in, int64_t R, int64_t Ch, int64_t I, float* scale,
+                                  int32_t mode, int8_t* out, void* stream) {
+  if (!in || !scale) return SSDI8_ERR_NULL;
+  if (mode < 0 || mode > 2) return SSDI8_ERR_UNSUPPORTED;
+  if (!out && mode != 2) return SSDI8_ERR_NULL;
+  if (R < 0 || Ch <= 0 || I <= 0) return SSDI8_ERR_SHAPE;
+  if (!(I == 1 || I % 4 == 0) || (Ch * I) % 4 != 0) return SSDI8_ERR_SHAPE;
+  if (R * Ch * I >= ((int64_t)1 << 33)) return SSDI8_ERR_SHAPE;
+  if (!aligned16(in) || (out && !aligned16(out)) || !aligned16(scale)) return SSDI8_ERR_ALIGN;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_quantize(in, R, Ch, I, scale, mode, out, static_cast<cudaStream_t>(stream));
+}
+
+ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a,
+                                    uint32_t flags, void* workspace, size_t workspace_bytes,
+                                    void* stream) {
+  if (!dims || !a) return SSDI8_ERR_NULL;
+  if ((flags & ~(uint32_t)SSDI8_PHASE_ALL) != 0) return SSDI8_ERR_UNSUPPORTED;
+  const uint32_t ph = (flags & SSDI8_PHASE_ALL) ? (flags & SSDI8_PHASE_ALL) : (uint32_t)SSDI8_PHASE_ALL;
+  if (!dims_supported(dims, true)) return SSDI8_ERR_SHAPE;
+  if (!a->xq || !a->Bq || !a->Cq || !a->s_x || !a->s_B || !a->s_C || !a->dt || !a->A || !a->s_xs ||
+      !a->s_cb || !a->s_h || !a->y || !workspace)
+    return SSDI8_ERR_NULL;
+  const void* ptrs[] = {a->xq, a->Bq, a->Cq, a->dt, a->init_state, a->y, a->final_state,
+                        a->tap_cs, a->tap_acc_cb, a->tap_CBq, a->tap_Xsq, a->tap_acc_st, a->tap_loc,
+                        a->tap_prev, a->tap_hq, a->tap_acc_off, a->tap_Mq, a->tap_acc_diag};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return SSDI8_ERR_ALIGN;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SSDI8_ERR_ALIGN;
+  const Dims d = make_dims(dims);
+  const Workspace w = layout(d);
+  if (workspace_bytes < w.total) return SSDI8_ERR_WORKSPACE;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  float* cs = a->tap_cs ? a->tap_cs : reinterpret_cast<float*>(ws + w.cs);
+  float* gamma = reinterpret_cast<float*>(ws + w.gamma);
+  int8_t* cbq = a->tap_CBq ? a->tap_CBq : reinterpret_cast<int8_t*>(ws + w.cbq);
+  float* loc = a->tap_loc ? a->tap_loc : reinterpret_cast<float*>(ws + w.loc);
+  int8_t* hq = a->tap_hq ? a->tap_hq : reinterpret_cast<int8_t*>(ws + w.hq);
+  if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
+
+  if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, cs, gamma, st)) != SSDI8_OK)
+    return s;
+  if ((ph & SSDI8_PHASE_BMM) &&
+      (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, st)) !=
+          SSDI8_OK)
+    return s;
+  if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
+      (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->dt, cs, loc, a->tap_Xsq,
+                              a->tap_acc_st, nullptr, st)) != SSDI8_OK)
+    return s;
+  if ((ph & SSDI8_PHASE_STATE_PASSING) &&
+      (s = launch_state_passing(d, loc, gamma, a->init_state, a->s_h, a->tap_prev, a->final_state,
+                                hq, nullptr, st)) != SSDI8_OK)
+    return s;
+  if (ph & SSDI8_PHASE_SCAN) {
+    ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
+    return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, a->dt, cs,
+                             a->D, a->corr, a->y, taps, st);
+  }
+  return SSDI8_OK;
+}
+
+ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, float* s_xs,
+                               float* s_cb, float* s_h, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  if (!dims || !a) return SSDI8_ERR_NULL;
+  if (!dims_supported(dims, true)) return SSDI8_ERR_SHAPE;
+  if (!a->xq || !a->Bq || !a->Cq || !a->s_x || !a->s_B || !a->s_C || !a->dt || !a->A || !s_xs ||
+      !s_cb || !s_h || !workspace)
+    return SSDI8_ERR_NULL;
+  const void* ptrs[] = {a->xq, a->Bq, a->Cq, a->dt, a->init_state};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return SSDI8_ERR_ALIGN;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SSDI8_ERR_ALIGN;
+  const Dims d = make_dims(dims);
+  const Workspace w = layout(d);
+  if (workspace_bytes < w.total) return SSDI8_ERR_WORKSPACE;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  float* cs = reinterpret_cast<float*>(ws + w.cs);
+  float* gamma = reinterpret_cast<float*>(ws + w.gamma);
+  float* loc = reinterpret_cast<float*>(ws + w.loc);
+  const i64 nhp = (i64)d.H * d.P;
+  // the outputs double as the running maxima (bit patterns), finalised in place
+  SSDI8_CUDA_CHECK(cudaMemsetAsync(s_xs, 0, sizeof(float) * nhp, st));
+  SSDI8_CUDA_CHECK(cudaMemsetAsync(s_cb, 0, sizeof(float) * d.G, st));
+  SSDI8_CUDA_CHECK(cudaMemsetAsync(s_h, 0, sizeof(float) * nhp, st));
+  if ((s = launch_cumsum(d, a->dt, a->A, cs, gamma, st)) != SSDI8_OK) return s;
+  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, nullptr, a->s_B, a->dt, cs, nullptr, nullptr,
+                              nullptr, reinterpret_cast<uint32_t*>(s_xs), st)) != SSDI8_OK)
+    return s;
+  if ((s = launch_finalize_scales(s_xs, nhp, nullptr, nullptr, 0, st)) != SSDI8_OK) return s;
+  if ((s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, nullptr, nullptr, nullptr,
+                      reinterpret_cast<uint32_t*>(s_cb), st)) != SSDI8_OK)
+    return s;
+  if ((s = launch_finalize_scales(s_cb, d.G, a->s_C, a->s_B, 1, st)) != SSDI8_OK) return s;
+  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, s_xs, a->s_B, a->dt, cs, loc, nullptr,
+                              nullptr, nullptr, st)) != SSDI8_OK)
+    return s;
+  if ((s = launch_state_passing(d, loc, gamma, a->init_state, nullptr, nullptr, nullptr, nullptr,
+                                reinterpret_cast<uint32_t*>(s_h), st)) != SSDI8_OK)
+    return s;
+  return launch_finalize_scales(s_h, nhp, nullptr, nullptr, 0, st);
+}
+
+ssdi8_status_t ssdi8_state_passing(const ssdi8_dims_t* dims, const float* loc, const float* gamma,
+                                   const float* init_state, float* prev, float* final_state,
+                                   int8_t* hq, const float* s_h, void* stream) {
+  if (!dims || !loc || !gamma) return SSDI8_ERR_NULL;
+  if (!dims_supported(dims, true)) return SSDI8_ERR_SHAPE;
+  if (hq && !s_h) return SSDI8_ERR_NULL;
+  const void* ptrs[] = {loc, init_state, prev, final_state, hq};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return SSDI8_ERR_ALIGN;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_state_passing(make_dims(dims), loc, gamma, init_state, s_h, prev, final_state, hq,
+                              nullptr, static_cast<cudaStream_t>(stream));
+}
+
+ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const float* s_x,
+                              const int8_t* Bq, const float* s_B, const int8_t* Cq,
+                              const float* s_C, const float* dt, const float* A, const float* D,
+                              const float* corr, float* state, float* y, void* stream) {
+  if (!dims || !xq || !s_x || !Bq || !s_B || !Cq || !s_C || !dt || !A || !state || !y)
+    return SSDI8_ERR_NULL;
+  if (!dims_supported(dims, false)) return SSDI8_ERR_SHAPE;
+  const void* ptrs[] = {xq, Bq, Cq, state, y};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return SSDI8_ERR_ALIGN;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_ssd_step(make_dims(dims), xq, s_x, Bq, s_B, Cq, s_C, dt, A, D, corr, state, y,
+                         static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

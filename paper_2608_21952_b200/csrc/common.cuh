@@ -1,0 +1,76 @@
+// Shared device helpers of the SSDi8 kernels: the binary32 building blocks that
+// decide integer codes (never contracted, never approximated) and small utilities.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ssdi8.h"
+
+namespace ssdi8 {
+
+typedef long long i64;
+
+// round half to even, saturate to [-127, 127] (Eq. 1: 2^(b-1)-1 levels per side)
+__device__ __forceinline__ int rne_clamp(float v) {
+  float r = rintf(v);
+  r = fmaxf(r, -127.0f);  // fmaxf(NaN, a) = a
+  r = fminf(r, 127.0f);
+  return __float2int_rn(r);
+}
+
+// binary32 exponential with a fixed operation sequence (see ssdi8.h): Cody-Waite
+// reduction by ln 2, degree-7 Taylor polynomial (Horner, fmaf), scaling by 2^n
+// through the exponent field.  0 below -80, argument clamped at +80.
+__device__ __forceinline__ float exp32(float x) {
+  if (!(x >= -80.0f)) return 0.0f;
+  x = fminf(x, 80.0f);
+  const float LOG2E = __uint_as_float(0x3FB8AA3Bu);
+  const float LN2_HI = __uint_as_float(0x3F317200u);
+  const float LN2_LO = __uint_as_float(0x35BFBE8Eu);
+  float n = rintf(__fmul_rn(x, LOG2E));
+  float r = __fmaf_rn(n, -LN2_HI, x);
+  r = __fmaf_rn(n, -LN2_LO, r);
+  float p = __uint_as_float(0x39500D01u);                 // 1/5040
+  p = __fmaf_rn(p, r, __uint_as_float(0x3AB60B61u));      // 1/720
+  p = __fmaf_rn(p, r, __uint_as_float(0x3C088889u));      // 1/120
+  p = __fmaf_rn(p, r, __uint_as_float(0x3D2AAAABu));      // 1/24
+  p = __fmaf_rn(p, r, __uint_as_float(0x3E2AAAABu));      // 1/6
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  return __uint_as_float(__float_as_uint(p) + ((uint32_t)__float2int_rn(n) << 23));
+}
+
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+  return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
+         ((uint32_t)(d & 0xff) << 24);
+}
+
+__device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xff); }
+
+struct Dims {
+  int b, L, H, P, N, G, Q, c;
+};
+
+inline Dims make_dims(const ssdi8_dims_t* d) {
+  Dims r;
+  r.b = d->batch; r.L = d->seqlen; r.H = d->nheads; r.P = d->headdim; r.N = d->dstate;
+  r.G = d->ngroups; r.Q = d->chunk; r.c = d->chunk > 0 ? d->seqlen / d->chunk : 0;
+  return r;
+}
+
+#define SSDI8_CUDA_CHECK(expr)                         \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) return SSDI8_ERR_CUDA;     \
+  } while (0)
+
+#define SSDI8_LAUNCH_CHECK()                                       \
+  do {                                                             \
+    if (cudaPeekAtLastError() != cudaSuccess) {                    \
+      (void)cudaGetLastError();                                    \
+      return SSDI8_ERR_CUDA;                                       \
+    }                                                              \
+  } while (0)
+
+}  // namespace ssdi8

@@ -1,0 +1,53 @@
+// Host-side launchers of the SSDi8 kernels (internal to the library).
+#pragma once
+#include "common.cuh"
+
+namespace ssdi8 {
+
+ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
+                               int8_t* out, cudaStream_t st);
+
+// cs [b,H,c,Q], gamma [b,H,c]
+ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* cs,
+                             float* gamma, cudaStream_t st);
+
+// acc_cb (tap, may be NULL), CBq (may be NULL when s_cb is NULL), absmax_acc: per-group
+// running max of |acc_cb| over the causal half (calibration; may be NULL)
+ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, const float* s_C,
+                          const float* s_B, const float* s_cb, int8_t* CBq, int32_t* tap_acc,
+                          uint32_t* absmax_acc, cudaStream_t st);
+
+// absmax_xs: per-channel running max (as binary32 bits) of |x_scaled| (calibration; may be
+// NULL).  When absmax_xs is non-NULL only that is computed.
+ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t* Bq,
+                                  const float* s_x, const float* s_xs, const float* s_B,
+                                  const float* dt, const float* cs, float* loc, int8_t* tap_Xsq,
+                                  int32_t* tap_acc, uint32_t* absmax_xs, cudaStream_t st);
+
+// absmax_h: per-channel running max (binary32 bits) of |S| over init, prev and final
+ssdi8_status_t launch_state_passing(const Dims& d, const float* loc, const float* gamma,
+                                    const float* init, const float* s_h, float* prev,
+                                    float* final_state, int8_t* hq, uint32_t* absmax_h,
+                                    cudaStream_t st);
+
+struct ScanTaps {
+  int32_t* acc_off; float* rowmax; int8_t* Mq; int32_t* acc_diag;
+};
+
+ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* Cq,
+                                 const int8_t* CBq, const int8_t* hq, const float* s_x,
+                                 const float* s_C, const float* s_cb, const float* s_h,
+                                 const float* dt, const float* cs, const float* D,
+                                 const float* corr, float* y, const ScanTaps& taps,
+                                 cudaStream_t st);
+
+ssdi8_status_t launch_ssd_step(const Dims& d, const int8_t* xq, const float* s_x,
+                               const int8_t* Bq, const float* s_B, const int8_t* Cq,
+                               const float* s_C, const float* dt, const float* A, const float* D,
+                               const float* corr, float* state, float* y, cudaStream_t st);
+
+// scale[k] = bits[k] == 0 ? 1 : fdiv(as_float(bits[k]) [* mul], 127)   (in place)
+ssdi8_status_t launch_finalize_scales(float* scale_bits, i64 n, const float* mul_a,
+                                      const float* mul_b, int bits_are_int, cudaStream_t st);
+
+}  // namespace ssdi8

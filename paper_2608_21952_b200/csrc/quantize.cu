@@ -1,0 +1,191 @@
+// Activation quantiser (Eq. 1): uniform symmetric 8-bit with one step size per channel
+// of the view in[R][Ch][I].  HBM-bound: 16-byte loads, 4-byte packed stores, every warp
+// instruction fully coalesced; absmax by per-thread running maxima, warp shuffles and
+// one order-independent atomicMax on the (non-negative) binary32 bit pattern.
+#include "kernels.h"
+
+namespace ssdi8 {
+namespace {
+
+constexpr int QT = 256;      // threads per block
+constexpr int QUNROLL = 4;   // float4 loads in flight per thread
+
+// ---- quantise, I == 1: 4 consecutive elements are 4 consecutive channels
+__global__ void __launch_bounds__(QT) quant_ch_fastest(const float4* __restrict__ in,
+                                                       const float4* __restrict__ scale,
+                                                       uint32_t* __restrict__ out, uint32_t n4,
+                                                       uint32_t ch4) {
+  uint32_t base = blockIdx.x * (QT * QUNROLL) + threadIdx.x;
+  float4 v[QUNROLL];
+  float4 s[QUNROLL];
+#pragma unroll
+  for (int u = 0; u < QUNROLL; ++u) {
+    uint32_t e = base + u * QT;
+    if (e < n4) {
+      v[u] = __ldcs(in + e);
+      s[u] = __ldg(scale + e % ch4);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < QUNROLL; ++u) {
+    uint32_t e = base + u * QT;
+    if (e < n4)
+      out[e] = pack4(rne_clamp(__fdiv_rn(v[u].x, s[u].x)), rne_clamp(__fdiv_rn(v[u].y, s[u].y)),
+                     rne_clamp(__fdiv_rn(v[u].z, s[u].z)), rne_clamp(__fdiv_rn(v[u].w, s[u].w)));
+  }
+}
+
+// ---- quantise, I % 4 == 0: 4 consecutive elements share a channel
+__global__ void __launch_bounds__(QT) quant_inner(const float4* __restrict__ in,
+                                                  const float* __restrict__ scale,
+                                                  uint32_t* __restrict__ out, uint32_t n4,
+                                                  uint32_t I4, uint32_t Ch) {
+  uint32_t base = blockIdx.x * (QT * QUNROLL) + threadIdx.x;
+#pragma unroll
+  for (int u = 0; u < QUNROLL; ++u) {
+    uint32_t e = base + u * QT;
+    if (e < n4) {
+      float4 v = __ldcs(in + e);
+      float s = __ldg(scale + (e / I4) % Ch);
+      out[e] = pack4(rne_clamp(__fdiv_rn(v.x, s)), rne_clamp(__fdiv_rn(v.y, s)),
+                     rne_clamp(__fdiv_rn(v.z, s)), rne_clamp(__fdiv_rn(v.w, s)));
+    }
+  }
+}
+
+// ---- absmax, I == 1.  Thread owns 4 channels and walks rows; grid.y splits the rows.
+__global__ void __launch_bounds__(QT) absmax_ch_fastest(const float4* __restrict__ in,
+                                                        uint32_t* __restrict__ bits, i64 R, int ch4,
+                                                        int rows_per_block) {
+  int q = blockIdx.x * QT + threadIdx.x;
+  if (q >= ch4) return;
+  i64 r0 = (i64)blockIdx.y * rows_per_block;
+  i64 r1 = r0 + rows_per_block < R ? r0 + rows_per_block : R;
+  float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+  i64 r = r0;
+  for (; r + 4 <= r1; r += 4) {
+    float4 v0 = __ldg(in + (r + 0) * ch4 + q), v1 = __ldg(in + (r + 1) * ch4 + q);
+    float4 v2 = __ldg(in + (r + 2) * ch4 + q), v3 = __ldg(in + (r + 3) * ch4 + q);
+    m.x = fmaxf(fmaxf(fmaxf(m.x, fabsf(v0.x)), fmaxf(fabsf(v1.x), fabsf(v2.x))), fabsf(v3.x));
+    m.y = fmaxf(fmaxf(fmaxf(m.y, fabsf(v0.y)), fmaxf(fabsf(v1.y), fabsf(v2.y))), fabsf(v3.y));
+    m.z = fmaxf(fmaxf(fmaxf(m.z, fabsf(v0.z)), fmaxf(fabsf(v1.z), fabsf(v2.z))), fabsf(v3.z));
+    m.w = fmaxf(fmaxf(fmaxf(m.w, fabsf(v0.w)), fmaxf(fabsf(v1.w), fabsf(v2.w))), fabsf(v3.w));
+  }
+  for (; r < r1; ++r) {
+    float4 v = __ldg(in + r * ch4 + q);
+    m.x = fmaxf(m.x, fabsf(v.x)); m.y = fmaxf(m.y, fabsf(v.y));
+    m.z = fmaxf(m.z, fabsf(v.z)); m.w = fmaxf(m.w, fabsf(v.w));
+  }
+  // step size of this partial maximum: fdiv by a positive constant is monotone, so the
+  // maximum of the step sizes is the step size of the maximum
+  atomicMax(bits + 4 * q + 0, __float_as_uint(__fdiv_rn(m.x, 127.0f)));
+  atomicMax(bits + 4 * q + 1, __float_as_uint(__fdiv_rn(m.y, 127.0f)));
+  atomicMax(bits + 4 * q + 2, __float_as_uint(__fdiv_rn(m.z, 127.0f)));
+  atomicMax(bits + 4 * q + 3, __float_as_uint(__fdiv_rn(m.w, 127.0f)));
+}
+
+// ---- absmax, I % 4 == 0.  Block (x = row split, y = channel) reduces its rows of one channel.
+__global__ void __launch_bounds__(QT) absmax_inner(const float4* __restrict__ in,
+                                                   uint32_t* __restrict__ bits, i64 R, int Ch, int I4,
+                                                   int rows_per_block) {
+  __shared__ float red[QT / 32];
+  int ch = blockIdx.y;
+  i64 r0 = (i64)blockIdx.x * rows_per_block;
+  i64 r1 = r0 + rows_per_block < R ? r0 + rows_per_block : R;
+  i64 cnt = (r1 - r0) * I4;
+  float m = 0.f;
+  for (i64 e = threadIdx.x; e < cnt; e += QT) {
+    i64 r = r0 + e / I4;
+    int i = (int)(e % I4);
+    float4 v = __ldg(in + (r * Ch + ch) * I4 + i);
+    m = fmaxf(fmaxf(fmaxf(m, fabsf(v.x)), fmaxf(fabsf(v.y), fabsf(v.z))), fabsf(v.w));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < QT / 32; ++w) m = fmaxf(m, red[w]);
+    atomicMax(bits + ch, __float_as_uint(__fdiv_rn(m, 127.0f)));
+  }
+}
+
+__global__ void finalize_alpha(uint32_t* bits, i64 n) {
+  i64 k = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < n && bits[k] == 0u) bits[k] = __float_as_uint(1.0f);  // all-zero channel: alpha = 1
+}
+
+}  // namespace
+
+ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
+                               int8_t* out, cudaStream_t st) {
+  const i64 n4 = R * Ch * I / 4;
+  if (n4 == 0) return SSDI8_OK;
+  uint32_t* bits = reinterpret_cast<uint32_t*>(scale);
+  if (mode == 1 || mode == 2) {
+    if (mode == 1) SSDI8_CUDA_CHECK(cudaMemsetAsync(scale, 0, sizeof(float) * Ch, st));
+    if (I == 1) {
+      int ch4 = (int)(Ch / 4);
+      int gx = (ch4 + QT - 1) / QT;
+      // enough row splits to fill the machine, at least 64 rows each
+      i64 want = (148 * 8 + gx - 1) / gx;
+      i64 rows = (R + want - 1) / want;
+      if (rows < 64) rows = 64;
+      int gy = (int)((R + rows - 1) / rows);
+      absmax_ch_fastest<<<dim3(gx, gy), QT, 0, st>>>(reinterpret_cast<const float4*>(in), bits, R,
+                                                      ch4, (int)rows);
+    } else {
+      int I4 = (int)(I / 4);
+      i64 want = (148 * 8 + Ch - 1) / Ch;
+      i64 rows = (R + want - 1) / want;
+      i64 min_rows = (QT * 4 + I4 - 1) / I4;
+      if (rows < min_rows) rows = min_rows;
+      int gx = (int)((R + rows - 1) / rows);
+      absmax_inner<<<dim3(gx, (unsigned)Ch), QT, 0, st>>>(reinterpret_cast<const float4*>(in), bits,
+                                                           R, (int)Ch, I4, (int)rows);
+    }
+    SSDI8_LAUNCH_CHECK();
+    if (mode == 1) {
+      finalize_alpha<<<(unsigned)((Ch + 255) / 256), 256, 0, st>>>(bits, Ch);
+      SSDI8_LAUNCH_CHECK();
+    }
+  }
+  if (!out) return SSDI8_OK;
+  unsigned grid = (unsigned)((n4 + QT * QUNROLL - 1) / (QT * QUNROLL));
+  if (I == 1)
+    quant_ch_fastest<<<grid, QT, 0, st>>>(reinterpret_cast<const float4*>(in),
+                                          reinterpret_cast<const float4*>(scale),
+                                          reinterpret_cast<uint32_t*>(out), (uint32_t)n4, (uint32_t)(Ch / 4));
+  else
+    quant_inner<<<grid, QT, 0, st>>>(reinterpret_cast<const float4*>(in), scale,
+                                     reinterpret_cast<uint32_t*>(out), (uint32_t)n4, (uint32_t)(I / 4),
+                                     (uint32_t)Ch);
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+// bits[k] holds either a binary32 absmax or (bits_are_int) an int32 absmax; the step size is
+// fdiv(fmul(value, fmul(mul_a[k], mul_b[k])), 127) (multipliers optional), 1 if the value is 0.
+namespace {
+__global__ void finalize_scales_k(float* s, i64 n, const float* mul_a, const float* mul_b,
+                                  int bits_are_int) {
+  i64 k = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= n) return;
+  uint32_t u = __float_as_uint(s[k]);
+  if (u == 0u) { s[k] = 1.0f; return; }
+  float v = bits_are_int ? (float)(int)u : s[k];
+  if (mul_a) v = __fmul_rn(v, __fmul_rn(mul_a[k], mul_b[k]));
+  s[k] = __fdiv_rn(v, 127.0f);
+}
+}  // namespace
+
+ssdi8_status_t launch_finalize_scales(float* scale_bits, i64 n, const float* mul_a,
+                                      const float* mul_b, int bits_are_int, cudaStream_t st) {
+  finalize_scales_k<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(scale_bits, n, mul_a, mul_b,
+                                                                 bits_are_int);
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+}  // namespace ssdi8

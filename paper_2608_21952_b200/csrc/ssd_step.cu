@@ -1,0 +1,87 @@
+// Recurrent-mode single-token step (the recurrence that Algorithm 2 unrolls; the paper has
+// no algorithm for it):  S <- exp(dt A) S + (dt s_x s_B) x B^T,  y = s_C C S + D s_x x + corr.
+// Pure streaming over the fp32 state [b,H,P,N]: one read and one write of the state per
+// token, 16-byte accesses, N/4 lanes per (b,h,p) row, ROWS rows per lane group in flight.
+#include "kernels.h"
+
+namespace ssdi8 {
+namespace {
+
+constexpr int ST_T = 256;
+constexpr int ROWS = 4;  // consecutive p per lane group
+
+template <int N4>  // lanes per row: 32 (N = 128) or 16 (N = 64)
+__global__ void __launch_bounds__(ST_T) ssd_step_kernel(
+    const int8_t* __restrict__ xq, const float* __restrict__ s_x, const uint32_t* __restrict__ Bq,
+    const float* __restrict__ s_B, const uint32_t* __restrict__ Cq, const float* __restrict__ s_C,
+    const float* __restrict__ dt, const float* __restrict__ A, const float* __restrict__ D,
+    const float* __restrict__ corr, float4* __restrict__ state, float* __restrict__ y, Dims d) {
+  const int lane = threadIdx.x % N4;
+  const i64 grp = ((i64)blockIdx.x * ST_T + threadIdx.x) / N4;  // over b*H*P/ROWS
+  const int pgroups = d.P / ROWS;
+  const i64 bh = grp / pgroups;
+  if (bh >= (i64)d.b * d.H) return;
+  const int p0 = (int)(grp % pgroups) * ROWS;
+  const int b = (int)(bh / d.H), h = (int)(bh % d.H);
+  const int g = h / (d.H / d.G);
+  float4* S = state + ((bh * d.P + p0) * N4 + lane);
+  float4 s[ROWS];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) s[r] = S[r * N4];
+  const float dtv = dt[bh];
+  const float a = expf(dtv * A[h]);
+  const uint32_t bw = Bq[((i64)b * d.G + g) * N4 + lane];
+  const uint32_t cw = Cq[((i64)b * d.G + g) * N4 + lane];
+  const float b0 = (float)sx8(bw, 0), b1 = (float)sx8(bw, 1), b2 = (float)sx8(bw, 2), b3 = (float)sx8(bw, 3);
+  const float c0 = (float)sx8(cw, 0), c1 = (float)sx8(cw, 1), c2 = (float)sx8(cw, 2), c3 = (float)sx8(cw, 3);
+  const float sB = s_B[g], sC = s_C[g];
+  float acc[ROWS];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    const int hp = h * d.P + p0 + r;
+    const float xv = s_x[hp] * (float)xq[bh * d.P + p0 + r];
+    const float u = dtv * xv * sB;
+    s[r].x = fmaf(a, s[r].x, u * b0);
+    s[r].y = fmaf(a, s[r].y, u * b1);
+    s[r].z = fmaf(a, s[r].z, u * b2);
+    s[r].w = fmaf(a, s[r].w, u * b3);
+    acc[r] = c0 * s[r].x + c1 * s[r].y + c2 * s[r].z + c3 * s[r].w;
+    S[r * N4] = s[r];
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+    for (int o = N4 / 2; o > 0; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+  if (lane < ROWS) {
+    float v = 0.f;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) if (lane == r) v = acc[r];
+    const int hp = h * d.P + p0 + lane;
+    v *= sC;
+    if (D) v += D[h] * s_x[hp] * (float)xq[bh * d.P + p0 + lane];
+    if (corr) v += corr[hp];
+    y[bh * d.P + p0 + lane] = v;
+  }
+}
+
+}  // namespace
+
+ssdi8_status_t launch_ssd_step(const Dims& d, const int8_t* xq, const float* s_x,
+                               const int8_t* Bq, const float* s_B, const int8_t* Cq,
+                               const float* s_C, const float* dt, const float* A, const float* D,
+                               const float* corr, float* state, float* y, cudaStream_t st) {
+  const int N4 = d.N / 4;
+  const i64 threads = (i64)d.b * d.H * (d.P / ROWS) * N4;
+  unsigned grid = (unsigned)((threads + ST_T - 1) / ST_T);
+  auto Bw = reinterpret_cast<const uint32_t*>(Bq);
+  auto Cw = reinterpret_cast<const uint32_t*>(Cq);
+  auto S4 = reinterpret_cast<float4*>(state);
+  if (N4 == 32)
+    ssd_step_kernel<32><<<grid, ST_T, 0, st>>>(xq, s_x, Bw, s_B, Cw, s_C, dt, A, D, corr, S4, y, d);
+  else
+    ssd_step_kernel<16><<<grid, ST_T, 0, st>>>(xq, s_x, Bw, s_B, Cw, s_C, dt, A, D, corr, S4, y, d);
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+}  // namespace ssdi8

@@ -1,0 +1,305 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle on seeded inputs.
+
+Bar: bit-exact on every int8 tensor and int32 accumulator and on the fp32 tensors that
+are defined operation by operation (cs, loc, states); max-abs error <= 1e-3 * RMS on
+the fp32 output y and on the final state.
+"""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2608_21952_b200 import inputs
+from paper_2608_21952_b200.inputs import CONFIGS, SSDConfig
+from helpers import rms
+
+pytestmark = pytest.mark.gpu
+
+Y_TOL = 1e-3  # max-abs error relative to the RMS of the reference output
+
+
+def _harness():
+    import gpu_harness
+    return gpu_harness
+
+
+def _causal(cfg):
+    return np.tril(np.ones((cfg.chunk, cfg.chunk), bool))
+
+
+def check_fwd(cfg, init=None, corr=None, use_D=True):
+    gh = _harness()
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t, init)
+    y_ref, fin_ref, ref = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"],
+                                        q["dt"], q["A"], q["D"] if use_D else None, corr, q["s_xs"],
+                                        q["s_cb"], q["s_h"], init, taps=gh.TAP_NAMES)
+    y, fin, got = gh.gpu_fwd(cfg, q, corr=corr, D="use" if use_D else None)
+    tril = _causal(cfg)
+    for name in ("cs", "Xsq", "acc_st", "loc", "prev", "hq", "acc_off", "rowmax", "Mq", "acc_diag"):
+        assert np.array_equal(got[name], ref[name]), name
+    for name in ("acc_cb", "CBq"):  # only the causal half is defined
+        assert np.array_equal(got[name][..., tril], ref[name][..., tril]), name
+    assert np.array_equal(fin, fin_ref)
+    assert np.abs(y - y_ref).max() <= Y_TOL * rms(y_ref)
+    return y, y_ref
+
+
+SMALL = [
+    CONFIGS["cfg0"],
+    SSDConfig("g2_n64_q128", 2, 256, 4, 64, 64, 2, 128, 0.02, 20.0, 21),
+    SSDConfig("n128_q256", 1, 512, 3, 64, 128, 1, 256, 0.02, 20.0, 22),
+    SSDConfig("g4_q64", 2, 128, 8, 64, 128, 4, 64, 0.02, 20.0, 23),
+    SSDConfig("one_chunk", 1, 128, 2, 64, 64, 1, 128, 0.02, 20.0, 24),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_fwd_all_taps_bit_exact(cfg):
+    check_fwd(cfg)
+
+
+def test_fwd_with_init_state_and_correction():
+    cfg = SMALL[1]
+    init = inputs.make_init_state(cfg, 0.5)
+    corr = (0.05 * np.random.default_rng(3).standard_normal(cfg.channels)).astype(np.float32)
+    check_fwd(cfg, init=init, corr=corr)
+
+
+def test_fwd_without_skip_weight():
+    check_fwd(SMALL[0], use_D=False)
+
+
+def test_fwd_cfg1_full():
+    check_fwd(CONFIGS["cfg1"])
+
+
+def test_fwd_degenerate_inputs():
+    """dt = 0 (every decay exactly 1, nothing enters the state) and x = 0 (all-zero rows of
+    the masked operand) run through the same path."""
+    gh = _harness()
+    cfg = SMALL[0]
+    t = inputs.make_prefill(cfg)
+    for case in ("dt0", "x0"):
+        tt = dict(t)
+        if case == "dt0":
+            tt["dt"] = np.zeros_like(t["dt"])
+        else:
+            tt["x"] = np.zeros_like(t["x"])
+        q = orc.prepare_quantized(cfg, tt)
+        y_ref, fin_ref, ref = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"],
+                                            q["dt"], q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"],
+                                            None, taps=("Mq", "rowmax", "hq", "Xsq"))
+        y, fin, got = gh.gpu_fwd(cfg, q, taps=("Mq", "rowmax", "hq", "Xsq"))
+        for name in ("Mq", "rowmax", "hq", "Xsq"):
+            assert np.array_equal(got[name], ref[name]), (case, name)
+        assert np.array_equal(fin, fin_ref)
+        assert np.abs(y - y_ref).max() <= Y_TOL * max(rms(y_ref), 1e-30)
+
+
+def _sampled_problem(cfg, t, pairs):
+    """Scales for a full-size workload without running the oracle on all of it: Eq. 1 on the
+    whole input tensors, internal step sizes calibrated by the oracle on the sampled
+    (batch, head) pairs and reused for the other heads (any positive step size is a valid
+    static scale; codes beyond it saturate)."""
+    T = cfg.tokens
+    xq, s_x = orc.quantize(t["x"], T, cfg.channels, 1, mode=1)
+    Bq, s_B = orc.quantize(t["B"], T, cfg.ngroups, cfg.dstate, mode=1)
+    Cq, s_C = orc.quantize(t["C"], T, cfg.ngroups, cfg.dstate, mode=1)
+    P = cfg.headdim
+    hpg = cfg.nheads // cfg.ngroups
+    one = cfg.replace(batch=1, nheads=1, ngroups=1)
+    per_head = {}
+    for (b, h) in pairs:
+        g = h // hpg
+        sub = _slice(cfg, b, h, xq, Bq, Cq, s_x, s_B, s_C, t)
+        s_xs, s_cb, s_h = orc.calibrate(one, sub["xq"], sub["Bq"], sub["Cq"], sub["s_x"], sub["s_B"],
+                                        sub["s_C"], sub["dt"], sub["A"])
+        per_head[h] = (s_xs, s_h, g, s_cb)
+    hs = sorted(per_head)
+    s_xs = np.empty(cfg.channels, np.float32); s_h = np.empty(cfg.channels, np.float32)
+    s_cb = np.ones(cfg.ngroups, np.float32)
+    for h in range(cfg.nheads):
+        src = per_head[hs[h % len(hs)]]
+        ratio = s_x[h * P:(h + 1) * P] / s_x[hs[h % len(hs)] * P:(hs[h % len(hs)] + 1) * P]
+        s_xs[h * P:(h + 1) * P] = src[0] * ratio
+        s_h[h * P:(h + 1) * P] = src[1] * ratio
+    for g in range(cfg.ngroups):
+        c = [v[3][0] for v in per_head.values() if v[2] == g]
+        s_cb[g] = max(c) if c else max(v[3][0] for v in per_head.values())
+    return dict(xq=xq, Bq=Bq, Cq=Cq, s_x=s_x, s_B=s_B, s_C=s_C, dt=t["dt"], A=t["A"], D=t["D"],
+                s_xs=s_xs.astype(np.float32), s_cb=s_cb, s_h=s_h.astype(np.float32), init=None)
+
+
+def _slice(cfg, b, h, xq, Bq, Cq, s_x, s_B, s_C, t, extra=None):
+    P = cfg.headdim
+    g = h // (cfg.nheads // cfg.ngroups)
+    d = dict(xq=xq[b:b + 1, :, h:h + 1], Bq=Bq[b:b + 1, :, g:g + 1], Cq=Cq[b:b + 1, :, g:g + 1],
+             s_x=s_x[h * P:(h + 1) * P], s_B=s_B[g:g + 1], s_C=s_C[g:g + 1],
+             dt=t["dt"][b:b + 1, :, h:h + 1], A=t["A"][h:h + 1], D=t["D"][h:h + 1])
+    if extra:
+        d.update(s_xs=extra["s_xs"][h * P:(h + 1) * P], s_cb=extra["s_cb"][g:g + 1],
+                 s_h=extra["s_h"][h * P:(h + 1) * P])
+    return {k: np.ascontiguousarray(v) for k, v in d.items()}
+
+
+@pytest.mark.parametrize("name,npairs", [("cfg2", 4), ("cfg3", 3)])
+def test_fwd_full_size_sampled(name, npairs):
+    """Full-size workloads in the launch configuration the benchmark times (no taps); the
+    oracle recomputes sampled (batch, head) pairs one by one."""
+    gh = _harness()
+    cfg = CONFIGS[name]
+    t = inputs.make_prefill(cfg)
+    rng = np.random.default_rng(100 + cfg.seed)
+    pairs = [(0, 0), (cfg.batch - 1, cfg.nheads - 1)]
+    while len(pairs) < npairs:
+        pr = (int(rng.integers(cfg.batch)), int(rng.integers(cfg.nheads)))
+        if pr not in pairs:
+            pairs.append(pr)
+    q = _sampled_problem(cfg, t, pairs)
+    y, fin, _ = gh.gpu_fwd(cfg, q, taps=())
+    assert np.all(np.isfinite(y)) and np.all(np.isfinite(fin))
+    one = cfg.replace(batch=1, nheads=1, ngroups=1)
+    for (b, h) in pairs:
+        s = _slice(cfg, b, h, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], t, extra=q)
+        y_ref, fin_ref, _ = orc.ssdi8_fwd(one, s["xq"], s["Bq"], s["Cq"], s["s_x"], s["s_B"], s["s_C"],
+                                          s["dt"], s["A"], s["D"], None, s["s_xs"], s["s_cb"], s["s_h"])
+        assert np.array_equal(fin[b, h], fin_ref[0, 0]), (b, h)
+        assert np.abs(y[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
+
+
+# --------------------------------------------------------------------------- quantiser
+@pytest.mark.parametrize("R,Ch,I", [(512, 256, 1), (37, 8, 1), (1000, 5120, 1), (512, 1, 64),
+                                    (333, 8, 128), (4, 4, 4), (1, 4, 1)])
+def test_quantizer_bit_exact(R, Ch, I):
+    gh = _harness()
+    rng = np.random.default_rng(R + Ch + I)
+    v = (rng.standard_normal((R, Ch, I)) * rng.uniform(0.05, 40, (1, Ch, 1))).astype(np.float32)
+    v[:, Ch // 2, :] = 0 if Ch > 1 else v[:, 0, :]
+    q_ref, s_ref = orc.quantize(v, R, Ch, I, mode=1)
+    q, s = gh.gpu_quantize(v, R, Ch, I, mode=1)
+    assert np.array_equal(s, s_ref) and np.array_equal(q, q_ref)
+    # static mode with a step size that saturates part of the tensor
+    st = (s_ref * 0.5).astype(np.float32)
+    q_ref, _ = orc.quantize(v, R, Ch, I, scale=st, mode=0)
+    q, s2 = gh.gpu_quantize(v, R, Ch, I, scale=st, mode=0)
+    assert np.array_equal(q, q_ref) and np.array_equal(s2, st)
+    # observe mode keeps the running maximum and writes nothing else
+    _, s_obs_ref = orc.quantize(v * 0.5, R, Ch, I, scale=s_ref, mode=2, want_out=False)
+    _, s_obs = gh.gpu_quantize(v * 0.5, R, Ch, I, scale=s_ref, mode=2, want_out=False)
+    assert np.array_equal(s_obs, s_obs_ref) and np.array_equal(s_obs, s_ref)
+    _, s_obs_ref = orc.quantize(v * 3, R, Ch, I, scale=s_ref, mode=2, want_out=False)
+    _, s_obs = gh.gpu_quantize(v * 3, R, Ch, I, scale=s_ref, mode=2, want_out=False)
+    assert np.array_equal(s_obs, s_obs_ref)
+
+
+def test_quantizer_empty_input_is_a_no_op():
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    x = torch.zeros(16, device="cuda"); s = torch.ones(4, device="cuda")
+    o = torch.full((16,), 5, dtype=torch.int8, device="cuda")
+    bd.ssdi8_quantize_act(x, 0, 4, 1, s, 0, o)
+    torch.cuda.synchronize()
+    assert bool((o == 5).all())
+
+
+def test_quantizer_full_size_x_and_bc():
+    gh = _harness()
+    cfg = CONFIGS["cfg2"]
+    t = inputs.make_prefill(cfg)
+    for key, Ch, I in (("x", cfg.channels, 1), ("B", cfg.ngroups, cfg.dstate)):
+        q_ref, s_ref = orc.quantize(t[key], cfg.tokens, Ch, I, mode=1)
+        q, s = gh.gpu_quantize(t[key], cfg.tokens, Ch, I, mode=1)
+        assert np.array_equal(s, s_ref) and np.array_equal(q, q_ref)
+
+
+# --------------------------------------------------------------------------- calibration
+@pytest.mark.parametrize("cfg", SMALL[:3], ids=lambda c: c.name)
+def test_calibrate_bit_exact(cfg):
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A")}
+    args = bd.make_fwd_args(init_state=gh.dev(init), **dv)
+    s_xs = torch.empty(cfg.channels, device="cuda"); s_cb = torch.empty(cfg.ngroups, device="cuda")
+    s_h = torch.empty(cfg.channels, device="cuda")
+    ws = bd.alloc_workspace(dims)
+    bd.ssdi8_calibrate(dims, args, s_xs, s_cb, s_h, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(s_xs.cpu().numpy(), q["s_xs"])
+    assert np.array_equal(s_cb.cpu().numpy(), q["s_cb"])
+    assert np.array_equal(s_h.cpu().numpy(), q["s_h"])
+
+
+# --------------------------------------------------------------------------- state passing
+@pytest.mark.parametrize("alias", [False, True])
+def test_state_passing_standalone(alias):
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SSDConfig("sp", 2, 6 * 64, 3, 64, 128, 1, 64, 0, 1, 31)
+    rng = np.random.default_rng(31)
+    shp = (cfg.batch, cfg.nchunks, cfg.nheads, cfg.headdim, cfg.dstate)
+    loc = rng.standard_normal(shp).astype(np.float32)
+    gamma = rng.uniform(0.0, 1.0, (cfg.batch, cfg.nheads, cfg.nchunks)).astype(np.float32)
+    init = rng.standard_normal(shp[:1] + shp[2:]).astype(np.float32)
+    s_h = rng.uniform(0.01, 0.05, cfg.channels).astype(np.float32)
+    prev_ref, fin_ref, hq_ref = orc.state_passing(cfg, loc, gamma, init, s_h)
+    dloc = gh.dev(loc)
+    prev = dloc if alias else torch.empty_like(dloc)
+    fin = torch.empty(shp[:1] + shp[2:], device="cuda")
+    hq = torch.empty(shp, dtype=torch.int8, device="cuda")
+    bd.ssdi8_state_passing(bd.dims_of(cfg), dloc, gh.dev(gamma), gh.dev(init), prev, fin, hq, gh.dev(s_h))
+    torch.cuda.synchronize()
+    assert np.array_equal(prev.cpu().numpy(), prev_ref)
+    assert np.array_equal(fin.cpu().numpy(), fin_ref)
+    assert np.array_equal(hq.cpu().numpy(), hq_ref)
+
+
+# --------------------------------------------------------------------------- decode step
+def _decode_case(cfg, steps):
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    prm = inputs.make_decode_params(cfg)
+    raw = [inputs.make_decode_step(cfg, s) for s in range(steps)]
+    # static scales over all steps (Eq. 1, observe mode)
+    s_x = np.zeros(cfg.channels, np.float32); s_B = np.zeros(cfg.ngroups, np.float32)
+    s_C = np.zeros(cfg.ngroups, np.float32)
+    for r in raw:
+        _, s_x = orc.quantize(r["x"], cfg.batch, cfg.channels, 1, scale=s_x, mode=2, want_out=False)
+        _, s_B = orc.quantize(r["B"], cfg.batch, cfg.ngroups, cfg.dstate, scale=s_B, mode=2, want_out=False)
+        _, s_C = orc.quantize(r["C"], cfg.batch, cfg.ngroups, cfg.dstate, scale=s_C, mode=2, want_out=False)
+    corr = np.linspace(-0.2, 0.2, cfg.channels).astype(np.float32)
+    st_ref = np.zeros((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate))
+    state = torch.zeros(st_ref.shape, device="cuda")
+    y = torch.empty((cfg.batch, cfg.nheads, cfg.headdim), device="cuda")
+    dims = bd.dims_of(cfg)
+    d = {k: gh.dev(v) for k, v in dict(s_x=s_x, s_B=s_B, s_C=s_C, A=prm["A"], D=prm["D"], corr=corr).items()}
+    worst = 0.0
+    for r in raw:
+        xq, _ = orc.quantize(r["x"], cfg.batch, cfg.channels, 1, scale=s_x, mode=0)
+        Bq, _ = orc.quantize(r["B"], cfg.batch, cfg.ngroups, cfg.dstate, scale=s_B, mode=0)
+        Cq, _ = orc.quantize(r["C"], cfg.batch, cfg.ngroups, cfg.dstate, scale=s_C, mode=0)
+        y_ref = orc.ssd_step(cfg, xq, s_x, Bq, s_B, Cq, s_C, r["dt"], prm["A"], prm["D"], corr, st_ref)
+        bd.ssdi8_ssd_step(dims, gh.dev(xq), d["s_x"], gh.dev(Bq), d["s_B"], gh.dev(Cq), d["s_C"],
+                          gh.dev(r["dt"]), d["A"], d["D"], d["corr"], state, y)
+        worst = max(worst, np.abs(y.cpu().numpy() - y_ref).max() / rms(y_ref))
+    assert worst <= Y_TOL
+    got = state.cpu().numpy()
+    assert np.abs(got - st_ref).max() <= Y_TOL * rms(st_ref)
+
+
+def test_step_256_tokens_small_batch():
+    _decode_case(CONFIGS["cfg4"].replace(batch=2, nheads=8), 256)
+
+
+def test_step_n64_groups():
+    _decode_case(SSDConfig("dec64", 3, 1, 4, 64, 64, 2, 64, 0.02, 20.0, 41, decode_steps=16), 16)
+
+
+def test_step_full_size_batch():
+    _decode_case(CONFIGS["cfg4"], 8)
