@@ -141,7 +141,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
     return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, a->dt, cs,
-                             a->D, a->corr, a->y, taps, st);
+                             a->D, a->corr, a->y, a->status, taps, st);
   }
   return SSDI8_OK;
 }
