@@ -348,6 +348,16 @@ def run_ours(args):
         ms = float(tms.item())
     value = world * cfg.tokens / (ms * 1e-3)
 
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "quick": True,
+                              "config": workload_config(cfg, world), "clocks": clk.summary()}))
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
     # end to end: pinned host fp32 inputs -> device, the step, fp32 y -> pinned host
     for _ in range(2):
         layer.e2e_step()
@@ -409,6 +419,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
+    ap.add_argument("--quick", action="store_true",
+                    help="timed steps only: skip the end-to-end, per-module, decode and CPU legs (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 5:

@@ -132,7 +132,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
     return s;
   if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
       (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->dt, cs, loc, a->tap_Xsq,
-                              a->tap_acc_st, nullptr, st)) != SSDI8_OK)
+                              a->tap_acc_st, nullptr, a->status, st)) != SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_STATE_PASSING) &&
       (s = launch_state_passing(d, loc, gamma, a->init_state, a->s_h, a->tap_prev, a->final_state,
@@ -175,7 +175,7 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
   SSDI8_CUDA_CHECK(cudaMemsetAsync(s_h, 0, sizeof(float) * nhp, st));
   if ((s = launch_cumsum(d, a->dt, a->A, cs, gamma, st)) != SSDI8_OK) return s;
   if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, nullptr, a->s_B, a->dt, cs, nullptr, nullptr,
-                              nullptr, reinterpret_cast<uint32_t*>(s_xs), st)) != SSDI8_OK)
+                              nullptr, reinterpret_cast<uint32_t*>(s_xs), nullptr, st)) != SSDI8_OK)
     return s;
   if ((s = launch_finalize_scales(s_xs, nhp, nullptr, nullptr, 0, st)) != SSDI8_OK) return s;
   if ((s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, nullptr, nullptr, nullptr,
@@ -183,7 +183,7 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
     return s;
   if ((s = launch_finalize_scales(s_cb, d.G, a->s_C, a->s_B, 1, st)) != SSDI8_OK) return s;
   if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, s_xs, a->s_B, a->dt, cs, loc, nullptr,
-                              nullptr, nullptr, st)) != SSDI8_OK)
+                              nullptr, nullptr, nullptr, st)) != SSDI8_OK)
     return s;
   if ((s = launch_state_passing(d, loc, gamma, a->init_state, nullptr, nullptr, nullptr, nullptr,
                                 reinterpret_cast<uint32_t*>(s_h), st)) != SSDI8_OK)

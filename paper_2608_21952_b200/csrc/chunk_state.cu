@@ -1,96 +1,159 @@
-// ChunkState with the sparse-aware reformulation (Eq. 3) and the INT32 rescale (Eq. 4):
+// ChunkState with the sparse-aware reformulation (Eq. 3) and the INT32 rescale (Eq. 4) on
+// tcgen05 tensor cores.  One CTA per (batch, chunk, head):
 //   LUT_state[i] = fmul(dt_i, exp32(fsub(cs_last, cs_i)))
-//   Xs_q[i,p]    = rne(fmul(fmul(float(xq[i,p]), fdiv(s_x, s_xs)), LUT_state[i]))
-//   acc_st[p,n]  = sum_i Xs_q[i,p] Bq[i,n]   (contraction over the tokens of the chunk)
+//   Xs_q[i,p]    = rne(fmul(fmul(float(xq[i,p]), fdiv(s_x, s_xs)), LUT_state[i]))   in place in smem
+//   acc_st[n,p]  = sum_i Bq[i,n] Xs_q[i,p]     INT8 MMA over the tokens of the chunk, INT32 in TMEM
 //   loc[p,n]     = fmul(float(acc_st), fmul(s_xs[h,p], s_B[g]))
-// One block per (batch, chunk, head).
+// Both operands are token-major in HBM, i.e. MN-major for this contraction: TMA stages them
+// as they are and the MMA reads them through MN-major descriptors (no transposes anywhere).
+// The accumulator is held with the state index n on the TMEM lanes, so that each warp store
+// of the epilogue writes 32 consecutive n of one p: full 128-byte lines of loc[p][n].
 #include "kernels.h"
-#include "mma_s8.cuh"
+#include "sm100.cuh"
 
 namespace ssdi8 {
 namespace {
 
-__global__ void __launch_bounds__(256) chunk_state_kernel(
-    const int8_t* __restrict__ xq, const int8_t* __restrict__ Bq, const float* __restrict__ s_x,
-    const float* __restrict__ s_xs, const float* __restrict__ s_B, const float* __restrict__ dt,
-    const float* __restrict__ cs, float* __restrict__ loc, int8_t* __restrict__ tap_Xsq,
-    int32_t* __restrict__ tap_acc, uint32_t* __restrict__ absmax_xs, Dims d) {
-  extern __shared__ __align__(16) int8_t smem[];
-  const int Q = d.Q, P = d.P, N = d.N, ld = Q + 16;
+using namespace sm100;
+
+struct StateArgs {
+  const float* s_x; const float* s_xs; const float* s_B; const float* dt; const float* cs;
+  float* loc; int8_t* tap_Xsq; int32_t* tap_acc; uint32_t* absmax_xs; int32_t* status;
+  Dims d;
+};
+
+constexpr int kThreads = 256;
+constexpr uint32_t OFF_B = 0;        // [Q][N]  Bq rows (token-major)
+constexpr uint32_t OFF_X = 32768;    // [Q][64] xq rows -> Xs_q in place
+constexpr uint32_t OFF_F = 49152;    // lut[256], bars, tmem slot
+constexpr uint32_t SMEM_BYTES = OFF_F + 256 * 4 + 64;
+
+__global__ void __launch_bounds__(kThreads, 3)
+chunk_state_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
+               const StateArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const Dims& d = a.d;
+  const int Q = d.Q, N = d.N, P = d.P;
+  const int TQ = Q < 128 ? Q : 128;  // rows per TMA box
   const int h = blockIdx.x, k = blockIdx.y, b = blockIdx.z;
   const int g = h / (d.H / d.G);
-  int8_t* XsT = smem;                  // [P][ld]  Xs_q transposed: row p, token contiguous
-  int8_t* BT = smem + P * ld;          // [N][ld]
-  float* lut = reinterpret_cast<float*>(smem + (P + N) * ld);  // [Q]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-  const float* csk = cs + (((i64)b * d.H + h) * d.c + k) * Q;
-  const float cs_last = csk[Q - 1];
-  for (int i = threadIdx.x; i < Q; i += blockDim.x)
-    lut[i] = __fmul_rn(dt[(tok0 + i) * d.H + h], exp32(__fsub_rn(cs_last, csk[i])));
-  __syncthreads();
-  // --- prologue: X_scaled, re-quantised, written transposed
-  const int pw = P / 4;  // words per token
-  const int pq = threadIdx.x % pw;
-  float rx[4], sx[4];
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    sx[u] = s_x[h * P + 4 * pq + u];
-    rx[u] = absmax_xs ? sx[u] : __fdiv_rn(sx[u], s_xs[h * P + 4 * pq + u]);
+  uint8_t* sB = smem + OFF_B;
+  uint8_t* sX = smem + OFF_X;
+  float* lut = reinterpret_cast<float*>(smem + OFF_F);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lut + 256);  // [0] operands landed, [1] MMA done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
+  const bool calib = a.absmax_xs != nullptr;
+
+  if (tid == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tm_B);
+    tma_prefetch_desc(&tm_x);
   }
-  float mx[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int i = threadIdx.x / pw; i < Q; i += blockDim.x / pw) {
-    const i64 o = ((tok0 + i) * d.H + h) * P + 4 * pq;
-    const uint32_t w = *reinterpret_cast<const uint32_t*>(xq + o);
-    const float l = lut[i];
-    if (absmax_xs) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        mx[u] = fmaxf(mx[u], fabsf(__fmul_rn(__fmul_rn((float)sx8(w, u), rx[u]), l)));
-    } else {
-      int q[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        q[u] = rne_clamp(__fmul_rn(__fmul_rn((float)sx8(w, u), rx[u]), l));
-        XsT[(4 * pq + u) * ld + i] = (int8_t)q[u];
-      }
-      if (tap_Xsq) *reinterpret_cast<uint32_t*>(tap_Xsq + o) = pack4(q[0], q[1], q[2], q[3]);
+  if (warp == 1 && !calib) tmem_alloc(tmem_slot, 64);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (tid == 0) {
+    mbar_expect_tx(&bars[0], (uint32_t)(Q * 64 + (calib ? 0 : Q * N)));
+    for (int i0 = 0; i0 < Q; i0 += TQ) {
+      tma_load_3d(sX + i0 * 64, &tm_x, &bars[0], 0, h, (int)(tok0 + i0));
+      if (!calib) tma_load_3d(sB + i0 * N, &tm_B, &bars[0], 0, g, (int)(tok0 + i0));
     }
   }
-  if (absmax_xs) {
+  const float* csk = a.cs + (((i64)b * d.H + h) * d.c + k) * Q;
+  const float cs_last = csk[Q - 1];
+  if (tid < Q) lut[tid] = __fmul_rn(a.dt[(tok0 + tid) * d.H + h], exp32(__fsub_rn(cs_last, csk[tid])));
+  // per-column factors of this thread's 16 channels (16-byte chunk c of every row it visits)
+  const int c = tid & 3;
+  float rx[16];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) atomicMax(absmax_xs + h * P + 4 * pq + u, __float_as_uint(mx[u]));
-    return;
-  }
-  const int nw = N / 4;
-  for (int e = threadIdx.x; e < Q * nw; e += blockDim.x) {
-    const int i = e / nw, w4 = e % nw;
-    const uint32_t w = *reinterpret_cast<const uint32_t*>(Bq + ((tok0 + i) * d.G + g) * N + 4 * w4);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) BT[(4 * w4 + u) * ld + i] = (int8_t)sx8(w, u);
+  for (int e = 0; e < 16; ++e) {
+    const int hp = h * P + c * 16 + e;
+    rx[e] = calib ? a.s_x[hp] : __fdiv_rn(a.s_x[hp], a.s_xs[hp]);
   }
   __syncthreads();
-  // --- acc[p][n]: 8 warps = 4 row blocks of 16 p  x  2 column halves of N/2
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = (warp & 3) * 16, nh = N / 2, n0 = (warp >> 2) * nh;
-  const float sB = s_B[g];
-  const i64 obase = ((((i64)b * d.c + k) * d.H + h) * P) * N;
-  for (int nb = 0; nb < nh; nb += 32) {
-    int acc[4][4];
+  mbar_wait(&bars[0], 0, a.status);
+
+  // ---- X_scaled, re-quantised in place (thread: chunk c of rows tid/4, tid/4 + 64, ...)
+  float mx[16];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+  for (int e = 0; e < 16; ++e) mx[e] = 0.f;
+  for (int i = tid >> 2; i < Q; i += kThreads / 4) {
+    uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
+    const uint4 w4 = *ptr;
+    const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+    const float l = lut[i];
+    if (calib) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[a][e] = 0;
-    warp_gemm_s8<4>(acc, XsT, ld, row0, BT, ld, n0 + nb, Q);
+      for (int e = 0; e < 16; ++e)
+        mx[e] = fmaxf(mx[e], fabsf(__fmul_rn(__fmul_rn((float)sx8(ww[e >> 2], e & 3), rx[e]), l)));
+    } else {
+      uint32_t o[4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+      for (int w = 0; w < 4; ++w) {
+        int q4[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int p = row0 + (lane >> 2) + 8 * (e >> 1);
-        const int n = n0 + nb + 8 * a + 2 * (lane & 3) + (e & 1);
-        const i64 o = obase + (i64)p * N + n;
-        if (tap_acc) tap_acc[o] = acc[a][e];
-        loc[o] = __fmul_rn((float)acc[a][e], __fmul_rn(s_xs[h * P + p], sB));
+        for (int e = 0; e < 4; ++e)
+          q4[e] = rne_clamp(__fmul_rn(__fmul_rn((float)sx8(ww[w], e), rx[w * 4 + e]), l));
+        o[w] = pack4(q4[0], q4[1], q4[2], q4[3]);
       }
+      const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+      *ptr = v;
+      if (a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
+    }
+  }
+  if (calib) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e) atomicMax(a.absmax_xs + h * P + c * 16 + e, __float_as_uint(mx[e]));
+    return;
+  }
+  fence_async_smem();
+  __syncthreads();
+
+  // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]: A = Bq (MN-major, M = N states), B = Xs_q (MN-major)
+  const uint32_t tmem = *tmem_slot;
+  if (tid == 0) {
+    tc_fence_after();
+    const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+    for (int s = 0; s < Q / 32; ++s)
+      mma_s8_ss(tmem, tile_desc(smem_u32(sB) + 32 * s * N, (uint32_t)N),
+                tile_desc(smem_u32(sX) + 32 * s * 64, 64), idesc, s > 0);
+    mma_commit(&bars[1]);
+  }
+  __syncwarp();
+  mbar_wait(&bars[1], 0, a.status);
+  tc_fence_after();
+
+  // ---- epilogue.  M = 128: accumulator row n on TMEM lane n.  M = 64: row n on lane
+  // (n % 16) + 32 (n / 16), i.e. the first 16 lanes of each warp's quarter.
+  {
+    const int q = warp & 3, ch = warp >> 2;
+    int acc[32];
+    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), acc);
+    tmem_ld_wait();
+    const bool ok = (N == 128) || (lane < 16);
+    const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
+    if (ok) {
+      const float sB_g = a.s_B[g];
+      const i64 obase = ((((i64)b * d.c + k) * d.H + h) * P) * N + n;
+#pragma unroll
+      for (int pp = 0; pp < 32; ++pp) {
+        const int p = ch * 32 + pp;
+        a.loc[obase + (i64)p * N] = __fmul_rn((float)acc[pp], __fmul_rn(a.s_xs[h * P + p], sB_g));
+        if (a.tap_acc) a.tap_acc[obase + (i64)p * N] = acc[pp];
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 64);
   }
 }
 
@@ -99,17 +162,28 @@ __global__ void __launch_bounds__(256) chunk_state_kernel(
 ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t* Bq,
                                   const float* s_x, const float* s_xs, const float* s_B,
                                   const float* dt, const float* cs, float* loc, int8_t* tap_Xsq,
-                                  int32_t* tap_acc, uint32_t* absmax_xs, cudaStream_t st) {
-  dim3 grid(d.H, d.c, d.b);
-  size_t smem = (size_t)(d.P + d.N) * (d.Q + 16) + sizeof(float) * d.Q;
-  static bool attr_done = false;
-  if (!attr_done) {
-    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_kernel,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-    attr_done = true;
+                                  int32_t* tap_acc, uint32_t* absmax_xs, int32_t* status,
+                                  cudaStream_t st) {
+  const int TQ = d.Q < 128 ? d.Q : 128;
+  const uint64_t T = (uint64_t)d.b * d.L;
+  CUtensorMap tm_B, tm_x;
+  {
+    uint64_t dims[3] = {(uint64_t)d.N, (uint64_t)d.G, T};
+    uint64_t str[2] = {(uint64_t)d.N, (uint64_t)d.G * d.N};
+    uint32_t box[3] = {(uint32_t)d.N, 1, (uint32_t)TQ};
+    if (!encode_tensor_map(&tm_B, Bq, 1, 3, dims, str, box, d.N)) return SSDI8_ERR_CUDA;
   }
-  chunk_state_kernel<<<grid, 256, smem, st>>>(xq, Bq, s_x, s_xs, s_B, dt, cs, loc, tap_Xsq, tap_acc,
-                                              absmax_xs, d);
+  {
+    uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
+    uint64_t str[2] = {(uint64_t)d.P, (uint64_t)d.H * d.P};
+    uint32_t box[3] = {64, 1, (uint32_t)TQ};
+    if (!encode_tensor_map(&tm_x, xq, 1, 3, dims, str, box, 64)) return SSDI8_ERR_CUDA;
+  }
+  StateArgs a = {s_x, s_xs, s_B, dt, cs, loc, tap_Xsq, tap_acc, absmax_xs, status, d};
+  const size_t smem = SMEM_BYTES + 1024;
+  SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid(d.H, d.c, d.b);
+  chunk_state_tc<<<grid, kThreads, smem, st>>>(tm_B, tm_x, a);
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

@@ -22,7 +22,8 @@ ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, con
 ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t* Bq,
                                   const float* s_x, const float* s_xs, const float* s_B,
                                   const float* dt, const float* cs, float* loc, int8_t* tap_Xsq,
-                                  int32_t* tap_acc, uint32_t* absmax_xs, cudaStream_t st);
+                                  int32_t* tap_acc, uint32_t* absmax_xs, int32_t* status,
+                                  cudaStream_t st);
 
 // absmax_h: per-channel running max (binary32 bits) of |S| over init, prev and final
 ssdi8_status_t launch_state_passing(const Dims& d, const float* loc, const float* gamma,
