@@ -144,7 +144,9 @@ typedef struct {
  *                j <= i) is re-quantised per output row so that its product with int8 X is
  *                an integer GEMM.  With sub-blocks of SB = min(64, Q) tokens and je the last
  *                column of the sub-block of j:
- *                  same sub-block : w = fmul(dt_j, exp32(fsub(cs_i, cs_j))),  f = 1
+ *                  same sub-block : running product of the per-token decays
+ *                                   a_m = exp32(fsub(cs_m, cs_{m-1})): E[i,i] = 1,
+ *                                   E[i,j] = fmul(E[i,j+1], a_{j+1}); w = fmul(dt_j, E[i,j]), f = 1
  *                  earlier block  : w = fmul(dt_j, exp32(fsub(cs_je, cs_j))), f = exp32(fsub(cs_i, cs_je))
  *                  t = fmul(float(CBq[i,j]), w)
  *                  rowmax_i = max over sub-blocks of fmul(max_j |t|, f)

@@ -389,7 +389,9 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 //  diagonal: the masked operand CB o LUT_scan2 is re-quantised per output row i
 //  so that the product with int8 X is an integer GEMM.  With sub-blocks of
 //  SB = min(64, Q) tokens, je = last column of the sub-block of j:
-//     same sub-block:  w = fmul(dt_j, exp32(fsub(cs_i, cs_j))),  f = 1
+//     same sub-block:  the decay is the running product of the per-token decays
+//                      a_m = exp32(fsub(cs_m, cs_{m-1})):  E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1});
+//                      w = fmul(dt_j, E[i,j]),  f = 1
 //     earlier block :  w = fmul(dt_j, exp32(fsub(cs_je, cs_j))), f = exp32(fsub(cs_i, cs_je))
 //     t[i,j]   = fmul(float(CBq[i,j]), w)          (w f = dt_j exp(cs_i - cs_j); every exponent <= 0)
 //     rowmax_i = max over sub-blocks J of fmul(max_{j in J, j<=i} |t[i,j]|, f)
@@ -410,13 +412,15 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
   for (int b = 0; b < b_; ++b)
     for (int h = 0; h < H; ++h) {
       const int g = h / hpg;
-      std::vector<float> t(Q), f(Q / SB + 1);
+      std::vector<float> t(Q), f(Q / SB + 1), a_tok(Q);
       std::vector<int8_t> mq(Q);
       for (int k = 0; k < c; ++k) {
         const i64 t0 = (i64)b * L + (i64)k * Q;
         const float* csk = cs + (((i64)b * H + h) * c + k) * Q;
         const int8_t* cbk = CBq + (((i64)b * c + k) * G + g) * Q * Q;
         const int8_t* hqk = hq + (((i64)b * c + k) * H + h) * P * N;
+        a_tok[0] = 1.0f;  // never used: a_m enters only for m >= 1
+        for (int m = 1; m < Q; ++m) a_tok[m] = exp32(fsub(csk[m], csk[m - 1]));
         for (int i = 0; i < Q; ++i) {
           const int I = i / SB;
           float rmax = 0.0f;
@@ -424,8 +428,15 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
             const int je = J * SB + SB - 1;
             f[J] = (J == I) ? 1.0f : exp32(fsub(csk[i], csk[je]));
             float bmax = 0.0f;
-            for (int j = J * SB; j <= (J == I ? i : je); ++j) {
-              const float e = (J == I) ? exp32(fsub(csk[i], csk[j])) : exp32(fsub(csk[je], csk[j]));
+            float E = 1.0f;
+            for (int j = (J == I ? i : je); j >= J * SB; --j) {
+              float e;
+              if (J == I) {
+                if (j < i) E = fmul(E, a_tok[j + 1]);
+                e = E;
+              } else {
+                e = exp32(fsub(csk[je], csk[j]));
+              }
               const float w = fmul(dt[(t0 + j) * H + h], e);
               t[j] = fmul((float)cbk[(size_t)i * Q + j], w);
               const float a = std::fabs(t[j]);

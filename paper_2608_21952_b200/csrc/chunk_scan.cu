@@ -31,7 +31,7 @@ constexpr uint32_t OFF_H = 16384;         // [64][N]         hq tile, K-major
 constexpr uint32_t OFF_X = 24576;         // [256][64]       xq rows, MN-major
 constexpr uint32_t OFF_CB = 40960;        // 2 x [128][128]  CBq panels -> Mq in place -> y staging
 constexpr uint32_t OFF_F = 73728;         // float arrays
-constexpr uint32_t SMEM_BYTES = OFF_F + 4 * 256 * 4 + 3 * 64 * 4 + 64;
+constexpr uint32_t SMEM_BYTES = OFF_F + 5 * 256 * 4 + 3 * 64 * 4 + 64;
 constexpr uint32_t PANEL = 16384;
 
 __device__ __forceinline__ float unpack_s8(uint32_t w_xor, int k) {
@@ -73,7 +73,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   float* dt_s = cs_s + 256;
   float* woff_s = dt_s + 256;
   float* part_s = woff_s + 256;
-  float* colA = part_s + 256;  // s_C s_h[p]
+  float* atok_s = part_s + 256;  // per-token decay a_m = exp32(cs_m - cs_{m-1})
+  float* colA = atok_s + 256;  // s_C s_h[p]
   float* colB = colA + 64;     // s_x[p]
   float* colC = colB + 64;     // corr[p]
   uint64_t* bars = reinterpret_cast<uint64_t*>(colC + 64);  // [0] C+h, [1] CBq, [2] xq, [3] MMA done
@@ -117,7 +118,10 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   }
   __syncthreads();
   // weight of column j as seen from a later sub-block: dt_j exp(cs_je - cs_j), je = end of j's sub-block
-  if (tid < KJ) woff_s[tid] = __fmul_rn(dt_s[tid], exp32(__fsub_rn(cs_s[tid | 63], cs_s[tid])));
+  if (tid < KJ) {
+    woff_s[tid] = __fmul_rn(dt_s[tid], exp32(__fsub_rn(cs_s[tid | 63], cs_s[tid])));
+    atok_s[tid] = tid > 0 ? exp32(__fsub_rn(cs_s[tid], cs_s[tid - 1])) : 1.0f;
+  }
 
   // ---- ChunkScan1 MMA: acc_off = Cq * hq^T   (overlaps the mask computation below)
   if (tid == 0) {
@@ -148,19 +152,21 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   float fJ[3] = {0.f, 0.f, 0.f};
   float rpart = 0.f;
   if (row_ok && role == 0) {
+    // own sub-block, right to left: E[i,j] = E[i,j+1] a_{j+1}, starting from E[i,i] = 1
     const int ri = i & 63;
+    float E = 1.0f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 3; c >= 0; --c) {
       const uint4 w4 = *chunk_ptr(I * 4 + c);
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
 #pragma unroll
-      for (int e = 0; e < 16; ++e) {
+      for (int e = 15; e >= 0; --e) {
         const int jj = c * 16 + e;
         float t = 0.f;
         if (jj <= ri) {
           const int j = (I << 6) + jj;
-          const float w = __fmul_rn(dt_s[j], exp32(__fsub_rn(cs_i, cs_s[j])));
-          t = __fmul_rn(unpack_s8(ww[e >> 2], e & 3), w);
+          if (jj < ri) E = __fmul_rn(E, atok_s[j + 1]);
+          t = __fmul_rn(unpack_s8(ww[e >> 2], e & 3), __fmul_rn(dt_s[j], E));
         }
         tdiag[jj] = t;
         rpart = fmaxf(rpart, fabsf(t));
