@@ -165,6 +165,26 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
                                     uint32_t flags, void* workspace, size_t workspace_bytes,
                                     void* stream);
 
+/* The same forward pass for callers that can pass no workspace because they must not, or
+ * cannot, allocate device memory: processes whose device-memory budget is fully assigned at
+ * start-up, and latency-critical loops that must never reach cudaMalloc / cudaFree (both
+ * synchronise the device).  (The paper has no counterpart of this entry point; it exists for
+ * deployment only and computes exactly what ssdi8_chunk_scan_fwd computes.)
+ *  - The scratch is a fixed array of SSDI8_STATIC_WORKSPACE_BYTES inside the library, held by
+ *    every GPU that loads the library until the process exits.  Dimensions that need more
+ *    (ssdi8_workspace_bytes(dims, flags) > SSDI8_STATIC_WORKSPACE_BYTES) are rejected with
+ *    SSDI8_ERR_WORKSPACE; use ssdi8_chunk_scan_fwd with your own workspace for those.
+ *  - The call allocates nothing and frees nothing, on the host or on the device.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.
+ *    Nothing in it has to start at zero (every region is written before it is read), but two
+ *    calls that overlap on the GPU (different streams, no dependency) race on it: order them.
+ * Arguments as for ssdi8_chunk_scan_fwd, minus the workspace. */
+#define SSDI8_STATIC_WORKSPACE_BYTES (16u << 20)
+ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
+                                           uint32_t flags, void* stream);
+
 /* Static calibration of the internal step sizes (Eq. 1 applied once to the internal
  * tensors of this input; the paper calibrates offline, Section 5 "Quantization Setup"):
  *   s_xs[h,p] = absmax over (b,t) of |fmul(fmul(float(xq), s_x), LUT_state)| / 127

@@ -28,7 +28,9 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TI
 PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1 << k for k in range(8, 13))
 
 EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
-           "ssdi8_chunk_scan_fwd", "ssdi8_calibrate", "ssdi8_state_passing", "ssdi8_ssd_step")
+           "ssdi8_chunk_scan_fwd", "ssdi8_chunk_scan_fwd_static", "ssdi8_calibrate",
+           "ssdi8_state_passing", "ssdi8_ssd_step")
+STATIC_WORKSPACE_BYTES = 16 << 20
 
 
 class Dims(C.Structure):
@@ -56,6 +58,8 @@ _lib.ssdi8_quantize_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
 _lib.ssdi8_chunk_scan_fwd.restype = C.c_int32
 _lib.ssdi8_chunk_scan_fwd.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_uint32, C.c_void_p,
                                       C.c_size_t, C.c_void_p]
+_lib.ssdi8_chunk_scan_fwd_static.restype = C.c_int32
+_lib.ssdi8_chunk_scan_fwd_static.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_uint32, C.c_void_p]
 _lib.ssdi8_calibrate.restype = C.c_int32
 _lib.ssdi8_calibrate.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -121,6 +125,14 @@ def ssdi8_chunk_scan_fwd(dims: Dims, args: FwdArgs, workspace, flags: int = 0, s
     _check(_lib.ssdi8_chunk_scan_fwd(C.byref(dims), C.byref(args), flags, _ptr(workspace),
                                      workspace.numel() * workspace.element_size(), _stream(stream)),
            "ssdi8_chunk_scan_fwd")
+
+
+def ssdi8_chunk_scan_fwd_static(dims: Dims, args: FwdArgs, flags: int = 0, stream=None) -> None:
+    """Forward pass on the library's built-in scratch: no workspace argument, no allocation.
+    For callers that cannot allocate device memory; raises SSDi8Error(ERR_WORKSPACE) when the
+    dimensions need more than STATIC_WORKSPACE_BYTES."""
+    _check(_lib.ssdi8_chunk_scan_fwd_static(C.byref(dims), C.byref(args), flags, _stream(stream)),
+           "ssdi8_chunk_scan_fwd_static")
 
 
 def ssdi8_calibrate(dims: Dims, args: FwdArgs, s_xs, s_cb, s_h, workspace, stream=None) -> None:

@@ -222,4 +222,38 @@ ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const 
                          static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------
+// Forward pass with library-owned scratch (no allocation by anyone).
+//
+// Some callers cannot hand the library a workspace: a serving process whose whole device-memory
+// budget was carved up at start-up (weights, state caches) has no allocator left to ask, and a
+// latency-critical decode/prefill loop must not reach cudaMalloc or cudaFree at all, because both
+// synchronise the device.  For them the scratch of the layer forward lives in the array below,
+// which every GPU that loads this library holds from load until the process exits.
+//
+// g_static_ws is a device symbol.  Inside host code its name is only a host-side stand-in, not a
+// device address, so the address is looked up once per device with cudaGetSymbolAddress (with
+// that device current) and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_ws[SSDI8_STATIC_WORKSPACE_BYTES];
+
+ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
+                                           uint32_t flags, void* stream) {
+  if (!dims || !args) return SSDI8_ERR_NULL;
+  const size_t need = ssdi8_workspace_bytes(dims, flags);
+  if (need == 0) return (flags & ~(uint32_t)SSDI8_PHASE_ALL) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
+  if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
+  static void* ws_of_device[64];  // resolved address of g_static_ws, per device
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
+  if (!ws_of_device[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return SSDI8_ERR_CUDA;
+    }
+    ws_of_device[dev] = p;
+  }
+  return ssdi8_chunk_scan_fwd(dims, args, flags, ws_of_device[dev], SSDI8_STATIC_WORKSPACE_BYTES, stream);
+}
+
 }  // extern "C"
