@@ -319,9 +319,8 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2608_21952_b200 import binding as bd
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2608_21952_b200 import ranks
+    world, rank, local = ranks.env_world()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -329,8 +328,7 @@ def run_ours(args):
     layer = Layer(cfg, torch, bd)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -342,11 +340,8 @@ def run_ours(args):
         ms = layer.timed(layer.step, args.steps)
         torch.cuda.synchronize()
     barrier()
-    if world > 1:
-        tms = torch.tensor([ms], device="cuda")
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
-    value = world * cfg.tokens / (ms * 1e-3)
+    ms = ranks.max_over_ranks(ms, "cuda")
+    value = ranks.whole_job_tokens_per_s(cfg.tokens, world, ms)
 
     if args.quick:
         if rank == 0:
@@ -364,10 +359,7 @@ def run_ours(args):
     barrier()
     ms_e2e = layer.timed(layer.e2e_step, max(3, min(args.steps, 10)))
     barrier()
-    if world > 1:
-        tms = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms_e2e = float(tms.item())
+    ms_e2e = ranks.max_over_ranks(ms_e2e, "cuda")
 
     line = None
     if rank == 0:
@@ -395,7 +387,7 @@ def run_ours(args):
                 "vs_baseline": (value / paper) if (paper and world == 1) else None, "dtype": "s8",
                 "data": "synthetic", "config": workload_config(cfg, world),
                 "clocks": clk.summary(),
-                "e2e": {"value": world * cfg.tokens / (ms_e2e * 1e-3), "unit": UNIT,
+                "e2e": {"value": ranks.whole_job_tokens_per_s(cfg.tokens, world, ms_e2e), "unit": UNIT,
                         "h2d_bytes_per_step": layer.h2d_bytes(), "d2h_bytes_per_step": layer.d2h_bytes(),
                         "ms_per_step": ms_e2e},
                 "gpu_launches": Layer.LAUNCHES_PER_STEP * args.steps,
