@@ -40,14 +40,14 @@ ssdi8_status_t check_arch() {
 }
 
 struct Workspace {
-  size_t cs, gamma, cbq, loc, hq, total;
+  size_t pack, gamma, cbq, loc, hq, total;
 };
 
 Workspace layout(const Dims& d) {
   Workspace w;
   size_t o = 0;
   const size_t nst = (size_t)d.b * d.c * d.H * d.P * d.N;
-  w.cs = o;    o = align_up(o + sizeof(float) * (size_t)d.b * d.H * d.L, 256);
+  w.pack = o;  o = align_up(o + sizeof(float) * kPackRows * (size_t)d.b * d.H * d.L, 256);
   w.gamma = o; o = align_up(o + sizeof(float) * (size_t)d.b * d.H * d.c, 256);
   w.cbq = o;   o = align_up(o + (size_t)d.b * d.c * d.G * d.Q * d.Q, 256);
   w.loc = o;   o = align_up(o + sizeof(float) * nst, 256);
@@ -117,21 +117,21 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
   if (s != SSDI8_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
-  float* cs = a->tap_cs ? a->tap_cs : reinterpret_cast<float*>(ws + w.cs);
+  float* pack = reinterpret_cast<float*>(ws + w.pack);
   float* gamma = reinterpret_cast<float*>(ws + w.gamma);
   int8_t* cbq = a->tap_CBq ? a->tap_CBq : reinterpret_cast<int8_t*>(ws + w.cbq);
   float* loc = a->tap_loc ? a->tap_loc : reinterpret_cast<float*>(ws + w.loc);
   int8_t* hq = a->tap_hq ? a->tap_hq : reinterpret_cast<int8_t*>(ws + w.hq);
   if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
 
-  if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, cs, gamma, st)) != SSDI8_OK)
+  if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st)) != SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_BMM) &&
       (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, st)) !=
           SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
-      (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->dt, cs, loc, a->tap_Xsq,
+      (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, pack, loc, a->tap_Xsq,
                               a->tap_acc_st, nullptr, a->status, st)) != SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_STATE_PASSING) &&
@@ -140,7 +140,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
     return s;
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
-    return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, a->dt, cs,
+    return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack,
                              a->D, a->corr, a->y, a->status, taps, st);
   }
   return SSDI8_OK;
@@ -165,7 +165,7 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
   if (s != SSDI8_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
-  float* cs = reinterpret_cast<float*>(ws + w.cs);
+  float* pack = reinterpret_cast<float*>(ws + w.pack);
   float* gamma = reinterpret_cast<float*>(ws + w.gamma);
   float* loc = reinterpret_cast<float*>(ws + w.loc);
   const i64 nhp = (i64)d.H * d.P;
@@ -173,8 +173,8 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
   SSDI8_CUDA_CHECK(cudaMemsetAsync(s_xs, 0, sizeof(float) * nhp, st));
   SSDI8_CUDA_CHECK(cudaMemsetAsync(s_cb, 0, sizeof(float) * d.G, st));
   SSDI8_CUDA_CHECK(cudaMemsetAsync(s_h, 0, sizeof(float) * nhp, st));
-  if ((s = launch_cumsum(d, a->dt, a->A, cs, gamma, st)) != SSDI8_OK) return s;
-  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, nullptr, a->s_B, a->dt, cs, nullptr, nullptr,
+  if ((s = launch_cumsum(d, a->dt, a->A, pack, gamma, nullptr, st)) != SSDI8_OK) return s;
+  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, nullptr, a->s_B, pack, nullptr, nullptr,
                               nullptr, reinterpret_cast<uint32_t*>(s_xs), nullptr, st)) != SSDI8_OK)
     return s;
   if ((s = launch_finalize_scales(s_xs, nhp, nullptr, nullptr, 0, st)) != SSDI8_OK) return s;
@@ -182,7 +182,7 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
                       reinterpret_cast<uint32_t*>(s_cb), st)) != SSDI8_OK)
     return s;
   if ((s = launch_finalize_scales(s_cb, d.G, a->s_C, a->s_B, 1, st)) != SSDI8_OK) return s;
-  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, s_xs, a->s_B, a->dt, cs, loc, nullptr,
+  if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, s_xs, a->s_B, pack, loc, nullptr,
                               nullptr, nullptr, nullptr, st)) != SSDI8_OK)
     return s;
   if ((s = launch_state_passing(d, loc, gamma, a->init_state, nullptr, nullptr, nullptr, nullptr,

@@ -1,6 +1,6 @@
 // ChunkState with the sparse-aware reformulation (Eq. 3) and the INT32 rescale (Eq. 4) on
 // tcgen05 tensor cores.  One CTA per (batch, chunk, head):
-//   LUT_state[i] = fmul(dt_i, exp32(fsub(cs_last, cs_i)))
+//   LUT_state[i] = fmul(dt_i, exp32(fsub(cs_last, cs_i)))        (row 4 of the ChunkCumsum pack)
 //   Xs_q[i,p]    = rne(fmul(fmul(float(xq[i,p]), fdiv(s_x, s_xs)), LUT_state[i]))   in place in smem
 //   acc_st[n,p]  = sum_i Bq[i,n] Xs_q[i,p]     INT8 MMA over the tokens of the chunk, INT32 in TMEM
 //   loc[p,n]     = fmul(float(acc_st), fmul(s_xs[h,p], s_B[g]))
@@ -17,7 +17,7 @@ namespace {
 using namespace sm100;
 
 struct StateArgs {
-  const float* s_x; const float* s_xs; const float* s_B; const float* dt; const float* cs;
+  const float* s_x; const float* s_xs; const float* s_B; const float* pack;
   float* loc; int8_t* tap_Xsq; int32_t* tap_acc; uint32_t* absmax_xs; int32_t* status;
   Dims d;
 };
@@ -65,9 +65,7 @@ chunk_state_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__
       if (!calib) tma_load_3d(sB + i0 * N, &tm_B, &bars[0], 0, g, (int)(tok0 + i0));
     }
   }
-  const float* csk = a.cs + (((i64)b * d.H + h) * d.c + k) * Q;
-  const float cs_last = csk[Q - 1];
-  if (tid < Q) lut[tid] = __fmul_rn(a.dt[(tok0 + tid) * d.H + h], exp32(__fsub_rn(cs_last, csk[tid])));
+  if (tid < Q) lut[tid] = a.pack[((((i64)b * d.H + h) * d.c + k) * kPackRows + PACK_LUT) * Q + tid];
   // per-column factors of this thread's 16 channels (16-byte chunk c of every row it visits)
   const int c = tid & 3;
   float rx[16];
@@ -161,7 +159,7 @@ chunk_state_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__
 
 ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t* Bq,
                                   const float* s_x, const float* s_xs, const float* s_B,
-                                  const float* dt, const float* cs, float* loc, int8_t* tap_Xsq,
+                                  const float* pack, float* loc, int8_t* tap_Xsq,
                                   int32_t* tap_acc, uint32_t* absmax_xs, int32_t* status,
                                   cudaStream_t st) {
   const int TQ = d.Q < 128 ? d.Q : 128;
@@ -179,7 +177,7 @@ ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t*
     uint32_t box[3] = {64, 1, (uint32_t)TQ};
     if (!encode_tensor_map(&tm_x, xq, 1, 3, dims, str, box, 64)) return SSDI8_ERR_CUDA;
   }
-  StateArgs a = {s_x, s_xs, s_B, dt, cs, loc, tap_Xsq, tap_acc, absmax_xs, status, d};
+  StateArgs a = {s_x, s_xs, s_B, pack, loc, tap_Xsq, tap_acc, absmax_xs, status, d};
   const size_t smem = SMEM_BYTES + 1024;
   SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.H, d.c, d.b);

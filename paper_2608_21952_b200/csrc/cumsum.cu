@@ -1,27 +1,37 @@
-// ChunkCumsum (Algorithm 2, module 1): cs[b,h,k,i] = (float) sum_{i'<=i} (double)dt (double)A_h
-// in token order within chunk k, and Gamma[b,h,k] = exp32(cs[.., Q-1]) (Decay_pass, Eq. 5).
-// The sum order is part of the definition (it decides rounding downstream), so each
-// (b, chunk, head) is scanned sequentially by one thread; loads and stores go through a
-// shared-memory tile so that both the [b,L,H] reads and the [b,H,c,Q] writes coalesce.
+// ChunkCumsum (Algorithm 2, module 1) and the per-token scalars every later module derives
+// from it.  For each (batch, head, chunk) it writes one contiguous pack of 5 rows of Q floats:
+//   row 0  cs[i]    = (float) sum_{i'<=i} (double)dt (double)A_h, in token order   (dA_cs)
+//   row 1  dt[i]
+//   row 2  woff[i]  = fmul(dt_i, exp32(fsub(cs_ie, cs_i))), ie = last token of i's 64-token sub-block
+//   row 3  atok[i]  = exp32(fsub(cs_i, cs_{i-1}))  (1 for i = 0): the per-token decay
+//   row 4  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
+// and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
+// (it decides rounding downstream), so each (b, chunk, head) is scanned sequentially by one
+// thread; loads and stores go through shared memory so that the [b,L,H] reads and the row
+// writes coalesce.  Later kernels fetch a pack with one bulk copy and need no exponentials
+// per token.
 #include "kernels.h"
 
 namespace ssdi8 {
 namespace {
 
-constexpr int CH = 32;  // heads per block
+constexpr int CH = 16;  // heads per block
 
 __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ dt,
                                                      const float* __restrict__ A,
-                                                     float* __restrict__ cs,
-                                                     float* __restrict__ gamma, Dims d) {
-  extern __shared__ float tile[];  // [CH][Q+1]
+                                                     float* __restrict__ pack,
+                                                     float* __restrict__ gamma,
+                                                     float* __restrict__ tap_cs, Dims d) {
+  extern __shared__ float tile[];  // dt [CH][Q+1], cs [CH][Q+1]
   const int Q = d.Q, ld = Q + 1;
+  float* dts = tile;
+  float* css = tile + CH * ld;
   const int h0 = blockIdx.x * CH, k = blockIdx.y, b = blockIdx.z;
   const int nh = min(CH, d.H - h0);
   const i64 t0 = (i64)b * d.L + (i64)k * Q;
   for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
     int i = e / CH, hh = e % CH;
-    if (hh < nh) tile[hh * ld + i] = dt[(t0 + i) * d.H + h0 + hh];
+    if (hh < nh) dts[hh * ld + i] = dt[(t0 + i) * d.H + h0 + hh];
   }
   __syncthreads();
   if (threadIdx.x < nh) {
@@ -30,26 +40,36 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     double acc = 0.0;
     float last = 0.f;
     for (int i = 0; i < Q; ++i) {
-      acc += (double)tile[hh * ld + i] * a;
+      acc += (double)dts[hh * ld + i] * a;
       last = (float)acc;
-      tile[hh * ld + i] = last;
+      css[hh * ld + i] = last;
     }
     gamma[((i64)b * d.H + h0 + hh) * d.c + k] = exp32(last);
   }
   __syncthreads();
   for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
-    int hh = e / Q, i = e % Q;
-    if (hh < nh) cs[(((i64)b * d.H + h0 + hh) * d.c + k) * Q + i] = tile[hh * ld + i];
+    const int hh = e / Q, i = e % Q;
+    if (hh >= nh) continue;
+    const float* c = css + hh * ld;
+    const float ci = c[i], di = dts[hh * ld + i];
+    const i64 u = ((i64)b * d.H + h0 + hh) * d.c + k;
+    float* p = pack + u * kPackRows * Q + i;
+    p[0] = ci;
+    p[Q] = di;
+    p[2 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[i | 63], ci)));
+    p[3 * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
+    p[4 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
+    if (tap_cs) tap_cs[u * Q + i] = ci;
   }
 }
 
 }  // namespace
 
-ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* cs,
-                             float* gamma, cudaStream_t st) {
+ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
+                             float* gamma, float* tap_cs, cudaStream_t st) {
   dim3 grid((d.H + CH - 1) / CH, d.c, d.b);
-  size_t smem = sizeof(float) * CH * (d.Q + 1);
-  cumsum_kernel<<<grid, 256, smem, st>>>(dt, A, cs, gamma, d);
+  size_t smem = sizeof(float) * 2 * CH * (d.Q + 1);
+  cumsum_kernel<<<grid, 256, smem, st>>>(dt, A, pack, gamma, tap_cs, d);
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

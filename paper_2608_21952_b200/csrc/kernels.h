@@ -7,9 +7,14 @@ namespace ssdi8 {
 ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
                                int8_t* out, cudaStream_t st);
 
-// cs [b,H,c,Q], gamma [b,H,c]
-ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* cs,
-                             float* gamma, cudaStream_t st);
+// Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, lut (see
+// cumsum.cu); element (u, row, i) at pack[(u * kPackRows + row) * Q + i], u = (b*H + h)*c + k.
+constexpr int kPackRows = 5;
+enum { PACK_CS = 0, PACK_DT = 1, PACK_WOFF = 2, PACK_ATOK = 3, PACK_LUT = 4 };
+
+// pack [b,H,c,5,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
+ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
+                             float* gamma, float* tap_cs, cudaStream_t st);
 
 // acc_cb (tap, may be NULL), CBq (may be NULL when s_cb is NULL), absmax_acc: per-group
 // running max of |acc_cb| over the causal half (calibration; may be NULL)
@@ -21,7 +26,7 @@ ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, con
 // NULL).  When absmax_xs is non-NULL only that is computed.
 ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t* Bq,
                                   const float* s_x, const float* s_xs, const float* s_B,
-                                  const float* dt, const float* cs, float* loc, int8_t* tap_Xsq,
+                                  const float* pack, float* loc, int8_t* tap_Xsq,
                                   int32_t* tap_acc, uint32_t* absmax_xs, int32_t* status,
                                   cudaStream_t st);
 
@@ -38,7 +43,7 @@ struct ScanTaps {
 ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* Cq,
                                  const int8_t* CBq, const int8_t* hq, const float* s_x,
                                  const float* s_C, const float* s_cb, const float* s_h,
-                                 const float* dt, const float* cs, const float* D,
+                                 const float* pack, const float* D,
                                  const float* corr, float* y, int32_t* status,
                                  const ScanTaps& taps, cudaStream_t st);
 

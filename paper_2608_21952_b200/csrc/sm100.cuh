@@ -24,6 +24,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -35,13 +38,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: every try_wait already blocks for a hardware-defined interval, so the cap
-// corresponds to seconds.  On expiry the caller's status word is set and the wait returns;
-// the kernel then runs to its normal end (tensor memory is freed) with undefined results.
-constexpr uint32_t kWaitCap = 1u << 22;
+// Bounded wait.  Every try_wait already blocks for a hardware-defined interval, so the cap is of
+// the order of a second.  On expiry the caller's status word is set and the wait returns; once
+// the word is set, every later wait of the grid gives up after a few polls, so the kernel runs
+// to its normal end (tensor memory is freed) quickly, with undefined results.
+constexpr uint32_t kWaitCap = 1u << 20;
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
-  for (uint32_t it = 0; it < kWaitCap; ++it)
+  for (uint32_t it = 0; it < kWaitCap; ++it) {
     if (mbar_try_wait(bar, parity)) return;
+    if ((it & 63u) == 63u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
+  }
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
 }
 
@@ -69,6 +75,12 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, ui
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
+}
+// untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, const void* src, int x, int y, int z) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
