@@ -142,7 +142,7 @@ typedef struct {
  *                y_off = exp(cs_i) s_C s_h acc_off   (decay only; no dt factor)
  *  ChunkScan2    the masked operand CB o LUT_scan2 (LUT_scan2[i,j] = dt_j exp(cs_i - cs_j),
  *                j <= i) is re-quantised per output row so that its product with int8 X is
- *                an integer GEMM.  With sub-blocks of SB = min(64, Q) tokens and je the last
+ *                an integer GEMM.  With sub-blocks of SB = 16 tokens and je the last
  *                column of the sub-block of j:
  *                  same sub-block : running product of the per-token decays
  *                                   a_m = exp32(fsub(cs_m, cs_{m-1})): E[i,i] = 1,

@@ -93,7 +93,7 @@ inline float exp32(float x) {
   return f_from_bits(u);
 }
 
-inline int sub_block(int Q) { return Q < 64 ? Q : 64; }
+inline int sub_block(int Q) { return Q < 16 ? Q : 16; }
 
 }  // namespace
 
@@ -388,7 +388,7 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 //                 y_off = exp(cs_i) s_C s_h[h,p] acc_off   (decay applied after the product)
 //  diagonal: the masked operand CB o LUT_scan2 is re-quantised per output row i
 //  so that the product with int8 X is an integer GEMM.  With sub-blocks of
-//  SB = min(64, Q) tokens, je = last column of the sub-block of j:
+//  SB = min(16, Q) tokens, je = last column of the sub-block of j:
 //     same sub-block:  the decay is the running product of the per-token decays
 //                      a_m = exp32(fsub(cs_m, cs_{m-1})):  E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1});
 //                      w = fmul(dt_j, E[i,j]),  f = 1

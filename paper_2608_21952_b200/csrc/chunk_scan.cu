@@ -1,15 +1,18 @@
 // ChunkScan1 + ChunkScan2 + output sum (Algorithm 2 modules 5, 6) on tcgen05 tensor cores:
-// a persistent, warp-specialised kernel, one CTA per SM, two pipeline stages.
+// a persistent, warp-specialised kernel, one CTA per SM.
 // Per (batch, chunk, head) and 128-row tile of the chunk:
 //   acc_off[i,p]  = sum_n Cq[i,n] hq[p,n]                 INT8 MMA, INT32 accumulator in TMEM
 //   Mq[i,j]       = per-row re-quantised CBq[i,j] dt_j exp(cs_i - cs_j), j <= i   (see ssdi8.h)
 //   acc_diag[i,p] = sum_j Mq[i,j] xq[j,p]                 INT8 MMA, second TMEM accumulator
 //   y = exp(cs_i) s_C s_h acc_off + (s_cb rowmax_i / 127) s_x acc_diag + D s_x xq + corr
-// Roles: warp 0 issues TMA loads (Cq, hq, CBq K-major; xq MN-major; the per-token scalar pack of
-// ChunkCumsum by one bulk copy); warp 1 issues the MMAs; warps 2-5 and 6-9 build Mq in place
-// over CBq for even and odd tiles (one thread per output row, no exchange between threads);
-// warps 10-13 read the accumulators, form y and store it through swizzled staging with TMA.
-// No multicast; every wait is bounded.
+// Roles (28 warps): warps 0, 2, 3 issue the TMA loads (CBq K-major and the per-token scalar pack
+// of ChunkCumsum; Cq, hq K-major; xq MN-major), each stream on its own ring; warp 1 issues the
+// MMAs; warps 4-19 build Mq in place over CBq (four threads per output row, 16-column chunks
+// dealt round robin); warps 20-27 read the accumulators, form y and store it through swizzled
+// staging with TMA.  Every buffer has its own "free" barrier, released by whoever reads it last
+// (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
+// hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
+// because every role executes different code at the same time.  No multicast; bounded waits.
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -27,44 +30,69 @@ struct ScanArgs {
   int ntiles, per_cta;
 };
 
-constexpr int kThreads = 14 * 32;
-constexpr uint32_t kTmemCols = 256;  // stage s: acc_off at 128 s, acc_diag at 128 s + 64
-// shared memory (bytes, from a 1024-byte aligned base); per stage:
-constexpr uint32_t OFF_C = 0;          // [128][N]        Cq tile, K-major
-constexpr uint32_t OFF_H = 16384;      // [64][N]         hq tile, K-major
-constexpr uint32_t OFF_X = 24576;      // [256][64]       xq rows, MN-major
-constexpr uint32_t OFF_CB = 40960;     // 2 x [128][128]  CBq panels -> Mq in place
-constexpr uint32_t OFF_TOK = 73728;    // 4 x Q floats: cs, dt, woff, atok (rows 0..3 of the pack)
-constexpr uint32_t OFF_PART = 77824;   // [128] rowmax
-constexpr uint32_t STAGE = 78848;      // 77 KB
-constexpr uint32_t PANEL = 16384;
-// after the two stages:
-constexpr uint32_t OFF_YST = 2 * STAGE;           // 4 warps x 2 halves x [32][128 B] y staging
-constexpr uint32_t OFF_COL = OFF_YST + 32768;     // 4 warps x 4 x [64] per-column factors
-constexpr uint32_t OFF_BAR = OFF_COL + 4096;
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr int kWarps = 28, kThreads = kWarps * 32;
+constexpr int kMaskWarp0 = 4, kMaskWarps = 16, kMaskThreads = kMaskWarps * 32;
+constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
+constexpr uint32_t kTmemCols = 256;  // accumulator pair a: acc_off at 128 a, acc_diag at 128 a + 64
+constexpr uint32_t PANEL = 16384;    // [128][128] int8
+// shared memory (bytes, from a 1024-byte aligned base)
+constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1-panel buffers
+constexpr uint32_t OFF_C = 98304;       // [128][N]
+constexpr uint32_t OFF_H = 114688;      // [64][N]
+constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
+constexpr uint32_t OFF_TOK = 155648;    // ring of 3 x (4 Q floats: cs, dt, woff, atok; 4 x [128] partial row maxima)
+constexpr uint32_t TOK_BYTES = 6144;
+constexpr uint32_t OFF_YST = 174080;    // 8 warps x [32][128 B] y staging
+constexpr uint32_t OFF_BAR = OFF_YST + 32768;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
-enum { B_FULL_CH = 0, B_FULL_CB = 2, B_FULL_X = 4, B_MQ = 6, B_ACC = 8, B_ACC_FREE = 10, B_STAGE_FREE = 12,
-       B_COUNT = 14 };
+__device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
+  return OFF_CB + (idx < 2 ? (uint32_t)idx * 32768u : 65536u + (uint32_t)(idx - 2) * 16384u);
+}
+// which CBq buffer tile n of this CTA uses: with two tiles per chunk the second (two panels)
+// alternates between buffers 0,1 and the first (one panel) between 2,3; otherwise all four rotate
+__device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
+  return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
+}
 
-__device__ __forceinline__ float unpack_s8(uint32_t w_xor, int k) {
-  // w_xor = word ^ 0x80808080: byte + 128 goes into the mantissa of 1.5 * 2^23
-  return __fadd_rn(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)), -12583040.0f);
+enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
+       B_TOK_FULL = 18, B_TOK_FREE = 21, B_ACC = 24, B_ACC_FREE = 26, B_COUNT = 28 };
+
+constexpr float kMagicIn = 12583040.0f;   // 1.5 * 2^23 + 128
+constexpr float kMagicOut = 12582912.0f;  // 1.5 * 2^23
+
+// two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
+__device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
+  const float2 m = make_float2(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)),
+                               __uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7651u + k)));
+  return __fadd2_rn(m, make_float2(-kMagicIn, -kMagicIn));
 }
 // rne(v) for |v| < 2^22 sits in the low bits of (v + 1.5 * 2^23); callers guarantee |v| < 127.5
-__device__ __forceinline__ uint32_t rne_bits(float v) { return __float_as_uint(__fadd_rn(v, 12582912.0f)); }
-__device__ __forceinline__ uint32_t pack4_bits(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
+__device__ __forceinline__ uint32_t pack4_rne(float2 a, float2 b) {
+  const float2 ra = __fadd2_rn(a, make_float2(kMagicOut, kMagicOut));
+  const float2 rb = __fadd2_rn(b, make_float2(kMagicOut, kMagicOut));
+  return __byte_perm(__byte_perm(__float_as_uint(ra.x), __float_as_uint(ra.y), 0x0040u),
+                     __byte_perm(__float_as_uint(rb.x), __float_as_uint(rb.y), 0x0040u), 0x5410u);
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
 }
 
 struct Tile {
   int b, k, h, g, it, KJ;
   i64 tok0, unit;  // unit = (b*H + h)*c + k
 };
-__device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntile_per_unit) {
+__device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntpu) {
   Tile x;
-  x.it = t % ntile_per_unit;
-  int u = t / ntile_per_unit;
+  x.it = t % ntpu;
+  int u = t / ntpu;
   x.h = u % d.H; u /= d.H;
   x.k = u % d.c;
   x.b = u / d.c;
@@ -75,111 +103,107 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
   return x;
 }
 
-// ---- one output row of the masked operand, in place over CBq (thread r of the mask group)
-__device__ __forceinline__ void mask_row(uint8_t* sCB, const float* tok, float* part_s, int r, int TM,
-                                         uint32_t RBQ, const Tile& t, const ScanArgs& a) {
+// ---- the masked operand of one tile, in place over CBq.  Four threads per output row; the
+// row's 16-column chunks (sub-blocks of the decay factorisation) are dealt round robin:
+// thread q handles chunks c = q, q + 4, ...  Chunk I16 = i / 16 is the row's own sub-block
+// (running product of per-token decays), earlier chunks use the column weights woff and one
+// factor f = exp32(cs_i - cs_ce) per chunk, later chunks are zero.
+__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int wtid, int TM, uint32_t RBQ,
+                                          const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
-  const float* cs_s = tok;
-  const float* dt_s = tok + Q;
-  const float* woff_s = tok + 2 * Q;
-  const float* atok_s = tok + 3 * Q;
-  if (r >= TM) return;
+  const float* cs_s = tokbuf;
+  const float* dt_s = tokbuf + Q;
+  const float* woff_s = tokbuf + 2 * Q;
+  const float* atok_s = tokbuf + 3 * Q;
+  float* part_s = tokbuf + 1024;  // [4][128]
+  const int r = wtid & 127, q4 = wtid >> 7;
+  const bool row_ok = r < TM;
   const int i = t.it * TM + r;       // row within the chunk
-  const int I = i >> 6;              // its 64-token sub-block
-  const int nblk = t.KJ >> 6;        // sub-blocks in the contraction range
-  const uint32_t cpp = RBQ >> 4;     // 16-byte chunks per panel row
-  auto chunk_ptr = [&](int j16) -> uint4* {
-    const uint32_t pn = (uint32_t)j16 / cpp, c = (uint32_t)j16 % cpp;
-    return reinterpret_cast<uint4*>(sCB + pn * PANEL + swz_off((uint32_t)r, c, RBQ));
+  const int I16 = i >> 4, ri = i & 15;
+  const int nch = t.KJ >> 4;         // 16-column chunks in the contraction range
+  const uint32_t cpp = RBQ >> 4;     // chunks per panel row
+  auto chunk_ptr = [&](int c) -> uint4* {
+    const uint32_t pn = (uint32_t)c / cpp, cc = (uint32_t)c % cpp;
+    return reinterpret_cast<uint4*>(sCB + pn * PANEL + swz_off((uint32_t)r, cc, RBQ));
   };
-  const float cs_i = cs_s[i];
-  float fJ[3] = {0.f, 0.f, 0.f};
-  float rowmax = 0.f;
-  // earlier sub-blocks: t = cb * woff_j, scaled as a block by f = exp32(cs_i - cs_je)
-#pragma unroll
-  for (int J = 0; J < 3; ++J) {
-    if (J >= I) break;
-    const float f = exp32(__fsub_rn(cs_i, cs_s[J * 64 + 63]));
-    fJ[J] = f;
-    float bmax = 0.f;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint4 w4 = *chunk_ptr(J * 4 + c);
+  const float cs_i = row_ok ? cs_s[i] : 0.f;
+  float tv[16];                      // t of the row's own sub-block (kept by the thread that owns it)
+  float rpart = 0.f;
+  if (row_ok) {
+#pragma unroll 1
+    for (int c = q4; c <= I16; c += 4) {
+      const uint4 w4 = *chunk_ptr(c);
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float* wo = woff_s + J * 64 + c * 16;
+      if (c < I16) {
+        const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
+        const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
+        float bmax = 0.f;
 #pragma unroll
-      for (int e = 0; e < 16; ++e) bmax = fmaxf(bmax, fabsf(__fmul_rn(unpack_s8(ww[e >> 2], e & 3), wo[e])));
-    }
-    rowmax = fmaxf(rowmax, __fmul_rn(bmax, f));
-  }
-  // own sub-block, right to left: E[i,j] = E[i,j+1] a_{j+1}, starting from E[i,i] = 1
-  float tdiag[64];
-  {
-    const int ri = i & 63;
-    float E = 1.0f;
-#pragma unroll
-    for (int c = 3; c >= 0; --c) {
-      const uint4 w4 = *chunk_ptr(I * 4 + c);
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-#pragma unroll
-      for (int e = 15; e >= 0; --e) {
-        const int jj = c * 16 + e;
-        float tv = 0.f;
-        if (jj <= ri) {
-          const int j = (I << 6) + jj;
-          if (jj < ri) E = __fmul_rn(E, atok_s[j + 1]);
-          tv = __fmul_rn(unpack_s8(ww[e >> 2], e & 3), __fmul_rn(dt_s[j], E));
+        for (int w = 0; w < 4; ++w) {
+          const float4 o = wo[w];
+          const float2 t0 = __fmul2_rn(unpack2(ww[w], 0), make_float2(o.x, o.y));
+          const float2 t1 = __fmul2_rn(unpack2(ww[w], 2), make_float2(o.z, o.w));
+          bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
+          bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
         }
-        tdiag[jj] = tv;
-        rowmax = fmaxf(rowmax, fabsf(tv));
+        rpart = fmaxf(rpart, __fmul_rn(bmax, f));
+      } else {
+        // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+        const float* dtc = dt_s + c * 16;
+        const float* atc = atok_s + c * 16 + 1;
+        float E = 1.0f;
+#pragma unroll
+        for (int e = 15; e >= 0; --e) {
+          float v = 0.f;
+          if (e <= ri) {
+            if (e < ri) E = __fmul_rn(E, atc[e]);
+            const float cb = __fadd_rn(__uint_as_float(__byte_perm(ww[e >> 2], 0x4B400000u, 0x7650u + (e & 3))), -kMagicIn);
+            v = __fmul_rn(cb, __fmul_rn(dtc[e], E));
+          }
+          tv[e] = v;
+          rpart = fmaxf(rpart, fabsf(v));
+        }
       }
     }
   }
-  part_s[r] = rowmax;
+  part_s[q4 * 128 + r] = rpart;
+  asm volatile("bar.sync 1, %0;" ::"n"(kMaskThreads) : "memory");
+  const float rowmax = fmaxf(fmaxf(part_s[r], part_s[128 + r]), fmaxf(part_s[256 + r], part_s[384 + r]));
+  if (!row_ok) return;
   const float inv = (rowmax >= 1e-30f) ? __fdiv_rn(127.0f, rowmax) : 0.f;
   int8_t* mq_tap = nullptr;
   if (a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
-  if (a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
-#pragma unroll
-  for (int J = 0; J < 3; ++J) {
-    if (J >= I) break;
-    const float gq = __fmul_rn(fJ[J], inv);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint4* ptr = chunk_ptr(J * 4 + c);
+  if (q4 == 0 && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+#pragma unroll 1
+  for (int c = q4; c < nch; c += 4) {
+    uint4* ptr = chunk_ptr(c);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);  // chunks after the row's own contribute nothing
+    if (c < I16) {
+      const float g = __fmul_rn(exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])), inv);
+      const float2 g2 = make_float2(g, g);
       const uint4 w4 = *ptr;
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float* wo = woff_s + J * 64 + c * 16;
+      const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
       uint32_t o[4];
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        uint32_t q4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          q4[e] = rne_bits(__fmul_rn(__fmul_rn(unpack_s8(ww[w], e), wo[w * 4 + e]), gq));
-        o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
+        const float4 f = wo[w];
+        o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(f.x, f.y)), g2),
+                         __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(f.z, f.w)), g2));
       }
-      const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
-      *ptr = v;
-      if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + J * 64 + c * 16) = v;
+      v = make_uint4(o[0], o[1], o[2], o[3]);
+    } else if (c == I16) {
+      const float2 inv2 = make_float2(inv, inv);
+      uint32_t o[4];
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        o[w] = pack4_rne(__fmul2_rn(make_float2(tv[w * 4], tv[w * 4 + 1]), inv2),
+                         __fmul2_rn(make_float2(tv[w * 4 + 2], tv[w * 4 + 3]), inv2));
+      v = make_uint4(o[0], o[1], o[2], o[3]);
     }
+    *ptr = v;
+    if (mq_tap && c <= I16) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
   }
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    uint32_t o[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const int e = c * 16 + w * 4;
-      o[w] = pack4_bits(rne_bits(__fmul_rn(tdiag[e], inv)), rne_bits(__fmul_rn(tdiag[e + 1], inv)),
-                        rne_bits(__fmul_rn(tdiag[e + 2], inv)), rne_bits(__fmul_rn(tdiag[e + 3], inv)));
-    }
-    const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
-    *chunk_ptr(I * 4 + c) = v;
-    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + I * 64 + c * 16) = v;
-  }
-  for (int J = I + 1; J < nblk; ++J)  // columns after the row's own sub-block contribute nothing
-#pragma unroll
-    for (int c = 0; c < 4; ++c) *chunk_ptr(J * 4 + c) = make_uint4(0u, 0u, 0u, 0u);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -200,14 +224,22 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
 
   if (tid == 0) {
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&bars[B_CB_FULL + s], 1);
+      mbar_init(&bars[B_CB_FREE + s], 1);
+      mbar_init(&bars[B_MQ + s], kMaskWarps);
+    }
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(&bars[B_TOK_FULL + s], 1);
+      mbar_init(&bars[B_TOK_FREE + s], kEpiWarps);
+    }
+    mbar_init(&bars[B_CH_FULL], 1);
+    mbar_init(&bars[B_CH_FREE], 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&bars[B_FULL_CH + s], 1);
-      mbar_init(&bars[B_FULL_CB + s], 1);
-      mbar_init(&bars[B_FULL_X + s], 1);
-      mbar_init(&bars[B_MQ + s], 4);
+      mbar_init(&bars[B_X_FULL + s], 1);
+      mbar_init(&bars[B_X_FREE + s], kEpiWarps);
       mbar_init(&bars[B_ACC + s], 1);
-      mbar_init(&bars[B_ACC_FREE + s], 4);
-      mbar_init(&bars[B_STAGE_FREE + s], 4);
+      mbar_init(&bars[B_ACC_FREE + s], kEpiWarps);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
@@ -220,142 +252,168 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
     if (lane == 0) {
+#pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const int s = n & 1, ph = (n >> 1) & 1;
-        uint8_t* st = smem + s * STAGE;
         const Tile t = decode_tile(tix, d, TM, ntpu);
-        mbar_wait(&bars[B_STAGE_FREE + s], ph ^ 1, a.status);
-        mbar_expect_tx(&bars[B_FULL_CH + s], (uint32_t)(TM * N + 64 * N));
-        tma_load_3d(st + OFF_C, &tm_C, &bars[B_FULL_CH + s], 0, t.g, (int)(t.tok0 + t.it * TM));
-        tma_load_2d(st + OFF_H, &tm_h, &bars[B_FULL_CH + s], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
+        const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
+        const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
+        mbar_wait(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
         const int npanel = t.KJ / (int)RBQ;
-        mbar_expect_tx(&bars[B_FULL_CB + s], (uint32_t)(npanel * TM * RBQ + 4 * Q * 4));
-        bulk_load(st + OFF_TOK, a.pack + t.unit * kPackRows * Q, (uint32_t)(4 * Q * 4), &bars[B_FULL_CB + s]);
+        mbar_expect_tx(&bars[B_CB_FULL + ci], (uint32_t)(npanel * TM * RBQ));
         for (int pn = 0; pn < npanel; ++pn)
-          tma_load_2d(st + OFF_CB + pn * PANEL, &tm_cb, &bars[B_FULL_CB + s], pn * (int)RBQ,
+          tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
                       (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
-        mbar_expect_tx(&bars[B_FULL_X + s], (uint32_t)(t.KJ * 64));
+        mbar_wait(&bars[B_TOK_FREE + t3], ph3 ^ 1, a.status);
+        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(4 * Q * 4));
+        bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(4 * Q * 4),
+                  &bars[B_TOK_FULL + t3]);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ TMA producer: Cq, hq
+    if (lane == 0) {
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
+        const Tile t = decode_tile(tix, d, TM, ntpu);
+        mbar_wait(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
+        mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
+        tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
+        tma_load_2d(smem + OFF_H, &tm_h, &bars[B_CH_FULL], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------ TMA producer: xq rows
+    if (lane == 0) {
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
+        const Tile t = decode_tile(tix, d, TM, ntpu);
+        const int s2 = n & 1;
+        const uint32_t ph2 = (n >> 1) & 1;
+        mbar_wait(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
+        mbar_expect_tx(&bars[B_X_FULL + s2], (uint32_t)(t.KJ * 64));
         for (int j0 = 0; j0 < t.KJ; j0 += TM)
-          tma_load_3d(st + OFF_X + j0 * 64, &tm_x, &bars[B_FULL_X + s], 0, t.h, (int)(t.tok0 + j0));
+          tma_load_3d(smem + OFF_X + s2 * 16384 + j0 * 64, &tm_x, &bars[B_X_FULL + s2], 0, t.h, (int)(t.tok0 + j0));
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc_off = idesc_s8(128, 64, 0, 0), idesc_diag = idesc_s8(128, 64, 0, 1);
+      const uint32_t sbase = smem_u32(smem);
+#pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const int s = n & 1, ph = (n >> 1) & 1;
-        const uint32_t sbase = smem_u32(smem + s * STAGE);
-        const int KJ = ((tix % ntpu) + 1) * TM;
-        const uint32_t acc = tmem + (uint32_t)s * 128u;
-        mbar_wait(&bars[B_ACC_FREE + s], ph ^ 1, a.status);
-        mbar_wait(&bars[B_FULL_CH + s], ph, a.status);
+        const int it = tix % ntpu;
+        const int ci = cb_index(n, it, ntpu), s2 = n & 1;
+        const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
+        const int KJ = (it + 1) * TM;
+        const uint32_t acc = tmem + (uint32_t)s2 * 128u;
+        mbar_wait(&bars[B_ACC_FREE + s2], ph2 ^ 1, a.status);
+        mbar_wait(&bars[B_CH_FULL], n & 1, a.status);
         tc_fence_after();
+#pragma unroll 1
         for (int q = 0; q < N / 32; ++q)
           mma_s8_ss(acc, tile_desc(sbase + OFF_C + 32 * q, RBN), tile_desc(sbase + OFF_H + 32 * q, RBN),
                     idesc_off, q > 0);
-        mbar_wait(&bars[B_MQ + s], ph, a.status);
-        mbar_wait(&bars[B_FULL_X + s], ph, a.status);
+        mma_commit(&bars[B_CH_FREE]);
+        mbar_wait(&bars[B_MQ + ci], ph4, a.status);
+        mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);
         tc_fence_after();
+#pragma unroll 1
         for (int q = 0; q < KJ / 32; ++q) {
           const uint32_t k0 = 32u * q;
-          mma_s8_ss(acc + 64, tile_desc(sbase + OFF_CB + (k0 / RBQ) * PANEL + (k0 % RBQ), RBQ),
-                    tile_desc(sbase + OFF_X + k0 * 64, 64), idesc_diag, q > 0);
+          mma_s8_ss(acc + 64, tile_desc(sbase + cb_offset(ci) + (k0 / RBQ) * PANEL + (k0 % RBQ), RBQ),
+                    tile_desc(sbase + OFF_X + s2 * 16384 + k0 * 64, 64), idesc_diag, q > 0);
         }
-        mma_commit(&bars[B_ACC + s]);
+        mma_commit(&bars[B_CB_FREE + ci]);
+        mma_commit(&bars[B_ACC + s2]);
       }
     }
-  } else if (warp < 10) {
-    // ------------------------------------------------------------ mask groups (stage = group)
-    const int grp = (warp - 2) >> 2;
-    const int r = ((warp - 2) & 3) * 32 + lane;
-    uint8_t* st = smem + grp * STAGE;
-    for (int tix = t_begin + grp, n = grp; tix < t_end; tix += 2, n += 2) {
-      const int ph = (n >> 1) & 1;
+  } else if (warp < kEpiWarp0) {
+    // ------------------------------------------------------------ mask warps
+    const int wtid = tid - kMaskWarp0 * 32;
+#pragma unroll 1
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
       const Tile t = decode_tile(tix, d, TM, ntpu);
-      mbar_wait(&bars[B_FULL_CB + grp], ph, a.status);
-      mask_row(st + OFF_CB, reinterpret_cast<const float*>(st + OFF_TOK),
-               reinterpret_cast<float*>(st + OFF_PART), r, TM, RBQ, t, a);
+      const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
+      const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
+      mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);
+      mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
+      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), wtid, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars[B_MQ + grp]);
+      if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
     }
   } else {
-    // ------------------------------------------------------------ epilogue warps
-    const int ew = warp - 10;
+    // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
+    const int ew = warp - kEpiWarp0;
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int ch = ew >> 2;                 // column half
     const int er = q * 32 + lane;           // row of the tile
-    uint8_t* ystage = smem + OFF_YST + ew * 8192;
-    float* col = reinterpret_cast<float*>(smem + OFF_COL + ew * 1024);  // A, B, D, C x [64]
-    int cur_h = -1;
+    uint8_t* ystage = smem + OFF_YST + ew * 4096;
+#pragma unroll 1
     for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-      const int s = n & 1, ph = (n >> 1) & 1;
-      const uint8_t* st = smem + s * STAGE;
       const Tile t = decode_tile(tix, d, TM, ntpu);
-      if (t.h != cur_h) {
-        cur_h = t.h;
-        __syncwarp();
-        const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f;
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int p = lane + 32 * e, hp = t.h * P + p;
-          const float sx = a.s_x[hp];
-          col[p] = sC * a.s_h[hp];
-          col[64 + p] = sx;
-          col[128 + p] = Dh * sx;
-          col[192 + p] = a.corr ? a.corr[hp] : 0.f;
-        }
-        __syncwarp();
-      }
-      mbar_wait(&bars[B_ACC + s], ph, a.status);
-      mbar_wait(&bars[B_MQ + s], ph, a.status);       // rowmax written by the mask group
-      mbar_wait(&bars[B_FULL_X + s], ph, a.status);   // xq rows (skip term)
-      mbar_wait(&bars[B_FULL_CB + s], ph, a.status);  // cs
+      const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n % 3;
+      const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n / 3) & 1;
+      const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
+      const uint8_t* sX = smem + OFF_X + s2 * 16384;
+      const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f, scb = a.s_cb[t.g];
+      const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
+      const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
+      const float4* gco = a.corr ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
+      mbar_wait(&bars[B_ACC + s2], ph2, a.status);
+      mbar_wait(&bars[B_MQ + ci], ph4, a.status);        // partial row maxima written by the mask warps
+      mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);    // xq rows (skip term)
+      mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);  // cs
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
-      const float* tok = reinterpret_cast<const float*>(st + OFF_TOK);
-      const float* part = reinterpret_cast<const float*>(st + OFF_PART);
-      const float dec = ok ? exp32(tok[ei]) : 0.f;
-      const float sm = ok ? a.s_cb[t.g] * part[er] * (1.0f / 127.0f) : 0.f;
-      if (lane == 0 && n > 0) tma_store_wait_read();  // staging of the previous tile has been read
+      const float* part = tok + 1024;
+      const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
+      const float sm = ok ? scb * fmaxf(fmaxf(part[er], part[128 + er]), fmaxf(part[256 + er], part[384 + er])) *
+                                (1.0f / 127.0f)
+                          : 0.f;
+      const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
+      if (lane == 0) tma_store_wait_read();  // last tile's store has finished reading the staging tile
       __syncwarp();
-#pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        int acc_o[32], acc_d[32];
-        const uint32_t taddr = tmem + (uint32_t)s * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32);
-        tmem_ld32(taddr, acc_o);
-        tmem_ld32(taddr + 64, acc_d);
+      uint8_t* srow = ystage + lane * 128;
+#pragma unroll 1
+      for (int pc = 0; pc < 2; ++pc) {       // 16 columns at a time
+        int acc_o[16], acc_d[16];
+        const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 16);
+        tmem_ld16(taddr, acc_o);
+        tmem_ld16(taddr + 64, acc_d);
         tmem_ld_wait();
         if (ok) {
-          const uint4 x0 = *reinterpret_cast<const uint4*>(st + OFF_X + swz_off((uint32_t)ei, (uint32_t)(ch * 2), 64));
-          const uint4 x1 = *reinterpret_cast<const uint4*>(st + OFF_X + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + 1), 64));
-          const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-          uint8_t* srow = ystage + ch * 4096 + lane * 128;
+          const uint4 xr = *reinterpret_cast<const uint4*>(sX + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + pc), 64));
+          const uint32_t xw[4] = {xr.x ^ 0x80808080u, xr.y ^ 0x80808080u, xr.z ^ 0x80808080u, xr.w ^ 0x80808080u};
 #pragma unroll
-          for (int cc = 0; cc < 8; ++cc) {
-            const int p0 = ch * 32 + cc * 4;
-            const float4 cA = *reinterpret_cast<const float4*>(col + p0);
-            const float4 cB = *reinterpret_cast<const float4*>(col + 64 + p0);
-            const float4 cD = *reinterpret_cast<const float4*>(col + 128 + p0);
-            const float4 cC = *reinterpret_cast<const float4*>(col + 192 + p0);
-            const float A4[4] = {cA.x, cA.y, cA.z, cA.w}, B4[4] = {cB.x, cB.y, cB.z, cB.w};
-            const float D4[4] = {cD.x, cD.y, cD.z, cD.w}, C4[4] = {cC.x, cC.y, cC.z, cC.w};
-            float v[4];
+          for (int cc = 0; cc < 4; ++cc) {
+            const float4 sx4 = __ldg(gsx + pc * 4 + cc), sh4 = __ldg(gsh + pc * 4 + cc);
+            const float4 co4 = gco ? __ldg(gco + pc * 4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float2 v[2];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int pp = cc * 4 + e;
-              const float xv = (float)sx8(xw[pp >> 2], pp & 3);
-              v[e] = fmaf(dec * A4[e], (float)acc_o[pp], fmaf(sm * B4[e], (float)acc_d[pp], fmaf(D4[e], xv, C4[e])));
+            for (int e2 = 0; e2 < 2; ++e2) {
+              const int pp = cc * 4 + e2 * 2;
+              const float2 sx2 = e2 ? make_float2(sx4.z, sx4.w) : make_float2(sx4.x, sx4.y);
+              const float2 sh2 = e2 ? make_float2(sh4.z, sh4.w) : make_float2(sh4.x, sh4.y);
+              const float2 co2 = e2 ? make_float2(co4.z, co4.w) : make_float2(co4.x, co4.y);
+              const float2 xv = unpack2(xw[cc], e2 * 2);
+              const float2 ao = make_float2((float)acc_o[pp], (float)acc_o[pp + 1]);
+              const float2 ad = make_float2((float)acc_d[pp], (float)acc_d[pp + 1]);
+              float2 r2 = __ffma2_rn(__fmul2_rn(Dh2, sx2), xv, co2);
+              r2 = __ffma2_rn(__fmul2_rn(sm2, sx2), ad, r2);
+              v[e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
             }
-            *reinterpret_cast<float4*>(srow + ((cc ^ (lane & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(srow + (((pc * 4 + cc) ^ (lane & 7)) << 4)) =
+                make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
           }
           if (a.taps.acc_off || a.taps.acc_diag) {
-            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32;
+            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 16;
 #pragma unroll
-            for (int pp = 0; pp < 32; ++pp) {
+            for (int pp = 0; pp < 16; ++pp) {
               if (a.taps.acc_off) a.taps.acc_off[o + pp] = acc_o[pp];
               if (a.taps.acc_diag) a.taps.acc_diag[o + pp] = acc_d[pp];
             }
@@ -366,12 +424,11 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       fence_async_smem();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(&bars[B_ACC_FREE + s]);
-        mbar_arrive(&bars[B_STAGE_FREE + s]);
+        mbar_arrive(&bars[B_ACC_FREE + s2]);
+        mbar_arrive(&bars[B_X_FREE + s2]);
+        mbar_arrive(&bars[B_TOK_FREE + t3]);
         if (q * 32 < TM) {
-          const int row0 = (int)(t.tok0 + t.it * TM + q * 32);
-          tma_store_3d(&tm_y, ystage, 0, t.h, row0);
-          tma_store_3d(&tm_y, ystage + 4096, 32, t.h, row0);
+          tma_store_3d(&tm_y, ystage, ch * 32, t.h, (int)(t.tok0 + t.it * TM + q * 32));
           tma_store_commit();
         }
       }
@@ -432,7 +489,8 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   const int ntiles = (int)((i64)d.b * d.c * d.H * (d.Q / TM));
   const int ctas = ntiles < sms ? ntiles : sms;
-  const int per_cta = (ntiles + ctas - 1) / ctas;
+  int per_cta = (ntiles + ctas - 1) / ctas;
+  if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
   ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta};
   const size_t smem = SMEM_BYTES + 1024;
   SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

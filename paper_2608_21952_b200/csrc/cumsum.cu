@@ -2,7 +2,7 @@
 // from it.  For each (batch, head, chunk) it writes one contiguous pack of 5 rows of Q floats:
 //   row 0  cs[i]    = (float) sum_{i'<=i} (double)dt (double)A_h, in token order   (dA_cs)
 //   row 1  dt[i]
-//   row 2  woff[i]  = fmul(dt_i, exp32(fsub(cs_ie, cs_i))), ie = last token of i's 64-token sub-block
+//   row 2  woff[i]  = fmul(dt_i, exp32(fsub(cs_ie, cs_i))), ie = last token of i's 16-token sub-block
 //   row 3  atok[i]  = exp32(fsub(cs_i, cs_{i-1}))  (1 for i = 0): the per-token decay
 //   row 4  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
 // and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     float* p = pack + u * kPackRows * Q + i;
     p[0] = ci;
     p[Q] = di;
-    p[2 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[i | 63], ci)));
+    p[2 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[i | 15], ci)));
     p[3 * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
     p[4 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
     if (tap_cs) tap_cs[u * Q + i] = ci;

@@ -46,7 +46,7 @@ constexpr uint32_t kWaitCap = 1u << 20;
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
   for (uint32_t it = 0; it < kWaitCap; ++it) {
     if (mbar_try_wait(bar, parity)) return;
-    if ((it & 63u) == 63u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
+    if ((it & 8191u) == 8191u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
   }
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
 }
