@@ -43,7 +43,8 @@ constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
 constexpr uint32_t OFF_TOK = 155648;    // ring of 3 x (4 Q floats: cs, dt, woff, atok; 4 x [128] partial row maxima)
 constexpr uint32_t TOK_BYTES = 6144;
 constexpr uint32_t OFF_YST = 174080;    // 8 warps x [32][128 B] y staging
-constexpr uint32_t OFF_BAR = OFF_YST + 32768;
+constexpr uint32_t OFF_FBUF = OFF_YST + 32768;   // [128][16] decay factors f of the tile being masked (thread-private slots)
+constexpr uint32_t OFF_BAR = OFF_FBUF + 8192;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
 __device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
@@ -89,6 +90,20 @@ struct Tile {
   int b, k, h, g, it, KJ;
   i64 tok0, unit;  // unit = (b*H + h)*c + k
 };
+// the tile after x in (it, h, k, b) order, without divisions
+__device__ __forceinline__ void next_tile(Tile& x, const Dims& d, int TM, int ntpu) {
+  if (++x.it == ntpu) {
+    x.it = 0;
+    if (++x.h == d.H) {
+      x.h = 0;
+      if (++x.k == d.c) { x.k = 0; ++x.b; }
+    }
+    x.g = x.h / (d.H / d.G);
+    x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
+    x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
+  }
+  x.KJ = (x.it + 1) * TM;
+}
 __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntpu) {
   Tile x;
   x.it = t % ntpu;
@@ -108,8 +123,8 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
 // thread q handles chunks c = q, q + 4, ...  Chunk I16 = i / 16 is the row's own sub-block
 // (running product of per-token decays), earlier chunks use the column weights woff and one
 // factor f = exp32(cs_i - cs_ce) per chunk, later chunks are zero.
-__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int wtid, int TM, uint32_t RBQ,
-                                          const Tile& t, const ScanArgs& a) {
+__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fbuf, int wtid, int TM,
+                                          uint32_t RBQ, const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
   const float* cs_s = tokbuf;
   const float* dt_s = tokbuf + Q;
@@ -121,11 +136,14 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int wtid,
   const int i = t.it * TM + r;       // row within the chunk
   const int I16 = i >> 4, ri = i & 15;
   const int nch = t.KJ >> 4;         // 16-column chunks in the contraction range
-  const uint32_t cpp = RBQ >> 4;     // chunks per panel row
+  const uint32_t cshift = RBQ == 128 ? 3u : 2u;  // log2(chunks per panel row)
+  uint8_t* const rowbase = sCB + (RBQ == 128 ? (uint32_t)r * 128u : (uint32_t)r * 64u);
+  const uint32_t rx = RBQ == 128 ? ((uint32_t)r & 7u) : (((uint32_t)r >> 1) & 3u);  // swizzle term of the row
   auto chunk_ptr = [&](int c) -> uint4* {
-    const uint32_t pn = (uint32_t)c / cpp, cc = (uint32_t)c % cpp;
-    return reinterpret_cast<uint4*>(sCB + pn * PANEL + swz_off((uint32_t)r, cc, RBQ));
+    const uint32_t pn = (uint32_t)c >> cshift, cc = (uint32_t)c & ((1u << cshift) - 1u);
+    return reinterpret_cast<uint4*>(rowbase + pn * PANEL + ((cc ^ rx) << 4));
   };
+  float* frow = fbuf + r * 16;
   const float cs_i = row_ok ? cs_s[i] : 0.f;
   float tv[16];                      // t of the row's own sub-block (kept by the thread that owns it)
   float rpart = 0.f;
@@ -136,6 +154,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int wtid,
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
       if (c < I16) {
         const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
+        frow[c] = f;
         const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
         float bmax = 0.f;
 #pragma unroll
@@ -179,7 +198,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int wtid,
     uint4* ptr = chunk_ptr(c);
     uint4 v = make_uint4(0u, 0u, 0u, 0u);  // chunks after the row's own contribute nothing
     if (c < I16) {
-      const float g = __fmul_rn(exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])), inv);
+      const float g = __fmul_rn(frow[c], inv);
       const float2 g2 = make_float2(g, g);
       const uint4 w4 = *ptr;
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
@@ -255,8 +274,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
     if (lane == 0) {
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const Tile t = decode_tile(tix, d, TM, ntpu);
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
         const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
         mbar_wait(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
@@ -275,8 +294,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     // ------------------------------------------------------------ TMA producer: Cq, hq
     if (lane == 0) {
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const Tile t = decode_tile(tix, d, TM, ntpu);
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         mbar_wait(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
         mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
         tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
@@ -287,8 +306,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     // ------------------------------------------------------------ TMA producer: xq rows
     if (lane == 0) {
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const Tile t = decode_tile(tix, d, TM, ntpu);
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int s2 = n & 1;
         const uint32_t ph2 = (n >> 1) & 1;
         mbar_wait(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
@@ -334,13 +353,14 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     // ------------------------------------------------------------ mask warps
     const int wtid = tid - kMaskWarp0 * 32;
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-      const Tile t = decode_tile(tix, d, TM, ntpu);
+    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
       const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
       mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);
       mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
-      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), wtid, TM, RBQ, t, a);
+      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES),
+                reinterpret_cast<float*>(smem + OFF_FBUF), wtid, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
@@ -353,8 +373,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     const int er = q * 32 + lane;           // row of the tile
     uint8_t* ystage = smem + OFF_YST + ew * 4096;
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-      const Tile t = decode_tile(tix, d, TM, ntpu);
+    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
       const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n % 3;
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n / 3) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);

@@ -27,26 +27,28 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One attempt: the thread is suspended by the hardware until the phase completes or the
+// suspend-time hint (about 20 us here) runs out, so a waiting warp does not burn issue slots.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Every try_wait already blocks for a hardware-defined interval, so the cap is of
-// the order of a second.  On expiry the caller's status word is set and the wait returns; once
+// Bounded wait.  Every try_wait blocks for up to its suspend-time hint, so the cap is of the
+// order of a second.  On expiry the caller's status word is set and the wait returns; once
 // the word is set, every later wait of the grid gives up after a few polls, so the kernel runs
 // to its normal end (tensor memory is freed) quickly, with undefined results.
-constexpr uint32_t kWaitCap = 1u << 20;
+constexpr uint32_t kWaitCap = 1u << 17;
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
   for (uint32_t it = 0; it < kWaitCap; ++it) {
     if (mbar_try_wait(bar, parity)) return;
-    if ((it & 8191u) == 8191u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
+    if ((it & 255u) == 255u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
   }
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
 }
