@@ -366,8 +366,8 @@ def run_ours(args):
         peaks = measured_peaks()
         # per-module device time (CUDA events around partial runs of the same call)
         phases = {"quantize": lambda: layer.quantize(0), "cumsum": lambda: layer.fwd(bd.PHASE_CUMSUM),
-                  "bmm": lambda: layer.fwd(bd.PHASE_BMM), "chunk_state": lambda: layer.fwd(bd.PHASE_CHUNK_STATE),
-                  "state_passing": lambda: layer.fwd(bd.PHASE_STATE_PASSING),
+                  "bmm": lambda: layer.fwd(bd.PHASE_BMM),
+                  "chunk_state_passing": lambda: layer.fwd(bd.PHASE_CHUNK_STATE | bd.PHASE_STATE_PASSING),
                   "chunk_scan": lambda: layer.fwd(bd.PHASE_SCAN)}
         layer.step(); torch.cuda.synchronize()
         kernel_ms = {k: layer.timed(fn, max(5, min(args.steps, 20))) for k, fn in phases.items()}

@@ -130,14 +130,22 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
       (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, st)) !=
           SSDI8_OK)
     return s;
-  if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
-      (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, pack, loc, a->tap_Xsq,
-                              a->tap_acc_st, nullptr, a->status, st)) != SSDI8_OK)
-    return s;
-  if ((ph & SSDI8_PHASE_STATE_PASSING) &&
-      (s = launch_state_passing(d, loc, gamma, a->init_state, a->s_h, a->tap_prev, a->final_state,
-                                hq, nullptr, st)) != SSDI8_OK)
-    return s;
+  if ((ph & SSDI8_PHASE_CHUNK_STATE) && (ph & SSDI8_PHASE_STATE_PASSING)) {
+    // both modules: the fused chunk-sequential kernel (the fp32 chunk-local states stay on chip)
+    if ((s = launch_chunk_state_passing(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->s_h, pack, gamma,
+                                        a->init_state, hq, a->final_state, a->tap_loc, a->tap_prev,
+                                        a->tap_Xsq, a->tap_acc_st, a->status, st)) != SSDI8_OK)
+      return s;
+  } else {
+    if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
+        (s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, pack, loc, a->tap_Xsq,
+                                a->tap_acc_st, nullptr, a->status, st)) != SSDI8_OK)
+      return s;
+    if ((ph & SSDI8_PHASE_STATE_PASSING) &&
+        (s = launch_state_passing(d, loc, gamma, a->init_state, a->s_h, a->tap_prev, a->final_state,
+                                  hq, nullptr, st)) != SSDI8_OK)
+      return s;
+  }
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
     return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack,

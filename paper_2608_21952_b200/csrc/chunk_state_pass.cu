@@ -1,0 +1,242 @@
+// ChunkState + StatePassing fused, chunk-sequential per (batch, head): the fp32 chunk-local
+// state never goes to HBM.  For chunk k = 0 .. c-1 of one (b, h):
+//   Xs_q[i,p]   = rne(fmul(fmul(float(xq[i,p]), fdiv(s_x, s_xs)), LUT_state[i]))       (Eq. 3)
+//   acc_st[n,p] = sum_i Bq[i,n] Xs_q[i,p]            INT8 MMA over the chunk's tokens, INT32 in TMEM
+//   loc[p,n]    = fmul(float(acc_st), fmul(s_xs[h,p], s_B[g]))                         (Eq. 4 rescale)
+//   hq[k][p,n]  = rne(fmul(S[p,n], fdiv(1, s_h[h,p])))     (state entering chunk k, int8 for ChunkScan1)
+//   S[p,n]      = fmaf(Gamma_k, S[p,n], loc[p,n])                                      (Eq. 6)
+// and final_state = S after the last chunk.  The running state lives in registers: the
+// accumulator has the state index n on the TMEM lanes, so thread (lane n) keeps S[., n] for its
+// 32 channels p.  Operand tiles arrive by TMA, double-buffered across chunks; hq leaves through
+// a shared-memory tile and one TMA store per chunk.  Same arithmetic, operation for operation,
+// as the separate kernels (chunk_state.cu, state_passing.cu).
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace ssdi8 {
+namespace {
+
+using namespace sm100;
+
+struct FusedArgs {
+  const float* s_x; const float* s_xs; const float* s_B; const float* s_h; const float* pack;
+  const float* gamma; const float* init; float* final_state;
+  float* tap_loc; float* tap_prev; int8_t* tap_Xsq; int32_t* tap_acc; int32_t* status;
+  Dims d;
+};
+
+constexpr int kThreads = 256;
+constexpr uint32_t STAGE = 49152;      // per stage: Bq rows [Q][N] (32 KB) + xq rows [Q][64] (16 KB)
+constexpr uint32_t OFF_B = 0;
+constexpr uint32_t OFF_X = 32768;
+constexpr uint32_t OFF_HQ = 2 * STAGE;            // [64 p][N] int8 staging of hq
+constexpr uint32_t OFF_LUT = OFF_HQ + 8192;       // 2 x [256] floats
+constexpr uint32_t OFF_COL = OFF_LUT + 2048;       // [64] s_xs s_B, [64] 1 / s_h
+constexpr uint32_t OFF_BAR = OFF_COL + 512;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
+
+__global__ void __launch_bounds__(kThreads, 2)
+chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
+                    const __grid_constant__ CUtensorMap tm_hq, const FusedArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const Dims& d = a.d;
+  const int Q = d.Q, N = d.N, P = d.P;
+  const int TQ = Q < 128 ? Q : 128;  // rows per TMA box
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int g = h / (d.H / d.G);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);  // [0,1] operands landed, [2] MMA done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
+  uint8_t* sHQ = smem + OFF_HQ;
+
+  if (tid == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    mbar_init(&bars[2], 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tm_B);
+    tma_prefetch_desc(&tm_x);
+    tma_prefetch_desc(&tm_hq);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, 64);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  auto issue_loads = [&](int k) {  // thread 0 only
+    const int s = k & 1;
+    uint8_t* st = smem + s * STAGE;
+    const i64 tok0 = (i64)b * d.L + (i64)k * Q;
+    mbar_expect_tx(&bars[s], (uint32_t)(Q * 64 + Q * N));
+    for (int i0 = 0; i0 < Q; i0 += TQ) {
+      tma_load_3d(st + OFF_X + i0 * 64, &tm_x, &bars[s], 0, h, (int)(tok0 + i0));
+      tma_load_3d(st + OFF_B + i0 * N, &tm_B, &bars[s], 0, g, (int)(tok0 + i0));
+    }
+  };
+  if (tid == 0) issue_loads(0);
+
+  // epilogue geometry: M = 128: accumulator row n on TMEM lane n; M = 64: row n on lane
+  // (n % 16) + 32 (n / 16), i.e. the first 16 lanes of each warp's quarter
+  const int q = warp & 3, ch = warp >> 2;
+  const bool ok = (N == 128) || (lane < 16);
+  const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
+  const i64 bh = (i64)b * d.H + h;
+  float S[32];
+#pragma unroll
+  for (int pp = 0; pp < 32; ++pp)
+    S[pp] = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
+  // per-column factors of the re-quantisation (thread: 16-byte chunk c of every row it visits)
+  const int c = tid & 3;
+  float rx[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    const int hp = h * P + c * 16 + e;
+    rx[e] = __fdiv_rn(a.s_x[hp], a.s_xs[hp]);
+  }
+  float* col_scale = reinterpret_cast<float*>(smem + OFF_COL);
+  float* col_invh = col_scale + 64;
+  if (tid < 64) {
+    col_scale[tid] = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]);
+    col_invh[tid] = __fdiv_rn(1.0f, a.s_h[h * P + tid]);
+  }
+  const i64 unit0 = bh * d.c;
+
+#pragma unroll 1
+  for (int k = 0; k < d.c; ++k) {
+    const int s = k & 1;
+    uint8_t* sB = smem + s * STAGE + OFF_B;
+    uint8_t* sX = smem + s * STAGE + OFF_X;
+    float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
+    const i64 tok0 = (i64)b * d.L + (i64)k * Q;
+    if (tid < Q) lut[tid] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + tid];
+    const float gam = a.gamma[unit0 + k];
+    __syncthreads();  // lut visible; the other stage (chunk k-1) is no longer read by anyone
+    if (tid == 0 && k + 1 < d.c) issue_loads(k + 1);
+    mbar_wait(&bars[s], (k >> 1) & 1, a.status);
+
+    // ---- X_scaled, re-quantised in place (thread: chunk c of rows tid/4, tid/4 + 64, ...)
+    for (int i = tid >> 2; i < Q; i += kThreads / 4) {
+      uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
+      const uint4 w4 = *ptr;
+      const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+      const float l = lut[i];
+      uint32_t o[4];
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        int q4[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          q4[e] = rne_clamp(__fmul_rn(__fmul_rn((float)sx8(ww[w], e), rx[w * 4 + e]), l));
+        o[w] = pack4(q4[0], q4[1], q4[2], q4[3]);
+      }
+      const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+      *ptr = v;
+      if (a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
+    }
+    fence_async_smem();
+    __syncthreads();
+
+    // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+      for (int st = 0; st < Q / 32; ++st)
+        mma_s8_ss(tmem, tile_desc(smem_u32(sB) + 32 * st * N, (uint32_t)N),
+                  tile_desc(smem_u32(sX) + 32 * st * 64, 64), idesc, st > 0);
+      mma_commit(&bars[2]);
+    }
+
+    // ---- while the MMA runs: hq[k] = codes of the state entering this chunk (and the prev tap)
+    if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
+    __syncthreads();
+    if (ok) {
+      const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+#pragma unroll
+      for (int pp = 0; pp < 32; ++pp) {
+        const int p = ch * 32 + pp;
+        sHQ[p * N + n] = (uint8_t)(int8_t)rne_clamp(__fmul_rn(S[pp], col_invh[p]));
+        if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
+      }
+    }
+    fence_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
+      tma_store_commit();
+    }
+
+    // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc)
+    mbar_wait(&bars[2], k & 1, a.status);
+    tc_fence_after();
+    {
+      int acc[32];
+      tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), acc);
+      tmem_ld_wait();
+      if (ok) {
+        const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+#pragma unroll
+        for (int pp = 0; pp < 32; ++pp) {
+          const int p = ch * 32 + pp;
+          const float loc = __fmul_rn((float)acc[pp], col_scale[p]);
+          if (a.tap_loc) a.tap_loc[obase + (i64)pp * N] = loc;
+          if (a.tap_acc) a.tap_acc[obase + (i64)pp * N] = acc[pp];
+          S[pp] = __fmaf_rn(gam, S[pp], loc);
+        }
+      }
+    }
+    tc_fence_before();  // the next chunk's MMA overwrites the accumulator after the next __syncthreads
+  }
+  if (a.final_state && ok) {
+#pragma unroll
+    for (int pp = 0; pp < 32; ++pp) a.final_state[(bh * P + ch * 32 + pp) * N + n] = S[pp];
+  }
+  if (tid == 0) tma_store_wait_read();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 64);
+  }
+}
+
+}  // namespace
+
+ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const int8_t* Bq,
+                                          const float* s_x, const float* s_xs, const float* s_B,
+                                          const float* s_h, const float* pack, const float* gamma,
+                                          const float* init, int8_t* hq, float* final_state,
+                                          float* tap_loc, float* tap_prev, int8_t* tap_Xsq,
+                                          int32_t* tap_acc, int32_t* status, cudaStream_t st) {
+  const int TQ = d.Q < 128 ? d.Q : 128;
+  const uint64_t T = (uint64_t)d.b * d.L;
+  CUtensorMap tm_B, tm_x, tm_hq;
+  {
+    uint64_t dims[3] = {(uint64_t)d.N, (uint64_t)d.G, T};
+    uint64_t str[2] = {(uint64_t)d.N, (uint64_t)d.G * d.N};
+    uint32_t box[3] = {(uint32_t)d.N, 1, (uint32_t)TQ};
+    if (!encode_tensor_map(&tm_B, Bq, 1, 3, dims, str, box, d.N)) return SSDI8_ERR_CUDA;
+  }
+  {
+    uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
+    uint64_t str[2] = {(uint64_t)d.P, (uint64_t)d.H * d.P};
+    uint32_t box[3] = {64, 1, (uint32_t)TQ};
+    if (!encode_tensor_map(&tm_x, xq, 1, 3, dims, str, box, 64)) return SSDI8_ERR_CUDA;
+  }
+  {
+    uint64_t dims[2] = {(uint64_t)d.N, (uint64_t)d.b * d.c * d.H * d.P};
+    uint64_t str[1] = {(uint64_t)d.N};
+    uint32_t box[2] = {(uint32_t)d.N, 64};
+    if (!encode_tensor_map(&tm_hq, hq, 1, 2, dims, str, box, 0)) return SSDI8_ERR_CUDA;
+  }
+  FusedArgs a = {s_x, s_xs, s_B, s_h, pack, gamma, init, final_state, tap_loc, tap_prev, tap_Xsq, tap_acc,
+                 status, d};
+  const size_t smem = SMEM_BYTES + 1024;
+  SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid(d.H, d.b);
+  chunk_state_pass_tc<<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+}  // namespace ssdi8

@@ -30,6 +30,14 @@ ssdi8_status_t launch_chunk_state(const Dims& d, const int8_t* xq, const int8_t*
                                   int32_t* tap_acc, uint32_t* absmax_xs, int32_t* status,
                                   cudaStream_t st);
 
+// ChunkState and StatePassing in one chunk-sequential kernel (loc never leaves the chip)
+ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const int8_t* Bq,
+                                          const float* s_x, const float* s_xs, const float* s_B,
+                                          const float* s_h, const float* pack, const float* gamma,
+                                          const float* init, int8_t* hq, float* final_state,
+                                          float* tap_loc, float* tap_prev, int8_t* tap_Xsq,
+                                          int32_t* tap_acc, int32_t* status, cudaStream_t st);
+
 // absmax_h: per-channel running max (binary32 bits) of |S| over init, prev and final
 ssdi8_status_t launch_state_passing(const Dims& d, const float* loc, const float* gamma,
                                     const float* init, const float* s_h, float* prev,
