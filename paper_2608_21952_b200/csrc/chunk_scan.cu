@@ -59,8 +59,6 @@ __device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
        B_TOK_FULL = 18, B_TOK_FREE = 21, B_ACC = 24, B_ACC_FREE = 26, B_COUNT = 28 };
 
-constexpr float kMagicIn = 12583040.0f;   // 1.5 * 2^23 + 128
-constexpr float kMagicOut = 12582912.0f;  // 1.5 * 2^23
 
 // two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
 __device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {

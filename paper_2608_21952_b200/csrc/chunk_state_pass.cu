@@ -120,16 +120,16 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     for (int i = tid >> 2; i < Q; i += kThreads / 4) {
       uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
       const uint4 w4 = *ptr;
-      const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
       const float l = lut[i];
       uint32_t o[4];
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        int q4[4];
+        uint32_t q4[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-          q4[e] = rne_clamp(__fmul_rn(__fmul_rn((float)sx8(ww[w], e), rx[w * 4 + e]), l));
-        o[w] = pack4(q4[0], q4[1], q4[2], q4[3]);
+          q4[e] = rne_clamp_bits(__fmul_rn(__fmul_rn(s8_to_f32(ww[w], e), rx[w * 4 + e]), l));
+        o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
       }
       const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
       *ptr = v;
@@ -156,7 +156,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
 #pragma unroll
       for (int pp = 0; pp < 32; ++pp) {
         const int p = ch * 32 + pp;
-        sHQ[p * N + n] = (uint8_t)(int8_t)rne_clamp(__fmul_rn(S[pp], col_invh[p]));
+        sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
         if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
       }
     }
@@ -179,7 +179,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
 #pragma unroll
         for (int pp = 0; pp < 32; ++pp) {
           const int p = ch * 32 + pp;
-          const float loc = __fmul_rn((float)acc[pp], col_scale[p]);
+          const float loc = __fmul_rn(i22_to_f32(acc[pp]), col_scale[p]);
           if (a.tap_loc) a.tap_loc[obase + (i64)pp * N] = loc;
           if (a.tap_acc) a.tap_acc[obase + (i64)pp * N] = acc[pp];
           S[pp] = __fmaf_rn(gam, S[pp], loc);

@@ -41,6 +41,27 @@ __device__ __forceinline__ float exp32(float x) {
   return __uint_as_float(__float_as_uint(p) + ((uint32_t)__float2int_rn(n) << 23));
 }
 
+// ---- conversions that stay off the quarter-rate conversion pipe (all exact)
+constexpr float kMagicIn = 12583040.0f;   // 1.5 * 2^23 + 128
+constexpr float kMagicOut = 12582912.0f;  // 1.5 * 2^23
+// int8 byte k of w_xor (= word ^ 0x80808080) as a float: the byte + 128 is placed in the mantissa
+// of 1.5 * 2^23 and the offset subtracted
+__device__ __forceinline__ float s8_to_f32(uint32_t w_xor, int k) {
+  return __fadd_rn(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)), -kMagicIn);
+}
+// int32 with |v| < 2^22 as a float
+__device__ __forceinline__ float i22_to_f32(int v) {
+  return __fadd_rn(__int_as_float(v + 0x4B400000), -kMagicOut);
+}
+// bits whose low byte is the int8 code rne(v) saturated to [-127, 127] (NaN -> -127): clamping
+// before rounding equals rounding before clamping, and (v + 1.5 * 2^23) rounds to nearest even
+__device__ __forceinline__ uint32_t rne_clamp_bits(float v) {
+  return __float_as_uint(__fadd_rn(fminf(fmaxf(v, -127.0f), 127.0f), kMagicOut));
+}
+__device__ __forceinline__ uint32_t pack4_bits(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
+}
+
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
   return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
          ((uint32_t)(d & 0xff) << 24);
