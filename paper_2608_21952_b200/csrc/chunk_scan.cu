@@ -271,8 +271,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
     if (lane == 0) {
-#pragma unroll 1
       Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
         const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
@@ -291,8 +291,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   } else if (warp == 2) {
     // ------------------------------------------------------------ TMA producer: Cq, hq
     if (lane == 0) {
-#pragma unroll 1
       Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         mbar_wait(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
         mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
@@ -303,8 +303,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   } else if (warp == 3) {
     // ------------------------------------------------------------ TMA producer: xq rows
     if (lane == 0) {
-#pragma unroll 1
       Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int s2 = n & 1;
         const uint32_t ph2 = (n >> 1) & 1;
@@ -350,8 +350,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------ mask warps
     const int wtid = tid - kMaskWarp0 * 32;
-#pragma unroll 1
     Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
     for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
       const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
@@ -370,8 +370,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     const int ch = ew >> 2;                 // column half
     const int er = q * 32 + lane;           // row of the tile
     uint8_t* ystage = smem + OFF_YST + ew * 4096;
-#pragma unroll 1
     Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
     for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
       const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n % 3;
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n / 3) & 1;

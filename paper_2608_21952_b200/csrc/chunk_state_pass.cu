@@ -112,8 +112,20 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     const i64 tok0 = (i64)b * d.L + (i64)k * Q;
     if (tid < Q) lut[tid] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + tid];
     const float gam = a.gamma[unit0 + k];
-    __syncthreads();  // lut visible; the other stage (chunk k-1) is no longer read by anyone
+    if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
+    __syncthreads();  // lut visible; stage (k+1)&1 and the hq staging tile are no longer read by anyone
     if (tid == 0 && k + 1 < d.c) issue_loads(k + 1);
+
+    // ---- hq[k] = codes of the state entering this chunk (and the prev tap)
+    if (ok) {
+      const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+#pragma unroll
+      for (int pp = 0; pp < 32; ++pp) {
+        const int p = ch * 32 + pp;
+        sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
+        if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
+      }
+    }
     mbar_wait(&bars[s], (k >> 1) & 1, a.status);
 
     // ---- X_scaled, re-quantised in place (thread: chunk c of rows tid/4, tid/4 + 64, ...)
@@ -138,7 +150,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     fence_async_smem();
     __syncthreads();
 
-    // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]
+    // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]; hq[k] leaves by TMA while the MMA runs
     if (tid == 0) {
       tc_fence_after();
       const uint32_t idesc = idesc_s8(N, 64, 1, 1);
@@ -146,23 +158,6 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
         mma_s8_ss(tmem, tile_desc(smem_u32(sB) + 32 * st * N, (uint32_t)N),
                   tile_desc(smem_u32(sX) + 32 * st * 64, 64), idesc, st > 0);
       mma_commit(&bars[2]);
-    }
-
-    // ---- while the MMA runs: hq[k] = codes of the state entering this chunk (and the prev tap)
-    if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
-    __syncthreads();
-    if (ok) {
-      const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
-#pragma unroll
-      for (int pp = 0; pp < 32; ++pp) {
-        const int p = ch * 32 + pp;
-        sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
-        if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
-      }
-    }
-    fence_async_smem();
-    __syncthreads();
-    if (tid == 0) {
       tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
       tma_store_commit();
     }
