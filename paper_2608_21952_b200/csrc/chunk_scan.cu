@@ -40,9 +40,9 @@ constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1
 constexpr uint32_t OFF_C = 98304;       // [128][N]
 constexpr uint32_t OFF_H = 114688;      // [64][N]
 constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
-constexpr uint32_t OFF_TOK = 155648;    // ring of 3 x (4 Q floats: cs, dt, woff, atok; 4 x [128] partial row maxima)
-constexpr uint32_t TOK_BYTES = 6144;
-constexpr uint32_t OFF_YST = 174080;    // 8 warps x [32][128 B] y staging
+constexpr uint32_t OFF_TOK = 155648;    // ring of 3 x (5 Q floats: cs, dt, woff, atok, wmax; 4 x [128] partial row maxima)
+constexpr uint32_t TOK_BYTES = 7168;
+constexpr uint32_t OFF_YST = 177152;    // 8 warps x [32][128 B] y staging
 constexpr uint32_t OFF_FBUF = OFF_YST + 32768;   // [128][16] decay factors f of the tile being masked (thread-private slots)
 constexpr uint32_t OFF_BAR = OFF_FBUF + 8192;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
@@ -128,7 +128,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
   const float* dt_s = tokbuf + Q;
   const float* woff_s = tokbuf + 2 * Q;
   const float* atok_s = tokbuf + 3 * Q;
-  float* part_s = tokbuf + 1024;  // [4][128]
+  const float* wmax_s = tokbuf + 4 * Q;
+  float* part_s = tokbuf + 1280;  // [4][128]
   const int r = wtid & 127, q4 = wtid >> 7;
   const bool row_ok = r < TM;
   const int i = t.it * TM + r;       // row within the chunk
@@ -146,13 +147,16 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
   float tv[16];                      // t of the row's own sub-block (kept by the thread that owns it)
   float rpart = 0.f;
   if (row_ok) {
+    // nearest chunks first: they carry the largest weights, so the running maximum soon exceeds
+    // the bound 127 wmax_c f of the far chunks, which are then skipped (they cannot be the maximum)
 #pragma unroll 1
-    for (int c = q4; c <= I16; c += 4) {
-      const uint4 w4 = *chunk_ptr(c);
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+    for (int c = I16 - ((I16 - q4) & 3); c >= 0; c -= 4) {
       if (c < I16) {
         const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
         frow[c] = f;
+        if (__fmul_rn(__fmul_rn(127.0f, wmax_s[c]), f) <= rpart) continue;
+        const uint4 w4 = *chunk_ptr(c);
+        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
         const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
         float bmax = 0.f;
 #pragma unroll
@@ -166,6 +170,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
         rpart = fmaxf(rpart, __fmul_rn(bmax, f));
       } else {
         // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+        const uint4 w4 = *chunk_ptr(c);
+        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
         const float* dtc = dt_s + c * 16;
         const float* atc = atok_s + c * 16 + 1;
         float E = 1.0f;
@@ -174,8 +180,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
           float v = 0.f;
           if (e <= ri) {
             if (e < ri) E = __fmul_rn(E, atc[e]);
-            const float cb = __fadd_rn(__uint_as_float(__byte_perm(ww[e >> 2], 0x4B400000u, 0x7650u + (e & 3))), -kMagicIn);
-            v = __fmul_rn(cb, __fmul_rn(dtc[e], E));
+            v = __fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E));
           }
           tv[e] = v;
           rpart = fmaxf(rpart, fabsf(v));
@@ -197,6 +202,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
     uint4 v = make_uint4(0u, 0u, 0u, 0u);  // chunks after the row's own contribute nothing
     if (c < I16) {
       const float g = __fmul_rn(frow[c], inv);
+      // every |cb woff g| <= 127 wmax_c g: below one half the whole chunk rounds to zero
+      if (__fmul_rn(__fmul_rn(127.0f, wmax_s[c]), g) >= 0.5f) {
       const float2 g2 = make_float2(g, g);
       const uint4 w4 = *ptr;
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
@@ -209,6 +216,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
                          __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(f.z, f.w)), g2));
       }
       v = make_uint4(o[0], o[1], o[2], o[3]);
+      }
     } else if (c == I16) {
       const float2 inv2 = make_float2(inv, inv);
       uint32_t o[4];
@@ -283,8 +291,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
           tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
                       (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
         mbar_wait(&bars[B_TOK_FREE + t3], ph3 ^ 1, a.status);
-        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(4 * Q * 4));
-        bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(4 * Q * 4),
+        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4));
+        bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4),
                   &bars[B_TOK_FULL + t3]);
       }
     }
@@ -388,7 +396,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
-      const float* part = tok + 1024;
+      const float* part = tok + 1280;
       const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
       const float sm = ok ? scb * fmaxf(fmaxf(part[er], part[128 + er]), fmaxf(part[256 + er], part[384 + er])) *
                                 (1.0f / 127.0f)

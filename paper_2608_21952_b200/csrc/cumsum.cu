@@ -1,10 +1,12 @@
 // ChunkCumsum (Algorithm 2, module 1) and the per-token scalars every later module derives
-// from it.  For each (batch, head, chunk) it writes one contiguous pack of 5 rows of Q floats:
+// from it.  For each (batch, head, chunk) it writes one contiguous pack of 6 rows of Q floats:
 //   row 0  cs[i]    = (float) sum_{i'<=i} (double)dt (double)A_h, in token order   (dA_cs)
 //   row 1  dt[i]
 //   row 2  woff[i]  = fmul(dt_i, exp32(fsub(cs_ie, cs_i))), ie = last token of i's 16-token sub-block
 //   row 3  atok[i]  = exp32(fsub(cs_i, cs_{i-1}))  (1 for i = 0): the per-token decay
-//   row 4  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
+//   row 4  wmax[c]  = max of woff over the 16-token sub-block c (first Q/16 entries; the rest 0):
+//                     an upper bound that lets the scan kernel skip sub-blocks that cannot matter
+//   row 5  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
 // and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
 // (it decides rounding downstream), so each (b, chunk, head) is scanned sequentially by one
 // thread; loads and stores go through shared memory so that the [b,L,H] reads and the row
@@ -15,17 +17,18 @@
 namespace ssdi8 {
 namespace {
 
-constexpr int CH = 16;  // heads per block
+constexpr int CH = 8;  // heads per block
 
 __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ dt,
                                                      const float* __restrict__ A,
                                                      float* __restrict__ pack,
                                                      float* __restrict__ gamma,
                                                      float* __restrict__ tap_cs, Dims d) {
-  extern __shared__ float tile[];  // dt [CH][Q+1], cs [CH][Q+1]
+  extern __shared__ float tile[];  // dt [CH][Q+1], cs [CH][Q+1], woff [CH][Q+1]
   const int Q = d.Q, ld = Q + 1;
   float* dts = tile;
   float* css = tile + CH * ld;
+  float* wos = tile + 2 * CH * ld;
   const int h0 = blockIdx.x * CH, k = blockIdx.y, b = blockIdx.z;
   const int nh = min(CH, d.H - h0);
   const i64 t0 = (i64)b * d.L + (i64)k * Q;
@@ -56,10 +59,21 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     float* p = pack + u * kPackRows * Q + i;
     p[0] = ci;
     p[Q] = di;
-    p[2 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[i | 15], ci)));
-    p[3 * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
-    p[4 * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
+    const float wo = __fmul_rn(di, exp32(__fsub_rn(c[i | 15], ci)));
+    wos[hh * ld + i] = wo;
+    p[PACK_WOFF * Q] = wo;
+    p[PACK_ATOK * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
+    p[PACK_LUT * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
     if (tap_cs) tap_cs[u * Q + i] = ci;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
+    const int hh = e / Q, i = e % Q;
+    if (hh >= nh) continue;
+    float m = 0.f;
+    if (i < Q / 16)
+      for (int j = 0; j < 16; ++j) m = fmaxf(m, wos[hh * ld + i * 16 + j]);
+    pack[((((i64)b * d.H + h0 + hh) * d.c + k) * kPackRows + PACK_WMAX) * Q + i] = m;
   }
 }
 
@@ -68,7 +82,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
                              float* gamma, float* tap_cs, cudaStream_t st) {
   dim3 grid((d.H + CH - 1) / CH, d.c, d.b);
-  size_t smem = sizeof(float) * 2 * CH * (d.Q + 1);
+  size_t smem = sizeof(float) * 3 * CH * (d.Q + 1);
   cumsum_kernel<<<grid, 256, smem, st>>>(dt, A, pack, gamma, tap_cs, d);
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;

@@ -7,12 +7,12 @@ namespace ssdi8 {
 ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
                                int8_t* out, cudaStream_t st);
 
-// Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, lut (see
+// Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, wmax, lut (see
 // cumsum.cu); element (u, row, i) at pack[(u * kPackRows + row) * Q + i], u = (b*H + h)*c + k.
-constexpr int kPackRows = 5;
-enum { PACK_CS = 0, PACK_DT = 1, PACK_WOFF = 2, PACK_ATOK = 3, PACK_LUT = 4 };
+constexpr int kPackRows = 6;
+enum { PACK_CS = 0, PACK_DT = 1, PACK_WOFF = 2, PACK_ATOK = 3, PACK_WMAX = 4, PACK_LUT = 5 };
 
-// pack [b,H,c,5,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
+// pack [b,H,c,6,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
                              float* gamma, float* tap_cs, cudaStream_t st);
 
