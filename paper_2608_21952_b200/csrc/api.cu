@@ -127,7 +127,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
   if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st)) != SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_BMM) &&
-      (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, st)) !=
+      (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, a->status, st)) !=
           SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_CHUNK_STATE) && (ph & SSDI8_PHASE_STATE_PASSING)) {
@@ -187,7 +187,7 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
     return s;
   if ((s = launch_finalize_scales(s_xs, nhp, nullptr, nullptr, 0, st)) != SSDI8_OK) return s;
   if ((s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, nullptr, nullptr, nullptr,
-                      reinterpret_cast<uint32_t*>(s_cb), st)) != SSDI8_OK)
+                      reinterpret_cast<uint32_t*>(s_cb), nullptr, st)) != SSDI8_OK)
     return s;
   if ((s = launch_finalize_scales(s_cb, d.G, a->s_C, a->s_B, 1, st)) != SSDI8_OK) return s;
   if ((s = launch_chunk_state(d, a->xq, a->Bq, a->s_x, s_xs, a->s_B, pack, loc, nullptr,

@@ -20,7 +20,7 @@ ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, flo
 // running max of |acc_cb| over the causal half (calibration; may be NULL)
 ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, const float* s_C,
                           const float* s_B, const float* s_cb, int8_t* CBq, int32_t* tap_acc,
-                          uint32_t* absmax_acc, cudaStream_t st);
+                          uint32_t* absmax_acc, int32_t* status, cudaStream_t st);
 
 // absmax_xs: per-channel running max (as binary32 bits) of |x_scaled| (calibration; may be
 // NULL).  When absmax_xs is non-NULL only that is computed.
