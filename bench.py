@@ -3,8 +3,8 @@
 
 One step = one pass of the whole hot path over one batch of seeded synthetic input:
 Eq. 1 quantisation of fp32 x, B, C with static step sizes (3 launches), then the
-five-kernel layer forward (ChunkCumsum, ChunkBMM, ChunkState, StatePassing,
-ChunkScan) from int8 x, B, C to the fp32 output y and the final state.
+layer forward (ChunkCumsum, ChunkBMM, fused ChunkState+StatePassing, ChunkScan)
+from int8 x, B, C to the fp32 output y and the final state.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
 
@@ -238,7 +238,7 @@ class Layer:
         self.quantize(0)
         self.fwd()
 
-    LAUNCHES_PER_STEP = 8  # 3 quantiser + 5 layer kernels
+    LAUNCHES_PER_STEP = 7  # 3 quantiser + cumsum, BMM, fused chunk state / state passing, chunk scan
 
     def e2e_step(self):
         for k in ("x", "B", "C", "dt"):
