@@ -168,8 +168,23 @@ TAP_SPECS = {
 }
 
 
+FLAG_INT8_STATE = 2
+
+
+def state_passing_int8(cfg, acc_st, gamma, init, s_xs, s_B, s_h):
+    """Eq. 4 + Eq. 7: persistent INT8 states with the fixed-point decay.  Returns (hq int8, final fp32)."""
+    d = dims_of(cfg)
+    shp = (cfg.batch, cfg.nchunks, cfg.nheads, cfg.headdim, cfg.dstate)
+    acc = np.ascontiguousarray(acc_st, dtype=np.int32)
+    hq = np.empty(shp, np.int8)
+    fin = np.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), np.float32)
+    _lib.orc_state_passing_int8(C.byref(d), _p(acc), _p(_f32(gamma)), _p(_f32(init)), _p(_f32(s_xs)),
+                                _p(_f32(s_B)), _p(_f32(s_h)), _p(hq), _p(fin))
+    return hq, fin
+
+
 def ssdi8_fwd(cfg, xq, Bq, Cq, s_x, s_B, s_C, dt, A, D, corr, s_xs, s_cb, s_h, init=None,
-              taps=()):
+              taps=(), flags=0):
     """L2 forward.  Returns (y fp64, final fp32, {tap name: array})."""
     d = dims_of(cfg)
     y = np.empty((cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim), np.float64)
@@ -183,7 +198,7 @@ def ssdi8_fwd(cfg, xq, Bq, Cq, s_x, s_B, s_C, dt, A, D, corr, s_xs, s_cb, s_h, i
     _lib.orc_ssdi8_fwd(C.byref(d), _p(_i8(xq)), _p(_i8(Bq)), _p(_i8(Cq)), _p(_f32(s_x)),
                        _p(_f32(s_B)), _p(_f32(s_C)), _p(_f32(dt)), _p(_f32(A)), _p(_f32(D)),
                        _p(_f32(corr)), _p(_f32(s_xs)), _p(_f32(s_cb)), _p(_f32(s_h)),
-                       _p(_f32(init)), _p(y), _p(fin), C.byref(t))
+                       _p(_f32(init)), _p(y), _p(fin), C.byref(t), C.c_uint32(flags))
     return y, fin, out
 
 

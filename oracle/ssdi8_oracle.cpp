@@ -10,7 +10,8 @@
 //       of Section 3.2 with the zero-order-hold step dt):
 //         h_t = exp(dt_t A) h_{t-1} + dt_t B_t x_t^T ,  y_t = C_t h_t + D x_t
 //   L1  chunked (dual) form of Algorithm 2 in fp64, no internal quantisation
-//   L2  SSDi8: Algorithm 2 with the INT8 path of Section 4.2 (Eq. 1, 3, 4)
+//   L2  SSDi8: Algorithm 2 with the INT8 path of Section 4.2 (Eq. 1, 3, 4); inter-chunk states
+//       either fp32 or, as in the paper, persistent INT8 with a fixed-point decay (Eq. 7)
 //   L3  single-token recurrent step (L0 restated per token, state in place)
 //
 // Precision.  Everything is fp64 with exact integer products, except the
@@ -376,6 +377,47 @@ void orc_state_passing(const Dims* d, const float* loc, const float* gamma, cons
       }
 }
 
+// ---------------------------------------------------------------------------
+// L2 stage, the paper's own state format: persistent INT8 states with a fixed-point decay
+// (Section 4.2 "Persistent INT8 Representation of Recurrent States", Eq. 4 and Eq. 7).
+//   r_st[h,p] = fdiv(fmul(s_xs[h,p], s_B[g]), s_h[h,p])        (Eq. 4: s_x s_b q_max / s_s)
+//   locq_k    = round(fmul(float(acc_st_k), r_st))             INT32 -> INT8, per-(H,P) scale s_h
+//   Gq_k      = round(fmul(Gamma_k, 128))  in [0, 128]         Q(Decay), S = 2^7
+//   Sq_k      = sat(locq_k + ((Gq_k * Sq_{k-1} + 64) >> 7))    Eq. 7: multiply, shift by k = 7 with
+//               rounding (floor((v + 64) / 128)), saturate to [-127, 127]
+//   Sq_{-1}   = round(fmul(init, fdiv(1, s_h))) or 0;  hq[k] = Sq_{k-1};  final = fmul(float(Sq_{c-1}), s_h)
+// All states of all chunks share the one scale s_h[h,p], which is what makes the shift exact.
+void orc_state_passing_int8(const Dims* d, const int32_t* acc_st, const float* gamma,
+                            const float* init, const float* s_xs, const float* s_B,
+                            const float* s_h, int8_t* hq, float* final_state) {
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
+            G = d->ngroups, Q = d->chunk, c = L / Q, hpg = H / G;
+#pragma omp parallel for collapse(2)
+  for (int b = 0; b < b_; ++b)
+    for (int h = 0; h < H; ++h)
+      for (int p = 0; p < P; ++p) {
+        const float sh = s_h[h * P + p];
+        const float r_st = fdiv(fmul(s_xs[h * P + p], s_B[h / hpg]), sh);
+        const float inv_h = fdiv(1.0f, sh);
+        for (int n = 0; n < N; ++n) {
+          int Sq = init ? (int)rne_clamp(fmul(init[(((i64)b * H + h) * P + p) * N + n], inv_h)) : 0;
+          for (int k = 0; k < c; ++k) {
+            const i64 o = ((((i64)b * c + k) * H + h) * P + p) * N + n;
+            hq[o] = (int8_t)Sq;
+            const int locq = (int)rne_clamp(fmul((float)acc_st[o], r_st));
+            const int Gq = (int)std::nearbyintf(fmul(gamma[((i64)b * H + h) * c + k], 128.0f));
+            const int v = Gq * Sq + 64;
+            const int shifted = (v >= 0) ? (v / 128) : -((-v + 127) / 128);  // floor(v / 128)
+            int Sn = locq + shifted;
+            if (Sn > 127) Sn = 127;
+            if (Sn < -127) Sn = -127;
+            Sq = Sn;
+          }
+          if (final_state) final_state[(((i64)b * H + h) * P + p) * N + n] = fmul((float)Sq, sh);
+        }
+      }
+}
+
 // Gamma[b,h,k] = exp32(cs[b,h,k,Q-1])   (Decay_pass of Eq. 5)
 void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
   const int b_ = d->batch, L = d->seqlen, H = d->nheads, Q = d->chunk, c = L / Q;
@@ -551,11 +593,13 @@ struct Taps {
   float* prev; int8_t* hq; int32_t* acc_off; float* rowmax; int8_t* Mq; int32_t* acc_diag;
 };
 
+// flags bit 1 (value 2): the paper's persistent INT8 states (orc_state_passing_int8) instead of
+// fp32 states; the loc and prev taps are not produced in that mode.
 void orc_ssdi8_fwd(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8_t* Cq,
                    const float* s_x, const float* s_B, const float* s_C, const float* dt,
                    const float* A, const float* D, const float* corr, const float* s_xs,
                    const float* s_cb, const float* s_h, const float* init, double* y,
-                   float* final_state, const Taps* taps) {
+                   float* final_state, const Taps* taps, uint32_t flags) {
   const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
             G = d->ngroups, Q = d->chunk, c = L / Q;
   Taps none;
@@ -578,8 +622,16 @@ void orc_ssdi8_fwd(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8
   orc_chunk_cumsum(d, dt, A, cs);
   orc_chunk_decay(d, cs, gamma.data());
   orc_chunk_bmm(d, Cq, Bq, s_C, s_B, s_cb, tp->acc_cb, CBq);
-  orc_chunk_state(d, xq, Bq, s_x, s_xs, s_B, dt, cs, tp->Xsq, tp->acc_st, loc);
-  orc_state_passing(d, loc, gamma.data(), init, s_h, prev, final_state, hq);
+  if (flags & 2u) {
+    std::vector<int32_t> acc_v;
+    int32_t* acc = tp->acc_st;
+    if (!acc) { acc_v.resize(nst); acc = acc_v.data(); }
+    orc_chunk_state(d, xq, Bq, s_x, s_xs, s_B, dt, cs, tp->Xsq, acc, nullptr);
+    orc_state_passing_int8(d, acc, gamma.data(), init, s_xs, s_B, s_h, hq, final_state);
+  } else {
+    orc_chunk_state(d, xq, Bq, s_x, s_xs, s_B, dt, cs, tp->Xsq, tp->acc_st, loc);
+    orc_state_passing(d, loc, gamma.data(), init, s_h, prev, final_state, hq);
+  }
   orc_chunk_scan(d, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D, corr, tp->acc_off,
                  tp->rowmax, tp->Mq, tp->acc_diag, y);
 }

@@ -400,3 +400,68 @@ def test_oracle_reproduces_stored_digests():
                 assert abs(got[k] - v) <= 1e-9 * abs(v), (name, k)
             else:
                 assert got[k] == v, (name, k)
+
+
+# --------------------------------------------------------------------------- Eq. 4 + Eq. 7: persistent INT8 states
+def _int8_state_case(cfg, init=None):
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t, init)
+    y, fin, taps = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"], q["A"],
+                                 q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], init,
+                                 taps=("cs", "acc_st", "hq", "acc_off"), flags=orc.FLAG_INT8_STATE)
+    return t, q, y, fin, taps
+
+
+@pytest.mark.parametrize("cfg", [TINY, CONFIGS["cfg0"]], ids=lambda c: c.name)
+def test_int8_state_tracks_the_fp32_recurrence_within_its_error_bound(cfg):
+    """Each step adds at most 1.5 code units (rounding of loc, rounding of the shift, quantisation of
+    the decay to 1/128) on top of Gamma times the previous error, so the INT8 state stays within
+    1.5 (k + 1) + 0.5 codes of the fp32 recurrence on the same integer chunk states."""
+    rng = np.random.default_rng(8)
+    init = (0.2 * rng.standard_normal((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate))).astype(np.float32)
+    t, q, y, fin, taps = _int8_state_case(cfg, init)
+    H, P, G = cfg.nheads, cfg.headdim, cfg.ngroups
+    hg = np.arange(H) // (H // G)
+    s_h = q["s_h"].astype(np.float64).reshape(H, P)[None, :, :, None]
+    scale = (q["s_xs"].astype(np.float64).reshape(H, P) * q["s_B"].astype(np.float64)[hg][:, None])[None, :, :, None]
+    gam = np.exp(taps["cs"][..., -1].astype(np.float64))                   # [b,H,c]
+    S = init.astype(np.float64)
+    saturated = np.zeros(S.shape, bool)
+    for k in range(cfg.nchunks):
+        codes = taps["hq"][:, k].astype(np.float64)
+        saturated |= np.abs(codes) >= 127
+        assert np.all((np.abs(codes - S / s_h) <= 1.5 * k + 0.5 + 1e-6) | saturated), k
+        loc = taps["acc_st"][:, k] * scale
+        saturated |= np.abs(loc / s_h) >= 127          # Eq. 4 saturates the chunk-local code itself
+        S = loc + gam[:, :, k, None, None] * S
+    assert np.all((np.abs(fin / s_h - S / s_h) <= 1.5 * cfg.nchunks + 0.5 + 1e-6) | saturated)
+    assert saturated.mean() < 0.05   # the bound is checked on (nearly) all elements
+    assert np.abs(taps["hq"].astype(int)).max() <= 127
+
+
+def test_int8_state_with_unit_decay_is_a_saturating_integer_sum():
+    """Gamma = 1 quantises to 128, (128 S + 64) >> 7 = S exactly: the recurrence is sat(sum of codes)."""
+    cfg = TINY
+    rng = np.random.default_rng(9)
+    shp = (cfg.batch, cfg.nchunks, cfg.nheads, cfg.headdim, cfg.dstate)
+    acc = rng.integers(-40, 41, shp).astype(np.int32)
+    ones = np.ones(cfg.channels, np.float32)
+    gamma = np.ones((cfg.batch, cfg.nheads, cfg.nchunks), np.float32)
+    hq, fin = orc.state_passing_int8(cfg, acc, gamma, None, ones, np.ones(cfg.ngroups, np.float32), ones)
+    run = np.zeros(shp[:1] + shp[2:], np.int64)
+    for k in range(cfg.nchunks):
+        assert np.array_equal(hq[:, k], run)
+        run = np.clip(run + acc[:, k], -127, 127)
+    assert np.array_equal(fin, run.astype(np.float32))
+    # zero decay forgets the past entirely
+    hq0, fin0 = orc.state_passing_int8(cfg, acc, np.zeros_like(gamma), None, ones, np.ones(cfg.ngroups, np.float32), ones)
+    assert np.array_equal(hq0[:, 1:], np.clip(acc[:, :-1], -127, 127))
+
+
+def test_int8_state_forward_stays_close_to_the_dual_form():
+    cfg = CONFIGS["cfg0"]
+    t, q, y, fin, taps = _int8_state_case(cfg)
+    xh, Bh, Ch = dequant(cfg, q)
+    y1, f1 = orc.ssd_chunked(cfg, xh, Bh, Ch, t["dt"], t["A"], t["D"])
+    assert np.sqrt(((y - y1) ** 2).sum() / (y1 ** 2).sum()) < 5e-2
+    assert np.sqrt(((fin - f1) ** 2).sum() / (f1 ** 2).sum()) < 8e-2
