@@ -69,6 +69,9 @@ enum {
   SSDI8_PHASE_ALL = 0x1f00u
 };
 
+/* state format bit of ssdi8_chunk_scan_fwd's flags */
+enum { SSDI8_FLAG_INT8_STATE = 1u << 1 };
+
 /* host, pure: static string for a status code */
 const char* ssdi8_status_string(ssdi8_status_t s);
 
@@ -155,7 +158,14 @@ typedef struct {
  *                acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p], INT32;
  *                y_diag = (s_cb rowmax_i / 127) s_x acc_diag
  *  Output        y = y_off + y_diag + D s_x xq + corr
- * flags: bit 0 is reserved for the paper's FP16 ChunkScan2 operand and must be 0.  Bits 8-12
+ * flags: bit 0 is reserved for the paper's FP16 ChunkScan2 operand and must be 0.
+ * SSDI8_FLAG_INT8_STATE selects the paper's own inter-chunk state format (Section 4.2, Eq. 4, 7)
+ * instead of fp32 states: the chunk-local state goes INT32 -> INT8 in registers and the
+ * recurrence is integer with a fixed-point decay, all states sharing the scale s_h[h,p]:
+ *   locq = rne(fmul(float(acc_st), fdiv(fmul(s_xs, s_B), s_h)));   Gq = rne(fmul(Gamma_k, 128))
+ *   Sq_k = sat(locq + ((Gq * Sq_{k-1} + 64) >> 7)),  Sq_{-1} = rne(fmul(init_state, fdiv(1, s_h)))
+ *   hq[k] = Sq_{k-1};  final_state = fmul(float(Sq_{c-1}), s_h);  tap_loc, tap_prev are not written.
+ * Bits 8-12
  * select modules (SSDI8_PHASE_*); 0 in those bits runs all five in order.  A partial run
  * reads the intermediates a previous call left in the same workspace (per-module timing,
  * tests); any other bit set gives SSDI8_ERR_UNSUPPORTED.

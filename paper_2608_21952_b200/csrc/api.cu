@@ -76,7 +76,7 @@ const char* ssdi8_status_string(ssdi8_status_t s) {
 }
 
 size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
-  if ((flags & ~(uint32_t)SSDI8_PHASE_ALL) != 0 || !dims_supported(dims, true)) return 0;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) != 0 || !dims_supported(dims, true)) return 0;
   return layout(make_dims(dims)).total;
 }
 
@@ -98,8 +98,12 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
                                     uint32_t flags, void* workspace, size_t workspace_bytes,
                                     void* stream) {
   if (!dims || !a) return SSDI8_ERR_NULL;
-  if ((flags & ~(uint32_t)SSDI8_PHASE_ALL) != 0) return SSDI8_ERR_UNSUPPORTED;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) != 0) return SSDI8_ERR_UNSUPPORTED;
+  const bool i8s = (flags & SSDI8_FLAG_INT8_STATE) != 0;
   const uint32_t ph = (flags & SSDI8_PHASE_ALL) ? (flags & SSDI8_PHASE_ALL) : (uint32_t)SSDI8_PHASE_ALL;
+  // the INT8 state lives inside the fused ChunkState + StatePassing kernel only
+  if (i8s && ((ph & SSDI8_PHASE_CHUNK_STATE) != 0) != ((ph & SSDI8_PHASE_STATE_PASSING) != 0))
+    return SSDI8_ERR_UNSUPPORTED;
   if (!dims_supported(dims, true)) return SSDI8_ERR_SHAPE;
   if (!a->xq || !a->Bq || !a->Cq || !a->s_x || !a->s_B || !a->s_C || !a->dt || !a->A || !a->s_xs ||
       !a->s_cb || !a->s_h || !a->y || !workspace)
@@ -134,7 +138,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
     // both modules: the fused chunk-sequential kernel (the fp32 chunk-local states stay on chip)
     if ((s = launch_chunk_state_passing(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->s_h, pack, gamma,
                                         a->init_state, hq, a->final_state, a->tap_loc, a->tap_prev,
-                                        a->tap_Xsq, a->tap_acc_st, a->status, st)) != SSDI8_OK)
+                                        a->tap_Xsq, a->tap_acc_st, a->status, i8s, st)) != SSDI8_OK)
       return s;
   } else {
     if ((ph & SSDI8_PHASE_CHUNK_STATE) &&
@@ -248,7 +252,8 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
                                            uint32_t flags, void* stream) {
   if (!dims || !args) return SSDI8_ERR_NULL;
   const size_t need = ssdi8_workspace_bytes(dims, flags);
-  if (need == 0) return (flags & ~(uint32_t)SSDI8_PHASE_ALL) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
+  if (need == 0)
+    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
   if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
   static void* ws_of_device[64];  // resolved address of g_static_ws, per device
   int dev = 0;

@@ -10,6 +10,11 @@
 // 32 channels p.  Operand tiles arrive by TMA, double-buffered across chunks; hq leaves through
 // a shared-memory tile and one TMA store per chunk.  Same arithmetic, operation for operation,
 // as the separate kernels (chunk_state.cu, state_passing.cu).
+// I8S = true selects the paper's own state format (Section 4.2, Eq. 4 and Eq. 7): the state is an
+// int8 code with the one per-(H,P) scale s_h, the chunk-local state goes INT32 -> INT8 in
+// registers, and the recurrence is integer with a fixed-point decay:
+//   locq = rne(fmul(float(acc_st), fdiv(fmul(s_xs, s_B), s_h)));  Gq = rne(fmul(Gamma_k, 128))
+//   Sq   = sat(locq + ((Gq * Sq + 64) >> 7));  hq[k] = Sq before the update;  final = fmul(float(Sq), s_h)
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -31,10 +36,11 @@ constexpr uint32_t OFF_B = 0;
 constexpr uint32_t OFF_X = 32768;
 constexpr uint32_t OFF_HQ = 2 * STAGE;            // [64 p][N] int8 staging of hq
 constexpr uint32_t OFF_LUT = OFF_HQ + 8192;       // 2 x [256] floats
-constexpr uint32_t OFF_COL = OFF_LUT + 2048;       // [64] s_xs s_B, [64] 1 / s_h
-constexpr uint32_t OFF_BAR = OFF_COL + 512;
+constexpr uint32_t OFF_COL = OFF_LUT + 2048;       // [64] loc scale, [64] 1 / s_h, [64] s_h
+constexpr uint32_t OFF_BAR = OFF_COL + 768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
 
+template <bool I8S>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
                     const __grid_constant__ CUtensorMap tm_hq, const FusedArgs a) {
@@ -83,10 +89,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   const bool ok = (N == 128) || (lane < 16);
   const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
   const i64 bh = (i64)b * d.H + h;
-  float S[32];
-#pragma unroll
-  for (int pp = 0; pp < 32; ++pp)
-    S[pp] = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
+  float S[32];  // fp32 state, or (I8S) the bit pattern of the integer code
   // per-column factors of the re-quantisation (thread: 16-byte chunk c of every row it visits)
   const int c = tid & 3;
   float rx[16];
@@ -97,9 +100,22 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   }
   float* col_scale = reinterpret_cast<float*>(smem + OFF_COL);
   float* col_invh = col_scale + 64;
+  float* col_sh = col_invh + 64;
   if (tid < 64) {
-    col_scale[tid] = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]);
-    col_invh[tid] = __fdiv_rn(1.0f, a.s_h[h * P + tid]);
+    const float sxb = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]), sh = a.s_h[h * P + tid];
+    col_scale[tid] = I8S ? __fdiv_rn(sxb, sh) : sxb;
+    col_invh[tid] = __fdiv_rn(1.0f, sh);
+    col_sh[tid] = sh;
+  }
+#pragma unroll
+  for (int pp = 0; pp < 32; ++pp) {
+    const float v = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
+    if (I8S) {
+      const float ih = __fdiv_rn(1.0f, a.s_h[h * P + ch * 32 + pp]);
+      S[pp] = __int_as_float((int)(int8_t)(rne_clamp_bits(__fmul_rn(v, ih)) & 0xffu));
+    } else {
+      S[pp] = v;
+    }
   }
   const i64 unit0 = bh * d.c;
 
@@ -122,8 +138,12 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
 #pragma unroll
       for (int pp = 0; pp < 32; ++pp) {
         const int p = ch * 32 + pp;
-        sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
-        if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
+        if (I8S) {
+          sHQ[p * N + n] = (uint8_t)__float_as_int(S[pp]);
+        } else {
+          sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
+          if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
+        }
       }
     }
     mbar_wait(&bars[s], (k >> 1) & 1, a.status);
@@ -175,9 +195,16 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
         for (int pp = 0; pp < 32; ++pp) {
           const int p = ch * 32 + pp;
           const float loc = __fmul_rn(i22_to_f32(acc[pp]), col_scale[p]);
-          if (a.tap_loc) a.tap_loc[obase + (i64)pp * N] = loc;
           if (a.tap_acc) a.tap_acc[obase + (i64)pp * N] = acc[pp];
-          S[pp] = __fmaf_rn(gam, S[pp], loc);
+          if (I8S) {
+            const int locq = (int)(int8_t)(rne_clamp_bits(loc) & 0xffu);
+            const int Gq = __float2int_rn(__fmul_rn(gam, 128.0f));
+            const int Sn = locq + ((Gq * __float_as_int(S[pp]) + 64) >> 7);
+            S[pp] = __int_as_float(max(-127, min(127, Sn)));
+          } else {
+            if (a.tap_loc) a.tap_loc[obase + (i64)pp * N] = loc;
+            S[pp] = __fmaf_rn(gam, S[pp], loc);
+          }
         }
       }
     }
@@ -185,7 +212,9 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   }
   if (a.final_state && ok) {
 #pragma unroll
-    for (int pp = 0; pp < 32; ++pp) a.final_state[(bh * P + ch * 32 + pp) * N + n] = S[pp];
+    for (int pp = 0; pp < 32; ++pp)
+      a.final_state[(bh * P + ch * 32 + pp) * N + n] =
+          I8S ? __fmul_rn((float)__float_as_int(S[pp]), col_sh[ch * 32 + pp]) : S[pp];
   }
   if (tid == 0) tma_store_wait_read();
   __syncthreads();
@@ -202,7 +231,8 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
                                           const float* s_h, const float* pack, const float* gamma,
                                           const float* init, int8_t* hq, float* final_state,
                                           float* tap_loc, float* tap_prev, int8_t* tap_Xsq,
-                                          int32_t* tap_acc, int32_t* status, cudaStream_t st) {
+                                          int32_t* tap_acc, int32_t* status, bool int8_state,
+                                          cudaStream_t st) {
   const int TQ = d.Q < 128 ? d.Q : 128;
   const uint64_t T = (uint64_t)d.b * d.L;
   CUtensorMap tm_B, tm_x, tm_hq;
@@ -227,9 +257,14 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
   FusedArgs a = {s_x, s_xs, s_B, s_h, pack, gamma, init, final_state, tap_loc, tap_prev, tap_Xsq, tap_acc,
                  status, d};
   const size_t smem = SMEM_BYTES + 1024;
-  SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.H, d.b);
-  chunk_state_pass_tc<<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
+  if (int8_state) {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    chunk_state_pass_tc<true><<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
+  } else {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    chunk_state_pass_tc<false><<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
+  }
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

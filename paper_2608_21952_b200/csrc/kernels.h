@@ -36,7 +36,8 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
                                           const float* s_h, const float* pack, const float* gamma,
                                           const float* init, int8_t* hq, float* final_state,
                                           float* tap_loc, float* tap_prev, int8_t* tap_Xsq,
-                                          int32_t* tap_acc, int32_t* status, cudaStream_t st);
+                                          int32_t* tap_acc, int32_t* status, bool int8_state,
+                                          cudaStream_t st);
 
 // absmax_h: per-channel running max (binary32 bits) of |S| over init, prev and final
 ssdi8_status_t launch_state_passing(const Dims& d, const float* loc, const float* gamma,

@@ -26,7 +26,7 @@ def tap_shapes(cfg):
     }
 
 
-def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use"):
+def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use", flags=0):
     """q: dict with xq,Bq,Cq,s_x,s_B,s_C,dt,A,D,s_xs,s_cb,s_h,init (numpy).  Returns y, final, taps."""
     dims = bd.dims_of(cfg)
     t = {k: dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "s_xs", "s_cb", "s_h")}
@@ -43,7 +43,7 @@ def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use"):
         tp["tap_" + name] = torch.zeros(shp, dtype=_NP2T[dt_], device="cuda")
     ws = bd.alloc_workspace(dims)
     args = bd.make_fwd_args(y=y, final_state=fin, status=status, **t, **tp)
-    bd.ssdi8_chunk_scan_fwd(dims, args, ws)
+    bd.ssdi8_chunk_scan_fwd(dims, args, ws, flags=flags)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     return y.cpu().numpy(), fin.cpu().numpy(), {k[4:]: v.cpu().numpy() for k, v in tp.items()}

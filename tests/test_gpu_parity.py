@@ -167,6 +167,34 @@ def test_fwd_full_size_sampled(name, npairs):
         assert np.abs(y[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
 
 
+# --------------------------------------------------------------------------- persistent INT8 states (Eq. 4, 7)
+@pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[2]], ids=lambda c: c.name)
+def test_fwd_int8_state_mode_bit_exact(cfg):
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    names = ("cs", "Xsq", "acc_st", "hq", "acc_off", "rowmax", "Mq", "acc_diag")
+    y_ref, fin_ref, ref = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                        q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], init, taps=names,
+                                        flags=orc.FLAG_INT8_STATE)
+    y, fin, got = gh.gpu_fwd(cfg, q, taps=names, flags=bd.FLAG_INT8_STATE)
+    for name in names:
+        assert np.array_equal(got[name], ref[name]), name
+    assert np.array_equal(fin, fin_ref)
+    assert np.abs(y - y_ref).max() <= Y_TOL * rms(y_ref)
+
+
+def test_int8_state_flag_needs_the_fused_state_kernel():
+    from paper_2608_21952_b200 import binding as bd
+    a = bd.FwdArgs()
+    d = bd.dims_of(SMALL[0])
+    import ctypes as C
+    rc = bd._lib.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), bd.FLAG_INT8_STATE | bd.PHASE_CHUNK_STATE, None, 0, None)
+    assert rc == bd.ERR_UNSUPPORTED
+
+
 # --------------------------------------------------------------------------- quantiser
 @pytest.mark.parametrize("R,Ch,I", [(512, 256, 1), (37, 8, 1), (1000, 5120, 1), (512, 1, 64),
                                     (333, 8, 128), (4, 4, 4), (1, 4, 1)])
