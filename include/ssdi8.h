@@ -206,6 +206,19 @@ ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t*
                                float* s_xs, float* s_cb, float* s_h, void* workspace,
                                size_t workspace_bytes, void* stream);
 
+/* Estimation of the mean-correction vector (Eq. 8): the least-squares optimal per-channel
+ * correction of a quantised output is the channel-wise mean of its error, damped by eta (0.15 in
+ * the paper's setup):  corr[ch] = eta * mean over r of (y_ref[r][ch] - y_q[r][ch]).
+ * y_ref, y_q: [R][Ch] fp32 (for the SSD output R = B*L, Ch = H*P), 16-byte aligned, Ch % 4 == 0.
+ * corr: [Ch].  Sums are carried in fp64 in a fixed order (deterministic).  workspace: at least
+ * ssdi8_mean_correction_workspace_bytes(Ch) bytes, 16-byte aligned.  The result can be passed as
+ * `corr` to ssdi8_chunk_scan_fwd / ssdi8_ssd_step.  (The multi-layer sequential update of
+ * Algorithm 1 needs a whole model and is outside this library.) */
+size_t ssdi8_mean_correction_workspace_bytes(int64_t Ch);
+ssdi8_status_t ssdi8_mean_correction(const float* y_ref, const float* y_q, int64_t R, int64_t Ch,
+                                     float eta, float* corr, void* workspace, size_t workspace_bytes,
+                                     void* stream);
+
 /* StatePassing alone (Eq. 5-6; Algorithm 2 module 3) on fp32 states.
  *   S_k = fmaf(gamma[b,h,k], S_{k-1}, loc[b,k,h,p,n]),  S_{-1} = init_state or 0
  *   prev[b,k] = S_{k-1} (may be NULL; may alias loc), final_state = S_{c-1} (may be NULL),

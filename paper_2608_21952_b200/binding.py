@@ -30,7 +30,8 @@ PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1
 
 EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
            "ssdi8_chunk_scan_fwd", "ssdi8_chunk_scan_fwd_static", "ssdi8_calibrate",
-           "ssdi8_state_passing", "ssdi8_ssd_step")
+           "ssdi8_state_passing", "ssdi8_ssd_step", "ssdi8_mean_correction",
+           "ssdi8_mean_correction_workspace_bytes")
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 
@@ -64,6 +65,11 @@ _lib.ssdi8_chunk_scan_fwd_static.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs)
 _lib.ssdi8_calibrate.restype = C.c_int32
 _lib.ssdi8_calibrate.argtypes = [C.POINTER(Dims), C.POINTER(FwdArgs), C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.ssdi8_mean_correction_workspace_bytes.restype = C.c_size_t
+_lib.ssdi8_mean_correction_workspace_bytes.argtypes = [C.c_int64]
+_lib.ssdi8_mean_correction.restype = C.c_int32
+_lib.ssdi8_mean_correction.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
+                                       C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.ssdi8_state_passing.restype = C.c_int32
 _lib.ssdi8_state_passing.argtypes = [C.POINTER(Dims)] + [C.c_void_p] * 8
 _lib.ssdi8_ssd_step.restype = C.c_int32
@@ -140,6 +146,16 @@ def ssdi8_calibrate(dims: Dims, args: FwdArgs, s_xs, s_cb, s_h, workspace, strea
     _check(_lib.ssdi8_calibrate(C.byref(dims), C.byref(args), _ptr(s_xs), _ptr(s_cb), _ptr(s_h),
                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
                                 _stream(stream)), "ssdi8_calibrate")
+
+
+def ssdi8_mean_correction_workspace_bytes(Ch: int) -> int:
+    return int(_lib.ssdi8_mean_correction_workspace_bytes(Ch))
+
+
+def ssdi8_mean_correction(y_ref, y_q, R: int, Ch: int, eta: float, corr, workspace, stream=None) -> None:
+    _check(_lib.ssdi8_mean_correction(_ptr(y_ref), _ptr(y_q), R, Ch, eta, _ptr(corr), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)),
+           "ssdi8_mean_correction")
 
 
 def ssdi8_state_passing(dims: Dims, loc, gamma, init_state, prev, final_state, hq, s_h,

@@ -234,6 +234,22 @@ ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const 
                          static_cast<cudaStream_t>(stream));
 }
 
+size_t ssdi8_mean_correction_workspace_bytes(int64_t Ch) {
+  return Ch > 0 ? sizeof(double) * (size_t)kMeanCorrMaxSlabs * (size_t)Ch : 0;
+}
+
+ssdi8_status_t ssdi8_mean_correction(const float* y_ref, const float* y_q, int64_t R, int64_t Ch, float eta,
+                                     float* corr, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!y_ref || !y_q || !corr || !workspace) return SSDI8_ERR_NULL;
+  if (R <= 0 || Ch <= 0 || Ch % 4 != 0) return SSDI8_ERR_SHAPE;
+  if (!aligned16(y_ref) || !aligned16(y_q) || !aligned16(workspace)) return SSDI8_ERR_ALIGN;
+  if (workspace_bytes < ssdi8_mean_correction_workspace_bytes(Ch)) return SSDI8_ERR_WORKSPACE;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_mean_correction(y_ref, y_q, R, Ch, eta, corr, static_cast<double*>(workspace),
+                                static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------
 // Forward pass with library-owned scratch (no allocation by anyone).
 //

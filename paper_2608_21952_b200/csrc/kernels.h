@@ -61,6 +61,12 @@ ssdi8_status_t launch_ssd_step(const Dims& d, const int8_t* xq, const float* s_x
                                const float* s_C, const float* dt, const float* A, const float* D,
                                const float* corr, float* state, float* y, cudaStream_t st);
 
+// Eq. 8: corr[ch] = eta * mean_r (y[r][ch] - yq[r][ch]); partial holds kMeanCorrMaxSlabs * Ch doubles
+constexpr int kMeanCorrMaxSlabs = 256;
+int mean_correction_slabs(i64 R);
+ssdi8_status_t launch_mean_correction(const float* y, const float* yq, i64 R, i64 Ch, float eta, float* corr,
+                                      double* partial, cudaStream_t st);
+
 // scale[k] = bits[k] == 0 ? 1 : fdiv(as_float(bits[k]) [* mul], 127)   (in place)
 ssdi8_status_t launch_finalize_scales(float* scale_bits, i64 n, const float* mul_a,
                                       const float* mul_b, int bits_are_int, cudaStream_t st);
