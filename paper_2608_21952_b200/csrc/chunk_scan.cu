@@ -74,16 +74,6 @@ __device__ __forceinline__ uint32_t pack4_rne(float2 a, float2 b) {
                      __byte_perm(__float_as_uint(rb.x), __float_as_uint(rb.y), 0x0040u), 0x5410u);
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
-
 struct Tile {
   int b, k, h, g, it, KJ;
   i64 tok0, unit;  // unit = (b*H + h)*c + k

@@ -30,15 +30,23 @@ struct FusedArgs {
   Dims d;
 };
 
-constexpr int kThreads = 256;
+constexpr int kStateThreads = 256;   // warps 0-7: running state, hq, MMA issue, TMA
+constexpr int kQuantThreads = 128;   // warps 8-11: Q(X_scaled) of the next chunk, one chunk ahead
+constexpr int kThreads = kStateThreads + kQuantThreads;
 constexpr uint32_t STAGE = 49152;      // per stage: Bq rows [Q][N] (32 KB) + xq rows [Q][64] (16 KB)
 constexpr uint32_t OFF_B = 0;
 constexpr uint32_t OFF_X = 32768;
 constexpr uint32_t OFF_HQ = 2 * STAGE;            // [64 p][N] int8 staging of hq
 constexpr uint32_t OFF_LUT = OFF_HQ + 8192;       // 2 x [256] floats
-constexpr uint32_t OFF_COL = OFF_LUT + 2048;       // [64] loc scale, [64] 1 / s_h, [64] s_h
+constexpr uint32_t OFF_COL = OFF_LUT + 2048;      // [64] loc scale, [64] 1 / s_h, [64] s_h
 constexpr uint32_t OFF_BAR = OFF_COL + 768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
+
+enum { B_FULL = 0, B_RQ = 2, B_MMA = 4, B_COUNT = 5 };
+
+__device__ __forceinline__ void named_bar(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 
 template <bool I8S>
 __global__ void __launch_bounds__(kThreads, 2)
@@ -52,20 +60,33 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   const int h = blockIdx.x, b = blockIdx.y;
   const int g = h / (d.H / d.G);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);  // [0,1] operands landed, [2] MMA done
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   uint8_t* sHQ = smem + OFF_HQ;
+  float* col_scale = reinterpret_cast<float*>(smem + OFF_COL);
+  float* col_invh = col_scale + 64;
+  float* col_sh = col_invh + 64;
+  const i64 bh = (i64)b * d.H + h;
+  const i64 unit0 = bh * d.c;
 
   if (tid == 0) {
-    mbar_init(&bars[0], 1);
-    mbar_init(&bars[1], 1);
-    mbar_init(&bars[2], 1);
+    mbar_init(&bars[B_FULL], 1);
+    mbar_init(&bars[B_FULL + 1], 1);
+    mbar_init(&bars[B_RQ], kQuantThreads / 32);
+    mbar_init(&bars[B_RQ + 1], kQuantThreads / 32);
+    mbar_init(&bars[B_MMA], 1);
     fence_mbar_init();
     tma_prefetch_desc(&tm_B);
     tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_hq);
   }
   if (warp == 1) tmem_alloc(tmem_slot, 64);
+  if (tid < 64) {
+    const float sxb = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]), sh = a.s_h[h * P + tid];
+    col_scale[tid] = I8S ? __fdiv_rn(sxb, sh) : sxb;
+    col_invh[tid] = __fdiv_rn(1.0f, sh);
+    col_sh[tid] = sh;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -75,148 +96,160 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     const int s = k & 1;
     uint8_t* st = smem + s * STAGE;
     const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-    mbar_expect_tx(&bars[s], (uint32_t)(Q * 64 + Q * N));
+    mbar_expect_tx(&bars[B_FULL + s], (uint32_t)(Q * 64 + Q * N));
     for (int i0 = 0; i0 < Q; i0 += TQ) {
-      tma_load_3d(st + OFF_X + i0 * 64, &tm_x, &bars[s], 0, h, (int)(tok0 + i0));
-      tma_load_3d(st + OFF_B + i0 * N, &tm_B, &bars[s], 0, g, (int)(tok0 + i0));
+      tma_load_3d(st + OFF_X + i0 * 64, &tm_x, &bars[B_FULL + s], 0, h, (int)(tok0 + i0));
+      tma_load_3d(st + OFF_B + i0 * N, &tm_B, &bars[B_FULL + s], 0, g, (int)(tok0 + i0));
     }
   };
-  if (tid == 0) issue_loads(0);
 
-  // epilogue geometry: M = 128: accumulator row n on TMEM lane n; M = 64: row n on lane
-  // (n % 16) + 32 (n / 16), i.e. the first 16 lanes of each warp's quarter
-  const int q = warp & 3, ch = warp >> 2;
-  const bool ok = (N == 128) || (lane < 16);
-  const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
-  const i64 bh = (i64)b * d.H + h;
-  float S[32];  // fp32 state, or (I8S) the bit pattern of the integer code
-  // per-column factors of the re-quantisation (thread: 16-byte chunk c of every row it visits)
-  const int c = tid & 3;
-  float rx[16];
+  if (tid >= kStateThreads) {
+    // ------------------------------------------------------------ Q(X_scaled), one chunk ahead of the state warps
+    const int qt = tid - kStateThreads;
+    const int c = qt & 3;  // 16-byte chunk (16 channels) of every row this thread visits
+    float rx[16];
 #pragma unroll
-  for (int e = 0; e < 16; ++e) {
-    const int hp = h * P + c * 16 + e;
-    rx[e] = __fdiv_rn(a.s_x[hp], a.s_xs[hp]);
-  }
-  float* col_scale = reinterpret_cast<float*>(smem + OFF_COL);
-  float* col_invh = col_scale + 64;
-  float* col_sh = col_invh + 64;
-  if (tid < 64) {
-    const float sxb = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]), sh = a.s_h[h * P + tid];
-    col_scale[tid] = I8S ? __fdiv_rn(sxb, sh) : sxb;
-    col_invh[tid] = __fdiv_rn(1.0f, sh);
-    col_sh[tid] = sh;
-  }
-#pragma unroll
-  for (int pp = 0; pp < 32; ++pp) {
-    const float v = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
-    if (I8S) {
-      const float ih = __fdiv_rn(1.0f, a.s_h[h * P + ch * 32 + pp]);
-      S[pp] = __int_as_float((int)(int8_t)(rne_clamp_bits(__fmul_rn(v, ih)) & 0xffu));
-    } else {
-      S[pp] = v;
+    for (int e = 0; e < 16; ++e) {
+      const int hp = h * P + c * 16 + e;
+      rx[e] = __fdiv_rn(a.s_x[hp], a.s_xs[hp]);
     }
-  }
-  const i64 unit0 = bh * d.c;
-
 #pragma unroll 1
-  for (int k = 0; k < d.c; ++k) {
-    const int s = k & 1;
-    uint8_t* sB = smem + s * STAGE + OFF_B;
-    uint8_t* sX = smem + s * STAGE + OFF_X;
-    float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
-    const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-    if (tid < Q) lut[tid] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + tid];
-    const float gam = a.gamma[unit0 + k];
-    if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
-    __syncthreads();  // lut visible; stage (k+1)&1 and the hq staging tile are no longer read by anyone
-    if (tid == 0 && k + 1 < d.c) issue_loads(k + 1);
-
-    // ---- hq[k] = codes of the state entering this chunk (and the prev tap)
-    if (ok) {
-      const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+    for (int k = 0; k < d.c; ++k) {
+      const int s = k & 1;
+      uint8_t* sX = smem + s * STAGE + OFF_X;
+      float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
+      const i64 tok0 = (i64)b * d.L + (i64)k * Q;
+      // lut[s] was last read for chunk k-2, which every thread of this group has left
+      for (int i = qt; i < Q; i += kQuantThreads) lut[i] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + i];
+      named_bar(2, kQuantThreads);
+      mbar_wait(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+#pragma unroll 1
+      for (int i = qt >> 2; i < Q; i += kQuantThreads / 4) {
+        uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
+        const uint4 w4 = *ptr;
+        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+        const float l = lut[i];
+        uint32_t o[4];
 #pragma unroll
-      for (int pp = 0; pp < 32; ++pp) {
-        const int p = ch * 32 + pp;
-        if (I8S) {
-          sHQ[p * N + n] = (uint8_t)__float_as_int(S[pp]);
-        } else {
-          sHQ[p * N + n] = (uint8_t)rne_clamp_bits(__fmul_rn(S[pp], col_invh[p]));
-          if (a.tap_prev) a.tap_prev[obase + (i64)pp * N] = S[pp];
+        for (int w = 0; w < 4; ++w) {
+          uint32_t q4[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            q4[e] = rne_clamp_bits(__fmul_rn(__fmul_rn(s8_to_f32(ww[w], e), rx[w * 4 + e]), l));
+          o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
         }
+        const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+        *ptr = v;
+        if (a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
       }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars[B_RQ + s]);
     }
-    mbar_wait(&bars[s], (k >> 1) & 1, a.status);
-
-    // ---- X_scaled, re-quantised in place (thread: chunk c of rows tid/4, tid/4 + 64, ...)
-    for (int i = tid >> 2; i < Q; i += kThreads / 4) {
-      uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
-      const uint4 w4 = *ptr;
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float l = lut[i];
-      uint32_t o[4];
+  } else {
+    // ------------------------------------------------------------ state warps
+    // M = 128: accumulator row n on TMEM lane n; M = 64: row n on lane (n % 16) + 32 (n / 16),
+    // i.e. the first 16 lanes of each warp's quarter
+    const int q = warp & 3, ch = warp >> 2;
+    const bool ok = (N == 128) || (lane < 16);
+    const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
+    float S[32];  // fp32 state, or (I8S) the bit pattern of the integer code
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        uint32_t q4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          q4[e] = rne_clamp_bits(__fmul_rn(__fmul_rn(s8_to_f32(ww[w], e), rx[w * 4 + e]), l));
-        o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
-      }
-      const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
-      *ptr = v;
-      if (a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
+    for (int pp = 0; pp < 32; ++pp) {
+      const float v = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
+      if (I8S)
+        S[pp] = __int_as_float((int)(int8_t)(rne_clamp_bits(__fmul_rn(v, col_invh[ch * 32 + pp])) & 0xffu));
+      else
+        S[pp] = v;
     }
-    fence_async_smem();
-    __syncthreads();
-
-    // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]; hq[k] leaves by TMA while the MMA runs
     if (tid == 0) {
-      tc_fence_after();
-      const uint32_t idesc = idesc_s8(N, 64, 1, 1);
-      for (int st = 0; st < Q / 32; ++st)
-        mma_s8_ss(tmem, tile_desc(smem_u32(sB) + 32 * st * N, (uint32_t)N),
-                  tile_desc(smem_u32(sX) + 32 * st * 64, 64), idesc, st > 0);
-      mma_commit(&bars[2]);
-      tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
-      tma_store_commit();
+      issue_loads(0);
+      if (d.c > 1) issue_loads(1);
     }
-
-    // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc)
-    mbar_wait(&bars[2], k & 1, a.status);
-    tc_fence_after();
-    {
-      int acc[32];
-      tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), acc);
-      tmem_ld_wait();
+#pragma unroll 1
+    for (int k = 0; k < d.c; ++k) {
+      const int s = k & 1;
+      const float gam = a.gamma[unit0 + k];
+      if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
+      named_bar(1, kStateThreads);  // also: every state thread has read the accumulator of chunk k-1
+      // ---- hq[k] = codes of the state entering this chunk (and the prev tap)
       if (ok) {
         const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+        // batches of 8: all loads of a batch before its byte stores (a byte store may alias anything,
+        // so interleaving them would serialise the loop on shared-memory latency)
 #pragma unroll
-        for (int pp = 0; pp < 32; ++pp) {
-          const int p = ch * 32 + pp;
-          const float loc = __fmul_rn(i22_to_f32(acc[pp]), col_scale[p]);
-          if (a.tap_acc) a.tap_acc[obase + (i64)pp * N] = acc[pp];
-          if (I8S) {
-            const int locq = (int)(int8_t)(rne_clamp_bits(loc) & 0xffu);
-            const int Gq = __float2int_rn(__fmul_rn(gam, 128.0f));
-            const int Sn = locq + ((Gq * __float_as_int(S[pp]) + 64) >> 7);
-            S[pp] = __int_as_float(max(-127, min(127, Sn)));
-          } else {
-            if (a.tap_loc) a.tap_loc[obase + (i64)pp * N] = loc;
-            S[pp] = __fmaf_rn(gam, S[pp], loc);
+        for (int p0 = 0; p0 < 32; p0 += 8) {
+          uint32_t code[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int pp = p0 + e;
+            code[e] = I8S ? (uint32_t)__float_as_int(S[pp])
+                          : rne_clamp_bits(__fmul_rn(S[pp], col_invh[ch * 32 + pp]));
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) sHQ[(ch * 32 + p0 + e) * N + n] = (uint8_t)code[e];
+        }
+        if (!I8S && a.tap_prev) {
+#pragma unroll
+          for (int pp = 0; pp < 32; ++pp) a.tap_prev[obase + (i64)pp * N] = S[pp];
+        }
+      }
+      fence_async_smem();
+      named_bar(1, kStateThreads);
+      // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]; hq[k] leaves by TMA while the MMA runs
+      if (tid == 0) {
+        mbar_wait(&bars[B_RQ + s], (k >> 1) & 1, a.status);
+        tc_fence_after();
+        const uint32_t sB = smem_u32(smem + s * STAGE + OFF_B), sX = smem_u32(smem + s * STAGE + OFF_X);
+        const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+#pragma unroll 1
+        for (int st = 0; st < Q / 32; ++st)
+          mma_s8_ss(tmem, tile_desc(sB + 32 * st * N, (uint32_t)N), tile_desc(sX + 32 * st * 64, 64), idesc, st > 0);
+        mma_commit(&bars[B_MMA]);
+        tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
+        tma_store_commit();
+      }
+      // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 16 channels at a time
+      mbar_wait(&bars[B_MMA], k & 1, a.status);
+      tc_fence_after();
+      if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        int acc[16];
+        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + hf * 16), acc);
+        tmem_ld_wait();
+        if (ok) {
+          const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32 + hf * 16) * N + n;
+          float cscale[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) cscale[e] = col_scale[ch * 32 + hf * 16 + e];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int pp = hf * 16 + e;
+            const float loc = __fmul_rn(i22_to_f32(acc[e]), cscale[e]);
+            if (a.tap_acc) a.tap_acc[obase + (i64)e * N] = acc[e];
+            if (I8S) {
+              const int locq = (int)(int8_t)(rne_clamp_bits(loc) & 0xffu);
+              const int Gq = __float2int_rn(__fmul_rn(gam, 128.0f));
+              const int Sn = locq + ((Gq * __float_as_int(S[pp]) + 64) >> 7);
+              S[pp] = __int_as_float(max(-127, min(127, Sn)));
+            } else {
+              if (a.tap_loc) a.tap_loc[obase + (i64)e * N] = loc;
+              S[pp] = __fmaf_rn(gam, S[pp], loc);
+            }
           }
         }
       }
+      tc_fence_before();  // ordered before the next chunk's MMA by the next named barrier
     }
-    tc_fence_before();  // the next chunk's MMA overwrites the accumulator after the next __syncthreads
-  }
-  if (a.final_state && ok) {
+    if (a.final_state && ok) {
 #pragma unroll
-    for (int pp = 0; pp < 32; ++pp)
-      a.final_state[(bh * P + ch * 32 + pp) * N + n] =
-          I8S ? __fmul_rn((float)__float_as_int(S[pp]), col_sh[ch * 32 + pp]) : S[pp];
+      for (int pp = 0; pp < 32; ++pp)
+        a.final_state[(bh * P + ch * 32 + pp) * N + n] =
+            I8S ? __fmul_rn((float)__float_as_int(S[pp]), col_sh[ch * 32 + pp]) : S[pp];
+    }
+    if (tid == 0) tma_store_wait_read();
   }
-  if (tid == 0) tma_store_wait_read();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
