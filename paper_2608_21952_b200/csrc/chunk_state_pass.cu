@@ -42,7 +42,7 @@ constexpr uint32_t OFF_COL = OFF_LUT + 2048;      // [64] loc scale, [64] 1 / s_
 constexpr uint32_t OFF_BAR = OFF_COL + 768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
 
-enum { B_FULL = 0, B_RQ = 2, B_MMA = 4, B_COUNT = 5 };
+enum { B_FULL = 0, B_RQ = 2, B_MMA = 4, B_ACC_FREE = 5, B_COUNT = 6 };
 
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -75,6 +75,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     mbar_init(&bars[B_RQ], kQuantThreads / 32);
     mbar_init(&bars[B_RQ + 1], kQuantThreads / 32);
     mbar_init(&bars[B_MMA], 1);
+    mbar_init(&bars[B_ACC_FREE], kStateThreads / 32);
     fence_mbar_init();
     tma_prefetch_desc(&tm_B);
     tma_prefetch_desc(&tm_x);
@@ -129,13 +130,21 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
         const uint4 w4 = *ptr;
         const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
         const float l = lut[i];
+        const float2 l2 = make_float2(l, l);
         uint32_t o[4];
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           uint32_t q4[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            q4[e] = rne_clamp_bits(__fmul_rn(__fmul_rn(s8_to_f32(ww[w], e), rx[w * 4 + e]), l));
+          for (int e = 0; e < 4; e += 2) {
+            const float2 xf = __fadd2_rn(
+                make_float2(__uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7650u + e)),
+                            __uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7651u + e))),
+                make_float2(-kMagicIn, -kMagicIn));
+            const float2 v2 = __fmul2_rn(__fmul2_rn(xf, make_float2(rx[w * 4 + e], rx[w * 4 + e + 1])), l2);
+            q4[e] = rne_clamp_bits(v2.x);
+            q4[e + 1] = rne_clamp_bits(v2.y);
+          }
           o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
         }
         const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
@@ -145,6 +154,20 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_RQ + s]);
+      // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p], issued as soon as the whole tile is re-quantised
+      // and the state warps have read the previous accumulator (overlaps their hq staging)
+      if (qt == 0) {
+        mbar_wait(&bars[B_RQ + s], (k >> 1) & 1, a.status);
+        mbar_wait(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);
+        tc_fence_after();
+        const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
+        const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+#pragma unroll 1
+        for (int st = 0; st < Q / 32; ++st)
+          mma_s8_ss(tmem, tile_desc(sBa + 32 * st * N, (uint32_t)N), tile_desc(sXa + 32 * st * 64, 64), idesc, st > 0);
+        mma_commit(&bars[B_MMA]);
+      }
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------ state warps
@@ -168,7 +191,6 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     }
 #pragma unroll 1
     for (int k = 0; k < d.c; ++k) {
-      const int s = k & 1;
       const float gam = a.gamma[unit0 + k];
       if (tid == 0 && k > 0) tma_store_wait_read();  // last chunk's hq store has read the staging tile
       named_bar(1, kStateThreads);  // also: every state thread has read the accumulator of chunk k-1
@@ -196,16 +218,8 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       }
       fence_async_smem();
       named_bar(1, kStateThreads);
-      // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p]; hq[k] leaves by TMA while the MMA runs
+      // ---- hq[k] leaves by TMA
       if (tid == 0) {
-        mbar_wait(&bars[B_RQ + s], (k >> 1) & 1, a.status);
-        tc_fence_after();
-        const uint32_t sB = smem_u32(smem + s * STAGE + OFF_B), sX = smem_u32(smem + s * STAGE + OFF_X);
-        const uint32_t idesc = idesc_s8(N, 64, 1, 1);
-#pragma unroll 1
-        for (int st = 0; st < Q / 32; ++st)
-          mma_s8_ss(tmem, tile_desc(sB + 32 * st * N, (uint32_t)N), tile_desc(sX + 32 * st * 64, 64), idesc, st > 0);
-        mma_commit(&bars[B_MMA]);
         tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
         tma_store_commit();
       }
@@ -240,7 +254,9 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
           }
         }
       }
-      tc_fence_before();  // ordered before the next chunk's MMA by the next named barrier
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars[B_ACC_FREE]);  // this warp has read the accumulator of chunk k
     }
     if (a.final_state && ok) {
 #pragma unroll
