@@ -93,6 +93,17 @@ size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags);
 ssdi8_status_t ssdi8_quantize_act(const float* in, int64_t R, int64_t Ch, int64_t I,
                                   float* scale, int32_t mode, int8_t* out, void* stream);
 
+/* Entry quantiser: the convolution output of a Mamba-2 block is one tensor xBC [T][D + 2 G N]
+ * (x, B, C along the last axis; T = B*L, D = H*P).  One pass writes xq [T][D], Bq [T][G*N] and
+ * Cq [T][G*N] with static step sizes (Eq. 1, q = rne(fdiv(float(v), alpha)) saturated): x per
+ * channel (s_x[D]), B and C per group (s_B[G], s_C[G]), i.e. B and C are quantised once on the
+ * group axis at layer entry and the int8 tensors are reused by every module (Section 4.2,
+ * "Quantization of B,C").  dtype of xBC: 0 = fp32, 1 = fp16, 2 = bf16 (the conversion to binary32
+ * is exact).  D % 4 == 0, N % 4 == 0; xBC, s_x and the outputs 16-byte aligned. */
+ssdi8_status_t ssdi8_quantize_entry(const void* xBC, int32_t dtype, int64_t T, int32_t D, int32_t G,
+                                    int32_t N, const float* s_x, const float* s_B, const float* s_C,
+                                    int8_t* xq, int8_t* Bq, int8_t* Cq, void* stream);
+
 typedef struct {
   /* layer inputs */
   const int8_t* xq;        /* [B,L,H,P]  per-channel codes of X                         */

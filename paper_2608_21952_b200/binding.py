@@ -31,7 +31,7 @@ PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1
 EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
            "ssdi8_chunk_scan_fwd", "ssdi8_chunk_scan_fwd_static", "ssdi8_calibrate",
            "ssdi8_state_passing", "ssdi8_ssd_step", "ssdi8_mean_correction",
-           "ssdi8_mean_correction_workspace_bytes")
+           "ssdi8_mean_correction_workspace_bytes", "ssdi8_quantize_entry")
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 
@@ -70,6 +70,9 @@ _lib.ssdi8_mean_correction_workspace_bytes.argtypes = [C.c_int64]
 _lib.ssdi8_mean_correction.restype = C.c_int32
 _lib.ssdi8_mean_correction.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.ssdi8_quantize_entry.restype = C.c_int32
+_lib.ssdi8_quantize_entry.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int32, C.c_int32, C.c_int32] + \
+    [C.c_void_p] * 7
 _lib.ssdi8_state_passing.restype = C.c_int32
 _lib.ssdi8_state_passing.argtypes = [C.POINTER(Dims)] + [C.c_void_p] * 8
 _lib.ssdi8_ssd_step.restype = C.c_int32
@@ -146,6 +149,15 @@ def ssdi8_calibrate(dims: Dims, args: FwdArgs, s_xs, s_cb, s_h, workspace, strea
     _check(_lib.ssdi8_calibrate(C.byref(dims), C.byref(args), _ptr(s_xs), _ptr(s_cb), _ptr(s_h),
                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
                                 _stream(stream)), "ssdi8_calibrate")
+
+
+_ENTRY_DTYPES = {torch.float32: 0, torch.float16: 1, torch.bfloat16: 2}
+
+
+def ssdi8_quantize_entry(xBC, T: int, D: int, G: int, N: int, s_x, s_B, s_C, xq, Bq, Cq, stream=None) -> None:
+    _check(_lib.ssdi8_quantize_entry(_ptr(xBC), _ENTRY_DTYPES[xBC.dtype], T, D, G, N, _ptr(s_x), _ptr(s_B),
+                                     _ptr(s_C), _ptr(xq), _ptr(Bq), _ptr(Cq), _stream(stream)),
+           "ssdi8_quantize_entry")
 
 
 def ssdi8_mean_correction_workspace_bytes(Ch: int) -> int:

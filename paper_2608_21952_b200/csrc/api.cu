@@ -234,6 +234,20 @@ ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const 
                          static_cast<cudaStream_t>(stream));
 }
 
+ssdi8_status_t ssdi8_quantize_entry(const void* xBC, int32_t dtype, int64_t T, int32_t D, int32_t G, int32_t N,
+                                    const float* s_x, const float* s_B, const float* s_C, int8_t* xq,
+                                    int8_t* Bq, int8_t* Cq, void* stream) {
+  if (!xBC || !s_x || !s_B || !s_C || !xq || !Bq || !Cq) return SSDI8_ERR_NULL;
+  if (dtype < 0 || dtype > 2) return SSDI8_ERR_UNSUPPORTED;
+  if (T < 0 || D <= 0 || G <= 0 || N <= 0 || D % 4 != 0 || N % 4 != 0) return SSDI8_ERR_SHAPE;
+  const void* ptrs[] = {xBC, s_x, xq, Bq, Cq};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return SSDI8_ERR_ALIGN;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_quantize_entry(xBC, dtype, T, D, G, N, s_x, s_B, s_C, xq, Bq, Cq, static_cast<cudaStream_t>(stream));
+}
+
 size_t ssdi8_mean_correction_workspace_bytes(int64_t Ch) {
   return Ch > 0 ? sizeof(double) * (size_t)kMeanCorrMaxSlabs * (size_t)Ch : 0;
 }

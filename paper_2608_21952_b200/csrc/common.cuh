@@ -62,6 +62,35 @@ __device__ __forceinline__ uint32_t pack4_bits(uint32_t a, uint32_t b, uint32_t 
   return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
 }
 
+// Eq. 1 codes without a division per element.  With rcp = frcp_rn(alpha), t = fmul(v, rcp) and
+// d = fdiv_rn(v, alpha) differ by at most 1.5 * 2^-23 |v / alpha| < 2.3e-5 wherever the code is not
+// saturated, so rne(t) = rne(d) unless t lies that close to a rounding boundary k + 1/2 (ties
+// included).  Those elements (about one in 10^4) take the division, and so does every element of a
+// step size whose reciprocal may not be a normal number, so the code always equals
+// rne(fdiv_rn(v, alpha)) saturated.  quant_code_bits returns bits whose low byte is the code.
+struct QuantStep {
+  float alpha, rcp, thr;
+};
+__device__ __forceinline__ QuantStep quant_step(float alpha) {
+  QuantStep s;
+  s.alpha = alpha;
+  s.rcp = __frcp_rn(alpha);
+  s.thr = (alpha >= 1e-30f && alpha <= 1e30f) ? 0.49994f : -1.0f;
+  return s;
+}
+__device__ __forceinline__ uint32_t quant_code_bits(float v, const QuantStep& s) {
+  const float tc = fminf(fmaxf(__fmul_rn(v, s.rcp), -127.0f), 127.0f);
+  const float m = __fadd_rn(tc, kMagicOut);
+  const float e = __fsub_rn(tc, __fsub_rn(m, kMagicOut));
+  if (fabsf(e) > s.thr) return rne_clamp_bits(__fdiv_rn(v, s.alpha));
+  return __float_as_uint(m);
+}
+__device__ __forceinline__ uint32_t quant_code4(const float4& v, const QuantStep& a, const QuantStep& b,
+                                                const QuantStep& c, const QuantStep& d) {
+  return pack4_bits(quant_code_bits(v.x, a), quant_code_bits(v.y, b), quant_code_bits(v.z, c),
+                    quant_code_bits(v.w, d));
+}
+
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
   return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
          ((uint32_t)(d & 0xff) << 24);

@@ -12,6 +12,11 @@ ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* sca
 constexpr int kPackRows = 6;
 enum { PACK_CS = 0, PACK_DT = 1, PACK_WOFF = 2, PACK_ATOK = 3, PACK_WMAX = 4, PACK_LUT = 5 };
 
+// xBC [T][D + 2 G N] (dtype 0 fp32, 1 fp16, 2 bf16) -> xq [T][D], Bq, Cq [T][G N], static step sizes
+ssdi8_status_t launch_quantize_entry(const void* xBC, int dtype, i64 T_, int D, int G, int N, const float* s_x,
+                                     const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq, int8_t* Cq,
+                                     cudaStream_t st);
+
 // pack [b,H,c,6,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
                              float* gamma, float* tap_cs, cudaStream_t st);

@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(128) quant_ch_fastest(const float4* __restrict
   const int q = blockIdx.x * 128 + threadIdx.x;
   if (q >= ch4) return;
   const float4 s = __ldg(scale + q);
+  const QuantStep sx = quant_step(s.x), sy = quant_step(s.y), sz = quant_step(s.z), sw = quant_step(s.w);
   const i64 r0 = (i64)blockIdx.y * rows_per_block;
   const i64 r1 = r0 + rows_per_block < R ? r0 + rows_per_block : R;
   i64 r = r0;
@@ -30,14 +31,11 @@ __global__ void __launch_bounds__(128) quant_ch_fastest(const float4* __restrict
     for (int u = 0; u < QROWS; ++u) v[u] = __ldcs(in + (r + u) * ch4 + q);
 #pragma unroll
     for (int u = 0; u < QROWS; ++u)
-      __stcs(out + (r + u) * ch4 + q,
-             pack4(rne_clamp(__fdiv_rn(v[u].x, s.x)), rne_clamp(__fdiv_rn(v[u].y, s.y)),
-                   rne_clamp(__fdiv_rn(v[u].z, s.z)), rne_clamp(__fdiv_rn(v[u].w, s.w))));
+      __stcs(out + (r + u) * ch4 + q, quant_code4(v[u], sx, sy, sz, sw));
   }
   for (; r < r1; ++r) {
     const float4 v = __ldcs(in + r * ch4 + q);
-    __stcs(out + r * ch4 + q, pack4(rne_clamp(__fdiv_rn(v.x, s.x)), rne_clamp(__fdiv_rn(v.y, s.y)),
-                                    rne_clamp(__fdiv_rn(v.z, s.z)), rne_clamp(__fdiv_rn(v.w, s.w))));
+    __stcs(out + r * ch4 + q, quant_code4(v, sx, sy, sz, sw));
   }
 }
 
@@ -52,9 +50,8 @@ __global__ void __launch_bounds__(QT) quant_inner(const float4* __restrict__ in,
     uint32_t e = base + u * QT;
     if (e < n4) {
       float4 v = __ldcs(in + e);
-      float s = __ldg(scale + (e / I4) % Ch);
-      out[e] = pack4(rne_clamp(__fdiv_rn(v.x, s)), rne_clamp(__fdiv_rn(v.y, s)),
-                     rne_clamp(__fdiv_rn(v.z, s)), rne_clamp(__fdiv_rn(v.w, s)));
+      const QuantStep s = quant_step(__ldg(scale + (e / I4) % Ch));
+      out[e] = quant_code4(v, s, s, s, s);
     }
   }
 }

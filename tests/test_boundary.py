@@ -103,3 +103,26 @@ def test_binding_raises_on_error_code():
     with pytest.raises(bd.SSDi8Error) as e:
         bd._check(bd.ERR_SHAPE, "x")
     assert e.value.code == bd.ERR_SHAPE and "dimensions" in str(e.value)
+
+
+def test_reciprocal_fast_path_of_the_quantiser_is_exact():
+    """The quantiser kernels replace fdiv(v, alpha) by fmul(v, frcp(alpha)) for every element whose
+    product lies farther than 6e-5 from a rounding boundary k + 1/2 and divide for the rest.  Checked
+    here in numpy binary32 on values placed on and next to the boundaries: outside the guard band
+    both roundings give the same code, and the band catches every element where they differ."""
+    import numpy as np
+    rng = np.random.default_rng(5)
+    alpha = np.concatenate([rng.uniform(1e-3, 10, 2000), 10.0 ** rng.uniform(-29, 29, 2000)]).astype(np.float32)
+    k = rng.integers(-128, 128, (alpha.size, 512)).astype(np.float64) + 0.5
+    off = rng.choice([0.0, 1e-7, -1e-7, 1e-6, -1e-6, 1e-5, -1e-5, 5e-5, -5e-5, 1e-4, 0.3], k.shape)
+    v = ((k + off) * alpha[:, None].astype(np.float64)).astype(np.float32)
+    v[:, :64] = (rng.standard_normal((alpha.size, 64)) * 60).astype(np.float32) * alpha[:, None]
+    a = np.broadcast_to(alpha[:, None], v.shape)
+    d = np.clip(np.rint(v / a), -127, 127)                       # float32 division, rne, saturate
+    rcp = (np.float32(1.0) / alpha).astype(np.float32)
+    t = np.clip(v * rcp[:, None], np.float32(-127), np.float32(127)).astype(np.float32)
+    kf = np.rint(t)
+    e = np.abs(t - kf)
+    fast = e <= np.float32(0.49994)
+    assert np.array_equal(kf[fast], d[fast])
+    assert 0.2 < fast.mean() < 1.0 and (~fast).sum() > 1000      # both paths exercised

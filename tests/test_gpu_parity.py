@@ -240,6 +240,37 @@ def test_quantizer_full_size_x_and_bc():
         assert np.array_equal(s, s_ref) and np.array_equal(q, q_ref)
 
 
+@pytest.mark.parametrize("dtype", ["float32", "float16", "bfloat16"])
+@pytest.mark.parametrize("T,H,P,G,N", [(333, 3, 8, 1, 16), (1000, 4, 64, 2, 64), (4096, 24, 64, 1, 128)])
+def test_entry_quantizer_bit_exact(dtype, T, H, P, G, N):
+    """xBC [T][D + 2GN] in one pass == the Eq. 1 oracle on its three slices (static step sizes)."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    D, GN = H * P, G * N
+    rng = np.random.default_rng([T, D, GN])
+    xBC = (rng.standard_normal((T, D + 2 * GN)) * rng.uniform(0.05, 20, (1, D + 2 * GN))).astype(np.float32)
+    td = getattr(torch, dtype)
+    dv = torch.from_numpy(xBC).to(td).cuda()
+    v = dv.float().cpu().numpy()          # the values the kernel sees (the widening is exact)
+    s_x = (np.abs(v[:, :D]).max(0) / 200).astype(np.float32)     # saturates part of every channel
+    s_x[D // 2] = 1.0
+    s_B = rng.uniform(0.01, 0.2, G).astype(np.float32)
+    s_C = rng.uniform(0.01, 0.2, G).astype(np.float32)
+    xq = torch.empty((T, D), dtype=torch.int8, device="cuda")
+    Bq = torch.empty((T, GN), dtype=torch.int8, device="cuda")
+    Cq = torch.empty((T, GN), dtype=torch.int8, device="cuda")
+    bd.ssdi8_quantize_entry(dv, T, D, G, N, torch.from_numpy(s_x).cuda(), torch.from_numpy(s_B).cuda(),
+                            torch.from_numpy(s_C).cuda(), xq, Bq, Cq)
+    torch.cuda.synchronize()
+    x_ref, _ = orc.quantize(np.ascontiguousarray(v[:, :D]), T, D, 1, scale=s_x, mode=0)
+    B_ref, _ = orc.quantize(np.ascontiguousarray(v[:, D:D + GN]), T, G, N, scale=s_B, mode=0)
+    C_ref, _ = orc.quantize(np.ascontiguousarray(v[:, D + GN:]), T, G, N, scale=s_C, mode=0)
+    assert np.array_equal(xq.cpu().numpy(), x_ref)
+    assert np.array_equal(Bq.cpu().numpy(), B_ref)
+    assert np.array_equal(Cq.cpu().numpy(), C_ref)
+    assert np.abs(x_ref).max() == 127
+
+
 # --------------------------------------------------------------------------- calibration
 @pytest.mark.parametrize("cfg", SMALL[:3], ids=lambda c: c.name)
 def test_calibrate_bit_exact(cfg):
