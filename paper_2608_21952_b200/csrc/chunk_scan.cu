@@ -221,6 +221,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
   }
 }
 
+template <bool CORR>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
               const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
@@ -274,13 +275,13 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
         const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
-        mbar_wait(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
+        mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
         const int npanel = t.KJ / (int)RBQ;
         mbar_expect_tx(&bars[B_CB_FULL + ci], (uint32_t)(npanel * TM * RBQ));
         for (int pn = 0; pn < npanel; ++pn)
           tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
                       (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
-        mbar_wait(&bars[B_TOK_FREE + t3], ph3 ^ 1, a.status);
+        mbar_wait_relaxed(&bars[B_TOK_FREE + t3], ph3 ^ 1, a.status);
         mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4));
         bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4),
                   &bars[B_TOK_FULL + t3]);
@@ -292,7 +293,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       Tile t = decode_tile(t_begin, d, TM, ntpu);
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-        mbar_wait(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
+        mbar_wait_relaxed(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
         mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
         tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
         tma_load_2d(smem + OFF_H, &tm_h, &bars[B_CH_FULL], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
@@ -306,7 +307,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int s2 = n & 1;
         const uint32_t ph2 = (n >> 1) & 1;
-        mbar_wait(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
+        mbar_wait_relaxed(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
         mbar_expect_tx(&bars[B_X_FULL + s2], (uint32_t)(t.KJ * 64));
         for (int j0 = 0; j0 < t.KJ; j0 += TM)
           tma_load_3d(smem + OFF_X + s2 * 16384 + j0 * 64, &tm_x, &bars[B_X_FULL + s2], 0, t.h, (int)(t.tok0 + j0));
@@ -378,8 +379,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f, scb = a.s_cb[t.g];
       const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
       const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
-      const float4* gco = a.corr ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
-      mbar_wait(&bars[B_ACC + s2], ph2, a.status);
+      const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
+      mbar_wait_relaxed(&bars[B_ACC + s2], ph2, a.status);
       mbar_wait(&bars[B_MQ + ci], ph4, a.status);        // partial row maxima written by the mask warps
       mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);    // xq rows (skip term)
       mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);  // cs
@@ -396,19 +397,20 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       __syncwarp();
       uint8_t* srow = ystage + lane * 128;
 #pragma unroll 1
-      for (int pc = 0; pc < 2; ++pc) {       // 16 columns at a time
-        int acc_o[16], acc_d[16];
-        const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 16);
-        tmem_ld16(taddr, acc_o);
-        tmem_ld16(taddr + 64, acc_d);
+      for (int pc = 0; pc < 4; ++pc) {       // 8 columns at a time (keeps the accumulators in registers)
+        int acc_o[8], acc_d[8];
+        const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 8);
+        tmem_ld8(taddr, acc_o);
+        tmem_ld8(taddr + 64, acc_d);
         tmem_ld_wait();
         if (ok) {
-          const uint4 xr = *reinterpret_cast<const uint4*>(sX + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + pc), 64));
-          const uint32_t xw[4] = {xr.x ^ 0x80808080u, xr.y ^ 0x80808080u, xr.z ^ 0x80808080u, xr.w ^ 0x80808080u};
+          const uint2 xr = *reinterpret_cast<const uint2*>(
+              sX + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + (pc >> 1)), 64) + (pc & 1) * 8);
+          const uint32_t xw[2] = {xr.x ^ 0x80808080u, xr.y ^ 0x80808080u};
 #pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            const float4 sx4 = __ldg(gsx + pc * 4 + cc), sh4 = __ldg(gsh + pc * 4 + cc);
-            const float4 co4 = gco ? __ldg(gco + pc * 4 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int cc = 0; cc < 2; ++cc) {
+            const float4 sx4 = __ldg(gsx + pc * 2 + cc), sh4 = __ldg(gsh + pc * 2 + cc);
+            const float4 co4 = CORR ? __ldg(gco + pc * 2 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
             float2 v[2];
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
@@ -423,13 +425,13 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
               r2 = __ffma2_rn(__fmul2_rn(sm2, sx2), ad, r2);
               v[e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
             }
-            *reinterpret_cast<float4*>(srow + (((pc * 4 + cc) ^ (lane & 7)) << 4)) =
+            *reinterpret_cast<float4*>(srow + (((pc * 2 + cc) ^ (lane & 7)) << 4)) =
                 make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
           }
           if (a.taps.acc_off || a.taps.acc_diag) {
-            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 16;
+            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 8;
 #pragma unroll
-            for (int pp = 0; pp < 16; ++pp) {
+            for (int pp = 0; pp < 8; ++pp) {
               if (a.taps.acc_off) a.taps.acc_off[o + pp] = acc_o[pp];
               if (a.taps.acc_diag) a.taps.acc_diag[o + pp] = acc_d[pp];
             }
@@ -509,9 +511,14 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
   ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta};
   const size_t smem = SMEM_BYTES + 1024;
-  SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
-  chunk_scan_tc<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
+  if (corr) {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    chunk_scan_tc<true><<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
+  } else {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    chunk_scan_tc<false><<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
+  }
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

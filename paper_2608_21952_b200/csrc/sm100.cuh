@@ -53,6 +53,18 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
 }
 
+// The same bounded wait for warps whose wait is long and off the critical path (producers waiting
+// for a free slot, epilogue warps waiting for an accumulator): a failed poll is followed by a short
+// sleep, so the polling loop leaves the issue slots to the warps that compute.
+__device__ __forceinline__ void mbar_wait_relaxed(uint64_t* bar, uint32_t parity, int32_t* status) {
+  for (uint32_t it = 0; it < kWaitCap; ++it) {
+    if (mbar_try_wait(bar, parity)) return;
+    __nanosleep(256);
+    if ((it & 255u) == 255u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
+  }
+  if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
+}
+
 // ------------------------------------------------------------------ proxies and fences
 __device__ __forceinline__ void fence_async_smem() {  // generic-proxy smem writes -> async proxy
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -134,6 +146,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
       : "r"(taddr)
       : "memory");
 }
