@@ -7,9 +7,10 @@
 //   y = exp(cs_i) s_C s_h acc_off + (s_cb rowmax_i / 127) s_x acc_diag + D s_x xq + corr
 // Roles (28 warps): warps 0, 2, 3 issue the TMA loads (CBq K-major and the per-token scalar pack
 // of ChunkCumsum; Cq, hq K-major; xq MN-major), each stream on its own ring; warp 1 issues the
-// MMAs; warps 4-19 build Mq in place over CBq (four threads per output row, 16-column chunks
-// dealt round robin); warps 20-27 read the accumulators, form y and store it through swizzled
-// staging with TMA.  Every buffer has its own "free" barrier, released by whoever reads it last
+// MMAs; warps 4-19 build Mq in place over CBq, as two groups of 8 warps that take alternate tiles
+// (two threads per output row, 16-column chunks dealt alternately: the per-row fixed work is done
+// twice, not four times, and two tiles are in flight); warps 20-27 read the accumulators, form y
+// and store it through swizzled staging with TMA.  Every buffer has its own "free" barrier, released by whoever reads it last
 // (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
 // hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
 // because every role executes different code at the same time.  No multicast; bounded waits.
@@ -31,7 +32,7 @@ struct ScanArgs {
 };
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
-constexpr int kMaskWarp0 = 4, kMaskWarps = 16, kMaskThreads = kMaskWarps * 32;
+constexpr int kMaskWarp0 = 4, kMaskWarps = 16, kGroupWarps = 8, kGroupThreads = kGroupWarps * 32;
 constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 256;  // accumulator pair a: acc_off at 128 a, acc_diag at 128 a + 64
 constexpr uint32_t PANEL = 16384;    // [128][128] int8
@@ -40,11 +41,10 @@ constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1
 constexpr uint32_t OFF_C = 98304;       // [128][N]
 constexpr uint32_t OFF_H = 114688;      // [64][N]
 constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
-constexpr uint32_t OFF_TOK = 155648;    // ring of 3 x (5 Q floats: cs, dt, woff, atok, wmax; 4 x [128] partial row maxima)
-constexpr uint32_t TOK_BYTES = 7168;
-constexpr uint32_t OFF_YST = 177152;    // 8 warps x [32][128 B] y staging
-constexpr uint32_t OFF_FBUF = OFF_YST + 32768;   // [128][16] decay factors f of the tile being masked (thread-private slots)
-constexpr uint32_t OFF_BAR = OFF_FBUF + 8192;
+constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds; 2 x [128] partial row maxima)
+constexpr uint32_t TOK_BYTES = 6144;
+constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][128 B] y staging
+constexpr uint32_t OFF_BAR = OFF_YST + 32768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
 __device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
@@ -57,7 +57,7 @@ __device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
 }
 
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
-       B_TOK_FULL = 18, B_TOK_FREE = 21, B_ACC = 24, B_ACC_FREE = 26, B_COUNT = 28 };
+       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_COUNT = 30 };
 
 
 // two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
@@ -106,21 +106,30 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
   return x;
 }
 
-// ---- the masked operand of one tile, in place over CBq.  Four threads per output row; the
-// row's 16-column chunks (sub-blocks of the decay factorisation) are dealt round robin:
-// thread q handles chunks c = q, q + 4, ...  Chunk I16 = i / 16 is the row's own sub-block
-// (running product of per-token decays), earlier chunks use the column weights woff and one
-// factor f = exp32(cs_i - cs_ce) per chunk, later chunks are zero.
-__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fbuf, int wtid, int TM,
+// ---- the masked operand of one tile, in place over CBq.  Two threads per output row; the
+// row's 16-column chunks (sub-blocks of the decay factorisation) are dealt alternately: thread q
+// handles chunks c = q, q + 2, ...  Chunk I16 = i / 16 is the row's own sub-block (running
+// product of per-token decays), earlier chunks use the column weights woff and one factor
+// f = exp32(cs_i - cs_ce) per chunk, later chunks are zero.
+//
+// Work that decides no output bit is skipped, nearest chunk first.  b127[c] bounds |cb woff| of
+// chunk c, so a chunk with fmul(b127[c], f) <= (running maximum) cannot raise the row maximum,
+// and one with fmul(b127[c], f inv) < 1/2 rounds to zero everywhere.  p127[c] bounds b127 of
+// chunks 0..c with a 1e-5 slack; where cs does not increase along the chunk, f of a farther
+// chunk is at most f of a nearer one (up to the few 1e-7 of exp32's error, inside the slack),
+// so the same two tests on p127[c] end the walk for all farther chunks at once.  (p127 is +inf
+// where cs is not monotone: the walk then visits every chunk.)
+__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid, int group, int TM,
                                           uint32_t RBQ, const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
   const float* cs_s = tokbuf;
   const float* dt_s = tokbuf + Q;
   const float* woff_s = tokbuf + 2 * Q;
   const float* atok_s = tokbuf + 3 * Q;
-  const float* wmax_s = tokbuf + 4 * Q;
-  float* part_s = tokbuf + 1280;  // [4][128]
-  const int r = wtid & 127, q4 = wtid >> 7;
+  const float* b127_s = tokbuf + 4 * Q;
+  const float* p127_s = b127_s + 16;
+  float* part_s = tokbuf + 1280;  // [2][128]
+  const int r = gtid & 127, q2 = gtid >> 7;
   const bool row_ok = r < TM;
   const int i = t.it * TM + r;       // row within the chunk
   const int I16 = i >> 4, ri = i & 15;
@@ -132,68 +141,87 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
     const uint32_t pn = (uint32_t)c >> cshift, cc = (uint32_t)c & ((1u << cshift) - 1u);
     return reinterpret_cast<uint4*>(rowbase + pn * PANEL + ((cc ^ rx) << 4));
   };
-  float* frow = fbuf + r * 16;
   const float cs_i = row_ok ? cs_s[i] : 0.f;
+  const bool own = (I16 & 1) == q2;  // this thread holds the row's own sub-block
+  const int c_first = I16 - 1 - ((I16 - 1 - q2) & 1);  // nearest earlier chunk of this thread (may be < 0)
   float tv[16];                      // t of the row's own sub-block (kept by the thread that owns it)
   float rpart = 0.f;
+  float f0 = 0.f, f1 = 0.f;          // f of the first two chunks visited
+  int nv = 0;                        // chunks whose f the first pass computed
   if (row_ok) {
-    // nearest chunks first: they carry the largest weights, so the running maximum soon exceeds
-    // the bound 127 wmax_c f of the far chunks, which are then skipped (they cannot be the maximum)
-#pragma unroll 1
-    for (int c = I16 - ((I16 - q4) & 3); c >= 0; c -= 4) {
-      if (c < I16) {
-        const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
-        frow[c] = f;
-        if (__fmul_rn(__fmul_rn(127.0f, wmax_s[c]), f) <= rpart) continue;
-        const uint4 w4 = *chunk_ptr(c);
-        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-        const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
-        float bmax = 0.f;
+    if (own) {
+      // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+      const uint4 w4 = *chunk_ptr(I16);
+      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+      const float* dtc = dt_s + I16 * 16;
+      const float* atc = atok_s + I16 * 16 + 1;
+      float E = 1.0f;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const float4 o = wo[w];
-          const float2 t0 = __fmul2_rn(unpack2(ww[w], 0), make_float2(o.x, o.y));
-          const float2 t1 = __fmul2_rn(unpack2(ww[w], 2), make_float2(o.z, o.w));
-          bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
-          bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
+      for (int e = 15; e >= 0; --e) {
+        float v = 0.f;
+        if (e <= ri) {
+          if (e < ri) E = __fmul_rn(E, atc[e]);
+          v = __fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E));
         }
-        rpart = fmaxf(rpart, __fmul_rn(bmax, f));
-      } else {
-        // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
-        const uint4 w4 = *chunk_ptr(c);
-        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-        const float* dtc = dt_s + c * 16;
-        const float* atc = atok_s + c * 16 + 1;
-        float E = 1.0f;
-#pragma unroll
-        for (int e = 15; e >= 0; --e) {
-          float v = 0.f;
-          if (e <= ri) {
-            if (e < ri) E = __fmul_rn(E, atc[e]);
-            v = __fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E));
-          }
-          tv[e] = v;
-          rpart = fmaxf(rpart, fabsf(v));
-        }
+        tv[e] = v;
+        rpart = fmaxf(rpart, fabsf(v));
       }
     }
+#pragma unroll 1
+    for (int c = c_first; c >= 0; c -= 2) {
+      const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
+      if (nv == 0) f0 = f;
+      if (nv == 1) f1 = f;
+      ++nv;
+      if (rpart >= 1e-30f && __fmul_rn(p127_s[c], f) <= rpart) break;  // nor can any farther chunk
+      if (__fmul_rn(b127_s[c], f) <= rpart) continue;
+      const uint4 w4 = *chunk_ptr(c);
+      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+      const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
+      float bmax = 0.f;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float4 o = wo[w];
+        const float2 t0 = __fmul2_rn(unpack2(ww[w], 0), make_float2(o.x, o.y));
+        const float2 t1 = __fmul2_rn(unpack2(ww[w], 2), make_float2(o.z, o.w));
+        bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
+        bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
+      }
+      rpart = fmaxf(rpart, __fmul_rn(bmax, f));
+    }
   }
-  part_s[q4 * 128 + r] = rpart;
-  asm volatile("bar.sync 1, %0;" ::"n"(kMaskThreads) : "memory");
-  const float rowmax = fmaxf(fmaxf(part_s[r], part_s[128 + r]), fmaxf(part_s[256 + r], part_s[384 + r]));
+  part_s[q2 * 128 + r] = rpart;
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGroupThreads) : "memory");
+  const float rowmax = fmaxf(part_s[r], part_s[128 + r]);
   if (!row_ok) return;
   const float inv = (rowmax >= 1e-30f) ? __fdiv_rn(127.0f, rowmax) : 0.f;
   int8_t* mq_tap = nullptr;
   if (a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
-  if (q4 == 0 && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+  if (q2 == 0 && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  // chunks after the row's own contribute nothing
 #pragma unroll 1
-  for (int c = q4; c < nch; c += 4) {
+  for (int c = c_first + 2 + (own ? 2 : 0); c < nch; c += 2) *chunk_ptr(c) = zero4;
+  if (own) {
+    const float2 inv2 = make_float2(inv, inv);
+    uint32_t o[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      o[w] = pack4_rne(__fmul2_rn(make_float2(tv[w * 4], tv[w * 4 + 1]), inv2),
+                       __fmul2_rn(make_float2(tv[w * 4 + 2], tv[w * 4 + 3]), inv2));
+    const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+    *chunk_ptr(I16) = v;
+    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + I16 * 16) = v;
+  }
+  int c = c_first;
+#pragma unroll 1
+  for (int v2 = 0; c >= 0; c -= 2, ++v2) {
+    const float f = v2 >= nv || v2 > 1 ? exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])) : (v2 ? f1 : f0);
+    const float g = __fmul_rn(f, inv);
+    if (__fmul_rn(p127_s[c], g) < 0.5f) break;  // this chunk and every farther one round to zero
     uint4* ptr = chunk_ptr(c);
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);  // chunks after the row's own contribute nothing
-    if (c < I16) {
-      const float g = __fmul_rn(frow[c], inv);
-      // every |cb woff g| <= 127 wmax_c g: below one half the whole chunk rounds to zero
-      if (__fmul_rn(__fmul_rn(127.0f, wmax_s[c]), g) >= 0.5f) {
+    uint4 v = zero4;
+    if (__fmul_rn(b127_s[c], g) >= 0.5f) {
       const float2 g2 = make_float2(g, g);
       const uint4 w4 = *ptr;
       const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
@@ -201,23 +229,19 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, float* fb
       uint32_t o[4];
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        const float4 f = wo[w];
-        o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(f.x, f.y)), g2),
-                         __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(f.z, f.w)), g2));
+        const float4 fo = wo[w];
+        o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)), g2),
+                         __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2));
       }
-      v = make_uint4(o[0], o[1], o[2], o[3]);
-      }
-    } else if (c == I16) {
-      const float2 inv2 = make_float2(inv, inv);
-      uint32_t o[4];
-#pragma unroll
-      for (int w = 0; w < 4; ++w)
-        o[w] = pack4_rne(__fmul2_rn(make_float2(tv[w * 4], tv[w * 4 + 1]), inv2),
-                         __fmul2_rn(make_float2(tv[w * 4 + 2], tv[w * 4 + 3]), inv2));
       v = make_uint4(o[0], o[1], o[2], o[3]);
     }
     *ptr = v;
-    if (mq_tap && c <= I16) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
+    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
+  }
+#pragma unroll 1
+  for (; c >= 0; c -= 2) {
+    *chunk_ptr(c) = zero4;
+    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = zero4;
   }
 }
 
@@ -243,9 +267,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     for (int s = 0; s < 4; ++s) {
       mbar_init(&bars[B_CB_FULL + s], 1);
       mbar_init(&bars[B_CB_FREE + s], 1);
-      mbar_init(&bars[B_MQ + s], kMaskWarps);
-    }
-    for (int s = 0; s < 3; ++s) {
+      mbar_init(&bars[B_MQ + s], kGroupWarps);
       mbar_init(&bars[B_TOK_FULL + s], 1);
       mbar_init(&bars[B_TOK_FREE + s], kEpiWarps);
     }
@@ -273,8 +295,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       Tile t = decode_tile(t_begin, d, TM, ntpu);
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-        const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
-        const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
+        const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+        const uint32_t ph4 = (n >> 2) & 1, ph3 = (n >> 2) & 1;
         mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
         const int npanel = t.KJ / (int)RBQ;
         mbar_expect_tx(&bars[B_CB_FULL + ci], (uint32_t)(npanel * TM * RBQ));
@@ -347,20 +369,23 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       }
     }
   } else if (warp < kEpiWarp0) {
-    // ------------------------------------------------------------ mask warps
-    const int wtid = tid - kMaskWarp0 * 32;
+    // ------------------------------------------------------------ mask warps: group g takes tiles n = g, g + 2, ...
+    const int g = (warp - kMaskWarp0) / kGroupWarps;
+    const int gtid = tid - (kMaskWarp0 + g * kGroupWarps) * 32;
     Tile t = decode_tile(t_begin, d, TM, ntpu);
+    if (g) next_tile(t, d, TM, ntpu);
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-      const int ci = cb_index(n, t.it, ntpu), t3 = n % 3;
-      const uint32_t ph4 = (n >> 2) & 1, ph3 = (n / 3) & 1;
-      mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);
+    for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
+      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+      const uint32_t ph4 = (n >> 2) & 1;
+      mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
       mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
-      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES),
-                reinterpret_cast<float*>(smem + OFF_FBUF), wtid, TM, RBQ, t, a);
+      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, g, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
+      next_tile(t, d, TM, ntpu);
+      next_tile(t, d, TM, ntpu);
     }
   } else {
     // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
@@ -372,8 +397,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     Tile t = decode_tile(t_begin, d, TM, ntpu);
 #pragma unroll 1
     for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-      const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n % 3;
-      const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n / 3) & 1;
+      const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n & 3;
+      const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n >> 2) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
       const uint8_t* sX = smem + OFF_X + s2 * 16384;
       const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f, scb = a.s_cb[t.g];
@@ -389,9 +414,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const int ei = t.it * TM + er;
       const float* part = tok + 1280;
       const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
-      const float sm = ok ? scb * fmaxf(fmaxf(part[er], part[128 + er]), fmaxf(part[256 + er], part[384 + er])) *
-                                (1.0f / 127.0f)
-                          : 0.f;
+      const float sm = ok ? scb * fmaxf(part[er], part[128 + er]) * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
       if (lane == 0) tma_store_wait_read();  // last tile's store has finished reading the staging tile
       __syncwarp();

@@ -4,8 +4,11 @@
 //   row 1  dt[i]
 //   row 2  woff[i]  = fmul(dt_i, exp32(fsub(cs_ie, cs_i))), ie = last token of i's 16-token sub-block
 //   row 3  atok[i]  = exp32(fsub(cs_i, cs_{i-1}))  (1 for i = 0): the per-token decay
-//   row 4  wmax[c]  = max of woff over the 16-token sub-block c (first Q/16 entries; the rest 0):
-//                     an upper bound that lets the scan kernel skip sub-blocks that cannot matter
+//   row 4  bounds that let the scan kernel skip sub-blocks that cannot matter (they decide no
+//          output bit): [c] = fmul(127, wmax_c), wmax_c the maximum of |woff| over the 16-token
+//          sub-block c; [16 + c] = the maximum of the former over sub-blocks 0..c, times
+//          1.00001, or +inf when cs is not non-increasing over the chunk (some dt A > 0), which
+//          switches the early exits of the scan kernel off
 //   row 5  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
 // and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
 // (it decides rounding downstream), so each (b, chunk, head) is scanned sequentially by one
@@ -42,11 +45,17 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     const double a = (double)A[h0 + hh];
     double acc = 0.0;
     float last = 0.f;
+    float dmin = 0.f, dmax = 0.f;  // every increment dt A <= 0  <=>  no dt has the sign of A
     for (int i = 0; i < Q; ++i) {
-      acc += (double)dts[hh * ld + i] * a;
+      const float dv = dts[hh * ld + i];
+      dmin = fminf(dmin, dv);
+      dmax = fmaxf(dmax, dv);
+      acc += (double)dv * a;
       last = (float)acc;
       css[hh * ld + i] = last;
     }
+    const bool mono = a > 0.0 ? dmax <= 0.f : (a < 0.0 ? dmin >= 0.f : true);
+    css[hh * ld + Q] = mono ? 1.0f : 0.0f;
     gamma[((i64)b * d.H + h0 + hh) * d.c + k] = exp32(last);
   }
   __syncthreads();
@@ -67,12 +76,25 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     if (tap_cs) tap_cs[u * Q + i] = ci;
   }
   __syncthreads();
+  // sub-block maxima of |woff| (dts is free now: it holds them, times 127)
+  for (int e = threadIdx.x; e < CH * 16; e += blockDim.x) {
+    const int hh = e >> 4, c = e & 15;
+    if (hh >= nh || c >= Q / 16) continue;
+    float m = 0.f;
+    for (int j = 0; j < 16; ++j) m = fmaxf(m, fabsf(wos[hh * ld + c * 16 + j]));
+    dts[hh * ld + c] = __fmul_rn(127.0f, m);
+  }
+  __syncthreads();
   for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
     const int hh = e / Q, i = e % Q;
     if (hh >= nh) continue;
     float m = 0.f;
-    if (i < Q / 16)
-      for (int j = 0; j < 16; ++j) m = fmaxf(m, wos[hh * ld + i * 16 + j]);
+    if (i < Q / 16) {
+      m = dts[hh * ld + i];
+    } else if (i >= 16 && i < 16 + Q / 16) {
+      for (int c = 0; c <= i - 16; ++c) m = fmaxf(m, dts[hh * ld + c]);
+      m = css[hh * ld + Q] != 0.f ? __fmul_rn(m, 1.00001f) : __int_as_float(0x7f800000);
+    }
     pack[((((i64)b * d.H + h0 + hh) * d.c + k) * kPackRows + PACK_WMAX) * Q + i] = m;
   }
 }

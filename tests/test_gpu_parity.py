@@ -26,9 +26,11 @@ def _causal(cfg):
     return np.tril(np.ones((cfg.chunk, cfg.chunk), bool))
 
 
-def check_fwd(cfg, init=None, corr=None, use_D=True):
+def check_fwd(cfg, init=None, corr=None, use_D=True, mutate=None):
     gh = _harness()
     t = inputs.make_prefill(cfg)
+    if mutate is not None:
+        mutate(t)
     q = orc.prepare_quantized(cfg, t, init)
     y_ref, fin_ref, ref = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"],
                                         q["dt"], q["A"], q["D"] if use_D else None, corr, q["s_xs"],
@@ -71,6 +73,35 @@ def test_fwd_without_skip_weight():
 
 def test_fwd_cfg1_full():
     check_fwd(CONFIGS["cfg1"])
+
+
+def _scale_A(f):
+    def m(t):
+        t["A"] = (t["A"] * np.float32(f)).astype(np.float32)
+    return m
+
+
+def _growing_head(t):
+    """Head 1 grows instead of decaying (A > 0, outside the model's range but inside the
+    interface's): the cumulative sums are not monotone there."""
+    t["A"] = t["A"].copy()
+    t["A"][1] = np.float32(0.25)
+
+
+def _mixed_sign_dt(t):
+    """dt of both signs: cs wanders, so no ordering of the decay factors may be assumed."""
+    t["dt"] = (t["dt"] * np.where(np.random.default_rng(9).random(t["dt"].shape) < 0.3, -1, 1)).astype(np.float32)
+
+
+@pytest.mark.parametrize("cfg", [SMALL[1], SMALL[2]], ids=lambda c: c.name)
+@pytest.mark.parametrize("regime", ["slow", "fast", "very_fast", "growing", "mixed_dt"])
+def test_fwd_decay_regimes_bit_exact(cfg, regime):
+    """The masked operand skips sub-blocks that cannot matter; the skipping must decide no bit
+    whether almost nothing decays (every sub-block of a row matters), almost everything does
+    (only the row's own sub-block survives), or the decay is not monotone (the walk may not stop early)."""
+    mutate = {"slow": _scale_A(0.01), "fast": _scale_A(8.0), "very_fast": _scale_A(200.0),
+              "growing": _growing_head, "mixed_dt": _mixed_sign_dt}[regime]
+    check_fwd(cfg, mutate=mutate)
 
 
 def test_fwd_degenerate_inputs():
