@@ -8,8 +8,8 @@
 // Roles (28 warps): warps 0, 2, 3 issue the TMA loads (CBq K-major and the per-token scalar pack
 // of ChunkCumsum; Cq, hq K-major; xq MN-major), each stream on its own ring; warp 1 issues the
 // MMAs; warps 4-19 build Mq in place over CBq, as two groups of 8 warps that take alternate tiles
-// (two threads per output row, 16-column chunks dealt alternately: the per-row fixed work is done
-// twice, not four times, and two tiles are in flight); warps 20-27 read the accumulators, form y
+// (two threads per output row in adjacent lanes, so each warp owns 16 rows and runs on its own,
+// without block barriers, and two tiles are in flight); warps 20-27 read the accumulators, form y
 // and store it through swizzled staging with TMA.  Every buffer has its own "free" barrier, released by whoever reads it last
 // (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
 // hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
@@ -32,7 +32,7 @@ struct ScanArgs {
 };
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
-constexpr int kMaskWarp0 = 4, kMaskWarps = 16, kGroupWarps = 8, kGroupThreads = kGroupWarps * 32;
+constexpr int kMaskWarp0 = 4, kGroupWarps = 8;
 constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 256;  // accumulator pair a: acc_off at 128 a, acc_diag at 128 a + 64
 constexpr uint32_t PANEL = 16384;    // [128][128] int8
@@ -41,7 +41,7 @@ constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1
 constexpr uint32_t OFF_C = 98304;       // [128][N]
 constexpr uint32_t OFF_H = 114688;      // [64][N]
 constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
-constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds; 2 x [128] partial row maxima)
+constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds; [128] row maxima)
 constexpr uint32_t TOK_BYTES = 6144;
 constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][128 B] y staging
 constexpr uint32_t OFF_BAR = OFF_YST + 32768;
@@ -106,11 +106,13 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
   return x;
 }
 
-// ---- the masked operand of one tile, in place over CBq.  Two threads per output row; the
-// row's 16-column chunks (sub-blocks of the decay factorisation) are dealt alternately: thread q
-// handles chunks c = q, q + 2, ...  Chunk I16 = i / 16 is the row's own sub-block (running
-// product of per-token decays), earlier chunks use the column weights woff and one factor
-// f = exp32(cs_i - cs_ce) per chunk, later chunks are zero.
+// ---- the masked operand of one tile, in place over CBq.  Two threads per output row, in
+// adjacent lanes, so a warp owns 16 rows that share their own sub-block I16 = i / 16 (the walk
+// below is warp-uniform up to the skip tests) and the row maximum needs one shuffle, no block
+// barrier.  Chunk I16 (16 columns) is the row's own sub-block: running product of per-token
+// decays, columns split 8/8 between the two threads (the one with the lower columns first runs
+// the product through the upper ones).  Earlier chunks use the column weights woff and one
+// factor f = exp32(cs_i - cs_ce) per chunk and are dealt alternately; later chunks are zero.
 //
 // Work that decides no output bit is skipped, nearest chunk first.  b127[c] bounds |cb woff| of
 // chunk c, so a chunk with fmul(b127[c], f) <= (running maximum) cannot raise the row maximum,
@@ -119,8 +121,8 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
 // chunk is at most f of a nearer one (up to the few 1e-7 of exp32's error, inside the slack),
 // so the same two tests on p127[c] end the walk for all farther chunks at once.  (p127 is +inf
 // where cs is not monotone: the walk then visits every chunk.)
-__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid, int group, int TM,
-                                          uint32_t RBQ, const Tile& t, const ScanArgs& a) {
+__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid, int TM, uint32_t RBQ,
+                                          const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
   const float* cs_s = tokbuf;
   const float* dt_s = tokbuf + Q;
@@ -128,9 +130,9 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
   const float* atok_s = tokbuf + 3 * Q;
   const float* b127_s = tokbuf + 4 * Q;
   const float* p127_s = b127_s + 16;
-  float* part_s = tokbuf + 1280;  // [2][128]
-  const int r = gtid & 127, q2 = gtid >> 7;
-  const bool row_ok = r < TM;
+  float* rowmax_s = tokbuf + 1280;   // [128], read by the epilogue warps
+  const int r = gtid >> 1, q2 = gtid & 1;
+  if (r >= TM) return;               // whole warps (TM is a multiple of 16)
   const int i = t.it * TM + r;       // row within the chunk
   const int I16 = i >> 4, ri = i & 15;
   const int nch = t.KJ >> 4;         // 16-column chunks in the contraction range
@@ -141,77 +143,79 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
     const uint32_t pn = (uint32_t)c >> cshift, cc = (uint32_t)c & ((1u << cshift) - 1u);
     return reinterpret_cast<uint4*>(rowbase + pn * PANEL + ((cc ^ rx) << 4));
   };
-  const float cs_i = row_ok ? cs_s[i] : 0.f;
-  const bool own = (I16 & 1) == q2;  // this thread holds the row's own sub-block
-  const int c_first = I16 - 1 - ((I16 - 1 - q2) & 1);  // nearest earlier chunk of this thread (may be < 0)
-  float tv[16];                      // t of the row's own sub-block (kept by the thread that owns it)
+  const float cs_i = cs_s[i];
+  const int c_first = I16 - 1 - q2;  // nearest earlier chunk of this thread (may be < 0)
+  float tv[8];                       // t of this thread's half of the row's own sub-block
   float rpart = 0.f;
   float f0 = 0.f, f1 = 0.f;          // f of the first two chunks visited
   int nv = 0;                        // chunks whose f the first pass computed
-  if (row_ok) {
-    if (own) {
-      // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
-      const uint4 w4 = *chunk_ptr(I16);
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float* dtc = dt_s + I16 * 16;
-      const float* atc = atok_s + I16 * 16 + 1;
-      float E = 1.0f;
+  uint2* const own_ptr = reinterpret_cast<uint2*>(chunk_ptr(I16)) + q2;
+  {
+    // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+    const uint2 w2 = *own_ptr;
+    const uint32_t ww[2] = {w2.x ^ 0x80808080u, w2.y ^ 0x80808080u};
+    const float* atc = atok_s + I16 * 16 + 1;
+    float E = 1.0f;
+    if (q2 == 0) {
 #pragma unroll
-      for (int e = 15; e >= 0; --e) {
-        float v = 0.f;
-        if (e <= ri) {
-          if (e < ri) E = __fmul_rn(E, atc[e]);
-          v = __fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E));
-        }
-        tv[e] = v;
-        rpart = fmaxf(rpart, fabsf(v));
-      }
+      for (int e = 15; e >= 8; --e)
+        if (e < ri) E = __fmul_rn(E, atc[e]);
     }
-#pragma unroll 1
-    for (int c = c_first; c >= 0; c -= 2) {
-      const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
-      if (nv == 0) f0 = f;
-      if (nv == 1) f1 = f;
-      ++nv;
-      if (rpart >= 1e-30f && __fmul_rn(p127_s[c], f) <= rpart) break;  // nor can any farther chunk
-      if (__fmul_rn(b127_s[c], f) <= rpart) continue;
-      const uint4 w4 = *chunk_ptr(c);
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
-      float bmax = 0.f;
+    const int e0 = q2 * 8;
+    const float* dtc = dt_s + I16 * 16 + e0;
+    atc += e0;
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const float4 o = wo[w];
-        const float2 t0 = __fmul2_rn(unpack2(ww[w], 0), make_float2(o.x, o.y));
-        const float2 t1 = __fmul2_rn(unpack2(ww[w], 2), make_float2(o.z, o.w));
-        bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
-        bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
+    for (int k = 7; k >= 0; --k) {
+      float v = 0.f;
+      if (e0 + k <= ri) {
+        if (e0 + k < ri) E = __fmul_rn(E, atc[k]);
+        v = __fmul_rn(s8_to_f32(ww[k >> 2], k & 3), __fmul_rn(dtc[k], E));
       }
-      rpart = fmaxf(rpart, __fmul_rn(bmax, f));
+      tv[k] = v;
+      rpart = fmaxf(rpart, fabsf(v));
     }
   }
-  part_s[q2 * 128 + r] = rpart;
-  asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGroupThreads) : "memory");
-  const float rowmax = fmaxf(part_s[r], part_s[128 + r]);
-  if (!row_ok) return;
+#pragma unroll 1
+  for (int c = c_first; c >= 0; c -= 2) {
+    const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
+    if (nv == 0) f0 = f;
+    if (nv == 1) f1 = f;
+    ++nv;
+    if (rpart >= 1e-30f && __fmul_rn(p127_s[c], f) <= rpart) break;  // nor can any farther chunk
+    if (__fmul_rn(b127_s[c], f) <= rpart) continue;
+    const uint4 w4 = *chunk_ptr(c);
+    const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+    const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
+    float bmax = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float4 o = wo[w];
+      const float2 t0 = __fmul2_rn(unpack2(ww[w], 0), make_float2(o.x, o.y));
+      const float2 t1 = __fmul2_rn(unpack2(ww[w], 2), make_float2(o.z, o.w));
+      bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
+      bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
+    }
+    rpart = fmaxf(rpart, __fmul_rn(bmax, f));
+  }
+  const float rowmax = fmaxf(rpart, __shfl_xor_sync(0xffffffffu, rpart, 1));
   const float inv = (rowmax >= 1e-30f) ? __fdiv_rn(127.0f, rowmax) : 0.f;
   int8_t* mq_tap = nullptr;
   if (a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
-  if (q2 == 0 && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+  if (q2 == 0) {
+    rowmax_s[r] = rowmax;
+    if (a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+  }
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
   // chunks after the row's own contribute nothing
 #pragma unroll 1
-  for (int c = c_first + 2 + (own ? 2 : 0); c < nch; c += 2) *chunk_ptr(c) = zero4;
-  if (own) {
+  for (int c = I16 + 1 + q2; c < nch; c += 2) *chunk_ptr(c) = zero4;
+  {
     const float2 inv2 = make_float2(inv, inv);
-    uint32_t o[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w)
-      o[w] = pack4_rne(__fmul2_rn(make_float2(tv[w * 4], tv[w * 4 + 1]), inv2),
-                       __fmul2_rn(make_float2(tv[w * 4 + 2], tv[w * 4 + 3]), inv2));
-    const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
-    *chunk_ptr(I16) = v;
-    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + I16 * 16) = v;
+    uint2 v;
+    v.x = pack4_rne(__fmul2_rn(make_float2(tv[0], tv[1]), inv2), __fmul2_rn(make_float2(tv[2], tv[3]), inv2));
+    v.y = pack4_rne(__fmul2_rn(make_float2(tv[4], tv[5]), inv2), __fmul2_rn(make_float2(tv[6], tv[7]), inv2));
+    *own_ptr = v;
+    if (mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
   }
   int c = c_first;
 #pragma unroll 1
@@ -380,7 +384,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const uint32_t ph4 = (n >> 2) & 1;
       mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
       mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
-      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, g, TM, RBQ, t, a);
+      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
@@ -405,18 +409,23 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
       const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
       const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
-      mbar_wait_relaxed(&bars[B_ACC + s2], ph2, a.status);
-      mbar_wait(&bars[B_MQ + ci], ph4, a.status);        // partial row maxima written by the mask warps
-      mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);    // xq rows (skip term)
-      mbar_wait(&bars[B_TOK_FULL + t3], ph3, a.status);  // cs
+      // four lanes wait side by side, one barrier each: the accumulators, the row maxima written by
+      // the mask warps, the xq rows (skip term) and the scalar pack (cs); the warp barrier passes
+      // what they acquired on to the other lanes
+      if (lane < 4) {
+        const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_MQ + ci : lane == 2 ? B_X_FULL + s2 : B_TOK_FULL + t3;
+        const uint32_t bp = lane == 0 || lane == 2 ? ph2 : (lane == 1 ? ph4 : ph3);
+        mbar_wait_relaxed(&bars[bi], bp, a.status);
+      }
+      __syncwarp();
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
       const float* part = tok + 1280;
       const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
-      const float sm = ok ? scb * fmaxf(part[er], part[128 + er]) * (1.0f / 127.0f) : 0.f;
+      const float sm = ok ? scb * part[er] * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
-      if (lane == 0) tma_store_wait_read();  // last tile's store has finished reading the staging tile
+      if (lane == 3) tma_store_wait_read();  // last tile's store has finished reading the staging tile
       __syncwarp();
       uint8_t* srow = ystage + lane * 128;
 #pragma unroll 1
@@ -464,17 +473,14 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       tc_fence_before();
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&bars[B_ACC_FREE + s2]);
-        mbar_arrive(&bars[B_X_FREE + s2]);
-        mbar_arrive(&bars[B_TOK_FREE + t3]);
-        if (q * 32 < TM) {
-          tma_store_3d(&tm_y, ystage, ch * 32, t.h, (int)(t.tok0 + t.it * TM + q * 32));
-          tma_store_commit();
-        }
+      if (lane < 3) {   // one release each, side by side
+        mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + s2 : B_TOK_FREE + t3]);
+      } else if (lane == 3 && q * 32 < TM) {
+        tma_store_3d(&tm_y, ystage, ch * 32, t.h, (int)(t.tok0 + t.it * TM + q * 32));
+        tma_store_commit();
       }
     }
-    if (lane == 0) tma_store_wait_read();
+    if (lane == 3) tma_store_wait_read();
   }
   tc_fence_before();
   __syncthreads();
