@@ -8,7 +8,7 @@
 //          output bit): [c] = fmul(127, wmax_c), wmax_c the maximum of |woff| over the 16-token
 //          sub-block c; [16 + c] = the maximum of the former over sub-blocks 0..c, times
 //          1.00001, or +inf when cs is not non-increasing over the chunk (some dt A > 0), which
-//          switches the early exits of the scan kernel off
+//          switches the early exits of the scan kernel off; entries from 32 on are not written
 //   row 5  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
 // and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
 // (it decides rounding downstream), so each (b, chunk, head) is scanned sequentially by one
@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
                                                      float* __restrict__ tap_cs, Dims d) {
   extern __shared__ float tile[];  // dt [CH][Q+1], cs [CH][Q+1], woff [CH][Q+1]
   const int Q = d.Q, ld = Q + 1;
+  const int lq = 31 - __clz(Q);  // Q is a power of two
   float* dts = tile;
   float* css = tile + CH * ld;
   float* wos = tile + 2 * CH * ld;
@@ -70,13 +71,14 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     gamma[((i64)b * d.H + h0 + hh) * d.c + k] = exp32(last);
   }
   __syncthreads();
+  const i64 u0 = ((i64)b * d.H + h0) * d.c + k;  // pack index of head h0; the next head is d.c further
   for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
-    const int hh = e / Q, i = e % Q;
+    const int hh = e >> lq, i = e & (Q - 1);
     if (hh >= nh) continue;
     const float* c = css + hh * ld;
     const float ci = c[i], di = dts[hh * ld + i];
-    const i64 u = ((i64)b * d.H + h0 + hh) * d.c + k;
-    float* p = pack + u * kPackRows * Q + i;
+    const i64 u = u0 + (i64)hh * d.c;
+    float* p = pack + ((u * kPackRows) << lq) + i;
     p[0] = ci;
     p[Q] = di;
     const float wo = __fmul_rn(di, exp32(__fsub_rn(c[i | 15], ci)));
@@ -84,7 +86,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     p[PACK_WOFF * Q] = wo;
     p[PACK_ATOK * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
     p[PACK_LUT * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
-    if (tap_cs) tap_cs[u * Q + i] = ci;
+    if (tap_cs) tap_cs[(u << lq) + i] = ci;
   }
   __syncthreads();
   // sub-block maxima of |woff| (dts is free now: it holds them, times 127)
@@ -96,8 +98,8 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
     dts[hh * ld + c] = __fmul_rn(127.0f, m);
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
-    const int hh = e / Q, i = e % Q;
+  for (int e = threadIdx.x; e < 32 * CH; e += blockDim.x) {   // the first 32 entries of the bounds row
+    const int hh = e >> 5, i = e & 31;
     if (hh >= nh) continue;
     float m = 0.f;
     if (i < Q / 16) {
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
       for (int c = 0; c <= i - 16; ++c) m = fmaxf(m, dts[hh * ld + c]);
       m = css[hh * ld + Q] != 0.f ? __fmul_rn(m, 1.00001f) : __int_as_float(0x7f800000);
     }
-    pack[((((i64)b * d.H + h0 + hh) * d.c + k) * kPackRows + PACK_WMAX) * Q + i] = m;
+    pack[(((u0 + (i64)hh * d.c) * kPackRows + PACK_WMAX) << lq) + i] = m;
   }
 }
 
