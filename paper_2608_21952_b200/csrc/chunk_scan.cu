@@ -121,6 +121,7 @@ __device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int nt
 // chunk is at most f of a nearer one (up to the few 1e-7 of exp32's error, inside the slack),
 // so the same two tests on p127[c] end the walk for all farther chunks at once.  (p127 is +inf
 // where cs is not monotone: the walk then visits every chunk.)
+template <bool TAPS>
 __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid, int TM, uint32_t RBQ,
                                           const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
@@ -200,10 +201,10 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
   const float rowmax = fmaxf(rpart, __shfl_xor_sync(0xffffffffu, rpart, 1));
   const float inv = (rowmax >= 1e-30f) ? __fdiv_rn(127.0f, rowmax) : 0.f;
   int8_t* mq_tap = nullptr;
-  if (a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
+  if (TAPS && a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
   if (q2 == 0) {
     rowmax_s[r] = rowmax;
-    if (a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
+    if (TAPS && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
   }
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
   // chunks after the row's own contribute nothing
@@ -215,7 +216,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
     v.x = pack4_rne(__fmul2_rn(make_float2(tv[0], tv[1]), inv2), __fmul2_rn(make_float2(tv[2], tv[3]), inv2));
     v.y = pack4_rne(__fmul2_rn(make_float2(tv[4], tv[5]), inv2), __fmul2_rn(make_float2(tv[6], tv[7]), inv2));
     *own_ptr = v;
-    if (mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
+    if (TAPS && mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
   }
   int c = c_first;
 #pragma unroll 1
@@ -240,16 +241,17 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
       v = make_uint4(o[0], o[1], o[2], o[3]);
     }
     *ptr = v;
-    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
+    if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
   }
 #pragma unroll 1
   for (; c >= 0; c -= 2) {
     *chunk_ptr(c) = zero4;
-    if (mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = zero4;
+    if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = zero4;
   }
 }
 
-template <bool CORR>
+// CORR: a mean-correction vector is given; TAPS: intermediate tensors are written out (tests)
+template <bool CORR, bool TAPS>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
               const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
@@ -384,7 +386,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const uint32_t ph4 = (n >> 2) & 1;
       mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
       mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
-      mask_tile(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, TM, RBQ, t, a);
+      mask_tile<TAPS>(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
@@ -460,7 +462,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
             *reinterpret_cast<float4*>(srow + (((pc * 2 + cc) ^ (lane & 7)) << 4)) =
                 make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
           }
-          if (a.taps.acc_off || a.taps.acc_diag) {
+          if (TAPS && (a.taps.acc_off || a.taps.acc_diag)) {
             const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 8;
 #pragma unroll
             for (int pp = 0; pp < 8; ++pp) {
@@ -541,13 +543,18 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta};
   const size_t smem = SMEM_BYTES + 1024;
   const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
-  if (corr) {
-    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    chunk_scan_tc<true><<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
-  } else {
-    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_scan_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    chunk_scan_tc<false><<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
-  }
+  const bool tp = taps.acc_off || taps.rowmax || taps.Mq || taps.acc_diag;
+  auto launch = [&](auto kernel) -> ssdi8_status_t {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
+    return SSDI8_OK;
+  };
+  ssdi8_status_t ls;
+  if (corr)
+    ls = tp ? launch(chunk_scan_tc<true, true>) : launch(chunk_scan_tc<true, false>);
+  else
+    ls = tp ? launch(chunk_scan_tc<false, true>) : launch(chunk_scan_tc<false, false>);
+  if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

@@ -48,7 +48,8 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-template <bool I8S>
+// TAPS: any of the intermediate-tensor taps is requested (tests); the production instance carries no tap code
+template <bool I8S, bool TAPS>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
                     const __grid_constant__ CUtensorMap tm_hq, const FusedArgs a) {
@@ -149,7 +150,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
         }
         const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
         *ptr = v;
-        if (a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
+        if (TAPS && a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
       }
       fence_async_smem();
       __syncwarp();
@@ -211,7 +212,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
 #pragma unroll
           for (int e = 0; e < 8; ++e) sHQ[(ch * 32 + p0 + e) * N + n] = (uint8_t)code[e];
         }
-        if (!I8S && a.tap_prev) {
+        if (TAPS && !I8S && a.tap_prev) {
 #pragma unroll
           for (int pp = 0; pp < 32; ++pp) a.tap_prev[obase + (i64)pp * N] = S[pp];
         }
@@ -228,27 +229,27 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       tc_fence_after();
       if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        int acc[16];
-        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + hf * 16), acc);
+      for (int hf = 0; hf < 4; ++hf) {       // 8 channels at a time
+        int acc[8];
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + hf * 8), acc);
         tmem_ld_wait();
         if (ok) {
-          const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32 + hf * 16) * N + n;
-          float cscale[16];
+          const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32 + hf * 8) * N + n;
+          float cscale[8];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) cscale[e] = col_scale[ch * 32 + hf * 16 + e];
+          for (int e = 0; e < 8; ++e) cscale[e] = col_scale[ch * 32 + hf * 8 + e];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int pp = hf * 16 + e;
+          for (int e = 0; e < 8; ++e) {
+            const int pp = hf * 8 + e;
             const float loc = __fmul_rn(i22_to_f32(acc[e]), cscale[e]);
-            if (a.tap_acc) a.tap_acc[obase + (i64)e * N] = acc[e];
+            if (TAPS && a.tap_acc) a.tap_acc[obase + (i64)e * N] = acc[e];
             if (I8S) {
               const int locq = (int)(int8_t)(rne_clamp_bits(loc) & 0xffu);
               const int Gq = __float2int_rn(__fmul_rn(gam, 128.0f));
               const int Sn = locq + ((Gq * __float_as_int(S[pp]) + 64) >> 7);
               S[pp] = __int_as_float(max(-127, min(127, Sn)));
             } else {
-              if (a.tap_loc) a.tap_loc[obase + (i64)e * N] = loc;
+              if (TAPS && a.tap_loc) a.tap_loc[obase + (i64)e * N] = loc;
               S[pp] = __fmaf_rn(gam, S[pp], loc);
             }
           }
@@ -307,13 +308,18 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
                  status, d};
   const size_t smem = SMEM_BYTES + 1024;
   dim3 grid(d.H, d.b);
-  if (int8_state) {
-    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    chunk_state_pass_tc<true><<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
-  } else {
-    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(chunk_state_pass_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    chunk_state_pass_tc<false><<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
-  }
+  const bool taps = tap_loc || tap_prev || tap_Xsq || tap_acc;
+  auto launch = [&](auto kernel) -> ssdi8_status_t {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
+    return SSDI8_OK;
+  };
+  ssdi8_status_t ls;
+  if (int8_state)
+    ls = taps ? launch(chunk_state_pass_tc<true, true>) : launch(chunk_state_pass_tc<true, false>);
+  else
+    ls = taps ? launch(chunk_state_pass_tc<false, true>) : launch(chunk_state_pass_tc<false, false>);
+  if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }
