@@ -1,0 +1,170 @@
+// Layer forward from HOST buffers: Eq. 1 quantisation of fp32 x, B, C with static step sizes and
+// the SSD layer forward (Algorithm 2), one batch element at a time.  Batch elements are
+// independent, so the host->device copies of element b+1 and the device->host copy of the
+// output of element b-1 run on two side streams while the kernels of element b run on the
+// caller's stream: the PCIe link is busy in both directions for the whole call instead of
+// idle during the kernels and one-directional during the copies.  Only stream and event
+// plumbing lives here; every arithmetic step is a kernel of this library.
+#include "kernels.h"
+
+namespace ssdi8 {
+namespace {
+
+constexpr int kStages = 2;
+
+struct StageBuf {
+  float *x, *B, *C, *dt, *y, *fin;
+  int8_t *xq, *Bq, *Cq;
+};
+struct Layout {
+  StageBuf st[kStages];
+  void* ws;
+  int32_t* status;
+  size_t ws_bytes, total;
+};
+
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+Layout make_layout(const ssdi8_dims_t& d1, uint8_t* base, uint32_t flags) {
+  Layout lo;
+  const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
+  const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { uint8_t* p = base + o; o = up256(o + bytes); return p; };
+  for (int s = 0; s < kStages; ++s) {
+    lo.st[s].x = reinterpret_cast<float*>(take(nx * 4));
+    lo.st[s].B = reinterpret_cast<float*>(take(nb * 4));
+    lo.st[s].C = reinterpret_cast<float*>(take(nb * 4));
+    lo.st[s].dt = reinterpret_cast<float*>(take(ndt * 4));
+    lo.st[s].y = reinterpret_cast<float*>(take(nx * 4));
+    lo.st[s].fin = reinterpret_cast<float*>(take(nfin * 4));
+    lo.st[s].xq = reinterpret_cast<int8_t*>(take(nx));
+    lo.st[s].Bq = reinterpret_cast<int8_t*>(take(nb));
+    lo.st[s].Cq = reinterpret_cast<int8_t*>(take(nb));
+  }
+  lo.status = reinterpret_cast<int32_t*>(take(256));
+  lo.ws_bytes = ssdi8_workspace_bytes(&d1, flags);
+  lo.ws = take(lo.ws_bytes);
+  lo.total = o;
+  return lo;
+}
+
+// side streams and events, made once per device and kept for the life of the process
+struct Plumbing {
+  bool ready = false;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t start = nullptr, in_done[kStages] = {}, cmp_done[kStages] = {}, out_done[kStages] = {};
+};
+Plumbing g_plumb[64];
+
+ssdi8_status_t get_plumbing(Plumbing** out) {
+  int dev = 0;
+  SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
+  Plumbing& p = g_plumb[dev];
+  if (!p.ready) {
+    SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
+    SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+    for (int s = 0; s < kStages; ++s) {
+      SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.in_done[s], cudaEventDisableTiming));
+      SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.cmp_done[s], cudaEventDisableTiming));
+      SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.out_done[s], cudaEventDisableTiming));
+    }
+    p.ready = true;
+  }
+  *out = &p;
+  return SSDI8_OK;
+}
+
+}  // namespace
+}  // namespace ssdi8
+
+using namespace ssdi8;
+
+extern "C" {
+
+size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
+  if (!dims || dims->batch <= 0) return 0;
+  ssdi8_dims_t d1 = *dims;
+  d1.batch = 1;
+  if (ssdi8_workspace_bytes(&d1, flags) == 0) return 0;
+  return make_layout(d1, nullptr, flags).total;
+}
+
+ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_host_args_t* a, void* scratch,
+                                    size_t scratch_bytes, uint32_t flags, void* stream) {
+  if (!dims || !a || !scratch) return SSDI8_ERR_NULL;
+  if (!a->x || !a->B || !a->C || !a->dt || !a->A || !a->s_x || !a->s_B || !a->s_C || !a->s_xs || !a->s_cb ||
+      !a->s_h || !a->y)
+    return SSDI8_ERR_NULL;
+  if (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE) return SSDI8_ERR_UNSUPPORTED;
+  const size_t need = ssdi8_layer_fwd_host_scratch_bytes(dims, flags);
+  if (need == 0) return SSDI8_ERR_SHAPE;
+  if (scratch_bytes < need) return SSDI8_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(scratch) & 255) return SSDI8_ERR_ALIGN;
+  ssdi8_dims_t d1 = *dims;
+  d1.batch = 1;
+  const Layout lo = make_layout(d1, static_cast<uint8_t*>(scratch), flags);
+  Plumbing* p = nullptr;
+  ssdi8_status_t s = get_plumbing(&p);
+  if (s != SSDI8_OK) return s;
+  cudaStream_t s_cmp = static_cast<cudaStream_t>(stream);
+  const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
+  const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
+  const int64_t T1 = d1.seqlen;
+
+  // everything below is ordered after the work already in the caller's stream
+  SSDI8_CUDA_CHECK(cudaMemsetAsync(lo.status, 0, sizeof(int32_t), s_cmp));
+  SSDI8_CUDA_CHECK(cudaEventRecord(p->start, s_cmp));
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_in, p->start, 0));
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_out, p->start, 0));
+
+  for (int b = 0; b < dims->batch; ++b) {
+    const int st = b % kStages;
+    const StageBuf& sb = lo.st[st];
+    // inputs of element b: the kernels of element b - kStages have finished with this stage
+    if (b >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_in, p->cmp_done[st], 0));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.x, a->x + (size_t)b * nx, nx * 4, cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.B, a->B + (size_t)b * nb, nb * 4, cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.C, a->C + (size_t)b * nb, nb * 4, cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.dt, a->dt + (size_t)b * ndt, ndt * 4, cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(cudaEventRecord(p->in_done[st], p->s_in));
+    // kernels of element b: its inputs have arrived, and y of element b - kStages has left
+    SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->in_done[st], 0));
+    if (b >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
+    s = ssdi8_quantize_act(sb.x, T1, (int64_t)d1.nheads * d1.headdim, 1, const_cast<float*>(a->s_x), 0, sb.xq, s_cmp);
+    if (s != SSDI8_OK) return s;
+    s = ssdi8_quantize_act(sb.B, T1, d1.ngroups, d1.dstate, const_cast<float*>(a->s_B), 0, sb.Bq, s_cmp);
+    if (s != SSDI8_OK) return s;
+    s = ssdi8_quantize_act(sb.C, T1, d1.ngroups, d1.dstate, const_cast<float*>(a->s_C), 0, sb.Cq, s_cmp);
+    if (s != SSDI8_OK) return s;
+    ssdi8_fwd_args_t f = {};
+    f.xq = sb.xq; f.Bq = sb.Bq; f.Cq = sb.Cq;
+    f.s_x = a->s_x; f.s_B = a->s_B; f.s_C = a->s_C;
+    f.dt = sb.dt; f.A = a->A; f.D = a->D; f.corr = a->corr;
+    f.s_xs = a->s_xs; f.s_cb = a->s_cb; f.s_h = a->s_h;
+    f.init_state = a->init_state ? a->init_state + (size_t)b * nfin : nullptr;
+    f.y = sb.y;
+    f.final_state = a->final_state ? sb.fin : nullptr;
+    f.status = lo.status;
+    s = ssdi8_chunk_scan_fwd(&d1, &f, flags, lo.ws, lo.ws_bytes, s_cmp);
+    if (s != SSDI8_OK) return s;
+    SSDI8_CUDA_CHECK(cudaEventRecord(p->cmp_done[st], s_cmp));
+    // outputs of element b
+    SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_out, p->cmp_done[st], 0));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->y + (size_t)b * nx, sb.y, nx * 4, cudaMemcpyDeviceToHost, p->s_out));
+    if (a->final_state)
+      SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->final_state + (size_t)b * nfin, sb.fin, nfin * 4, cudaMemcpyDeviceToHost,
+                                       p->s_out));
+    SSDI8_CUDA_CHECK(cudaEventRecord(p->out_done[st], p->s_out));
+  }
+  // the caller's stream ends after the last copies (the last kStages elements' events cover all)
+  for (int st = 0; st < kStages && st < dims->batch; ++st)
+    SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
+  if (a->status)
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->status, lo.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s_cmp));
+  return SSDI8_OK;
+}
+
+}  // extern "C"

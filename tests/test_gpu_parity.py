@@ -393,3 +393,54 @@ def test_step_n64_groups():
 
 def test_step_full_size_batch():
     _decode_case(CONFIGS["cfg4"], 8)
+
+
+# --------------------------------------------------------------------------- host-buffer entry point
+@pytest.mark.parametrize("flags", [0, 2])
+def test_layer_fwd_host_matches_the_device_path_bit_for_bit(flags):
+    """ssdi8_layer_fwd_host (pinned host tensors in, pipelined per batch element) == Eq. 1 quantiser +
+    ssdi8_chunk_scan_fwd on the whole batch, and the oracle agrees with both; twice in a row
+    (the second call reuses the side streams and both scratch stages)."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SSDConfig("host_b3", 3, 256, 4, 64, 64, 2, 128, 0.02, 20.0, 31)   # odd batch: both stages, ragged
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    y_ref, fin_ref, _ = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                      q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], init, flags=flags)
+    q["init"] = init
+    y_dev, fin_dev, _ = gh.gpu_fwd(cfg, q, taps=(), flags=flags)
+    dims = bd.dims_of(cfg)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    host = {k: pin(t[k]) for k in ("x", "B", "C", "dt")}
+    y = torch.empty(t["x"].shape).pin_memory()
+    fin = torch.empty(init.shape).pin_memory()
+    status = torch.full((1,), -99, dtype=torch.int32).pin_memory()
+    dv = {k: gh.dev(q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "A", "D")}
+    args = bd.make_host_args(y=y, final_state=fin, status=status, init_state=gh.dev(init), **host, **dv)
+    scratch = torch.empty(bd.ssdi8_layer_fwd_host_scratch_bytes(dims, flags), dtype=torch.uint8, device="cuda")
+    for rep in range(2):
+        y.fill_(float("nan")); fin.fill_(float("nan"))
+        bd.ssdi8_layer_fwd_host(dims, args, scratch, flags)
+        torch.cuda.synchronize()
+        assert int(status[0]) == 0
+        assert np.array_equal(fin.numpy(), fin_ref)
+        assert np.abs(y.numpy() - y_ref).max() <= Y_TOL * rms(y_ref)
+        assert np.array_equal(y.numpy(), y_dev) and np.array_equal(fin.numpy(), fin_dev)
+
+
+def test_layer_fwd_host_rejects_a_short_scratch():
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SMALL[0]
+    dims = bd.dims_of(cfg)
+    z = torch.zeros(16).pin_memory()
+    d = gh.dev(np.zeros(16, np.float32))
+    args = bd.make_host_args(x=z, B=z, C=z, dt=z, y=z, A=d, s_x=d, s_B=d, s_C=d, s_xs=d, s_cb=d, s_h=d)
+    scratch = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bd.SSDi8Error) as e:
+        bd.ssdi8_layer_fwd_host(dims, args, scratch)
+    assert e.value.code == bd.ERR_WORKSPACE
