@@ -206,33 +206,40 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
 ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
                                            uint32_t flags, void* stream);
 
-/* Layer forward from HOST buffers: Eq. 1 quantisation of fp32 x, B, C with the given static step
- * sizes (three ssdi8_quantize_act calls, mode 0) followed by ssdi8_chunk_scan_fwd, one batch
- * element at a time.  Batch elements are independent (Algorithm 2 has no cross-batch term), so
- * the host->device copies of element b+1 and the device->host copy of y of element b-1 run on two
- * side streams while the kernels of element b run on `stream`: both directions of the host link
- * stay busy for the whole call.  The result is bit-identical to quantising and running the whole
- * batch at once.  The paper has no counterpart (it measures with device-resident tensors).
- *   x, B, C, dt, y, final_state, status: HOST pointers (page-locked memory, or the copies neither
- *     overlap nor run asynchronously); layouts as in ssdi8_fwd_args_t; final_state, status may be NULL.
- *   A, D, corr, the six step-size vectors, init_state: DEVICE pointers (D, corr, init_state may be NULL).
- *   scratch: DEVICE, 256-byte aligned, ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes,
- *     owned by the caller (two stages of one batch element's tensors plus one workspace).
- * The call returns once everything is enqueued; `stream` is made to wait for the last copy, so
- * synchronising `stream` completes it.  flags: 0 or SSDI8_FLAG_INT8_STATE.  The side streams and
+/* The layer step as one call: Eq. 1 quantisation of fp32 x, B, C with the given static step sizes
+ * (ssdi8_quantize_act, mode 0) followed by ssdi8_chunk_scan_fwd.  The paper has no counterpart (its
+ * modules are separate kernels on device-resident tensors); the arithmetic is exactly that of
+ * the two calls it replaces, and so is the result.
+ *
+ * ssdi8_layer_fwd: every pointer is a DEVICE pointer.  The modules that do not depend on xq (the
+ *   quantisers of B and C, ChunkCumsum, ChunkBMM) run on a side stream under the quantiser of x;
+ *   the streams join before ChunkState.  workspace: 256-byte aligned,
+ *   ssdi8_layer_fwd_workspace_bytes(dims, flags) bytes (the int8 tensors plus ssdi8_workspace_bytes).
+ * ssdi8_layer_fwd_host: x, B, C, dt, y, final_state, status are HOST pointers (page-locked memory, or
+ *   the copies neither overlap nor run asynchronously), the rest DEVICE pointers.  One batch element
+ *   at a time (Algorithm 2 has no cross-batch term): the host->device copies of element b+1 and the
+ *   device->host copy of y of element b-1 run on two more side streams while the kernels of element
+ *   b run, so both directions of the host link stay busy.  scratch: DEVICE, 256-byte aligned,
+ *   ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes (two stages of one element's tensors).
+ * Layouts as in ssdi8_fwd_args_t; D, corr, init_state, final_state, status may be NULL.  Both calls
+ * return once everything is enqueued and leave `stream` waiting for the last piece of work, so
+ * synchronising `stream` completes them.  flags: 0 or SSDI8_FLAG_INT8_STATE.  The side streams and
  * events are created at the first call on each device and shared by later calls: calls on one
  * device must not overlap in time.  Errors: as ssdi8_quantize_act / ssdi8_chunk_scan_fwd, plus
- * SSDI8_ERR_WORKSPACE for a short scratch. */
+ * SSDI8_ERR_WORKSPACE for a short workspace or scratch. */
 typedef struct {
-  const float* x; const float* B; const float* C; const float* dt;            /* HOST   */
-  const float* A; const float* D; const float* corr;                          /* DEVICE */
-  const float* s_x; const float* s_B; const float* s_C;                       /* DEVICE */
-  const float* s_xs; const float* s_cb; const float* s_h;                     /* DEVICE */
-  const float* init_state;                                                    /* DEVICE */
-  float* y; float* final_state; int32_t* status;                              /* HOST   */
-} ssdi8_host_args_t;
+  const float* x; const float* B; const float* C; const float* dt;   /* [B,L,H,P], [B,L,G,N] x2, [B,L,H] */
+  const float* A; const float* D; const float* corr;                 /* [H], [H], [H*P]                   */
+  const float* s_x; const float* s_B; const float* s_C;              /* step sizes of x, B, C             */
+  const float* s_xs; const float* s_cb; const float* s_h;            /* internal step sizes               */
+  const float* init_state;                                           /* [B,H,P,N]                         */
+  float* y; float* final_state; int32_t* status;                     /* [B,L,H,P], [B,H,P,N], 1 word      */
+} ssdi8_layer_args_t;
+size_t ssdi8_layer_fwd_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags);
+ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_t* args, void* workspace,
+                               size_t workspace_bytes, uint32_t flags, void* stream);
 size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t flags);
-ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_host_args_t* args, void* scratch,
+ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_args_t* args, void* scratch,
                                     size_t scratch_bytes, uint32_t flags, void* stream);
 
 /* Static calibration of the internal step sizes (Eq. 1 applied once to the internal

@@ -32,6 +32,7 @@ EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
            "ssdi8_chunk_scan_fwd", "ssdi8_chunk_scan_fwd_static", "ssdi8_calibrate",
            "ssdi8_state_passing", "ssdi8_ssd_step", "ssdi8_mean_correction",
            "ssdi8_mean_correction_workspace_bytes", "ssdi8_quantize_entry",
+           "ssdi8_layer_fwd", "ssdi8_layer_fwd_workspace_bytes",
            "ssdi8_layer_fwd_host", "ssdi8_layer_fwd_host_scratch_bytes")
 STATIC_WORKSPACE_BYTES = 16 << 20
 
@@ -51,15 +52,15 @@ class FwdArgs(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in _FWD_FIELDS]
 
 
-_HOST_FIELDS = ("x", "B", "C", "dt", "A", "D", "corr", "s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h",
+_LAYER_FIELDS = ("x", "B", "C", "dt", "A", "D", "corr", "s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h",
                 "init_state", "y", "final_state", "status")
 
 
 _HOST_SIDE = ("x", "B", "C", "dt", "y", "final_state", "status")
 
 
-class HostArgs(C.Structure):
-    _fields_ = [(k, C.c_void_p) for k in _HOST_FIELDS]
+class LayerArgs(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in _LAYER_FIELDS]
 
 
 _lib.ssdi8_status_string.restype = C.c_char_p
@@ -165,18 +166,24 @@ def ssdi8_calibrate(dims: Dims, args: FwdArgs, s_xs, s_cb, s_h, workspace, strea
 
 _lib.ssdi8_layer_fwd_host_scratch_bytes.restype = C.c_size_t
 _lib.ssdi8_layer_fwd_host_scratch_bytes.argtypes = [C.POINTER(Dims), C.c_uint32]
+_lib.ssdi8_layer_fwd_workspace_bytes.restype = C.c_size_t
+_lib.ssdi8_layer_fwd_workspace_bytes.argtypes = [C.POINTER(Dims), C.c_uint32]
+_lib.ssdi8_layer_fwd.restype = C.c_int32
+_lib.ssdi8_layer_fwd.argtypes = [C.POINTER(Dims), C.POINTER(LayerArgs), C.c_void_p, C.c_size_t, C.c_uint32,
+                                 C.c_void_p]
 _lib.ssdi8_layer_fwd_host.restype = C.c_int32
-_lib.ssdi8_layer_fwd_host.argtypes = [C.POINTER(Dims), C.POINTER(HostArgs), C.c_void_p, C.c_size_t, C.c_uint32,
+_lib.ssdi8_layer_fwd_host.argtypes = [C.POINTER(Dims), C.POINTER(LayerArgs), C.c_void_p, C.c_size_t, C.c_uint32,
                                       C.c_void_p]
 
 
-def make_host_args(**tensors) -> HostArgs:
-    """x, B, C, dt, y, final_state, status: host tensors (pinned); the rest: device tensors."""
-    a = HostArgs()
+def make_layer_args(host: bool = False, **tensors) -> LayerArgs:
+    """Arguments of ssdi8_layer_fwd (host=False: all device tensors) or ssdi8_layer_fwd_host
+    (host=True: x, B, C, dt, y, final_state, status are host tensors, pinned; the rest device tensors)."""
+    a = LayerArgs()
     for k, v in tensors.items():
-        if k not in _HOST_FIELDS:
+        if k not in _LAYER_FIELDS:
             raise KeyError(k)
-        if k in _HOST_SIDE and v is not None:
+        if host and k in _HOST_SIDE and v is not None:
             assert not v.is_cuda and v.is_contiguous(), f"{k} must be a contiguous host tensor"
             setattr(a, k, v.data_ptr())
         else:
@@ -185,11 +192,25 @@ def make_host_args(**tensors) -> HostArgs:
     return a
 
 
+def make_host_args(**tensors) -> LayerArgs:
+    return make_layer_args(host=True, **tensors)
+
+
+def ssdi8_layer_fwd_workspace_bytes(dims: Dims, flags: int = 0) -> int:
+    return int(_lib.ssdi8_layer_fwd_workspace_bytes(C.byref(dims), flags))
+
+
+def ssdi8_layer_fwd(dims: Dims, args: LayerArgs, workspace, flags: int = 0, stream=None) -> None:
+    _check(_lib.ssdi8_layer_fwd(C.byref(dims), C.byref(args), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), flags, _stream(stream)),
+           "ssdi8_layer_fwd")
+
+
 def ssdi8_layer_fwd_host_scratch_bytes(dims: Dims, flags: int = 0) -> int:
     return int(_lib.ssdi8_layer_fwd_host_scratch_bytes(C.byref(dims), flags))
 
 
-def ssdi8_layer_fwd_host(dims: Dims, args: HostArgs, scratch, flags: int = 0, stream=None) -> None:
+def ssdi8_layer_fwd_host(dims: Dims, args: LayerArgs, scratch, flags: int = 0, stream=None) -> None:
     _check(_lib.ssdi8_layer_fwd_host(C.byref(dims), C.byref(args), _ptr(scratch),
                                      scratch.numel() * scratch.element_size(), flags, _stream(stream)),
            "ssdi8_layer_fwd_host")

@@ -97,6 +97,14 @@ ssdi8_status_t ssdi8_quantize_act(const float* in, int64_t R, int64_t Ch, int64_
 ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a,
                                     uint32_t flags, void* workspace, size_t workspace_bytes,
                                     void* stream) {
+  return ssdi8::fwd_phases(dims, a, flags, workspace, workspace_bytes, stream, true);
+}
+
+}  // extern "C"
+
+namespace ssdi8 {
+ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
+                          size_t workspace_bytes, void* stream, bool clear_status) {
   if (!dims || !a) return SSDI8_ERR_NULL;
   if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) != 0) return SSDI8_ERR_UNSUPPORTED;
   const bool i8s = (flags & SSDI8_FLAG_INT8_STATE) != 0;
@@ -126,7 +134,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
   int8_t* cbq = a->tap_CBq ? a->tap_CBq : reinterpret_cast<int8_t*>(ws + w.cbq);
   float* loc = a->tap_loc ? a->tap_loc : reinterpret_cast<float*>(ws + w.loc);
   int8_t* hq = a->tap_hq ? a->tap_hq : reinterpret_cast<int8_t*>(ws + w.hq);
-  if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
+  if (a->status && clear_status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
 
   if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st)) != SSDI8_OK)
     return s;
@@ -157,6 +165,9 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
   }
   return SSDI8_OK;
 }
+}  // namespace ssdi8
+
+extern "C" {
 
 ssdi8_status_t ssdi8_calibrate(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, float* s_xs,
                                float* s_cb, float* s_h, void* workspace, size_t workspace_bytes,

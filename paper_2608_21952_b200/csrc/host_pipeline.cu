@@ -1,5 +1,9 @@
-// Layer forward from HOST buffers: Eq. 1 quantisation of fp32 x, B, C with static step sizes and
-// the SSD layer forward (Algorithm 2), one batch element at a time.  Batch elements are
+// The layer step as one call: Eq. 1 quantisation of fp32 x, B, C with static step sizes and the SSD
+// layer forward (Algorithm 2).
+// ssdi8_layer_fwd (device buffers): the modules that do not depend on xq (the quantisers of B and C,
+// ChunkCumsum, ChunkBMM; all latency-bound) run on a side stream under the HBM-bound quantiser of
+// x, then the two streams join for ChunkState/StatePassing and ChunkScan.
+// ssdi8_layer_fwd_host (host buffers): the same, one batch element at a time.  Batch elements are
 // independent, so the host->device copies of element b+1 and the device->host copy of the
 // output of element b-1 run on two side streams while the kernels of element b run on the
 // caller's stream: the PCIe link is busy in both directions for the whole call instead of
@@ -52,8 +56,9 @@ Layout make_layout(const ssdi8_dims_t& d1, uint8_t* base, uint32_t flags) {
 // side streams and events, made once per device and kept for the life of the process
 struct Plumbing {
   bool ready = false;
-  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaStream_t s_in = nullptr, s_out = nullptr, s_side = nullptr;
   cudaEvent_t start = nullptr, in_done[kStages] = {}, cmp_done[kStages] = {}, out_done[kStages] = {};
+  cudaEvent_t fork = nullptr, join = nullptr;
 };
 Plumbing g_plumb[64];
 
@@ -65,7 +70,14 @@ ssdi8_status_t get_plumbing(Plumbing** out) {
   if (!p.ready) {
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+    // the side stream carries short latency-bound kernels: highest priority, so that their blocks are
+    // placed as soon as the bandwidth-bound quantiser of x frees a slot instead of behind its whole grid
+    int prio_lo = 0, prio_hi = 0;
+    SSDI8_CUDA_CHECK(cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
+    SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side, cudaStreamNonBlocking, prio_hi));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming));
+    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming));
     for (int s = 0; s < kStages; ++s) {
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.in_done[s], cudaEventDisableTiming));
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.cmp_done[s], cudaEventDisableTiming));
@@ -77,12 +89,91 @@ ssdi8_status_t get_plumbing(Plumbing** out) {
   return SSDI8_OK;
 }
 
+struct LayerWs {
+  int8_t *xq, *Bq, *Cq;
+  void* ws;
+  size_t ws_bytes, total;
+};
+LayerWs layer_ws(const ssdi8_dims_t& d, uint8_t* base, uint32_t flags) {
+  LayerWs w;
+  const size_t nx = (size_t)d.batch * d.seqlen * d.nheads * d.headdim;
+  const size_t nb = (size_t)d.batch * d.seqlen * d.ngroups * d.dstate;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { uint8_t* p = base + o; o = up256(o + bytes); return p; };
+  w.xq = reinterpret_cast<int8_t*>(take(nx));
+  w.Bq = reinterpret_cast<int8_t*>(take(nb));
+  w.Cq = reinterpret_cast<int8_t*>(take(nb));
+  w.ws_bytes = ssdi8_workspace_bytes(&d, flags);
+  w.ws = take(w.ws_bytes);
+  w.total = o;
+  return w;
+}
+
+// quantisers + forward on device tensors, int8 tensors and workspace given; status cleared by the caller
+ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, const float* x, const float* B,
+                          const float* C, const float* dt, const float* init, float* y, float* fin,
+                          int32_t* status, int8_t* xq, int8_t* Bq, int8_t* Cq, void* ws, size_t ws_bytes,
+                          uint32_t flags, Plumbing& p, cudaStream_t st) {
+  const int64_t T = (int64_t)d.batch * d.seqlen;
+  ssdi8_fwd_args_t f = {};
+  f.xq = xq; f.Bq = Bq; f.Cq = Cq;
+  f.s_x = a.s_x; f.s_B = a.s_B; f.s_C = a.s_C;
+  f.dt = dt; f.A = a.A; f.D = a.D; f.corr = a.corr;
+  f.s_xs = a.s_xs; f.s_cb = a.s_cb; f.s_h = a.s_h;
+  f.init_state = init; f.y = y; f.final_state = fin; f.status = status;
+  const uint32_t fl = flags & (uint32_t)SSDI8_FLAG_INT8_STATE;
+  ssdi8_status_t s;
+  SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork, 0));
+  // side stream: everything that does not need xq
+  if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, p.s_side)) != SSDI8_OK) return s;
+  if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, p.s_side)) != SSDI8_OK) return s;
+  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM | SSDI8_PHASE_BMM, ws, ws_bytes, p.s_side, false)) != SSDI8_OK)
+    return s;
+  SSDI8_CUDA_CHECK(cudaEventRecord(p.join, p.s_side));
+  // caller's stream: the quantiser of x, then the modules that need everything
+  if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
+    return s;
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join, 0));
+  return fwd_phases(&d, &f, fl | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING | SSDI8_PHASE_SCAN, ws,
+                    ws_bytes, st, false);
+}
+
+bool layer_args_ok(const ssdi8_layer_args_t* a) {
+  return a->x && a->B && a->C && a->dt && a->A && a->s_x && a->s_B && a->s_C && a->s_xs && a->s_cb && a->s_h && a->y;
+}
+
 }  // namespace
 }  // namespace ssdi8
 
 using namespace ssdi8;
 
 extern "C" {
+
+size_t ssdi8_layer_fwd_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
+  if (!dims || dims->batch <= 0 || (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE)) return 0;
+  if (ssdi8_workspace_bytes(dims, flags) == 0) return 0;
+  return layer_ws(*dims, nullptr, flags).total;
+}
+
+ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_t* a, void* workspace,
+                               size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (!dims || !a || !workspace) return SSDI8_ERR_NULL;
+  if (!layer_args_ok(a)) return SSDI8_ERR_NULL;
+  if (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE) return SSDI8_ERR_UNSUPPORTED;
+  const size_t need = ssdi8_layer_fwd_workspace_bytes(dims, flags);
+  if (need == 0) return SSDI8_ERR_SHAPE;
+  if (workspace_bytes < need) return SSDI8_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return SSDI8_ERR_ALIGN;
+  const LayerWs w = layer_ws(*dims, static_cast<uint8_t*>(workspace), flags);
+  Plumbing* p = nullptr;
+  ssdi8_status_t s = get_plumbing(&p);
+  if (s != SSDI8_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
+  return layer_step(*dims, *a, a->x, a->B, a->C, a->dt, a->init_state, a->y, a->final_state, a->status, w.xq, w.Bq,
+                    w.Cq, w.ws, w.ws_bytes, flags, *p, st);
+}
 
 size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
   if (!dims || dims->batch <= 0) return 0;
@@ -92,12 +183,10 @@ size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t fla
   return make_layout(d1, nullptr, flags).total;
 }
 
-ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_host_args_t* a, void* scratch,
+ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_args_t* a, void* scratch,
                                     size_t scratch_bytes, uint32_t flags, void* stream) {
   if (!dims || !a || !scratch) return SSDI8_ERR_NULL;
-  if (!a->x || !a->B || !a->C || !a->dt || !a->A || !a->s_x || !a->s_B || !a->s_C || !a->s_xs || !a->s_cb ||
-      !a->s_h || !a->y)
-    return SSDI8_ERR_NULL;
+  if (!layer_args_ok(a)) return SSDI8_ERR_NULL;
   if (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE) return SSDI8_ERR_UNSUPPORTED;
   const size_t need = ssdi8_layer_fwd_host_scratch_bytes(dims, flags);
   if (need == 0) return SSDI8_ERR_SHAPE;
@@ -112,7 +201,6 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_host_a
   cudaStream_t s_cmp = static_cast<cudaStream_t>(stream);
   const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
   const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
-  const int64_t T1 = d1.seqlen;
 
   // everything below is ordered after the work already in the caller's stream
   SSDI8_CUDA_CHECK(cudaMemsetAsync(lo.status, 0, sizeof(int32_t), s_cmp));
@@ -133,22 +221,9 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_host_a
     // kernels of element b: its inputs have arrived, and y of element b - kStages has left
     SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->in_done[st], 0));
     if (b >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
-    s = ssdi8_quantize_act(sb.x, T1, (int64_t)d1.nheads * d1.headdim, 1, const_cast<float*>(a->s_x), 0, sb.xq, s_cmp);
-    if (s != SSDI8_OK) return s;
-    s = ssdi8_quantize_act(sb.B, T1, d1.ngroups, d1.dstate, const_cast<float*>(a->s_B), 0, sb.Bq, s_cmp);
-    if (s != SSDI8_OK) return s;
-    s = ssdi8_quantize_act(sb.C, T1, d1.ngroups, d1.dstate, const_cast<float*>(a->s_C), 0, sb.Cq, s_cmp);
-    if (s != SSDI8_OK) return s;
-    ssdi8_fwd_args_t f = {};
-    f.xq = sb.xq; f.Bq = sb.Bq; f.Cq = sb.Cq;
-    f.s_x = a->s_x; f.s_B = a->s_B; f.s_C = a->s_C;
-    f.dt = sb.dt; f.A = a->A; f.D = a->D; f.corr = a->corr;
-    f.s_xs = a->s_xs; f.s_cb = a->s_cb; f.s_h = a->s_h;
-    f.init_state = a->init_state ? a->init_state + (size_t)b * nfin : nullptr;
-    f.y = sb.y;
-    f.final_state = a->final_state ? sb.fin : nullptr;
-    f.status = lo.status;
-    s = ssdi8_chunk_scan_fwd(&d1, &f, flags, lo.ws, lo.ws_bytes, s_cmp);
+    s = layer_step(d1, *a, sb.x, sb.B, sb.C, sb.dt, a->init_state ? a->init_state + (size_t)b * nfin : nullptr,
+                   sb.y, a->final_state ? sb.fin : nullptr, lo.status, sb.xq, sb.Bq, sb.Cq, lo.ws, lo.ws_bytes, flags,
+                   *p, s_cmp);
     if (s != SSDI8_OK) return s;
     SSDI8_CUDA_CHECK(cudaEventRecord(p->cmp_done[st], s_cmp));
     // outputs of element b

@@ -17,6 +17,11 @@ ssdi8_status_t launch_quantize_entry(const void* xBC, int dtype, i64 T_, int D, 
                                      const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq, int8_t* Cq,
                                      cudaStream_t st);
 
+// ssdi8_chunk_scan_fwd's body; clear_status = false leaves the status word alone (callers that run
+// the modules as several calls clear it once themselves)
+ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
+                          size_t workspace_bytes, void* stream, bool clear_status);
+
 // pack [b,H,c,6,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
                              float* gamma, float* tap_cs, cudaStream_t st);
