@@ -124,7 +124,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       // lut[s] was last read for chunk k-2, which every thread of this group has left
       for (int i = qt; i < Q; i += kQuantThreads) lut[i] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + i];
       named_bar(2, kQuantThreads);
-      mbar_wait(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+      mbar_wait_relaxed(&bars[B_FULL + s], (k >> 1) & 1, a.status);
 #pragma unroll 1
       for (int i = qt >> 2; i < Q; i += kQuantThreads / 4) {
         uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
@@ -159,7 +159,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       // and the state warps have read the previous accumulator (overlaps their hq staging)
       if (qt == 0) {
         mbar_wait(&bars[B_RQ + s], (k >> 1) & 1, a.status);
-        mbar_wait(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);
+        mbar_wait_relaxed(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);
         tc_fence_after();
         const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
         const uint32_t idesc = idesc_s8(N, 64, 1, 1);
@@ -225,7 +225,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
         tma_store_commit();
       }
       // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 16 channels at a time
-      mbar_wait(&bars[B_MMA], k & 1, a.status);
+      mbar_wait_relaxed(&bars[B_MMA], k & 1, a.status);
       tc_fence_after();
       if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
 #pragma unroll
