@@ -410,6 +410,12 @@ def run_ours(args):
         dom = max((k for k in kernel_ms if k != "quantize"), key=lambda k: kernel_ms[k])
         entry_ms = layer.entry_fused_ms(max(5, min(args.steps, 20)))
         ms_separate = layer.timed(layer.step_separate, max(5, min(args.steps, 20)))
+        # the scan kernel with the paper's 16-bit output format (beside the step, which keeps fp32 y)
+        y16 = torch.empty(layer.y.shape, dtype=torch.bfloat16, device="cuda")
+        args16 = bd.make_fwd_args(**{**layer.args._keepalive, "y": y16})
+        scan16 = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args16, layer.ws, flags=bd.PHASE_SCAN | bd.FLAG_Y_BF16)
+        scan16(); torch.cuda.synchronize()
+        kernel_ms["chunk_scan_bf16_y"] = layer.timed(scan16, max(5, min(args.steps, 20)))
         alg = scan_algorithmic_bytes(cfg)
         scan_gbs = alg / (kernel_ms["chunk_scan"] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "chunk_scan", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],

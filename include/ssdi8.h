@@ -72,6 +72,10 @@ enum {
 /* state format bit of ssdi8_chunk_scan_fwd's flags */
 enum { SSDI8_FLAG_INT8_STATE = 1u << 1 };
 
+/* output format bits (at most one): y is written as 16-bit elements, the paper's own output
+ * format being FP16 (Algorithm 2 keeps Y in half precision); default is binary32 */
+enum { SSDI8_FLAG_Y_FP16 = 1u << 2, SSDI8_FLAG_Y_BF16 = 1u << 3 };
+
 /* host, pure: static string for a status code */
 const char* ssdi8_status_string(ssdi8_status_t s);
 
@@ -170,6 +174,9 @@ typedef struct {
  *                y_diag = (s_cb rowmax_i / 127) s_x acc_diag
  *  Output        y = y_off + y_diag + D s_x xq + corr
  * flags: bit 0 is reserved for the paper's FP16 ChunkScan2 operand and must be 0.
+ * SSDI8_FLAG_Y_FP16 / SSDI8_FLAG_Y_BF16: `y` points to [B,L,H,P] 16-bit elements; each binary32
+ * output value is rounded to nearest even into that format (fp16 overflows to infinity) as it
+ * leaves the epilogue, which halves the largest byte stream of the layer.  Not combinable with taps.
  * SSDI8_FLAG_INT8_STATE selects the paper's own inter-chunk state format (Section 4.2, Eq. 4, 7)
  * instead of fp32 states: the chunk-local state goes INT32 -> INT8 in registers and the
  * recurrence is integer with a fixed-point decay, all states sharing the scale s_h[h,p]:
@@ -223,7 +230,8 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  *   ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes (two stages of one element's tensors).
  * Layouts as in ssdi8_fwd_args_t; D, corr, init_state, final_state, status may be NULL.  Both calls
  * return once everything is enqueued and leave `stream` waiting for the last piece of work, so
- * synchronising `stream` completes them.  flags: 0 or SSDI8_FLAG_INT8_STATE.  The side streams and
+ * synchronising `stream` completes them.  flags: any of SSDI8_FLAG_INT8_STATE, SSDI8_FLAG_Y_FP16,
+ * SSDI8_FLAG_Y_BF16 (`y` then points to 16-bit elements).  The side streams and
  * events are created at the first call on each device and shared by later calls: calls on one
  * device must not overlap in time.  Errors: as ssdi8_quantize_act / ssdi8_chunk_scan_fwd, plus
  * SSDI8_ERR_WORKSPACE for a short workspace or scratch. */

@@ -26,6 +26,7 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TI
     -1, -2, -3, -4, -5, -6, -7, -8
 
 FLAG_INT8_STATE = 1 << 1
+FLAG_Y_FP16, FLAG_Y_BF16 = 1 << 2, 1 << 3
 PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1 << k for k in range(8, 13))
 
 EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",

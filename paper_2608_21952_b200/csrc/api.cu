@@ -76,7 +76,7 @@ const char* ssdi8_status_string(ssdi8_status_t s) {
 }
 
 size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) != 0 || !dims_supported(dims, true)) return 0;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0 || !dims_supported(dims, true)) return 0;
   return layout(make_dims(dims)).total;
 }
 
@@ -106,8 +106,11 @@ namespace ssdi8 {
 ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
                           size_t workspace_bytes, void* stream, bool clear_status) {
   if (!dims || !a) return SSDI8_ERR_NULL;
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) != 0) return SSDI8_ERR_UNSUPPORTED;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0) return SSDI8_ERR_UNSUPPORTED;
   const bool i8s = (flags & SSDI8_FLAG_INT8_STATE) != 0;
+  if ((flags & SSDI8_FLAG_Y_FP16) && (flags & SSDI8_FLAG_Y_BF16)) return SSDI8_ERR_UNSUPPORTED;
+  const int ydt = (flags & SSDI8_FLAG_Y_FP16) ? 1 : (flags & SSDI8_FLAG_Y_BF16) ? 2 : 0;
+  if (ydt && (a->tap_acc_off || a->tap_rowmax || a->tap_Mq || a->tap_acc_diag)) return SSDI8_ERR_UNSUPPORTED;
   const uint32_t ph = (flags & SSDI8_PHASE_ALL) ? (flags & SSDI8_PHASE_ALL) : (uint32_t)SSDI8_PHASE_ALL;
   // the INT8 state lives inside the fused ChunkState + StatePassing kernel only
   if (i8s && ((ph & SSDI8_PHASE_CHUNK_STATE) != 0) != ((ph & SSDI8_PHASE_STATE_PASSING) != 0))
@@ -161,7 +164,7 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
     return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack,
-                             a->D, a->corr, a->y, a->status, taps, st);
+                             a->D, a->corr, a->y, ydt, a->status, taps, st);
   }
   return SSDI8_OK;
 }
@@ -294,7 +297,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
   if (!dims || !args) return SSDI8_ERR_NULL;
   const size_t need = ssdi8_workspace_bytes(dims, flags);
   if (need == 0)
-    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
+    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
   if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
   static void* ws_of_device[64];  // resolved address of g_static_ws, per device
   int dev = 0;

@@ -14,6 +14,9 @@
 // (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
 // hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
 // because every role executes different code at the same time.  No multicast; bounded waits.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -250,8 +253,9 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
   }
 }
 
-// CORR: a mean-correction vector is given; TAPS: intermediate tensors are written out (tests)
-template <bool CORR, bool TAPS>
+// CORR: a mean-correction vector is given; TAPS: intermediate tensors are written out (tests);
+// YT: format of y (0 binary32, 1 fp16, 2 bf16: rounded to nearest even on the way to the staging tile)
+template <bool CORR, bool TAPS, int YT>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
               const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
@@ -429,7 +433,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
       if (lane == 3) tma_store_wait_read();  // last tile's store has finished reading the staging tile
       __syncwarp();
-      uint8_t* srow = ystage + lane * 128;
+      uint8_t* srow = ystage + lane * (YT ? 64 : 128);
 #pragma unroll 1
       for (int pc = 0; pc < 4; ++pc) {       // 8 columns at a time (keeps the accumulators in registers)
         int acc_o[8], acc_d[8];
@@ -441,11 +445,11 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
           const uint2 xr = *reinterpret_cast<const uint2*>(
               sX + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + (pc >> 1)), 64) + (pc & 1) * 8);
           const uint32_t xw[2] = {xr.x ^ 0x80808080u, xr.y ^ 0x80808080u};
+          float2 v[4];
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
             const float4 sx4 = __ldg(gsx + pc * 2 + cc), sh4 = __ldg(gsh + pc * 2 + cc);
             const float4 co4 = CORR ? __ldg(gco + pc * 2 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
-            float2 v[2];
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
               const int pp = cc * 4 + e2 * 2;
@@ -457,10 +461,25 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
               const float2 ad = make_float2((float)acc_d[pp], (float)acc_d[pp + 1]);
               float2 r2 = __ffma2_rn(__fmul2_rn(Dh2, sx2), xv, co2);
               r2 = __ffma2_rn(__fmul2_rn(sm2, sx2), ad, r2);
-              v[e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
+              v[cc * 2 + e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
             }
-            *reinterpret_cast<float4*>(srow + (((pc * 2 + cc) ^ (lane & 7)) << 4)) =
-                make_float4(v[0].x, v[0].y, v[1].x, v[1].y);
+            if (YT == 0)
+              *reinterpret_cast<float4*>(srow + (((pc * 2 + cc) ^ (lane & 7)) << 4)) =
+                  make_float4(v[cc * 2].x, v[cc * 2].y, v[cc * 2 + 1].x, v[cc * 2 + 1].y);
+          }
+          if (YT != 0) {  // 8 values = one 16-byte chunk of the [32][64 B] staging tile (64-byte swizzle)
+            uint32_t h[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (YT == 1) {
+                const __half2 hv = __floats2half2_rn(v[e].x, v[e].y);
+                h[e] = *reinterpret_cast<const uint32_t*>(&hv);
+              } else {
+                const __nv_bfloat162 bv = __floats2bfloat162_rn(v[e].x, v[e].y);
+                h[e] = *reinterpret_cast<const uint32_t*>(&bv);
+              }
+            }
+            *reinterpret_cast<uint4*>(srow + ((pc ^ ((lane >> 1) & 3)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
           }
           if (TAPS && (a.taps.acc_off || a.taps.acc_diag)) {
             const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 8;
@@ -498,7 +517,7 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
                                  const int8_t* CBq, const int8_t* hq, const float* s_x,
                                  const float* s_C, const float* s_cb, const float* s_h,
                                  const float* pack, const float* D,
-                                 const float* corr, float* y, int32_t* status, const ScanTaps& taps,
+                                 const float* corr, void* y, int ydt, int32_t* status, const ScanTaps& taps,
                                  cudaStream_t st) {
   const int TM = d.Q < 128 ? d.Q : 128;
   const uint64_t T = (uint64_t)d.b * d.L;
@@ -528,10 +547,11 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
     if (!encode_tensor_map(&tm_cb, CBq, 1, 2, dims, str, box, TM)) return SSDI8_ERR_CUDA;
   }
   {
+    const uint64_t eb = ydt ? 2 : 4;  // bytes per element of y
     uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
-    uint64_t str[2] = {(uint64_t)d.P * 4, (uint64_t)d.H * d.P * 4};
+    uint64_t str[2] = {(uint64_t)d.P * eb, (uint64_t)d.H * d.P * eb};
     uint32_t box[3] = {32, 1, 32};
-    if (!encode_tensor_map(&tm_y, y, 4, 3, dims, str, box, 128)) return SSDI8_ERR_CUDA;
+    if (!encode_tensor_map(&tm_y, y, (int)eb, 3, dims, str, box, ydt ? 64 : 128)) return SSDI8_ERR_CUDA;
   }
   int dev = 0, sms = 0;
   SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
@@ -549,11 +569,16 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
     kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
     return SSDI8_OK;
   };
+  if (tp && ydt) return SSDI8_ERR_UNSUPPORTED;  // the taps come with binary32 y only
   ssdi8_status_t ls;
-  if (corr)
-    ls = tp ? launch(chunk_scan_tc<true, true>) : launch(chunk_scan_tc<true, false>);
+  if (tp)
+    ls = corr ? launch(chunk_scan_tc<true, true, 0>) : launch(chunk_scan_tc<false, true, 0>);
+  else if (ydt == 0)
+    ls = corr ? launch(chunk_scan_tc<true, false, 0>) : launch(chunk_scan_tc<false, false, 0>);
+  else if (ydt == 1)
+    ls = corr ? launch(chunk_scan_tc<true, false, 1>) : launch(chunk_scan_tc<false, false, 1>);
   else
-    ls = tp ? launch(chunk_scan_tc<false, true>) : launch(chunk_scan_tc<false, false>);
+    ls = corr ? launch(chunk_scan_tc<true, false, 2>) : launch(chunk_scan_tc<false, false, 2>);
   if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;

@@ -15,6 +15,7 @@ namespace ssdi8 {
 namespace {
 
 constexpr int kStages = 2;
+constexpr uint32_t kLayerFlags = SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16;
 
 struct StageBuf {
   float *x, *B, *C, *dt, *y, *fin;
@@ -121,7 +122,7 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
   f.dt = dt; f.A = a.A; f.D = a.D; f.corr = a.corr;
   f.s_xs = a.s_xs; f.s_cb = a.s_cb; f.s_h = a.s_h;
   f.init_state = init; f.y = y; f.final_state = fin; f.status = status;
-  const uint32_t fl = flags & (uint32_t)SSDI8_FLAG_INT8_STATE;
+  const uint32_t fl = flags & kLayerFlags;
   ssdi8_status_t s;
   SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork, 0));
@@ -151,7 +152,7 @@ using namespace ssdi8;
 extern "C" {
 
 size_t ssdi8_layer_fwd_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
-  if (!dims || dims->batch <= 0 || (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE)) return 0;
+  if (!dims || dims->batch <= 0 || (flags & ~kLayerFlags)) return 0;
   if (ssdi8_workspace_bytes(dims, flags) == 0) return 0;
   return layer_ws(*dims, nullptr, flags).total;
 }
@@ -160,7 +161,7 @@ ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_
                                size_t workspace_bytes, uint32_t flags, void* stream) {
   if (!dims || !a || !workspace) return SSDI8_ERR_NULL;
   if (!layer_args_ok(a)) return SSDI8_ERR_NULL;
-  if (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE) return SSDI8_ERR_UNSUPPORTED;
+  if (flags & ~kLayerFlags) return SSDI8_ERR_UNSUPPORTED;
   const size_t need = ssdi8_layer_fwd_workspace_bytes(dims, flags);
   if (need == 0) return SSDI8_ERR_SHAPE;
   if (workspace_bytes < need) return SSDI8_ERR_WORKSPACE;
@@ -187,7 +188,7 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
                                     size_t scratch_bytes, uint32_t flags, void* stream) {
   if (!dims || !a || !scratch) return SSDI8_ERR_NULL;
   if (!layer_args_ok(a)) return SSDI8_ERR_NULL;
-  if (flags & ~(uint32_t)SSDI8_FLAG_INT8_STATE) return SSDI8_ERR_UNSUPPORTED;
+  if (flags & ~kLayerFlags) return SSDI8_ERR_UNSUPPORTED;
   const size_t need = ssdi8_layer_fwd_host_scratch_bytes(dims, flags);
   if (need == 0) return SSDI8_ERR_SHAPE;
   if (scratch_bytes < need) return SSDI8_ERR_WORKSPACE;
@@ -202,6 +203,7 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
   const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
   const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
 
+  const size_t yb = (flags & (SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? 2 : 4;  // bytes per element of y
   // everything below is ordered after the work already in the caller's stream
   SSDI8_CUDA_CHECK(cudaMemsetAsync(lo.status, 0, sizeof(int32_t), s_cmp));
   SSDI8_CUDA_CHECK(cudaEventRecord(p->start, s_cmp));
@@ -228,7 +230,8 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
     SSDI8_CUDA_CHECK(cudaEventRecord(p->cmp_done[st], s_cmp));
     // outputs of element b
     SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_out, p->cmp_done[st], 0));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->y + (size_t)b * nx, sb.y, nx * 4, cudaMemcpyDeviceToHost, p->s_out));
+    SSDI8_CUDA_CHECK(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(a->y) + (size_t)b * nx * yb, sb.y, nx * yb,
+                                     cudaMemcpyDeviceToHost, p->s_out));
     if (a->final_state)
       SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->final_state + (size_t)b * nfin, sb.fin, nfin * 4, cudaMemcpyDeviceToHost,
                                        p->s_out));

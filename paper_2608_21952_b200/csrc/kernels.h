@@ -63,7 +63,7 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
                                  const int8_t* CBq, const int8_t* hq, const float* s_x,
                                  const float* s_C, const float* s_cb, const float* s_h,
                                  const float* pack, const float* D,
-                                 const float* corr, float* y, int32_t* status,
+                                 const float* corr, void* y, int ydt, int32_t* status,
                                  const ScanTaps& taps, cudaStream_t st);
 
 ssdi8_status_t launch_ssd_step(const Dims& d, const int8_t* xq, const float* s_x,

@@ -470,3 +470,58 @@ def test_layer_fwd_host_rejects_a_short_scratch():
     with pytest.raises(bd.SSDi8Error) as e:
         bd.ssdi8_layer_fwd_host(dims, args, scratch)
     assert e.value.code == bd.ERR_WORKSPACE
+
+
+# --------------------------------------------------------------------------- 16-bit y
+@pytest.mark.parametrize("fmt", ["float16", "bfloat16"])
+@pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[3]], ids=lambda c: c.name)
+def test_fwd_16_bit_y(cfg, fmt):
+    """SSDI8_FLAG_Y_FP16 / _BF16: y leaves the epilogue rounded to nearest even into the 16-bit
+    format.  Checked two ways: bit for bit against the kernel's own binary32 y converted by the
+    library routine, and against the oracle's y within the fp32 tolerance plus half a 16-bit ulp."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    y_ref, fin_ref, _ = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                      q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], None)
+    y32, fin32, _ = gh.gpu_fwd(cfg, q, taps=())
+    td = getattr(torch, fmt)
+    flag = bd.FLAG_Y_FP16 if fmt == "float16" else bd.FLAG_Y_BF16
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    y16 = torch.full(t["x"].shape, float("nan"), dtype=td, device="cuda")
+    fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_fwd_args(y=y16, final_state=fin, status=status, **dv)
+    bd.ssdi8_chunk_scan_fwd(dims, args, bd.alloc_workspace(dims), flags=flag)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(fin.cpu().numpy(), fin32)
+    want = torch.from_numpy(y32).to(td)
+    assert torch.equal(y16.cpu().view(torch.int16), want.view(torch.int16))
+    half_ulp = 2.0 ** -11 if fmt == "float16" else 2.0 ** -8
+    err = np.abs(y16.float().cpu().numpy() - y_ref)
+    assert np.all(err <= Y_TOL * rms(y_ref) + 1.01 * half_ulp * np.abs(y_ref) + 1e-7)
+
+
+def test_16_bit_y_flags_are_exclusive_and_without_taps():
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SMALL[0]
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    y16 = torch.empty(t["x"].shape, dtype=torch.float16, device="cuda")
+    ws = bd.alloc_workspace(dims)
+    with pytest.raises(bd.SSDi8Error) as e:
+        bd.ssdi8_chunk_scan_fwd(dims, bd.make_fwd_args(y=y16, **dv), ws, flags=bd.FLAG_Y_FP16 | bd.FLAG_Y_BF16)
+    assert e.value.code == bd.ERR_UNSUPPORTED
+    tap = torch.zeros((cfg.batch, cfg.seqlen, cfg.nheads), device="cuda")
+    with pytest.raises(bd.SSDi8Error) as e:
+        bd.ssdi8_chunk_scan_fwd(dims, bd.make_fwd_args(y=y16, tap_rowmax=tap, **dv), ws, flags=bd.FLAG_Y_FP16)
+    assert e.value.code == bd.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
