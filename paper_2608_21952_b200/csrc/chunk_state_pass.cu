@@ -28,6 +28,7 @@ struct FusedArgs {
   const float* gamma; const float* init; float* final_state;
   float* tap_loc; float* tap_prev; int8_t* tap_Xsq; int32_t* tap_acc; int32_t* status;
   Dims d;
+  int n_full;  // CTAs below this index own a whole (batch, head); the rest own one 16-channel quarter of one
 };
 
 constexpr int kStateThreads = 256;   // warps 0-7: running state, hq, MMA issue, TMA
@@ -49,16 +50,17 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
 }
 
 // TAPS: any of the intermediate-tensor taps is requested (tests); the production instance carries no tap code
-template <bool I8S, bool TAPS>
-__global__ void __launch_bounds__(kThreads, 2)
-chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
-                    const __grid_constant__ CUtensorMap tm_hq, const FusedArgs a) {
+// NCQ: 16-channel chunks of the head this CTA owns (4 = the whole head, 1 = one quarter)
+template <bool I8S, bool TAPS, int NCQ>
+__device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtensorMap& tm_x, const CUtensorMap& tm_hq,
+                                           const FusedArgs& a, const int unit, const int c0) {
   extern __shared__ uint8_t smem_raw[];
+  constexpr int ncq = NCQ;
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const Dims& d = a.d;
   const int Q = d.Q, N = d.N, P = d.P;
   const int TQ = Q < 128 ? Q : 128;  // rows per TMA box
-  const int h = blockIdx.x, b = blockIdx.y;
+  const int h = unit % d.H, b = unit / d.H;
   const int g = h / (d.H / d.G);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
@@ -108,7 +110,8 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   if (tid >= kStateThreads) {
     // ------------------------------------------------------------ Q(X_scaled), one chunk ahead of the state warps
     const int qt = tid - kStateThreads;
-    const int c = qt & 3;  // 16-byte chunk (16 channels) of every row this thread visits
+    constexpr int lq = ncq == 4 ? 2 : 0;  // log2(chunks per row in this CTA's range)
+    const int c = c0 + (qt & (ncq - 1));  // 16-byte chunk (16 channels) of every row this thread visits
     float rx[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
@@ -126,7 +129,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       named_bar(2, kQuantThreads);
       mbar_wait_relaxed(&bars[B_FULL + s], (k >> 1) & 1, a.status);
 #pragma unroll 1
-      for (int i = qt >> 2; i < Q; i += kQuantThreads / 4) {
+      for (int i = qt >> lq; i < Q; i += kQuantThreads >> lq) {
         uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
         const uint4 w4 = *ptr;
         const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
@@ -175,14 +178,16 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     // M = 128: accumulator row n on TMEM lane n; M = 64: row n on lane (n % 16) + 32 (n / 16),
     // i.e. the first 16 lanes of each warp's quarter
     const int q = warp & 3, ch = warp >> 2;
+    constexpr int npp = 8 * ncq;             // channels per thread
+    const int cb = 16 * c0 + ch * npp;       // first channel of this thread
     const bool ok = (N == 128) || (lane < 16);
     const int n = (N == 128) ? q * 32 + lane : q * 16 + lane;
     float S[32];  // fp32 state, or (I8S) the bit pattern of the integer code
 #pragma unroll
     for (int pp = 0; pp < 32; ++pp) {
-      const float v = (a.init && ok) ? a.init[(bh * P + ch * 32 + pp) * N + n] : 0.f;
+      const float v = (a.init && ok && pp < npp) ? a.init[(bh * P + cb + pp) * N + n] : 0.f;
       if (I8S)
-        S[pp] = __int_as_float((int)(int8_t)(rne_clamp_bits(__fmul_rn(v, col_invh[ch * 32 + pp])) & 0xffu));
+        S[pp] = __int_as_float((int)(int8_t)(rne_clamp_bits(__fmul_rn(v, col_invh[(cb + pp) & 63])) & 0xffu));
       else
         S[pp] = v;
     }
@@ -197,31 +202,35 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       named_bar(1, kStateThreads);  // also: every state thread has read the accumulator of chunk k-1
       // ---- hq[k] = codes of the state entering this chunk (and the prev tap)
       if (ok) {
-        const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32) * N + n;
+        const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + cb) * N + n;
         // batches of 8: all loads of a batch before its byte stores (a byte store may alias anything,
         // so interleaving them would serialise the loop on shared-memory latency)
 #pragma unroll
         for (int p0 = 0; p0 < 32; p0 += 8) {
+          if (p0 < npp) {
           uint32_t code[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const int pp = p0 + e;
             code[e] = I8S ? (uint32_t)__float_as_int(S[pp])
-                          : rne_clamp_bits(__fmul_rn(S[pp], col_invh[ch * 32 + pp]));
+                          : rne_clamp_bits(__fmul_rn(S[pp], col_invh[cb + pp]));
           }
 #pragma unroll
-          for (int e = 0; e < 8; ++e) sHQ[(ch * 32 + p0 + e) * N + n] = (uint8_t)code[e];
+          for (int e = 0; e < 8; ++e) sHQ[(cb + p0 + e) * N + n] = (uint8_t)code[e];
+        }
         }
         if (TAPS && !I8S && a.tap_prev) {
 #pragma unroll
-          for (int pp = 0; pp < 32; ++pp) a.tap_prev[obase + (i64)pp * N] = S[pp];
+          for (int pp = 0; pp < 32; ++pp)
+            if (pp < npp) a.tap_prev[obase + (i64)pp * N] = S[pp];
         }
       }
       fence_async_smem();
       named_bar(1, kStateThreads);
       // ---- hq[k] leaves by TMA
       if (tid == 0) {
-        tma_store_2d(&tm_hq, sHQ, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P)));
+        for (int j = c0; j < c0 + ncq; ++j)  // 16 channels (rows of hq) per store
+          tma_store_2d(&tm_hq, sHQ + 16 * j * N, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P) + 16 * j));
         tma_store_commit();
       }
       // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 16 channels at a time
@@ -230,14 +239,15 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
       if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
 #pragma unroll
       for (int hf = 0; hf < 4; ++hf) {       // 8 channels at a time
+        if (hf < ncq) {
         int acc[8];
-        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + hf * 8), acc);
+        tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(cb + hf * 8), acc);
         tmem_ld_wait();
         if (ok) {
-          const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + ch * 32 + hf * 8) * N + n;
+          const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + cb + hf * 8) * N + n;
           float cscale[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) cscale[e] = col_scale[ch * 32 + hf * 8 + e];
+          for (int e = 0; e < 8; ++e) cscale[e] = col_scale[cb + hf * 8 + e];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const int pp = hf * 8 + e;
@@ -255,6 +265,7 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
           }
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_ACC_FREE]);  // this warp has read the accumulator of chunk k
@@ -262,8 +273,9 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
     if (a.final_state && ok) {
 #pragma unroll
       for (int pp = 0; pp < 32; ++pp)
-        a.final_state[(bh * P + ch * 32 + pp) * N + n] =
-            I8S ? __fmul_rn((float)__float_as_int(S[pp]), col_sh[ch * 32 + pp]) : S[pp];
+        if (pp < npp)
+          a.final_state[(bh * P + cb + pp) * N + n] =
+              I8S ? __fmul_rn((float)__float_as_int(S[pp]), col_sh[cb + pp]) : S[pp];
     }
     if (tid == 0) tma_store_wait_read();
   }
@@ -271,6 +283,22 @@ chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_const
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 64);
+  }
+}
+
+// Column range of a CTA: 16-channel chunks c0 .. c0 + ncq - 1 of one head.  Whole heads first, then
+// the heads that would form a nearly empty last wave, split in quarters so that the tail of the
+// grid packs into the free slots (operand tiles and the MMA stay full width: only the
+// re-quantisation, the state update and the hq rows are restricted to the range).
+template <bool I8S, bool TAPS>
+__global__ void __launch_bounds__(kThreads, 2)
+chunk_state_pass_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__ CUtensorMap tm_x,
+                    const __grid_constant__ CUtensorMap tm_hq, const FusedArgs a) {
+  if ((int)blockIdx.x < a.n_full) {
+    fused_body<I8S, TAPS, 4>(tm_B, tm_x, tm_hq, a, (int)blockIdx.x, 0);
+  } else {
+    const int r = (int)blockIdx.x - a.n_full;
+    fused_body<I8S, TAPS, 1>(tm_B, tm_x, tm_hq, a, a.n_full + (r >> 2), r & 3);
   }
 }
 
@@ -301,13 +329,23 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
   {
     uint64_t dims[2] = {(uint64_t)d.N, (uint64_t)d.b * d.c * d.H * d.P};
     uint64_t str[1] = {(uint64_t)d.N};
-    uint32_t box[2] = {(uint32_t)d.N, 64};
+    uint32_t box[2] = {(uint32_t)d.N, 16};
     if (!encode_tensor_map(&tm_hq, hq, 1, 2, dims, str, box, 0)) return SSDI8_ERR_CUDA;
   }
+  // (batch, head) units over the CTA slots of the device (2 CTAs per SM): whole waves of whole
+  // units, and the units of a last, partly filled wave as four quarter-width CTAs each, which pack
+  // into that wave's free slots (a quarter costs about a third of a whole unit: the operand tiles
+  // and the MMA stay full width)
+  int dev = 0, sms = 0;
+  SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
+  SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int units = d.H * d.b, slots = 2 * sms;
+  int n_full = units / slots * slots;
+  if (4 * (units - n_full) > 3 * slots) n_full = units;  // a well filled last wave: leave it whole
   FusedArgs a = {s_x, s_xs, s_B, s_h, pack, gamma, init, final_state, tap_loc, tap_prev, tap_Xsq, tap_acc,
-                 status, d};
+                 status, d, n_full};
   const size_t smem = SMEM_BYTES + 1024;
-  dim3 grid(d.H, d.b);
+  const unsigned grid = (unsigned)(n_full + 4 * (units - n_full));
   const bool taps = tap_loc || tap_prev || tap_Xsq || tap_acc;
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
