@@ -1,14 +1,15 @@
 // Recurrent-mode single-token step (the recurrence that Algorithm 2 unrolls; the paper has
 // no algorithm for it):  S <- exp(dt A) S + (dt s_x s_B) x B^T,  y = s_C C S + D s_x x + corr.
 // Pure streaming over the fp32 state [b,H,P,N]: one read and one write of the state per
-// token, 16-byte accesses, N/4 lanes per (b,h,p) row, ROWS rows per lane group in flight.
+// token, 16-byte accesses, N/4 lanes per (b,h,p) row, ROWS rows (128 bytes per thread) in flight,
+// evict-first loads and stores (the state does not fit in L2 and is touched once per step).
 #include "kernels.h"
 
 namespace ssdi8 {
 namespace {
 
 constexpr int ST_T = 256;
-constexpr int ROWS = 4;  // consecutive p per lane group
+constexpr int ROWS = 8;  // consecutive p per lane group
 
 template <int N4>  // lanes per row: 32 (N = 128) or 16 (N = 64)
 __global__ void __launch_bounds__(ST_T) ssd_step_kernel(
@@ -27,7 +28,7 @@ __global__ void __launch_bounds__(ST_T) ssd_step_kernel(
   float4* S = state + ((bh * d.P + p0) * N4 + lane);
   float4 s[ROWS];
 #pragma unroll
-  for (int r = 0; r < ROWS; ++r) s[r] = S[r * N4];
+  for (int r = 0; r < ROWS; ++r) s[r] = __ldcs(S + r * N4);
   const float dtv = dt[bh];
   const float a = expf(dtv * A[h]);
   const uint32_t bw = Bq[((i64)b * d.G + g) * N4 + lane];
@@ -46,7 +47,7 @@ __global__ void __launch_bounds__(ST_T) ssd_step_kernel(
     s[r].z = fmaf(a, s[r].z, u * b2);
     s[r].w = fmaf(a, s[r].w, u * b3);
     acc[r] = c0 * s[r].x + c1 * s[r].y + c2 * s[r].z + c3 * s[r].w;
-    S[r * N4] = s[r];
+    __stcs(S + r * N4, s[r]);
   }
 #pragma unroll
   for (int r = 0; r < ROWS; ++r)
