@@ -100,7 +100,11 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
     const int s = k & 1;
     uint8_t* st = smem + s * STAGE;
     const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-    mbar_expect_tx(&bars[B_FULL + s], (uint32_t)(Q * 64 + Q * N));
+    mbar_expect_tx(&bars[B_FULL + s], (uint32_t)(Q * 64 + Q * N + Q * 4));
+    // LUT_state of the chunk arrives with the tiles (a global load here would sit on the
+    // re-quantisation group's critical path)
+    bulk_load(smem + OFF_LUT + s * 1024, a.pack + ((unit0 + k) * kPackRows + PACK_LUT) * Q, (uint32_t)(Q * 4),
+              &bars[B_FULL + s]);
     for (int i0 = 0; i0 < Q; i0 += TQ) {
       tma_load_3d(st + OFF_X + i0 * 64, &tm_x, &bars[B_FULL + s], 0, h, (int)(tok0 + i0));
       tma_load_3d(st + OFF_B + i0 * N, &tm_B, &bars[B_FULL + s], 0, g, (int)(tok0 + i0));
@@ -124,9 +128,6 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       uint8_t* sX = smem + s * STAGE + OFF_X;
       float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
       const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-      // lut[s] was last read for chunk k-2, which every thread of this group has left
-      for (int i = qt; i < Q; i += kQuantThreads) lut[i] = a.pack[((unit0 + k) * kPackRows + PACK_LUT) * Q + i];
-      named_bar(2, kQuantThreads);
       mbar_wait_relaxed(&bars[B_FULL + s], (k >> 1) & 1, a.status);
 #pragma unroll 1
       for (int i = qt >> lq; i < Q; i += kQuantThreads >> lq) {
