@@ -167,9 +167,12 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
         tc_fence_after();
         const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
         const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+        // descriptors advance by a constant per 32-token slab (their low bits are the address >> 4):
+        // the issuing thread is on this group's critical path, so the loop is kept to an add per operand
+        uint64_t da = tile_desc(sBa, (uint32_t)N), db = tile_desc(sXa, 64);
+        const uint64_t sa = (uint64_t)((32 * N) >> 4), sb = (uint64_t)((32 * 64) >> 4);
 #pragma unroll 1
-        for (int st = 0; st < Q / 32; ++st)
-          mma_s8_ss(tmem, tile_desc(sBa + 32 * st * N, (uint32_t)N), tile_desc(sXa + 32 * st * 64, 64), idesc, st > 0);
+        for (int st = 0; st < Q / 32; ++st, da += sa, db += sb) mma_s8_ss(tmem, da, db, idesc, st > 0);
         mma_commit(&bars[B_MMA]);
       }
       __syncwarp();
