@@ -53,6 +53,14 @@ def num_threads() -> int:
     return int(_lib.orc_num_threads())
 
 
+def round_half(v):
+    """Round-to-nearest-even to IEEE binary16, returned as float64 (the oracle's own routine)."""
+    v = np.ascontiguousarray(v, np.float64)
+    _lib.orc_round_half.restype = C.c_double
+    _lib.orc_round_half.argtypes = [C.c_double]
+    return np.array([_lib.orc_round_half(float(x)) for x in v.ravel()]).reshape(v.shape)
+
+
 def exp32(x):
     x = _f32(x)
     out = np.empty_like(x)
@@ -169,6 +177,7 @@ TAP_SPECS = {
 
 
 FLAG_INT8_STATE = 2
+FLAG_FP16_OPERAND = 1   # the paper's FP16 ChunkScan2 operand (no per-row re-quantisation)
 
 
 def state_passing_int8(cfg, acc_st, gamma, init, s_xs, s_B, s_h):

@@ -442,11 +442,29 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 //     acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p]    (exact)
 //     y_diag   = (s_cb rowmax_i / 127) s_x[h,p] acc_diag
 //  y = y_off + y_diag + D s_x xq + corr
+// Round to the nearest IEEE binary16 value, ties to even (11 significant bits, subnormal quantum
+// 2^-24, overflow to infinity), returned as a double.  Used by the paper's FP16 ChunkScan2 operand.
+double orc_round_half(double v) {
+  if (v == 0.0 || std::isnan(v) || std::isinf(v)) return v;
+  int e;
+  (void)std::frexp(std::fabs(v), &e);                  // |v| = m 2^e, m in [0.5, 1)
+  const int q = (e - 1 < -14) ? -24 : e - 11;          // exponent of the spacing around |v|
+  const double r = std::ldexp(std::nearbyint(std::ldexp(std::fabs(v), -q)), q);
+  const double out = (r >= 65520.0) ? INFINITY : r;    // 65520 = the midpoint above the largest half
+  return v < 0 ? -out : out;
+}
+
+// flags bit 0 (value 1): the paper's own ChunkScan2 operand (Section 4.2; Algorithm 2, module 6):
+// no per-row re-quantisation; the masked operand is kept in FP16 with the dequantisation scale of
+// CB fused into the look-up table,  M16[i,j] = half(s_cb CBq[i,j] dt_j exp(cs_i - cs_j)), j <= i,
+// X enters as the exact FP16 image of its int8 codes, and  y_diag = s_x sum_j M16[i,j] xq[j,p]
+// (accumulated here in binary64).  rowmax, Mq and acc_diag are not produced in that mode.
 void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int8_t* CBq,
                     const int8_t* hq, const float* s_x, const float* s_C, const float* s_cb,
                     const float* s_h, const float* dt, const float* cs, const float* D,
                     const float* corr, int32_t* acc_off, float* rowmax, int8_t* Mq,
-                    int32_t* acc_diag, double* y) {
+                    int32_t* acc_diag, double* y, uint32_t flags) {
+  const bool fp16_operand = (flags & 1u) != 0;
   const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
             G = d->ngroups, Q = d->chunk, c = L / Q, hpg = H / G;
   const int SB = sub_block(Q);
@@ -456,6 +474,7 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
       const int g = h / hpg;
       std::vector<float> t(Q), f(Q / SB + 1), a_tok(Q);
       std::vector<int8_t> mq(Q);
+      std::vector<double> m16(Q);
       for (int k = 0; k < c; ++k) {
         const i64 t0 = (i64)b * L + (i64)k * Q;
         const float* csk = cs + (((i64)b * H + h) * c + k) * Q;
@@ -464,6 +483,28 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
         a_tok[0] = 1.0f;  // never used: a_m enters only for m >= 1
         for (int m = 1; m < Q; ++m) a_tok[m] = exp32(fsub(csk[m], csk[m - 1]));
         for (int i = 0; i < Q; ++i) {
+          if (fp16_operand) {
+            for (int j = 0; j <= i; ++j)
+              m16[j] = orc_round_half((double)s_cb[g] * (double)cbk[(size_t)i * Q + j] *
+                                      (double)dt[(t0 + j) * H + h] *
+                                      std::exp((double)csk[i] - (double)csk[j]));
+            const double dec = std::exp((double)csk[i]);
+            for (int p = 0; p < P; ++p) {
+              int32_t ao = 0;
+              for (int n = 0; n < N; ++n)
+                ao += (int32_t)Cq[((t0 + i) * G + g) * N + n] * (int32_t)hqk[(size_t)p * N + n];
+              double ad = 0.0;
+              for (int j = 0; j <= i; ++j) ad += m16[j] * (double)xq[((t0 + j) * H + h) * P + p];
+              const i64 o = ((t0 + i) * H + h) * P + p;
+              if (acc_off) acc_off[o] = ao;
+              double v = dec * (double)s_C[g] * (double)s_h[h * P + p] * (double)ao +
+                         (double)s_x[h * P + p] * ad;
+              if (D) v += (double)D[h] * (double)s_x[h * P + p] * (double)xq[o];
+              if (corr) v += (double)corr[h * P + p];
+              y[o] = v;
+            }
+            continue;
+          }
           const int I = i / SB;
           float rmax = 0.0f;
           for (int J = 0; J <= I; ++J) {
@@ -593,6 +634,7 @@ struct Taps {
   float* prev; int8_t* hq; int32_t* acc_off; float* rowmax; int8_t* Mq; int32_t* acc_diag;
 };
 
+// flags bit 0 (value 1): the paper's FP16 ChunkScan2 operand (see orc_chunk_scan).
 // flags bit 1 (value 2): the paper's persistent INT8 states (orc_state_passing_int8) instead of
 // fp32 states; the loc and prev taps are not produced in that mode.
 void orc_ssdi8_fwd(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8_t* Cq,
@@ -633,7 +675,7 @@ void orc_ssdi8_fwd(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8
     orc_state_passing(d, loc, gamma.data(), init, s_h, prev, final_state, hq);
   }
   orc_chunk_scan(d, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D, corr, tp->acc_off,
-                 tp->rowmax, tp->Mq, tp->acc_diag, y);
+                 tp->rowmax, tp->Mq, tp->acc_diag, y, flags);
 }
 
 // ---------------------------------------------------------------------------

@@ -465,3 +465,55 @@ def test_int8_state_forward_stays_close_to_the_dual_form():
     y1, f1 = orc.ssd_chunked(cfg, xh, Bh, Ch, t["dt"], t["A"], t["D"])
     assert np.sqrt(((y - y1) ** 2).sum() / (y1 ** 2).sum()) < 5e-2
     assert np.sqrt(((fin - f1) ** 2).sum() / (f1 ** 2).sum()) < 8e-2
+
+
+# --------------------------------------------------------------------------- the paper's FP16 ChunkScan2 operand
+def test_round_half_is_ieee_binary16_round_to_nearest_even():
+    rng = np.random.default_rng(0)
+    v = np.concatenate([rng.standard_normal(3000) * 10.0 ** rng.uniform(-9, 5, 3000),
+                        [0.0, -0.0, 65504, 65519.9, 65520, 7e4, -7e4, 2.0 ** -24, 2.0 ** -25, 1.5 * 2.0 ** -25,
+                         2.0 ** -14, 1 + 2.0 ** -11, 1 + 3 * 2.0 ** -11, 1 + 2.0 ** -10]])
+    with np.errstate(over="ignore"):
+        want = v.astype(np.float16).astype(np.float64)
+    assert np.array_equal(orc.round_half(v), want)
+
+
+@pytest.mark.parametrize("cfg", [TINY, TWO_BLOCK], ids=lambda c: c.name)
+def test_fp16_operand_mode_against_numpy_half_arithmetic(cfg):
+    """flags bit 0: y differs from the int8-operand y only in the diagonal term, which must equal
+    s_x sum_j half(s_cb CBq dt_j exp(cs_i - cs_j)) xq[j] computed here with numpy's float16."""
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    args = (cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"], q["A"], q["D"], None,
+            q["s_xs"], q["s_cb"], q["s_h"], None)
+    y8, fin8, tp = orc.ssdi8_fwd(*args, taps=("cs", "CBq", "rowmax", "acc_diag"))
+    y16, fin16, _ = orc.ssdi8_fwd(*args, flags=orc.FLAG_FP16_OPERAND)
+    assert np.array_equal(fin8, fin16)
+    b_, L, H, P, G, Q = cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim, cfg.ngroups, cfg.chunk
+    c = L // Q
+    hg = np.arange(H) // (H // G)
+    s_x = q["s_x"].astype(np.float64).reshape(H, P)
+    s_m = q["s_cb"].astype(np.float64)[hg][None, None, :] * tp["rowmax"] / 127.0
+    diag8 = s_m[..., None] * s_x * tp["acc_diag"]                                  # [b, L, H, P]
+    cs = tp["cs"].astype(np.float64)                                               # [b, H, c, Q]
+    dt = q["dt"].astype(np.float64).reshape(b_, c, Q, H)
+    xq = q["xq"].astype(np.float64).reshape(b_, c, Q, H, P)
+    cbq = tp["CBq"].astype(np.float64)                                             # [b, c, G, Q, Q]
+    tril = np.tril(np.ones((Q, Q), bool))
+    diag16 = np.zeros((b_, c, Q, H, P))
+    for b in range(b_):
+        for k in range(c):
+            for h in range(H):
+                lut = dt[b, k, :, h][None, :] * np.exp(cs[b, h, k][:, None] - cs[b, h, k][None, :])
+                m = float(q["s_cb"][hg[h]]) * cbq[b, k, hg[h]] * lut
+                with np.errstate(over="ignore"):
+                    m16 = np.where(tril, m, 0.0).astype(np.float16).astype(np.float64)
+                diag16[b, k, :, h, :] = (m16 @ xq[b, k, :, h, :]) * s_x[h][None, :]
+    want = y8 - diag8 + diag16.reshape(b_, L, H, P)
+    assert np.abs(y16 - want).max() <= 1e-9 * max(1.0, np.abs(want).max())
+    # the paper's operand (11 significant bits) is the more accurate of the two (8 bits per row):
+    # both against the dual form on the same dequantised inputs
+    xh, Bh, Ch = dequant(cfg, q)
+    y_ref = orc.ssd_chunked(cfg, xh, Bh, Ch, q["dt"], q["A"], q["D"])
+    y_ref = y_ref[0] if isinstance(y_ref, tuple) else y_ref
+    assert rms(y16 - y_ref) <= rms(y8 - y_ref)
