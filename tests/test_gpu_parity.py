@@ -261,6 +261,16 @@ def test_quantizer_empty_input_is_a_no_op():
     assert bool((o == 5).all())
 
 
+def test_entry_quantizer_empty_input_is_a_no_op():
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    x = torch.zeros(64, dtype=torch.bfloat16, device="cuda"); s = torch.ones(16, device="cuda")
+    o = torch.full((64,), 5, dtype=torch.int8, device="cuda")
+    bd.ssdi8_quantize_entry(x, 0, 16, 1, 16, s, s, s, o, o, o)
+    torch.cuda.synchronize()
+    assert bool((o == 5).all())
+
+
 def test_quantizer_full_size_x_and_bc():
     gh = _harness()
     cfg = CONFIGS["cfg2"]
@@ -396,15 +406,16 @@ def test_step_full_size_batch():
 
 
 # --------------------------------------------------------------------------- host-buffer entry point
+@pytest.mark.parametrize("batch", [3, 1])
 @pytest.mark.parametrize("flags", [0, 2])
-def test_layer_fwd_host_matches_the_device_path_bit_for_bit(flags):
+def test_layer_fwd_host_matches_the_device_path_bit_for_bit(flags, batch):
     """ssdi8_layer_fwd_host (pinned host tensors in, pipelined per batch element) == Eq. 1 quantiser +
     ssdi8_chunk_scan_fwd on the whole batch, and the oracle agrees with both; twice in a row
     (the second call reuses the side streams and both scratch stages)."""
     import torch
     from paper_2608_21952_b200 import binding as bd
     gh = _harness()
-    cfg = SSDConfig("host_b3", 3, 256, 4, 64, 64, 2, 128, 0.02, 20.0, 31)   # odd batch: both stages, ragged
+    cfg = SSDConfig("host_b", batch, 256, 4, 64, 64, 2, 128, 0.02, 20.0, 31)   # odd batch: both stages, ragged; 1: one stage
     t = inputs.make_prefill(cfg)
     init = inputs.make_init_state(cfg, 0.3)
     q = orc.prepare_quantized(cfg, t, init)
