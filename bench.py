@@ -416,6 +416,16 @@ def run_ours(args):
         scan16 = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args16, layer.ws, flags=bd.PHASE_SCAN | bd.FLAG_Y_BF16)
         scan16(); torch.cuda.synchronize()
         kernel_ms["chunk_scan_bf16_y"] = layer.timed(scan16, max(5, min(args.steps, 20)))
+        # the paper's own ChunkScan2: FP16 masked operand (kind::f16 MMA) and FP16 y; includes the
+        # pass that writes the FP16 image of xq
+        y_h = torch.empty(layer.y.shape, dtype=torch.float16, device="cuda")
+        args_h = bd.make_fwd_args(**{**layer.args._keepalive, "y": y_h})
+        fl_h = bd.PHASE_SCAN | bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16
+        ws_h = bd.alloc_workspace(layer.dims, flags=bd.FLAG_FP16_OPERAND)
+        layer.fwd_into = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args_h, ws_h, flags=bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16)
+        layer.fwd_into(); torch.cuda.synchronize()
+        scan_h = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args_h, ws_h, flags=fl_h)
+        kernel_ms["chunk_scan_fp16_operand_fp16_y"] = layer.timed(scan_h, max(5, min(args.steps, 20)))
         alg = scan_algorithmic_bytes(cfg)
         scan_gbs = alg / (kernel_ms["chunk_scan"] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "chunk_scan", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],

@@ -69,6 +69,17 @@ enum {
   SSDI8_PHASE_ALL = 0x1f00u
 };
 
+/* operand format bit of ssdi8_chunk_scan_fwd's flags: the paper's own ChunkScan2 (Section 4.2;
+ * Algorithm 2, module 6) instead of the per-row int8 re-quantisation of the masked operand:
+ *   M16[i,j] = half(s_cb CBq[i,j] dt_j exp(cs_i - cs_j)), j <= i   (FP16, CB's scale fused into the LUT)
+ *   y_diag   = s_x sum_j M16[i,j] xq[j,p]      (FP16 tensor-core MMA, FP32 accumulation; X enters as
+ *                                               the exact FP16 image of its int8 codes)
+ * computed with one factor per 16-token sub-block as below (own sub-block: running product of the
+ * per-token decays; earlier: woff_j f), in binary32 before the rounding to FP16, so a value may
+ * differ from the definition by one FP16 unit in the last place.  Needs 2 bytes per element of x
+ * more workspace (ssdi8_workspace_bytes with the flag).  Not combinable with the scan taps. */
+enum { SSDI8_FLAG_FP16_OPERAND = 1u << 0 };
+
 /* state format bit of ssdi8_chunk_scan_fwd's flags */
 enum { SSDI8_FLAG_INT8_STATE = 1u << 1 };
 
@@ -173,7 +184,7 @@ typedef struct {
  *                acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p], INT32;
  *                y_diag = (s_cb rowmax_i / 127) s_x acc_diag
  *  Output        y = y_off + y_diag + D s_x xq + corr
- * flags: bit 0 is reserved for the paper's FP16 ChunkScan2 operand and must be 0.
+ * flags: SSDI8_FLAG_FP16_OPERAND selects the paper's FP16 ChunkScan2 operand (above).
  * SSDI8_FLAG_Y_FP16 / SSDI8_FLAG_Y_BF16: `y` points to [B,L,H,P] 16-bit elements; each binary32
  * output value is rounded to nearest even into that format (fp16 overflows to infinity) as it
  * leaves the epilogue, which halves the largest byte stream of the layer.  Not combinable with taps.
@@ -231,7 +242,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  * Layouts as in ssdi8_fwd_args_t; D, corr, init_state, final_state, status may be NULL.  Both calls
  * return once everything is enqueued and leave `stream` waiting for the last piece of work, so
  * synchronising `stream` completes them.  flags: any of SSDI8_FLAG_INT8_STATE, SSDI8_FLAG_Y_FP16,
- * SSDI8_FLAG_Y_BF16 (`y` then points to 16-bit elements).  The side streams and
+ * SSDI8_FLAG_Y_BF16 (`y` then points to 16-bit elements), SSDI8_FLAG_FP16_OPERAND.  The side streams and
  * events are created at the first call on each device and shared by later calls: calls on one
  * device must not overlap in time.  Errors: as ssdi8_quantize_act / ssdi8_chunk_scan_fwd, plus
  * SSDI8_ERR_WORKSPACE for a short workspace or scratch. */

@@ -458,7 +458,9 @@ double orc_round_half(double v) {
 // no per-row re-quantisation; the masked operand is kept in FP16 with the dequantisation scale of
 // CB fused into the look-up table,  M16[i,j] = half(s_cb CBq[i,j] dt_j exp(cs_i - cs_j)), j <= i,
 // X enters as the exact FP16 image of its int8 codes, and  y_diag = s_x sum_j M16[i,j] xq[j,p]
-// (accumulated here in binary64).  rowmax, Mq and acc_diag are not produced in that mode.
+// (accumulated here in binary64).  The value that is rounded to FP16 is the binary32 product
+// fmul(t[i,j], fmul(f, s_cb)) with t and f of the sub-block factorisation below (f = 1 in the
+// row's own sub-block).  rowmax, Mq and acc_diag are not produced in that mode.
 void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int8_t* CBq,
                     const int8_t* hq, const float* s_x, const float* s_C, const float* s_cb,
                     const float* s_h, const float* dt, const float* cs, const float* D,
@@ -483,28 +485,6 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
         a_tok[0] = 1.0f;  // never used: a_m enters only for m >= 1
         for (int m = 1; m < Q; ++m) a_tok[m] = exp32(fsub(csk[m], csk[m - 1]));
         for (int i = 0; i < Q; ++i) {
-          if (fp16_operand) {
-            for (int j = 0; j <= i; ++j)
-              m16[j] = orc_round_half((double)s_cb[g] * (double)cbk[(size_t)i * Q + j] *
-                                      (double)dt[(t0 + j) * H + h] *
-                                      std::exp((double)csk[i] - (double)csk[j]));
-            const double dec = std::exp((double)csk[i]);
-            for (int p = 0; p < P; ++p) {
-              int32_t ao = 0;
-              for (int n = 0; n < N; ++n)
-                ao += (int32_t)Cq[((t0 + i) * G + g) * N + n] * (int32_t)hqk[(size_t)p * N + n];
-              double ad = 0.0;
-              for (int j = 0; j <= i; ++j) ad += m16[j] * (double)xq[((t0 + j) * H + h) * P + p];
-              const i64 o = ((t0 + i) * H + h) * P + p;
-              if (acc_off) acc_off[o] = ao;
-              double v = dec * (double)s_C[g] * (double)s_h[h * P + p] * (double)ao +
-                         (double)s_x[h * P + p] * ad;
-              if (D) v += (double)D[h] * (double)s_x[h * P + p] * (double)xq[o];
-              if (corr) v += (double)corr[h * P + p];
-              y[o] = v;
-            }
-            continue;
-          }
           const int I = i / SB;
           float rmax = 0.0f;
           for (int J = 0; J <= I; ++J) {
@@ -527,6 +507,28 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
             }
             const float m = fmul(bmax, f[J]);
             if (m > rmax) rmax = m;
+          }
+          if (fp16_operand) {
+            // the value that is rounded to FP16 is formed in binary32 in this order (a rounding
+            // decision: both sides of a parity test must take it in the same precision)
+            for (int j = 0; j <= i; ++j)
+              m16[j] = orc_round_half((double)fmul(t[j], (j / SB == I) ? s_cb[g] : fmul(f[j / SB], s_cb[g])));
+            const double dec = std::exp((double)csk[i]);
+            for (int p = 0; p < P; ++p) {
+              int32_t ao = 0;
+              for (int n = 0; n < N; ++n)
+                ao += (int32_t)Cq[((t0 + i) * G + g) * N + n] * (int32_t)hqk[(size_t)p * N + n];
+              double ad = 0.0;
+              for (int j = 0; j <= i; ++j) ad += m16[j] * (double)xq[((t0 + j) * H + h) * P + p];
+              const i64 o = ((t0 + i) * H + h) * P + p;
+              if (acc_off) acc_off[o] = ao;
+              double v = dec * (double)s_C[g] * (double)s_h[h * P + p] * (double)ao +
+                         (double)s_x[h * P + p] * ad;
+              if (D) v += (double)D[h] * (double)s_x[h * P + p] * (double)xq[o];
+              if (corr) v += (double)corr[h * P + p];
+              y[o] = v;
+            }
+            continue;
           }
           const float inv = (rmax >= 1e-30f) ? fdiv(127.0f, rmax) : 0.0f;
           for (int j = 0; j < Q; ++j) mq[j] = 0;

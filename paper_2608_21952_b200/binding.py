@@ -25,6 +25,7 @@ OK = 0
 ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = \
     -1, -2, -3, -4, -5, -6, -7, -8
 
+FLAG_FP16_OPERAND = 1 << 0
 FLAG_INT8_STATE = 1 << 1
 FLAG_Y_FP16, FLAG_Y_BF16 = 1 << 2, 1 << 3
 PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1 << k for k in range(8, 13))
@@ -249,8 +250,8 @@ def ssdi8_ssd_step(dims: Dims, xq, s_x, Bq, s_B, Cq, s_C, dt, A, D, corr, state,
                                _stream(stream)), "ssdi8_ssd_step")
 
 
-def alloc_workspace(dims: Dims, device="cuda"):
-    n = ssdi8_workspace_bytes(dims)
+def alloc_workspace(dims: Dims, device="cuda", flags: int = 0):
+    n = ssdi8_workspace_bytes(dims, flags)
     if n == 0:
         raise SSDi8Error(ERR_SHAPE, "ssdi8_workspace_bytes")
     return torch.empty(n, dtype=torch.uint8, device=device)

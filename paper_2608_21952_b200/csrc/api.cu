@@ -40,10 +40,10 @@ ssdi8_status_t check_arch() {
 }
 
 struct Workspace {
-  size_t pack, gamma, cbq, loc, hq, total;
+  size_t pack, gamma, cbq, loc, hq, x16, total;
 };
 
-Workspace layout(const Dims& d) {
+Workspace layout(const Dims& d, bool fp16_operand = false) {
   Workspace w;
   size_t o = 0;
   const size_t nst = (size_t)d.b * d.c * d.H * d.P * d.N;
@@ -52,6 +52,8 @@ Workspace layout(const Dims& d) {
   w.cbq = o;   o = align_up(o + (size_t)d.b * d.c * d.G * d.Q * d.Q, 256);
   w.loc = o;   o = align_up(o + sizeof(float) * nst, 256);
   w.hq = o;    o = align_up(o + nst, 256);
+  w.x16 = o;   // FP16 image of xq, only for the paper's FP16 ChunkScan2 operand
+  if (fp16_operand) o = align_up(o + 2 * (size_t)d.b * d.L * d.H * d.P, 256);
   w.total = o;
   return w;
 }
@@ -76,8 +78,8 @@ const char* ssdi8_status_string(ssdi8_status_t s) {
 }
 
 size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0 || !dims_supported(dims, true)) return 0;
-  return layout(make_dims(dims)).total;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0 || !dims_supported(dims, true)) return 0;
+  return layout(make_dims(dims), (flags & SSDI8_FLAG_FP16_OPERAND) != 0).total;
 }
 
 ssdi8_status_t ssdi8_quantize_act(const float* in, int64_t R, int64_t Ch, int64_t I, float* scale,
@@ -106,11 +108,13 @@ namespace ssdi8 {
 ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
                           size_t workspace_bytes, void* stream, bool clear_status) {
   if (!dims || !a) return SSDI8_ERR_NULL;
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0) return SSDI8_ERR_UNSUPPORTED;
+  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0) return SSDI8_ERR_UNSUPPORTED;
   const bool i8s = (flags & SSDI8_FLAG_INT8_STATE) != 0;
   if ((flags & SSDI8_FLAG_Y_FP16) && (flags & SSDI8_FLAG_Y_BF16)) return SSDI8_ERR_UNSUPPORTED;
   const int ydt = (flags & SSDI8_FLAG_Y_FP16) ? 1 : (flags & SSDI8_FLAG_Y_BF16) ? 2 : 0;
   if (ydt && (a->tap_acc_off || a->tap_rowmax || a->tap_Mq || a->tap_acc_diag)) return SSDI8_ERR_UNSUPPORTED;
+  const bool f16op = (flags & SSDI8_FLAG_FP16_OPERAND) != 0;
+  if (f16op && (a->tap_acc_off || a->tap_rowmax || a->tap_Mq || a->tap_acc_diag)) return SSDI8_ERR_UNSUPPORTED;
   const uint32_t ph = (flags & SSDI8_PHASE_ALL) ? (flags & SSDI8_PHASE_ALL) : (uint32_t)SSDI8_PHASE_ALL;
   // the INT8 state lives inside the fused ChunkState + StatePassing kernel only
   if (i8s && ((ph & SSDI8_PHASE_CHUNK_STATE) != 0) != ((ph & SSDI8_PHASE_STATE_PASSING) != 0))
@@ -126,7 +130,7 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
     if (p && !aligned16(p)) return SSDI8_ERR_ALIGN;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SSDI8_ERR_ALIGN;
   const Dims d = make_dims(dims);
-  const Workspace w = layout(d);
+  const Workspace w = layout(d, f16op);
   if (workspace_bytes < w.total) return SSDI8_ERR_WORKSPACE;
   ssdi8_status_t s = check_arch();
   if (s != SSDI8_OK) return s;
@@ -161,6 +165,9 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
                                   hq, nullptr, st)) != SSDI8_OK)
       return s;
   }
+  if ((ph & SSDI8_PHASE_SCAN) && f16op)
+    return launch_chunk_scan_f16(d, a->xq, ws + w.x16, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack, a->D,
+                                 a->corr, a->y, ydt, a->status, st);
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};
     return launch_chunk_scan(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack,
@@ -297,7 +304,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
   if (!dims || !args) return SSDI8_ERR_NULL;
   const size_t need = ssdi8_workspace_bytes(dims, flags);
   if (need == 0)
-    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
+    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
   if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
   static void* ws_of_device[64];  // resolved address of g_static_ws, per device
   int dev = 0;

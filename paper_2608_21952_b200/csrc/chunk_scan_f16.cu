@@ -1,0 +1,546 @@
+// ChunkScan1 + ChunkScan2 + output sum with the paper's own ChunkScan2 operand (Section 4.2;
+// Algorithm 2, module 6): the masked operand stays in FP16 with the dequantisation scale of CB
+// fused into the look-up table,
+//   M16[i,j] = half(s_cb CBq[i,j] dt_j exp(cs_i - cs_j)), j <= i,      y_diag = s_x sum_j M16[i,j] xq[j,p],
+// instead of the per-row int8 re-quantisation of chunk_scan.cu.  Same persistent, warp-specialised
+// structure (28 warps: 3 TMA producers, 1 MMA warp, two mask groups of 8 warps on alternate
+// tiles, 8 epilogue warps), with these differences:
+//  * the mask warps write M16 straight into tensor memory (tcgen05.st, thread = row), from where
+//    tcgen05.mma.kind::f16 takes it as its A operand: the operand never exists in shared memory,
+//    there is no row maximum, no second pass and no zero fill of shared memory;
+//  * X enters as the exact FP16 image of its int8 codes (written once per call by a streaming
+//    kernel), TMA-staged MN-major with 128-byte rows; ChunkScan1 stays an int8 MMA;
+//  * tensor memory: two accumulator pairs (INT32 C h, FP32 M16 x) and two operand buffers, 512 columns.
+// One factor per 16-column sub-block as in chunk_scan.cu: own sub-block by the running product of
+// per-token decays, earlier ones woff_j f with f = exp32(cs_i - cs_je); a sub-block whose bound
+// says every |value| < 2^-25 (half of the smallest FP16 subnormal) is zero, and so is every
+// farther one where cs does not increase (p127, see cumsum.cu).  No multicast; bounded waits.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace ssdi8 {
+namespace {
+
+using namespace sm100;
+
+struct ScanArgs {
+  const float* s_x; const float* s_C; const float* s_cb; const float* s_h;
+  const float* pack; const float* D; const float* corr;
+  int32_t* status;
+  Dims d;
+  int ntiles, per_cta;
+};
+
+constexpr int kWarps = 28, kThreads = kWarps * 32;
+constexpr int kMaskWarp0 = 4, kGroupWarps = 8;
+constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
+constexpr uint32_t kTmemCols = 512;  // accumulator pair a at 128 a (+0 INT32 C h, +64 FP32 M16 x); operand buffer g at 256 + 128 g
+constexpr uint32_t PANEL = 16384;    // [128][128] int8
+// shared memory (bytes, from a 1024-byte aligned base)
+constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1-panel buffers
+constexpr uint32_t OFF_C = 98304;       // [128][N]
+constexpr uint32_t OFF_H = 114688;      // [64][N]
+constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64] fp16 (128-byte rows)
+constexpr uint32_t X_BYTES = 32768;
+constexpr uint32_t OFF_TOK = OFF_X + 2 * X_BYTES;   // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds)
+constexpr uint32_t TOK_BYTES = 6144;
+constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][64 B] y staging
+constexpr uint32_t OFF_BAR = OFF_YST + 16384;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
+
+__device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
+  return OFF_CB + (idx < 2 ? (uint32_t)idx * 32768u : 65536u + (uint32_t)(idx - 2) * 16384u);
+}
+__device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
+  return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
+}
+
+enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
+       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_COUNT = 32 };
+
+// two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
+__device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
+  const float2 m = make_float2(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)),
+                               __uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7651u + k)));
+  return __fadd2_rn(m, make_float2(-kMagicIn, -kMagicIn));
+}
+__device__ __forceinline__ uint32_t half2_bits(float2 v) {
+  const __half2 h = __floats2half2_rn(v.x, v.y);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem], FP16 operands, FP32 accumulator; issued by one thread
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// instruction descriptor for kind::f16: FP16 A (K-major, in tensor memory) and B, FP32 accumulator
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N, int b_mn_major) {
+  return (1u << 4) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct Tile {
+  int b, k, h, g, it, KJ;
+  i64 tok0, unit;  // unit = (b*H + h)*c + k
+};
+__device__ __forceinline__ void next_tile(Tile& x, const Dims& d, int TM, int ntpu) {
+  if (++x.it == ntpu) {
+    x.it = 0;
+    if (++x.h == d.H) {
+      x.h = 0;
+      if (++x.k == d.c) { x.k = 0; ++x.b; }
+    }
+    x.g = x.h / (d.H / d.G);
+    x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
+    x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
+  }
+  x.KJ = (x.it + 1) * TM;
+}
+__device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntpu) {
+  Tile x;
+  x.it = t % ntpu;
+  int u = t / ntpu;
+  x.h = u % d.H; u /= d.H;
+  x.k = u % d.c;
+  x.b = u / d.c;
+  x.g = x.h / (d.H / d.G);
+  x.KJ = (x.it + 1) * TM;
+  x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
+  x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
+  return x;
+}
+
+// ---- the FP16 operand of one tile, written to tensor memory.  A warp owns 32 rows (lane = row =
+// TMEM lane, warp index mod 4 = lane quarter) and the 16-column chunks of one parity q2; every
+// chunk of that parity in the contraction range gets one collective store of 8 packed words per
+// row (zeros where the chunk lies after the row's own, is skipped, or the row is idle).
+__device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* tokbuf, uint32_t a_tmem, int rq,
+                                              int q2, int lane, int TM, uint32_t RBQ, const Tile& t,
+                                              const ScanArgs& a) {
+  const int Q = a.d.Q;
+  const float* cs_s = tokbuf;
+  const float* dt_s = tokbuf + Q;
+  const float* woff_s = tokbuf + 2 * Q;
+  const float* atok_s = tokbuf + 3 * Q;
+  const float* b127_s = tokbuf + 4 * Q;
+  const float* p127_s = b127_s + 16;
+  const int r = rq * 32 + lane;
+  const bool row_ok = r < TM;
+  const int i = t.it * TM + r;       // row within the chunk
+  const int I16 = i >> 4, ri = i & 15;
+  const int nch = t.KJ >> 4;         // 16-column chunks in the contraction range
+  const uint32_t cshift = RBQ == 128 ? 3u : 2u;  // log2(chunks per panel row)
+  const uint8_t* const rowbase = sCB + (RBQ == 128 ? (uint32_t)r * 128u : (uint32_t)r * 64u);
+  const uint32_t rx = RBQ == 128 ? ((uint32_t)r & 7u) : (((uint32_t)r >> 1) & 3u);  // swizzle term of the row
+  auto chunk_ptr = [&](int c) -> const uint4* {
+    const uint32_t pn = (uint32_t)c >> cshift, cc = (uint32_t)c & ((1u << cshift) - 1u);
+    return reinterpret_cast<const uint4*>(rowbase + pn * PANEL + ((cc ^ rx) << 4));
+  };
+  const float cs_i = row_ok ? cs_s[i] : 0.f;
+  const float scb = a.s_cb[t.g];
+  const float kTiny = 2.9e-8f;       // below 2^-25 = 2.98e-8: rounds to zero in FP16
+  const uint32_t lane_addr = a_tmem + ((uint32_t)(rq * 32) << 16);
+  bool done = !row_ok;               // this row has nothing (more) to contribute
+#pragma unroll 1
+  for (int c = ((nch - 1 - q2) & ~1) + q2; c >= 0; c -= 2) {
+    uint32_t w8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+    if (!done && c <= I16) {
+      if (c == I16) {
+        // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+        const uint4 w4 = *chunk_ptr(c);
+        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+        const float* dtc = dt_s + c * 16;
+        const float* atc = atok_s + c * 16 + 1;
+        float E = 1.0f;
+        float tv[16];
+#pragma unroll
+        for (int e = 15; e >= 0; --e) {
+          float v = 0.f;
+          if (e <= ri) {
+            if (e < ri) E = __fmul_rn(E, atc[e]);
+            v = __fmul_rn(__fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E)), scb);
+          }
+          tv[e] = v;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w8[e] = half2_bits(make_float2(tv[2 * e], tv[2 * e + 1]));
+      } else {
+        const float g = __fmul_rn(exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])), scb);
+        if (__fmul_rn(p127_s[c], g) < kTiny) {
+          done = true;               // this chunk and every farther one round to zero
+        } else if (__fmul_rn(b127_s[c], g) >= kTiny) {
+          const float2 g2 = make_float2(g, g);
+          const uint4 w4 = *chunk_ptr(c);
+          const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+          const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const float4 fo = wo[w];
+            w8[2 * w] = half2_bits(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)), g2));
+            w8[2 * w + 1] = half2_bits(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2));
+          }
+        }
+      }
+    }
+    __syncwarp();
+    tmem_st8(lane_addr + (uint32_t)(c * 8), w8);
+  }
+  tmem_st_wait();
+}
+
+// CORR: a mean-correction vector is given; YT: format of y (0 binary32, 1 fp16, 2 bf16)
+template <bool CORR, int YT>
+__global__ void __launch_bounds__(kThreads, 1)
+chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
+                  const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
+                  const __grid_constant__ CUtensorMap tm_y, const ScanArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const Dims& d = a.d;
+  const int Q = d.Q, N = d.N, P = d.P;
+  const int TM = Q < 128 ? Q : 128;        // valid rows of a tile
+  const int ntpu = Q / TM;                 // tiles per (batch, chunk, head)
+  const uint32_t RBN = N, RBQ = TM;        // row bytes of the N-contracted and Q-contracted int8 tiles
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t_begin = blockIdx.x * a.per_cta;
+  const int t_end = min(a.ntiles, t_begin + a.per_cta);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+
+  if (tid == 0) {
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&bars[B_CB_FULL + s], 1);
+      mbar_init(&bars[B_CB_FREE + s], kGroupWarps);   // released by the mask group that read it
+      mbar_init(&bars[B_MQ + s], kGroupWarps);
+      mbar_init(&bars[B_TOK_FULL + s], 1);
+      mbar_init(&bars[B_TOK_FREE + s], kEpiWarps);
+    }
+    mbar_init(&bars[B_CH_FULL], 1);
+    mbar_init(&bars[B_CH_FREE], 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bars[B_X_FULL + s], 1);
+      mbar_init(&bars[B_X_FREE + s], kEpiWarps);
+      mbar_init(&bars[B_ACC + s], 1);
+      mbar_init(&bars[B_ACC_FREE + s], kEpiWarps);
+      mbar_init(&bars[B_AFREE + s], 1);
+    }
+    fence_mbar_init();
+    tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
+    tma_prefetch_desc(&tm_cb); tma_prefetch_desc(&tm_y);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
+    if (lane == 0) {
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+        const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+        const uint32_t ph4 = (n >> 2) & 1;
+        mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
+        const int npanel = t.KJ / (int)RBQ;
+        mbar_expect_tx(&bars[B_CB_FULL + ci], (uint32_t)(npanel * TM * RBQ));
+        for (int pn = 0; pn < npanel; ++pn)
+          tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
+                      (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
+        mbar_wait_relaxed(&bars[B_TOK_FREE + t3], ph4 ^ 1, a.status);
+        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4));
+        bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4),
+                  &bars[B_TOK_FULL + t3]);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ TMA producer: Cq, hq
+    if (lane == 0) {
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+        mbar_wait_relaxed(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
+        mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
+        tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
+        tma_load_2d(smem + OFF_H, &tm_h, &bars[B_CH_FULL], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------ TMA producer: FP16 x rows
+    if (lane == 0) {
+      Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+        const int s2 = n & 1;
+        const uint32_t ph2 = (n >> 1) & 1;
+        mbar_wait_relaxed(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
+        mbar_expect_tx(&bars[B_X_FULL + s2], (uint32_t)(t.KJ * 128));
+        for (int j0 = 0; j0 < t.KJ; j0 += TM)
+          tma_load_3d(smem + OFF_X + s2 * X_BYTES + j0 * 128, &tm_x, &bars[B_X_FULL + s2], 0, t.h, (int)(t.tok0 + j0));
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_off = idesc_s8(128, 64, 0, 0), idesc_diag = idesc_f16(128, 64, 1);
+      const uint32_t sbase = smem_u32(smem);
+#pragma unroll 1
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
+        const int it = tix % ntpu;
+        const int ci = cb_index(n, it, ntpu), s2 = n & 1;
+        const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
+        const int KJ = (it + 1) * TM;
+        const uint32_t acc = tmem + (uint32_t)s2 * 128u;
+        mbar_wait(&bars[B_ACC_FREE + s2], ph2 ^ 1, a.status);
+        mbar_wait(&bars[B_CH_FULL], n & 1, a.status);
+        tc_fence_after();
+#pragma unroll 1
+        for (int q = 0; q < N / 32; ++q)
+          mma_s8_ss(acc, tile_desc(sbase + OFF_C + 32 * q, RBN), tile_desc(sbase + OFF_H + 32 * q, RBN),
+                    idesc_off, q > 0);
+        mma_commit(&bars[B_CH_FREE]);
+        mbar_wait(&bars[B_MQ + ci], ph4, a.status);        // the operand of this tile is in tensor memory
+        mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);
+        tc_fence_after();
+        // 16 tokens per instruction: 8 operand columns and 16 rows of 128 bytes of x
+        uint64_t bd = smem_desc(sbase + OFF_X + s2 * X_BYTES, 16, 1024, SWZ_128B);
+        const uint32_t a_op = tmem + 256u + (uint32_t)s2 * 128u;
+#pragma unroll 1
+        for (int q = 0; q < KJ / 16; ++q, bd += (16 * 128) >> 4)
+          mma_f16_ts(acc + 64, a_op + (uint32_t)(q * 8), bd, idesc_diag, q > 0);
+        mma_commit(&bars[B_AFREE + s2]);
+        mma_commit(&bars[B_ACC + s2]);
+      }
+    }
+  } else if (warp < kEpiWarp0) {
+    // ------------------------------------------------------------ mask warps: group g takes tiles n = g, g + 2, ...
+    const int g = (warp - kMaskWarp0) / kGroupWarps;
+    const int wg = (warp - kMaskWarp0) % kGroupWarps;
+    const int rq = warp & 3;               // TMEM lane quarter of this warp = row quarter of the tile
+    const int q2 = wg >> 2;                // chunk parity of this warp
+    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    if (g) next_tile(t, d, TM, ntpu);
+#pragma unroll 1
+    for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
+      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+      const uint32_t ph4 = (n >> 2) & 1;
+      mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
+      mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
+      mbar_wait(&bars[B_AFREE + g], ((n >> 1) & 1) ^ 1, a.status);   // the MMAs of tile n - 2 have read the buffer
+      tc_fence_after();
+      mask_tile_f16(smem + cb_offset(ci), reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES),
+                    tmem + 256u + (uint32_t)g * 128u, rq, q2, lane, TM, RBQ, t, a);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&bars[B_MQ + ci]);
+        mbar_arrive(&bars[B_CB_FREE + ci]);
+      }
+      next_tile(t, d, TM, ntpu);
+      next_tile(t, d, TM, ntpu);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
+    const int ew = warp - kEpiWarp0;
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int ch = ew >> 2;                 // column half
+    const int er = q * 32 + lane;           // row of the tile
+    uint8_t* ystage = smem + OFF_YST + ew * 2048;   // [32][64 B], 64-byte swizzle
+    uint8_t* srow = ystage + lane * 64;
+    Tile t = decode_tile(t_begin, d, TM, ntpu);
+#pragma unroll 1
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      const int s2 = n & 1, t3 = n & 3;
+      const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
+      const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
+      const uint8_t* sX = smem + OFF_X + s2 * X_BYTES;
+      const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f;
+      const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
+      const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
+      const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
+      // three lanes wait side by side: the accumulators, the x rows (skip term), the scalar pack (cs)
+      if (lane < 3) {
+        const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_X_FULL + s2 : B_TOK_FULL + t3;
+        mbar_wait_relaxed(&bars[bi], lane == 2 ? ph4 : ph2, a.status);
+      }
+      __syncwarp();
+      tc_fence_after();
+      const bool ok = er < TM;
+      const int ei = t.it * TM + er;
+      const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
+      const float2 dec2 = make_float2(dec, dec), Dh2 = make_float2(Dh, Dh);
+#pragma unroll 1
+      for (int pc = 0; pc < 4; ++pc) {       // 8 columns at a time
+        int acc_o[8], acc_d[8];
+        const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 8);
+        tmem_ld8(taddr, acc_o);
+        tmem_ld8(taddr + 64, acc_d);
+        if (YT != 0 ? pc == 0 : (pc & 1) == 0) {
+          if (lane == 3) tma_store_wait_read();  // the last store has finished reading the staging tile
+          __syncwarp();
+        }
+        tmem_ld_wait();
+        if (ok) {
+          // 8 FP16 values of x (exact images of the int8 codes): one 16-byte chunk of the row
+          const uint4 xr = *reinterpret_cast<const uint4*>(sX + swz_off((uint32_t)ei, (uint32_t)(ch * 4 + pc), 128));
+          const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+          float2 v[4];
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const float4 sx4 = __ldg(gsx + pc * 2 + cc), sh4 = __ldg(gsh + pc * 2 + cc);
+            const float4 co4 = CORR ? __ldg(gco + pc * 2 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int e2 = 0; e2 < 2; ++e2) {
+              const int pp = cc * 4 + e2 * 2;
+              const float2 sx2 = e2 ? make_float2(sx4.z, sx4.w) : make_float2(sx4.x, sx4.y);
+              const float2 sh2 = e2 ? make_float2(sh4.z, sh4.w) : make_float2(sh4.x, sh4.y);
+              const float2 co2 = e2 ? make_float2(co4.z, co4.w) : make_float2(co4.x, co4.y);
+              const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(&xw[cc * 2 + e2]));
+              const float2 ao = make_float2((float)acc_o[pp], (float)acc_o[pp + 1]);
+              const float2 ad = make_float2(__int_as_float(acc_d[pp]), __int_as_float(acc_d[pp + 1]));
+              float2 r2 = __ffma2_rn(__fmul2_rn(Dh2, sx2), xv, co2);
+              r2 = __ffma2_rn(sx2, ad, r2);
+              v[cc * 2 + e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
+            }
+            if (YT == 0)
+              *reinterpret_cast<float4*>(srow + ((((pc & 1) * 2 + cc) ^ ((lane >> 1) & 3)) << 4)) =
+                  make_float4(v[cc * 2].x, v[cc * 2].y, v[cc * 2 + 1].x, v[cc * 2 + 1].y);
+          }
+          if (YT != 0) {  // 8 values = one 16-byte chunk of the staging row
+            uint32_t h[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              if (YT == 1) {
+                h[e] = half2_bits(v[e]);
+              } else {
+                const __nv_bfloat162 bv = __floats2bfloat162_rn(v[e].x, v[e].y);
+                h[e] = *reinterpret_cast<const uint32_t*>(&bv);
+              }
+            }
+            *reinterpret_cast<uint4*>(srow + ((pc ^ ((lane >> 1) & 3)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+          }
+        }
+        if (YT != 0 ? pc == 3 : (pc & 1) == 1) {   // a staging tile is full: 32 columns of 16-bit y, or 16 of binary32
+          if (pc == 3) tc_fence_before();
+          fence_async_smem();
+          __syncwarp();
+          if (pc == 3 && lane < 3) {
+            mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + s2 : B_TOK_FREE + t3]);
+          } else if (lane == 3 && q * 32 < TM) {
+            tma_store_3d(&tm_y, ystage, ch * 32 + (YT != 0 ? 0 : (pc >> 1) * 16), t.h,
+                         (int)(t.tok0 + t.it * TM + q * 32));
+            tma_store_commit();
+          }
+        }
+      }
+    }
+    if (lane == 3) tma_store_wait_read();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+__global__ void __launch_bounds__(256) x_to_half_kernel(const uint32_t* __restrict__ xq, uint2* __restrict__ x16,
+                                                        i64 n4) {
+  const i64 e = (i64)blockIdx.x * 256 + threadIdx.x;
+  if (e >= n4) return;
+  const uint32_t w = __ldcs(xq + e);
+  const __half2 lo = __floats2half2_rn((float)sx8(w, 0), (float)sx8(w, 1));
+  const __half2 hi = __floats2half2_rn((float)sx8(w, 2), (float)sx8(w, 3));
+  uint2 o;
+  o.x = *reinterpret_cast<const uint32_t*>(&lo);
+  o.y = *reinterpret_cast<const uint32_t*>(&hi);
+  __stcs(x16 + e, o);
+}
+
+}  // namespace
+
+ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16, const int8_t* Cq,
+                                     const int8_t* CBq, const int8_t* hq, const float* s_x, const float* s_C,
+                                     const float* s_cb, const float* s_h, const float* pack, const float* D,
+                                     const float* corr, void* y, int ydt, int32_t* status, cudaStream_t st) {
+  const int TM = d.Q < 128 ? d.Q : 128;
+  const uint64_t T = (uint64_t)d.b * d.L;
+  // X as FP16 (exact images of the int8 codes)
+  const i64 n4 = (i64)T * d.H * d.P / 4;
+  x_to_half_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(xq),
+                                                                 static_cast<uint2*>(x16), n4);
+  SSDI8_LAUNCH_CHECK();
+  CUtensorMap tm_C, tm_h, tm_x, tm_cb, tm_y;
+  {
+    uint64_t dims[3] = {(uint64_t)d.N, (uint64_t)d.G, T};
+    uint64_t str[2] = {(uint64_t)d.N, (uint64_t)d.G * d.N};
+    uint32_t box[3] = {(uint32_t)d.N, 1, (uint32_t)TM};
+    if (!encode_tensor_map(&tm_C, Cq, 1, 3, dims, str, box, d.N)) return SSDI8_ERR_CUDA;
+  }
+  {
+    uint64_t dims[2] = {(uint64_t)d.N, (uint64_t)d.b * d.c * d.H * d.P};
+    uint64_t str[1] = {(uint64_t)d.N};
+    uint32_t box[2] = {(uint32_t)d.N, 64};
+    if (!encode_tensor_map(&tm_h, hq, 1, 2, dims, str, box, d.N)) return SSDI8_ERR_CUDA;
+  }
+  {
+    uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
+    uint64_t str[2] = {(uint64_t)d.P * 2, (uint64_t)d.H * d.P * 2};
+    uint32_t box[3] = {64, 1, (uint32_t)TM};
+    if (!encode_tensor_map(&tm_x, x16, 2, 3, dims, str, box, 128)) return SSDI8_ERR_CUDA;
+  }
+  {
+    uint64_t dims[2] = {(uint64_t)d.Q, (uint64_t)d.b * d.c * d.G * d.Q};
+    uint64_t str[1] = {(uint64_t)d.Q};
+    uint32_t box[2] = {(uint32_t)TM, (uint32_t)TM};
+    if (!encode_tensor_map(&tm_cb, CBq, 1, 2, dims, str, box, TM)) return SSDI8_ERR_CUDA;
+  }
+  {
+    const uint64_t eb = ydt ? 2 : 4;  // bytes per element of y; the staging tile holds 64-byte rows either way
+    uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
+    uint64_t str[2] = {(uint64_t)d.P * eb, (uint64_t)d.H * d.P * eb};
+    uint32_t box[3] = {ydt ? 32u : 16u, 1, 32};
+    if (!encode_tensor_map(&tm_y, y, (int)eb, 3, dims, str, box, 64)) return SSDI8_ERR_CUDA;
+  }
+  int dev = 0, sms = 0;
+  SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
+  SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int ntiles = (int)((i64)d.b * d.c * d.H * (d.Q / TM));
+  const int ctas = ntiles < sms ? ntiles : sms;
+  int per_cta = (ntiles + ctas - 1) / ctas;
+  if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
+  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, d, ntiles, per_cta};
+  const size_t smem = SMEM_BYTES + 1024;
+  const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
+  auto launch = [&](auto kernel) -> ssdi8_status_t {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
+    return SSDI8_OK;
+  };
+  ssdi8_status_t ls;
+  if (ydt == 0)
+    ls = corr ? launch(chunk_scan_f16_tc<true, 0>) : launch(chunk_scan_f16_tc<false, 0>);
+  else if (ydt == 1)
+    ls = corr ? launch(chunk_scan_f16_tc<true, 1>) : launch(chunk_scan_f16_tc<false, 1>);
+  else
+    ls = corr ? launch(chunk_scan_f16_tc<true, 2>) : launch(chunk_scan_f16_tc<false, 2>);
+  if (ls != SSDI8_OK) return ls;
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+}  // namespace ssdi8

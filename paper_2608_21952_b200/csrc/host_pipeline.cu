@@ -15,7 +15,7 @@ namespace ssdi8 {
 namespace {
 
 constexpr int kStages = 2;
-constexpr uint32_t kLayerFlags = SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16;
+constexpr uint32_t kLayerFlags = SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16;
 
 struct StageBuf {
   float *x, *B, *C, *dt, *y, *fin;

@@ -41,7 +41,7 @@ def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use", flags=0):
     for name in taps:
         shp, dt_ = shapes[name]
         tp["tap_" + name] = torch.zeros(shp, dtype=_NP2T[dt_], device="cuda")
-    ws = bd.alloc_workspace(dims)
+    ws = bd.alloc_workspace(dims, flags=flags)
     args = bd.make_fwd_args(y=y, final_state=fin, status=status, **t, **tp)
     bd.ssdi8_chunk_scan_fwd(dims, args, ws, flags=flags)
     torch.cuda.synchronize()

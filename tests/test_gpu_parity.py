@@ -173,10 +173,12 @@ def _slice(cfg, b, h, xq, Bq, Cq, s_x, s_B, s_C, t, extra=None):
     return {k: np.ascontiguousarray(v) for k, v in d.items()}
 
 
+@pytest.mark.parametrize("flags", [0, 1], ids=["int8_operand", "fp16_operand"])
 @pytest.mark.parametrize("name,npairs", [("cfg2", 4), ("cfg3", 3)])
-def test_fwd_full_size_sampled(name, npairs):
+def test_fwd_full_size_sampled(name, npairs, flags):
     """Full-size workloads in the launch configuration the benchmark times (no taps); the
-    oracle recomputes sampled (batch, head) pairs one by one."""
+    oracle recomputes sampled (batch, head) pairs one by one.  flags = 1: the paper's FP16
+    ChunkScan2 operand on both sides."""
     gh = _harness()
     cfg = CONFIGS[name]
     t = inputs.make_prefill(cfg)
@@ -187,13 +189,14 @@ def test_fwd_full_size_sampled(name, npairs):
         if pr not in pairs:
             pairs.append(pr)
     q = _sampled_problem(cfg, t, pairs)
-    y, fin, _ = gh.gpu_fwd(cfg, q, taps=())
+    y, fin, _ = gh.gpu_fwd(cfg, q, taps=(), flags=flags)
     assert np.all(np.isfinite(y)) and np.all(np.isfinite(fin))
     one = cfg.replace(batch=1, nheads=1, ngroups=1)
     for (b, h) in pairs:
         s = _slice(cfg, b, h, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], t, extra=q)
         y_ref, fin_ref, _ = orc.ssdi8_fwd(one, s["xq"], s["Bq"], s["Cq"], s["s_x"], s["s_B"], s["s_C"],
-                                          s["dt"], s["A"], s["D"], None, s["s_xs"], s["s_cb"], s["s_h"])
+                                          s["dt"], s["A"], s["D"], None, s["s_xs"], s["s_cb"], s["s_h"],
+                                          flags=flags)
         assert np.array_equal(fin[b, h], fin_ref[0, 0]), (b, h)
         assert np.abs(y[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
 
@@ -536,3 +539,42 @@ def test_16_bit_y_flags_are_exclusive_and_without_taps():
         bd.ssdi8_chunk_scan_fwd(dims, bd.make_fwd_args(y=y16, tap_rowmax=tap, **dv), ws, flags=bd.FLAG_Y_FP16)
     assert e.value.code == bd.ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+# --------------------------------------------------------------------------- the paper's FP16 ChunkScan2 operand
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_fwd_fp16_operand_against_the_oracle_mode(cfg):
+    """SSDI8_FLAG_FP16_OPERAND: the masked operand in FP16 in tensor memory, kind::f16 MMA.  y within
+    the fp32 tolerance of the oracle's FP16-operand mode (the operand is formed in binary32 before its
+    rounding to FP16, the oracle forms it in binary64: single FP16 ulps may differ); the states, which
+    this mode does not touch, bit for bit."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    y_ref, fin_ref, _ = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                      q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], init,
+                                      flags=orc.FLAG_FP16_OPERAND)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    y = torch.full(t["x"].shape, float("nan"), device="cuda")
+    fin = torch.empty(init.shape, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_fwd_args(y=y, final_state=fin, status=status, init_state=gh.dev(init), **dv)
+    ws = bd.alloc_workspace(dims, flags=bd.FLAG_FP16_OPERAND)
+    for rep in range(2):
+        y.fill_(float("nan"))
+        bd.ssdi8_chunk_scan_fwd(dims, args, ws, flags=bd.FLAG_FP16_OPERAND)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(fin.cpu().numpy(), fin_ref)
+        err = np.abs(y.cpu().numpy() - y_ref).max()
+        assert err <= Y_TOL * rms(y_ref), err / rms(y_ref)
+    # with the paper's output format as well
+    y16 = torch.full(t["x"].shape, float("nan"), dtype=torch.float16, device="cuda")
+    args16 = bd.make_fwd_args(y=y16, final_state=fin, status=status, init_state=gh.dev(init), **dv)
+    bd.ssdi8_chunk_scan_fwd(dims, args16, ws, flags=bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16)
+    torch.cuda.synchronize()
+    assert torch.equal(y16.cpu().view(torch.int16), y.cpu().half().view(torch.int16))

@@ -510,7 +510,11 @@ def test_fp16_operand_mode_against_numpy_half_arithmetic(cfg):
                     m16 = np.where(tril, m, 0.0).astype(np.float16).astype(np.float64)
                 diag16[b, k, :, h, :] = (m16 @ xq[b, k, :, h, :]) * s_x[h][None, :]
     want = y8 - diag8 + diag16.reshape(b_, L, H, P)
-    assert np.abs(y16 - want).max() <= 1e-9 * max(1.0, np.abs(want).max())
+    # the oracle rounds the binary32 product of the sub-block factorisation, this restatement the
+    # binary64 product: about one operand element in a thousand lands on the neighbouring FP16 value
+    # (2^-11 of one term of one output); anything structural would be orders of magnitude larger
+    err = np.abs(y16 - want)
+    assert rms(err) <= 2e-5 * rms(want) and err.max() <= 2e-3 * rms(want)
     # the paper's operand (11 significant bits) is the more accurate of the two (8 bits per row):
     # both against the dual form on the same dequantised inputs
     xh, Bh, Ch = dequant(cfg, q)
