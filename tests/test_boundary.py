@@ -71,7 +71,8 @@ def test_host_side_argument_errors():
     a = bd.FwdArgs()
     assert L.ssdi8_chunk_scan_fwd(None, None, 0, None, 0, None) == bd.ERR_NULL
     assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 0, None, 0, None) == bd.ERR_NULL
-    assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 1, None, 0, None) == bd.ERR_UNSUPPORTED
+    assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 1, None, 0, None) == bd.ERR_NULL   # bit 0: FP16 operand, valid
+    assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), (1 << 2) | (1 << 3), None, 0, None) == bd.ERR_UNSUPPORTED
     assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 1 << 13, None, 0, None) == bd.ERR_UNSUPPORTED
     dbad = bd.dims_of(CONFIGS["cfg0"].replace(chunk=32))
     assert L.ssdi8_chunk_scan_fwd(C.byref(dbad), C.byref(a), 0, None, 0, None) == bd.ERR_SHAPE
