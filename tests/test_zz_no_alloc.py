@@ -29,7 +29,7 @@ def test_static_entry_rejects_what_does_not_fit_on_the_host():
     assert L.ssdi8_chunk_scan_fwd_static(None, None, 0, None) == bd.ERR_NULL
     bad = bd.dims_of(CONFIGS["cfg0"].replace(chunk=48))
     assert L.ssdi8_chunk_scan_fwd_static(C.byref(bad), C.byref(a), 0, None) == bd.ERR_SHAPE
-    assert L.ssdi8_chunk_scan_fwd_static(C.byref(big), C.byref(a), 1, None) == bd.ERR_UNSUPPORTED
+    assert L.ssdi8_chunk_scan_fwd_static(C.byref(big), C.byref(a), 1 << 13, None) == bd.ERR_UNSUPPORTED
     for name in ("cfg0", "cfg1"):
         assert bd.ssdi8_workspace_bytes(bd.dims_of(CONFIGS[name])) <= bd.STATIC_WORKSPACE_BYTES
 
