@@ -458,17 +458,28 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   }
 }
 
-__global__ void __launch_bounds__(256) x_to_half_kernel(const uint32_t* __restrict__ xq, uint2* __restrict__ x16,
-                                                        i64 n4) {
+// FP16 image of int8 codes, 16 codes per thread.  With u = code ^ 0x80 (0..255), the half with bits
+// 0x6400 | u is 1024 + u exactly, and subtracting 1152 gives the code: one byte permute and one
+// packed subtraction per two elements, no integer-to-float conversions.
+__global__ void __launch_bounds__(256) x_to_half_kernel(const uint4* __restrict__ xq, uint4* __restrict__ x16,
+                                                        i64 n16) {
   const i64 e = (i64)blockIdx.x * 256 + threadIdx.x;
-  if (e >= n4) return;
-  const uint32_t w = __ldcs(xq + e);
-  const __half2 lo = __floats2half2_rn((float)sx8(w, 0), (float)sx8(w, 1));
-  const __half2 hi = __floats2half2_rn((float)sx8(w, 2), (float)sx8(w, 3));
-  uint2 o;
-  o.x = *reinterpret_cast<const uint32_t*>(&lo);
-  o.y = *reinterpret_cast<const uint32_t*>(&hi);
-  __stcs(x16 + e, o);
+  if (e >= n16) return;
+  const uint4 w = __ldcs(xq + e);
+  const uint32_t ww[4] = {w.x ^ 0x80808080u, w.y ^ 0x80808080u, w.z ^ 0x80808080u, w.w ^ 0x80808080u};
+  const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+  uint32_t o[8];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      const uint32_t bits = __byte_perm(ww[k], 0x64646464u, p ? 0x7372u : 0x7170u);  // {0x64, b(2p+1), 0x64, b(2p)}
+      const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&bits), off);
+      o[k * 2 + p] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+  }
+  __stcs(x16 + 2 * e, make_uint4(o[0], o[1], o[2], o[3]));
+  __stcs(x16 + 2 * e + 1, make_uint4(o[4], o[5], o[6], o[7]));
 }
 
 }  // namespace
@@ -480,9 +491,9 @@ ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16,
   const int TM = d.Q < 128 ? d.Q : 128;
   const uint64_t T = (uint64_t)d.b * d.L;
   // X as FP16 (exact images of the int8 codes)
-  const i64 n4 = (i64)T * d.H * d.P / 4;
-  x_to_half_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(xq),
-                                                                 static_cast<uint2*>(x16), n4);
+  const i64 n16 = (i64)T * d.H * d.P / 16;   // P = 64: a multiple of 16
+  x_to_half_kernel<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint4*>(xq),
+                                                                  static_cast<uint4*>(x16), n16);
   SSDI8_LAUNCH_CHECK();
   CUtensorMap tm_C, tm_h, tm_x, tm_cb, tm_y;
   {
