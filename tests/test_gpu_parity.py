@@ -445,8 +445,9 @@ def test_layer_fwd_host_matches_the_device_path_bit_for_bit(flags, batch):
         assert np.array_equal(y.numpy(), y_dev) and np.array_equal(fin.numpy(), fin_dev)
 
 
+@pytest.mark.parametrize("flags", [0, 1, 3], ids=["default", "fp16_operand", "fp16_operand_int8_state"])
 @pytest.mark.parametrize("cfg", [SMALL[1], SMALL[3]], ids=lambda c: c.name)
-def test_layer_fwd_matches_the_separate_calls_bit_for_bit(cfg):
+def test_layer_fwd_matches_the_separate_calls_bit_for_bit(cfg, flags):
     """ssdi8_layer_fwd (fp32 device tensors in, side-stream overlap inside) == three quantiser calls +
     ssdi8_chunk_scan_fwd; run three times in a row on the same workspace."""
     import torch
@@ -454,7 +455,7 @@ def test_layer_fwd_matches_the_separate_calls_bit_for_bit(cfg):
     gh = _harness()
     t = inputs.make_prefill(cfg)
     q = orc.prepare_quantized(cfg, t)
-    y_dev, fin_dev, _ = gh.gpu_fwd(cfg, q, taps=())
+    y_dev, fin_dev, _ = gh.gpu_fwd(cfg, q, taps=(), flags=flags)
     dims = bd.dims_of(cfg)
     dv = {k: gh.dev(q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "A", "D")}
     dv.update({k: gh.dev(t[k]) for k in ("x", "B", "C", "dt")})
@@ -462,10 +463,10 @@ def test_layer_fwd_matches_the_separate_calls_bit_for_bit(cfg):
     fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     args = bd.make_layer_args(y=y, final_state=fin, status=status, **dv)
-    ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims, flags), dtype=torch.uint8, device="cuda")
     for rep in range(3):
         y.fill_(float("nan")); fin.fill_(float("nan"))
-        bd.ssdi8_layer_fwd(dims, args, ws)
+        bd.ssdi8_layer_fwd(dims, args, ws, flags)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert np.array_equal(y.cpu().numpy(), y_dev) and np.array_equal(fin.cpu().numpy(), fin_dev)
