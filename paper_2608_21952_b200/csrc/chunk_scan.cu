@@ -388,8 +388,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
       const uint32_t ph4 = (n >> 2) & 1;
-      mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
-      mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
+      mbar_wait_relaxed(&bars[B_TOK_FULL + t3], ph4, a.status);
+      mbar_wait_relaxed(&bars[B_CB_FULL + ci], ph4, a.status);
       mask_tile<TAPS>(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
