@@ -7,7 +7,9 @@
 //   S[p,n]      = fmaf(Gamma_k, S[p,n], loc[p,n])                                      (Eq. 6)
 // and final_state = S after the last chunk.  The running state lives in registers: the
 // accumulator has the state index n on the TMEM lanes, so thread (lane n) keeps S[., n] for its
-// 32 channels p.  Operand tiles arrive by TMA, double-buffered across chunks; hq leaves through
+// 32 channels p.  Operand tiles arrive by TMA, double-buffered across chunks; each re-quantisation
+// warp owns whole 32-token slabs and issues their MMAs itself (the accumulator is opened by the warp
+// that owns slab 0, the others order their MMAs after it through an mbarrier); hq leaves through
 // a shared-memory tile and one TMA store per chunk.  Same arithmetic, operation for operation,
 // as the separate kernels (chunk_state.cu, state_passing.cu).
 // I8S = true selects the paper's own state format (Section 4.2, Eq. 4 and Eq. 7): the state is an
@@ -43,7 +45,7 @@ constexpr uint32_t OFF_COL = OFF_LUT + 2048;      // [64] loc scale, [64] 1 / s_
 constexpr uint32_t OFF_BAR = OFF_COL + 768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
 
-enum { B_FULL = 0, B_RQ = 2, B_MMA = 4, B_ACC_FREE = 5, B_COUNT = 6 };
+enum { B_FULL = 0, B_OPEN = 2, B_MMA = 4, B_ACC_FREE = 5, B_COUNT = 6 };
 
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -75,9 +77,8 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
   if (tid == 0) {
     mbar_init(&bars[B_FULL], 1);
     mbar_init(&bars[B_FULL + 1], 1);
-    mbar_init(&bars[B_RQ], kQuantThreads / 32);
-    mbar_init(&bars[B_RQ + 1], kQuantThreads / 32);
-    mbar_init(&bars[B_MMA], 1);
+    mbar_init(&bars[B_OPEN], 1);
+    mbar_init(&bars[B_MMA], Q / 32 < kQuantThreads / 32 ? Q / 32 : kQuantThreads / 32);   // one commit per issuing warp
     mbar_init(&bars[B_ACC_FREE], kStateThreads / 32);
     fence_mbar_init();
     tma_prefetch_desc(&tm_B);
@@ -129,51 +130,61 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
       const i64 tok0 = (i64)b * d.L + (i64)k * Q;
       mbar_wait_relaxed(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+      // a warp owns whole 32-token slabs (slab = one MMA): rows of a slab are split over the lanes,
+      // and the warp's lane 0 issues the slab's MMA as soon as the warp has re-quantised it, so no
+      // warp waits for another.  The accumulator is opened by the MMA of slab 0 (accumulate = 0);
+      // the other issuing threads order their first MMA of the chunk after it through B_OPEN.
+      const int qw = qt >> 5;
+      const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
+      const uint32_t idesc = idesc_s8(N, 64, 1, 1);
 #pragma unroll 1
-      for (int i = qt >> lq; i < Q; i += kQuantThreads >> lq) {
-        uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
-        const uint4 w4 = *ptr;
-        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-        const float l = lut[i];
-        const float2 l2 = make_float2(l, l);
-        uint32_t o[4];
+      for (int sl = qw; sl < Q / 32; sl += kQuantThreads / 32) {
+#pragma unroll 1
+        for (int i = sl * 32 + (lane >> lq); i < sl * 32 + 32; i += 32 >> lq) {
+          uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
+          const uint4 w4 = *ptr;
+          const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+          const float l = lut[i];
+          const float2 l2 = make_float2(l, l);
+          uint32_t o[4];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          uint32_t q4[4];
+          for (int w = 0; w < 4; ++w) {
+            uint32_t q4[4];
 #pragma unroll
-          for (int e = 0; e < 4; e += 2) {
-            const float2 xf = __fadd2_rn(
-                make_float2(__uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7650u + e)),
-                            __uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7651u + e))),
-                make_float2(-kMagicIn, -kMagicIn));
-            const float2 v2 = __fmul2_rn(__fmul2_rn(xf, make_float2(rx[w * 4 + e], rx[w * 4 + e + 1])), l2);
-            q4[e] = rne_clamp_bits(v2.x);
-            q4[e + 1] = rne_clamp_bits(v2.y);
+            for (int e = 0; e < 4; e += 2) {
+              const float2 xf = __fadd2_rn(
+                  make_float2(__uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7650u + e)),
+                              __uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7651u + e))),
+                  make_float2(-kMagicIn, -kMagicIn));
+              const float2 v2 = __fmul2_rn(__fmul2_rn(xf, make_float2(rx[w * 4 + e], rx[w * 4 + e + 1])), l2);
+              q4[e] = rne_clamp_bits(v2.x);
+              q4[e + 1] = rne_clamp_bits(v2.y);
+            }
+            o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
           }
-          o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
+          const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+          *ptr = v;
+          if (TAPS && a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
         }
-        const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
-        *ptr = v;
-        if (TAPS && a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = v;
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars[B_RQ + s]);
-      // ---- acc[n][p] = sum_i Bq[i][n] Xs_q[i][p], issued as soon as the whole tile is re-quantised
-      // and the state warps have read the previous accumulator (overlaps their hq staging)
-      if (qt == 0) {
-        mbar_wait(&bars[B_RQ + s], (k >> 1) & 1, a.status);
-        mbar_wait_relaxed(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);
+      if (lane == 0 && qw < Q / 32) {
+        if (qw == 0) {
+          mbar_wait_relaxed(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
+        } else {
+          mbar_wait(&bars[B_OPEN], k & 1, a.status);
+        }
         tc_fence_after();
-        const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
-        const uint32_t idesc = idesc_s8(N, 64, 1, 1);
-        // descriptors advance by a constant per 32-token slab (their low bits are the address >> 4):
-        // the issuing thread is on this group's critical path, so the loop is kept to an add per operand
-        uint64_t da = tile_desc(sBa, (uint32_t)N), db = tile_desc(sXa, 64);
-        const uint64_t sa = (uint64_t)((32 * N) >> 4), sb = (uint64_t)((32 * 64) >> 4);
 #pragma unroll 1
-        for (int st = 0; st < Q / 32; ++st, da += sa, db += sb) mma_s8_ss(tmem, da, db, idesc, st > 0);
-        mma_commit(&bars[B_MMA]);
+        for (int sl = qw; sl < Q / 32; sl += kQuantThreads / 32) {
+          mma_s8_ss(tmem, tile_desc(sBa + 32 * sl * N, (uint32_t)N), tile_desc(sXa + 32 * sl * 64, 64), idesc, sl > 0);
+          if (sl == 0) {
+            tc_fence_before();
+            mbar_arrive(&bars[B_OPEN]);
+          }
+        }
+        mma_commit(&bars[B_MMA]);   // arrives when this thread's MMAs are done
       }
       __syncwarp();
     }
