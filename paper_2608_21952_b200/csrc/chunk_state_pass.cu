@@ -171,7 +171,7 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       __syncwarp();
       if (lane == 0 && qw < Q / 32) {
         if (qw == 0) {
-          mbar_wait_relaxed(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
+          mbar_wait(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
         } else {
           mbar_wait(&bars[B_OPEN], k & 1, a.status);
         }
