@@ -127,3 +127,34 @@ def test_reciprocal_fast_path_of_the_quantiser_is_exact():
     fast = e <= np.float32(0.49994)
     assert np.array_equal(kf[fast], d[fast])
     assert 0.2 < fast.mean() < 1.0 and (~fast).sum() > 1000      # both paths exercised
+
+
+def test_host_side_argument_errors_of_the_layer_and_entry_calls():
+    """The one-call layer entries and the entry quantiser validate on the host before any CUDA
+    call: these checks run without a device."""
+    from paper_2608_21952_b200 import binding as bd
+    from paper_2608_21952_b200.inputs import CONFIGS
+    L = bd._lib
+    d = bd.dims_of(CONFIGS["cfg0"])
+    a = bd.LayerArgs()
+    for fn in (L.ssdi8_layer_fwd, L.ssdi8_layer_fwd_host):
+        assert fn(None, None, None, 0, 0, None) == bd.ERR_NULL
+        assert fn(C.byref(d), C.byref(a), 4096, 1 << 40, 0, None) == bd.ERR_NULL          # no tensors
+    for k in ("x", "B", "C", "dt", "A", "s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "y"):
+        setattr(a, k, 4096)
+    for fn, size in ((L.ssdi8_layer_fwd, L.ssdi8_layer_fwd_workspace_bytes),
+                     (L.ssdi8_layer_fwd_host, L.ssdi8_layer_fwd_host_scratch_bytes)):
+        need = size(C.byref(d), 0)
+        assert need > 0
+        assert fn(C.byref(d), C.byref(a), 4096, need - 1, 0, None) == bd.ERR_WORKSPACE
+        assert fn(C.byref(d), C.byref(a), 4096 + 8, need, 0, None) == bd.ERR_ALIGN
+        assert fn(C.byref(d), C.byref(a), 4096, need, 1 << 13, None) == bd.ERR_UNSUPPORTED
+        assert size(C.byref(d), 1) > need                      # the FP16 operand needs the FP16 image of x
+        bad = bd.dims_of(CONFIGS["cfg0"].replace(chunk=48))
+        assert size(C.byref(bad), 0) == 0
+        assert fn(C.byref(bad), C.byref(a), 4096, 1 << 40, 0, None) == bd.ERR_SHAPE
+    q = L.ssdi8_quantize_entry
+    assert q(None, 0, 16, 64, 1, 16, 4096, 4096, 4096, 4096, 4096, 4096, None) == bd.ERR_NULL
+    assert q(4096, 3, 16, 64, 1, 16, 4096, 4096, 4096, 4096, 4096, 4096, None) == bd.ERR_UNSUPPORTED
+    assert q(4096, 0, 16, 62, 1, 16, 4096, 4096, 4096, 4096, 4096, 4096, None) == bd.ERR_SHAPE
+    assert q(4096 + 4, 0, 16, 64, 1, 16, 4096, 4096, 4096, 4096, 4096, 4096, None) == bd.ERR_ALIGN
