@@ -360,19 +360,29 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
         mbar_wait(&bars[B_ACC_FREE + s2], ph2 ^ 1, a.status);
         mbar_wait(&bars[B_CH_FULL], n & 1, a.status);
         tc_fence_after();
+        // descriptors advance by a constant per 32-byte K step (their low bits are the address >> 4):
+        // this thread's issue time is on the path from a freed accumulator to the next epilogue
+        {
+          uint64_t da = tile_desc(sbase + OFF_C, RBN), db = tile_desc(sbase + OFF_H, RBN);
 #pragma unroll 1
-        for (int q = 0; q < N / 32; ++q)
-          mma_s8_ss(acc, tile_desc(sbase + OFF_C + 32 * q, RBN), tile_desc(sbase + OFF_H + 32 * q, RBN),
-                    idesc_off, q > 0);
+          for (int q = 0; q < N / 32; ++q, da += 2, db += 2) mma_s8_ss(acc, da, db, idesc_off, q > 0);
+        }
         mma_commit(&bars[B_CH_FREE]);
         mbar_wait(&bars[B_MQ + ci], ph4, a.status);
         mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);
         tc_fence_after();
+        {
+          uint64_t db = tile_desc(sbase + OFF_X + s2 * 16384, 64);
+          uint32_t first = 0;
 #pragma unroll 1
-        for (int q = 0; q < KJ / 32; ++q) {
-          const uint32_t k0 = 32u * q;
-          mma_s8_ss(acc + 64, tile_desc(sbase + cb_offset(ci) + (k0 / RBQ) * PANEL + (k0 % RBQ), RBQ),
-                    tile_desc(sbase + OFF_X + s2 * 16384 + k0 * 64, 64), idesc_diag, q > 0);
+          for (uint32_t pn = 0; pn < (uint32_t)KJ / RBQ; ++pn) {     // panels of RBQ columns of Mq
+            uint64_t da = tile_desc(sbase + cb_offset(ci) + pn * PANEL, RBQ);
+#pragma unroll 1
+            for (uint32_t q = 0; q < RBQ / 32; ++q, da += 2, db += (32 * 64) >> 4) {
+              mma_s8_ss(acc + 64, da, db, idesc_diag, first);
+              first = 1;
+            }
+          }
         }
         mma_commit(&bars[B_CB_FREE + ci]);
         mma_commit(&bars[B_ACC + s2]);
