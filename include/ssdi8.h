@@ -234,11 +234,12 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  *   the streams join before ChunkState.  workspace: 256-byte aligned,
  *   ssdi8_layer_fwd_workspace_bytes(dims, flags) bytes (the int8 tensors plus ssdi8_workspace_bytes).
  * ssdi8_layer_fwd_host: x, B, C, dt, y, final_state, status are HOST pointers (page-locked memory, or
- *   the copies neither overlap nor run asynchronously), the rest DEVICE pointers.  One batch element
- *   at a time (Algorithm 2 has no cross-batch term): the host->device copies of element b+1 and the
- *   device->host copy of y of element b-1 run on two more side streams while the kernels of element
- *   b run, so both directions of the host link stay busy.  scratch: DEVICE, 256-byte aligned,
- *   ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes (two stages of one element's tensors).
+ *   the copies neither overlap nor run asynchronously), the rest DEVICE pointers.  One slice at a
+ *   time, a slice being a batch element or, when an element's x exceeds 96 MB, an equal range of its
+ *   heads (Algorithm 2 has no term across batch elements or heads): the host->device copies of slice
+ *   i+1 and the device->host copy of y of slice i-1 run on two more side streams while the kernels
+ *   of slice i run, so both directions of the host link stay busy.  scratch: DEVICE, 256-byte
+ *   aligned, ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes (two stages of one slice's tensors).
  * Layouts as in ssdi8_fwd_args_t; D, corr, init_state, final_state, status may be NULL.  Both calls
  * return once everything is enqueued and leave `stream` waiting for the last piece of work, so
  * synchronising `stream` completes them.  flags: any of SSDI8_FLAG_INT8_STATE, SSDI8_FLAG_Y_FP16,

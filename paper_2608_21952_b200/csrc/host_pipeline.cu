@@ -23,6 +23,7 @@ struct StageBuf {
 };
 struct Layout {
   StageBuf st[kStages];
+  float* dt_full[2];   // dt of a whole batch element (all heads), alternating by element
   void* ws;
   int32_t* status;
   size_t ws_bytes, total;
@@ -30,7 +31,7 @@ struct Layout {
 
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-Layout make_layout(const ssdi8_dims_t& d1, uint8_t* base, uint32_t flags) {
+Layout make_layout(const ssdi8_dims_t& d1, int full_heads, uint8_t* base, uint32_t flags) {
   Layout lo;
   const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
   const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
@@ -47,6 +48,7 @@ Layout make_layout(const ssdi8_dims_t& d1, uint8_t* base, uint32_t flags) {
     lo.st[s].Bq = reinterpret_cast<int8_t*>(take(nb));
     lo.st[s].Cq = reinterpret_cast<int8_t*>(take(nb));
   }
+  for (int e = 0; e < 2; ++e) lo.dt_full[e] = reinterpret_cast<float*>(take((size_t)d1.seqlen * full_heads * 4));
   lo.status = reinterpret_cast<int32_t*>(take(256));
   lo.ws_bytes = ssdi8_workspace_bytes(&d1, flags);
   lo.ws = take(lo.ws_bytes);
@@ -140,6 +142,37 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
                     ws_bytes, st, false);
 }
 
+// How many equal head ranges a batch element is cut into for the host pipeline: halved while a
+// slice's fp32 x is larger than 96 MB (below that the fixed cost of a copy outweighs the shorter
+// fill and drain of the pipeline: measured on PCIe 5 x16, a 21 MB copy runs at 47 GB/s, a 350 MB
+// copy at 55 GB/s), as long as the cut keeps groups whole (and their step-size
+// vectors 16-byte aligned) or there is a single group.
+int choose_parts(const ssdi8_dims_t& d) {
+  int np = 1;
+  auto can = [&](int n) {
+    if (d.nheads % n != 0) return false;
+    if (d.ngroups == 1) return true;
+    return d.ngroups % n == 0 && (d.ngroups / n) % 4 == 0;
+  };
+  const size_t x_bytes = (size_t)d.seqlen * d.nheads * d.headdim * 4;
+  while (np < 4 && can(np * 2) && x_bytes / np > ((size_t)96 << 20)) np *= 2;
+  return np;
+}
+ssdi8_dims_t slice_dims(const ssdi8_dims_t& d, int nparts) {
+  ssdi8_dims_t s = d;
+  s.batch = 1;
+  s.nheads = d.nheads / nparts;
+  s.ngroups = d.ngroups == 1 ? 1 : d.ngroups / nparts;
+  return s;
+}
+
+// rows of `width` bytes from one pitched buffer to another; one plain copy when both are compact
+cudaError_t copy_rows(void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, size_t rows,
+                      cudaMemcpyKind kind, cudaStream_t st) {
+  if (dpitch == width && spitch == width) return cudaMemcpyAsync(dst, src, width * rows, kind, st);
+  return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, rows, kind, st);
+}
+
 bool layer_args_ok(const ssdi8_layer_args_t* a) {
   return a->x && a->B && a->C && a->dt && a->A && a->s_x && a->s_B && a->s_C && a->s_xs && a->s_cb && a->s_h && a->y;
 }
@@ -178,10 +211,10 @@ ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_
 
 size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
   if (!dims || dims->batch <= 0) return 0;
-  ssdi8_dims_t d1 = *dims;
-  d1.batch = 1;
+  if (ssdi8_workspace_bytes(dims, flags) == 0) return 0;   // unsupported dimensions or flags
+  const ssdi8_dims_t d1 = slice_dims(*dims, choose_parts(*dims));
   if (ssdi8_workspace_bytes(&d1, flags) == 0) return 0;
-  return make_layout(d1, nullptr, flags).total;
+  return make_layout(d1, dims->nheads, nullptr, flags).total;
 }
 
 ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_args_t* a, void* scratch,
@@ -193,16 +226,18 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
   if (need == 0) return SSDI8_ERR_SHAPE;
   if (scratch_bytes < need) return SSDI8_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(scratch) & 255) return SSDI8_ERR_ALIGN;
-  ssdi8_dims_t d1 = *dims;
-  d1.batch = 1;
-  const Layout lo = make_layout(d1, static_cast<uint8_t*>(scratch), flags);
+  // a slice = one batch element, or an equal part of its heads when an element is large: the
+  // pipeline fills and drains with one slice's copies exposed, so smaller slices hide more
+  const int nparts = choose_parts(*dims);
+  const ssdi8_dims_t d1 = slice_dims(*dims, nparts);
+  const Layout lo = make_layout(d1, dims->nheads, static_cast<uint8_t*>(scratch), flags);
   Plumbing* p = nullptr;
   ssdi8_status_t s = get_plumbing(&p);
   if (s != SSDI8_OK) return s;
   cudaStream_t s_cmp = static_cast<cudaStream_t>(stream);
-  const size_t nx = (size_t)d1.seqlen * d1.nheads * d1.headdim, nb = (size_t)d1.seqlen * d1.ngroups * d1.dstate;
-  const size_t ndt = (size_t)d1.seqlen * d1.nheads, nfin = (size_t)d1.nheads * d1.headdim * d1.dstate;
-
+  const size_t L = dims->seqlen, H = dims->nheads, P = dims->headdim, N = dims->dstate, G = dims->ngroups;
+  const size_t Hs = d1.nheads, Gs = d1.ngroups;
+  const size_t nfin = Hs * P * N;
   const size_t yb = (flags & (SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? 2 : 4;  // bytes per element of y
   // everything below is ordered after the work already in the caller's stream
   SSDI8_CUDA_CHECK(cudaMemsetAsync(lo.status, 0, sizeof(int32_t), s_cmp));
@@ -210,35 +245,57 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_in, p->start, 0));
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_out, p->start, 0));
 
-  for (int b = 0; b < dims->batch; ++b) {
-    const int st = b % kStages;
+  const int nslices = dims->batch * nparts;
+  for (int i = 0; i < nslices; ++i) {
+    const size_t b = (size_t)(i / nparts), part = (size_t)(i % nparts);
+    const size_t h0 = part * Hs, g0 = (G == 1) ? 0 : part * Gs;   // first head and first group of the slice
+    const int st = i % kStages;
     const StageBuf& sb = lo.st[st];
-    // inputs of element b: the kernels of element b - kStages have finished with this stage
-    if (b >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_in, p->cmp_done[st], 0));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.x, a->x + (size_t)b * nx, nx * 4, cudaMemcpyHostToDevice, p->s_in));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.B, a->B + (size_t)b * nb, nb * 4, cudaMemcpyHostToDevice, p->s_in));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.C, a->C + (size_t)b * nb, nb * 4, cudaMemcpyHostToDevice, p->s_in));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.dt, a->dt + (size_t)b * ndt, ndt * 4, cudaMemcpyHostToDevice, p->s_in));
+    // inputs of the slice (rows of L tokens, strided in the host tensors, compact on the device):
+    // the kernels of slice i - kStages have finished with this stage
+    if (i >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_in, p->cmp_done[st], 0));
+    SSDI8_CUDA_CHECK(copy_rows(sb.x, Hs * P * 4, a->x + (b * L * H + h0) * P, H * P * 4, Hs * P * 4, L,
+                                       cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(copy_rows(sb.B, Gs * N * 4, a->B + (b * L * G + g0) * N, G * N * 4, Gs * N * 4, L,
+                                       cudaMemcpyHostToDevice, p->s_in));
+    SSDI8_CUDA_CHECK(copy_rows(sb.C, Gs * N * 4, a->C + (b * L * G + g0) * N, G * N * 4, Gs * N * 4, L,
+                                       cudaMemcpyHostToDevice, p->s_in));
+    // dt has short rows (4 bytes per head): it crosses the link once per element in one piece and is
+    // cut into head ranges on the device
+    if (nparts == 1) {
+      SSDI8_CUDA_CHECK(cudaMemcpyAsync(sb.dt, a->dt + b * L * H, L * H * 4, cudaMemcpyHostToDevice, p->s_in));
+    } else {
+      if (part == 0)
+        SSDI8_CUDA_CHECK(cudaMemcpyAsync(lo.dt_full[b & 1], a->dt + b * L * H, L * H * 4, cudaMemcpyHostToDevice, p->s_in));
+      SSDI8_CUDA_CHECK(copy_rows(sb.dt, Hs * 4, lo.dt_full[b & 1] + h0, H * 4, Hs * 4, L, cudaMemcpyDeviceToDevice,
+                                 p->s_in));
+    }
     SSDI8_CUDA_CHECK(cudaEventRecord(p->in_done[st], p->s_in));
-    // kernels of element b: its inputs have arrived, and y of element b - kStages has left
+    // kernels of the slice: its inputs have arrived, and y of slice i - kStages has left
     SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->in_done[st], 0));
-    if (b >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
-    s = layer_step(d1, *a, sb.x, sb.B, sb.C, sb.dt, a->init_state ? a->init_state + (size_t)b * nfin : nullptr,
-                   sb.y, a->final_state ? sb.fin : nullptr, lo.status, sb.xq, sb.Bq, sb.Cq, lo.ws, lo.ws_bytes, flags,
-                   *p, s_cmp);
+    if (i >= kStages) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
+    ssdi8_layer_args_t as = *a;   // per-head and per-group vectors of the slice
+    as.A = a->A + h0;
+    as.D = a->D ? a->D + h0 : nullptr;
+    as.corr = a->corr ? a->corr + h0 * P : nullptr;
+    as.s_x = a->s_x + h0 * P; as.s_xs = a->s_xs + h0 * P; as.s_h = a->s_h + h0 * P;
+    as.s_B = a->s_B + g0; as.s_C = a->s_C + g0; as.s_cb = a->s_cb + g0;
+    const size_t fin_off = (b * H + h0) * P * N;
+    s = layer_step(d1, as, sb.x, sb.B, sb.C, sb.dt, a->init_state ? a->init_state + fin_off : nullptr, sb.y,
+                   a->final_state ? sb.fin : nullptr, lo.status, sb.xq, sb.Bq, sb.Cq, lo.ws, lo.ws_bytes, flags, *p,
+                   s_cmp);
     if (s != SSDI8_OK) return s;
     SSDI8_CUDA_CHECK(cudaEventRecord(p->cmp_done[st], s_cmp));
-    // outputs of element b
+    // outputs of the slice
     SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p->s_out, p->cmp_done[st], 0));
-    SSDI8_CUDA_CHECK(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(a->y) + (size_t)b * nx * yb, sb.y, nx * yb,
-                                     cudaMemcpyDeviceToHost, p->s_out));
+    SSDI8_CUDA_CHECK(copy_rows(reinterpret_cast<uint8_t*>(a->y) + (b * L * H + h0) * P * yb, H * P * yb, sb.y,
+                                       Hs * P * yb, Hs * P * yb, L, cudaMemcpyDeviceToHost, p->s_out));
     if (a->final_state)
-      SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->final_state + (size_t)b * nfin, sb.fin, nfin * 4, cudaMemcpyDeviceToHost,
-                                       p->s_out));
+      SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->final_state + fin_off, sb.fin, nfin * 4, cudaMemcpyDeviceToHost, p->s_out));
     SSDI8_CUDA_CHECK(cudaEventRecord(p->out_done[st], p->s_out));
   }
-  // the caller's stream ends after the last copies (the last kStages elements' events cover all)
-  for (int st = 0; st < kStages && st < dims->batch; ++st)
+  // the caller's stream ends after the last copies (the last kStages slices' events cover all)
+  for (int st = 0; st < kStages && st < nslices; ++st)
     SSDI8_CUDA_CHECK(cudaStreamWaitEvent(s_cmp, p->out_done[st], 0));
   if (a->status)
     SSDI8_CUDA_CHECK(cudaMemcpyAsync(a->status, lo.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s_cmp));

@@ -579,3 +579,56 @@ def test_fwd_fp16_operand_against_the_oracle_mode(cfg):
     bd.ssdi8_chunk_scan_fwd(dims, args16, ws, flags=bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16)
     torch.cuda.synchronize()
     assert torch.equal(y16.cpu().view(torch.int16), y.cpu().half().view(torch.int16))
+
+
+@pytest.mark.parametrize("G", [1, 8])
+def test_layer_fwd_host_with_head_range_slices(G):
+    """A batch element whose x exceeds 96 MB is cut into head ranges by the host entry (strided
+    copies, offset step-size vectors, per-range groups): the result must equal the whole-batch
+    device call bit for bit.  Scales come from the library's own calibration (parity of every
+    kernel with the oracle is established by the tests above)."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    cfg = SSDConfig("host_wide", 2, 4096, 128, 64, 64, G, 256, 0.01, 50.0, 41)   # 134 MB of x per element
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.2)
+    dims = bd.dims_of(cfg)
+    dv = {k: torch.from_numpy(t[k]).cuda() for k in ("x", "B", "C", "dt", "A", "D")}
+    dinit = torch.from_numpy(init).cuda()
+    T = cfg.tokens
+    i8 = lambda k: torch.empty(t[k].shape, dtype=torch.int8, device="cuda")
+    xq, Bq, Cq = i8("x"), i8("B"), i8("C")
+    z = lambda n: torch.empty(n, device="cuda")
+    s_x, s_B, s_C = z(cfg.channels), z(cfg.ngroups), z(cfg.ngroups)
+    s_xs, s_cb, s_h = z(cfg.channels), z(cfg.ngroups), z(cfg.channels)
+    bd.ssdi8_quantize_act(dv["x"], T, cfg.channels, 1, s_x, 1, xq)
+    bd.ssdi8_quantize_act(dv["B"], T, cfg.ngroups, cfg.dstate, s_B, 1, Bq)
+    bd.ssdi8_quantize_act(dv["C"], T, cfg.ngroups, cfg.dstate, s_C, 1, Cq)
+    ws = bd.alloc_workspace(dims)
+    cal = bd.make_fwd_args(xq=xq, Bq=Bq, Cq=Cq, s_x=s_x, s_B=s_B, s_C=s_C, dt=dv["dt"], A=dv["A"], init_state=dinit)
+    bd.ssdi8_calibrate(dims, cal, s_xs, s_cb, s_h, ws)
+    scales = dict(s_x=s_x, s_B=s_B, s_C=s_C, s_xs=s_xs, s_cb=s_cb, s_h=s_h, A=dv["A"], D=dv["D"])
+    # whole-batch device call
+    y_d = torch.empty(t["x"].shape, device="cuda")
+    fin_d = torch.empty(init.shape, device="cuda")
+    st_d = torch.zeros(1, dtype=torch.int32, device="cuda")
+    a_d = bd.make_layer_args(x=dv["x"], B=dv["B"], C=dv["C"], dt=dv["dt"], init_state=dinit, y=y_d,
+                             final_state=fin_d, status=st_d, **scales)
+    lws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims), dtype=torch.uint8, device="cuda")
+    bd.ssdi8_layer_fwd(dims, a_d, lws)
+    # host call: two head ranges per batch element
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    host = {k: pin(t[k]) for k in ("x", "B", "C", "dt")}
+    y_h = torch.full(t["x"].shape, float("nan")).pin_memory()
+    fin_h = torch.full(init.shape, float("nan")).pin_memory()
+    st_h = torch.full((1,), -99, dtype=torch.int32).pin_memory()
+    a_h = bd.make_host_args(y=y_h, final_state=fin_h, status=st_h, init_state=dinit, **host, **scales)
+    need = bd.ssdi8_layer_fwd_host_scratch_bytes(dims)
+    # sized for half of the heads: well below the need of the same element at half the length, uncut
+    uncut = bd.ssdi8_layer_fwd_host_scratch_bytes(bd.dims_of(cfg.replace(seqlen=2048, nheads=64, ngroups=max(1, G // 2))))
+    assert need < 2.2 * uncut
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    bd.ssdi8_layer_fwd_host(dims, a_h, scratch)
+    torch.cuda.synchronize()
+    assert int(st_d.item()) == 0 and int(st_h[0]) == 0
+    assert torch.equal(y_h, y_d.cpu()) and torch.equal(fin_h, fin_d.cpu())
