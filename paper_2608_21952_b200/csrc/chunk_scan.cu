@@ -32,6 +32,7 @@ struct ScanArgs {
   ScanTaps taps;
   Dims d;
   int ntiles, per_cta;
+  int hpg;  // heads per group
 };
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
@@ -78,31 +79,36 @@ __device__ __forceinline__ uint32_t pack4_rne(float2 a, float2 b) {
 }
 
 struct Tile {
-  int b, k, h, g, it, KJ;
-  i64 tok0, unit;  // unit = (b*H + h)*c + k
+  int b, k, h, g, hg, it, KJ;  // hg = h - g * (heads per group)
+  i64 tok0, unit;              // unit = (b*H + h)*c + k
 };
-// the tile after x in (it, h, k, b) order, without divisions
-__device__ __forceinline__ void next_tile(Tile& x, const Dims& d, int TM, int ntpu) {
+// the tile after x in (it, h, k, b) order, without divisions (every role walks the tiles, so this
+// is inlined many times and runs once per tile on each role's critical path)
+__device__ __forceinline__ void next_tile(Tile& x, const ScanArgs& a, int TM, int ntpu) {
   if (++x.it == ntpu) {
     x.it = 0;
-    if (++x.h == d.H) {
-      x.h = 0;
-      if (++x.k == d.c) { x.k = 0; ++x.b; }
+    ++x.h;
+    if (++x.hg == a.hpg) { x.hg = 0; ++x.g; }
+    if (x.h == a.d.H) {
+      x.h = 0; x.g = 0; x.hg = 0;
+      x.tok0 += a.d.Q;               // (b, k) -> (b, k + 1) or (b + 1, 0): L = c Q
+      if (++x.k == a.d.c) { x.k = 0; ++x.b; }
     }
-    x.g = x.h / (d.H / d.G);
-    x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
-    x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
+    x.unit = ((i64)x.b * a.d.H + x.h) * a.d.c + x.k;
   }
   x.KJ = (x.it + 1) * TM;
 }
-__device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntpu) {
+// first tile of a CTA: computed once, by one thread, and handed to the roles through shared memory
+__device__ __forceinline__ Tile decode_tile(int t, const ScanArgs& a, int TM, int ntpu) {
+  const Dims& d = a.d;
   Tile x;
   x.it = t % ntpu;
   int u = t / ntpu;
   x.h = u % d.H; u /= d.H;
   x.k = u % d.c;
   x.b = u / d.c;
-  x.g = x.h / (d.H / d.G);
+  x.g = x.h / a.hpg;
+  x.hg = x.h - x.g * a.hpg;
   x.KJ = (x.it + 1) * TM;
   x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
   x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
@@ -272,6 +278,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   const int t_end = min(a.ntiles, t_begin + a.per_cta);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+  Tile* first_tile = reinterpret_cast<Tile*>(bars + B_COUNT + 2);
 
   if (tid == 0) {
     for (int s = 0; s < 4; ++s) {
@@ -292,6 +299,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     fence_mbar_init();
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_cb); tma_prefetch_desc(&tm_y);
+    *first_tile = decode_tile(t_begin, a, TM, ntpu);
   }
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
@@ -302,9 +310,9 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      Tile t = *first_tile;
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
         const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
         const uint32_t ph4 = (n >> 2) & 1, ph3 = (n >> 2) & 1;
         mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
@@ -322,9 +330,9 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   } else if (warp == 2) {
     // ------------------------------------------------------------ TMA producer: Cq, hq
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      Tile t = *first_tile;
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
         mbar_wait_relaxed(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
         mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
         tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
@@ -334,9 +342,9 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   } else if (warp == 3) {
     // ------------------------------------------------------------ TMA producer: xq rows
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      Tile t = *first_tile;
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
         const int s2 = n & 1;
         const uint32_t ph2 = (n >> 1) & 1;
         mbar_wait_relaxed(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
@@ -352,7 +360,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const uint32_t sbase = smem_u32(smem);
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
-        const int it = tix % ntpu;
+        const int it = ntpu == 1 ? 0 : (tix & 1);   // a CTA's first tile is the first of its chunk
         const int ci = cb_index(n, it, ntpu), s2 = n & 1;
         const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
         const int KJ = (it + 1) * TM;
@@ -392,8 +400,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     // ------------------------------------------------------------ mask warps: group g takes tiles n = g, g + 2, ...
     const int g = (warp - kMaskWarp0) / kGroupWarps;
     const int gtid = tid - (kMaskWarp0 + g * kGroupWarps) * 32;
-    Tile t = decode_tile(t_begin, d, TM, ntpu);
-    if (g) next_tile(t, d, TM, ntpu);
+    Tile t = *first_tile;
+    if (g) next_tile(t, a, TM, ntpu);
 #pragma unroll 1
     for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
@@ -404,8 +412,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
-      next_tile(t, d, TM, ntpu);
-      next_tile(t, d, TM, ntpu);
+      next_tile(t, a, TM, ntpu);
+      next_tile(t, a, TM, ntpu);
     }
   } else {
     // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
@@ -414,9 +422,9 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     const int ch = ew >> 2;                 // column half
     const int er = q * 32 + lane;           // row of the tile
     uint8_t* ystage = smem + OFF_YST + ew * 4096;
-    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    Tile t = *first_tile;
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
       const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n & 3;
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n >> 2) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
@@ -570,7 +578,7 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   const int ctas = ntiles < sms ? ntiles : sms;
   int per_cta = (ntiles + ctas - 1) / ctas;
   if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
-  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta};
+  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta, d.H / d.G};
   const size_t smem = SMEM_BYTES + 1024;
   const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
   const bool tp = taps.acc_off || taps.rowmax || taps.Mq || taps.acc_diag;

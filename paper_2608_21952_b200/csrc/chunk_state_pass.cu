@@ -129,7 +129,7 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       uint8_t* sX = smem + s * STAGE + OFF_X;
       float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
       const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-      mbar_wait_relaxed(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+      mbar_wait_inline<256>(&bars[B_FULL + s], (k >> 1) & 1, a.status);
       // a warp owns whole 32-token slabs (slab = one MMA): rows of a slab are split over the lanes,
       // and the warp's lane 0 issues the slab's MMA as soon as the warp has re-quantised it, so no
       // warp waits for another.  The accumulator is opened by the MMA of slab 0 (accumulate = 0);
@@ -171,9 +171,9 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       __syncwarp();
       if (lane == 0 && qw < Q / 32) {
         if (qw == 0) {
-          mbar_wait(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
+          mbar_wait_inline<0>(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
         } else {
-          mbar_wait(&bars[B_OPEN], k & 1, a.status);
+          mbar_wait_inline<0>(&bars[B_OPEN], k & 1, a.status);
         }
         tc_fence_after();
 #pragma unroll 1
@@ -249,7 +249,7 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
         tma_store_commit();
       }
       // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 16 channels at a time
-      mbar_wait_relaxed(&bars[B_MMA], k & 1, a.status);
+      mbar_wait_inline<256>(&bars[B_MMA], k & 1, a.status);
       tc_fence_after();
       if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
 #pragma unroll

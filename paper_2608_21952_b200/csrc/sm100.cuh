@@ -44,22 +44,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // order of a second.  On expiry the caller's status word is set and the wait returns; once
 // the word is set, every later wait of the grid gives up after a few polls, so the kernel runs
 // to its normal end (tensor memory is freed) quickly, with undefined results.
+// The polling loop is one out-of-line function: a call site is the first attempt and a branch, so
+// the many waits of a warp-specialised kernel do not bloat its instruction footprint.
 constexpr uint32_t kWaitCap = 1u << 17;
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
+static __device__ __noinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, int32_t* status,
+                                                   uint32_t sleep_ns) {
   for (uint32_t it = 0; it < kWaitCap; ++it) {
     if (mbar_try_wait(bar, parity)) return;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 255u) == 255u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
   }
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
+}
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
+  if (!mbar_try_wait(bar, parity)) mbar_wait_slow(bar, parity, status, 0u);
 }
 
 // The same bounded wait for warps whose wait is long and off the critical path (producers waiting
 // for a free slot, epilogue warps waiting for an accumulator): a failed poll is followed by a short
 // sleep, so the polling loop leaves the issue slots to the warps that compute.
 __device__ __forceinline__ void mbar_wait_relaxed(uint64_t* bar, uint32_t parity, int32_t* status) {
+  if (!mbar_try_wait(bar, parity)) mbar_wait_slow(bar, parity, status, 256u);
+}
+
+// Inline forms of both waits, for kernels with few wait sites and no registers to spare around a call.
+template <uint32_t SLEEP_NS>
+__device__ __forceinline__ void mbar_wait_inline(uint64_t* bar, uint32_t parity, int32_t* status) {
   for (uint32_t it = 0; it < kWaitCap; ++it) {
     if (mbar_try_wait(bar, parity)) return;
-    __nanosleep(256);
+    if (SLEEP_NS) __nanosleep(SLEEP_NS);
     if ((it & 255u) == 255u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
   }
   if (status) atomicExch(status, (int32_t)SSDI8_ERR_DEVICE_TIMEOUT);
