@@ -10,7 +10,11 @@
 // MMAs; warps 4-19 build Mq in place over CBq, as two groups of 8 warps that take alternate tiles
 // (two threads per output row in adjacent lanes, so each warp owns 16 rows and runs on its own,
 // without block barriers, and two tiles are in flight); warps 20-27 read the accumulators, form y
-// and store it through swizzled staging with TMA.  Every buffer has its own "free" barrier, released by whoever reads it last
+// and store it through a swizzled staging tile with coalesced 16-byte stores (a TMA store of rows this
+// short is slower and needs a proxy fence per tile), again as two groups (of 4 warps) on alternate
+// tiles, so one group's per-tile bookkeeping and waits run under the other's arithmetic.  Four
+// accumulator pairs and an xq buffer per chunk (shared by the chunk's two tiles) keep the MMAs of
+// the next tiles independent of the epilogue of the current ones.  Every buffer has its own "free" barrier, released by whoever reads it last
 // (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
 // hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
 // because every role executes different code at the same time.  No multicast; bounded waits.
@@ -28,6 +32,7 @@ using namespace sm100;
 struct ScanArgs {
   const float* s_x; const float* s_C; const float* s_cb; const float* s_h;
   const float* pack; const float* D; const float* corr;
+  uint8_t* y;       // [b*L][H][P] binary32 or 16-bit
   int32_t* status;
   ScanTaps taps;
   Dims d;
@@ -37,17 +42,22 @@ struct ScanArgs {
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
 constexpr int kMaskWarp0 = 4, kGroupWarps = 8;
-constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
-constexpr uint32_t kTmemCols = 256;  // accumulator pair a: acc_off at 128 a, acc_diag at 128 a + 64
+constexpr int kEpiWarp0 = 20, kEpiWarps = 8, kEpiGroupWarps = 4;
+constexpr uint32_t kTmemCols = 512;  // four accumulator pairs: acc_off at 128 a, acc_diag at 128 a + 64
 constexpr uint32_t PANEL = 16384;    // [128][128] int8
 // shared memory (bytes, from a 1024-byte aligned base)
 constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1-panel buffers
 constexpr uint32_t OFF_C = 98304;       // [128][N]
 constexpr uint32_t OFF_H = 114688;      // [64][N]
-constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]
-constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds; [128] row maxima)
-constexpr uint32_t TOK_BYTES = 6144;
-constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][128 B] y staging
+constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]: the xq rows of a chunk
+constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds), read by the mask warps
+constexpr uint32_t TOK_BYTES = 5120;
+// ring of 8 x what the epilogue needs of a tile: [128] row maxima and [128] exp(cs_i), written by the
+// mask warps, and the head's s_x, s_h and correction vectors ([64] each, bulk-loaded).  Eight deep so
+// that the mask of a tile never waits for the epilogue of an earlier one.
+constexpr uint32_t OFF_ROW = OFF_TOK + 4 * TOK_BYTES;
+constexpr uint32_t ROW_BYTES = 2048, ROW_COLS = 1024;
+constexpr uint32_t OFF_YST = OFF_ROW + 8 * ROW_BYTES;  // 8 warps x [32][128 B] y staging
 constexpr uint32_t OFF_BAR = OFF_YST + 32768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
@@ -60,8 +70,13 @@ __device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
   return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
 }
 
+// the xq buffer of tile n and the phase of its barriers: one buffer per chunk
+__device__ __forceinline__ int x_index(int n, int ntpu) { return ntpu == 1 ? (n & 1) : ((n >> 1) & 1); }
+__device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 ? ((n >> 1) & 1) : ((n >> 2) & 1); }
+
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
-       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_COUNT = 30 };
+       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 30, B_ROW_FULL = 34, B_ROW_FREE = 42,
+       B_COUNT = 50 };
 
 
 // two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
@@ -98,6 +113,11 @@ __device__ __forceinline__ void next_tile(Tile& x, const ScanArgs& a, int TM, in
   }
   x.KJ = (x.it + 1) * TM;
 }
+// the first tile of the next (batch, chunk, head)
+__device__ __forceinline__ void next_head(Tile& x, const ScanArgs& a, int TM, int ntpu) {
+  x.it = ntpu - 1;
+  next_tile(x, a, TM, ntpu);
+}
 // first tile of a CTA: computed once, by one thread, and handed to the roles through shared memory
 __device__ __forceinline__ Tile decode_tile(int t, const ScanArgs& a, int TM, int ntpu) {
   const Dims& d = a.d;
@@ -131,7 +151,7 @@ __device__ __forceinline__ Tile decode_tile(int t, const ScanArgs& a, int TM, in
 // so the same two tests on p127[c] end the walk for all farther chunks at once.  (p127 is +inf
 // where cs is not monotone: the walk then visits every chunk.)
 template <bool TAPS>
-__device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid, int TM, uint32_t RBQ,
+__device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, float* rowbuf, int rb, int lane, int TM, uint32_t RBQ,
                                           const Tile& t, const ScanArgs& a) {
   const int Q = a.d.Q;
   const float* cs_s = tokbuf;
@@ -140,8 +160,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
   const float* atok_s = tokbuf + 3 * Q;
   const float* b127_s = tokbuf + 4 * Q;
   const float* p127_s = b127_s + 16;
-  float* rowmax_s = tokbuf + 1280;   // [128], read by the epilogue warps
-  const int r = gtid >> 1, q2 = gtid & 1;
+  const int r = rb * 16 + (lane >> 1), q2 = lane & 1;   // the warp's block of 16 rows
   if (r >= TM) return;               // whole warps (TM is a multiple of 16)
   const int i = t.it * TM + r;       // row within the chunk
   const int I16 = i >> 4, ri = i & 15;
@@ -212,7 +231,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, float* tokbuf, int gtid,
   int8_t* mq_tap = nullptr;
   if (TAPS && a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
   if (q2 == 0) {
-    rowmax_s[r] = rowmax;
+    rowbuf[r] = rowmax;                 // read by the epilogue warps, with the decay of the
+    rowbuf[128 + r] = exp32(cs_i);      // off-diagonal term
     if (TAPS && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
   }
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
@@ -278,7 +298,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   const int t_end = min(a.ntiles, t_begin + a.per_cta);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
-  Tile* first_tile = reinterpret_cast<Tile*>(bars + B_COUNT + 2);
+  Tile* first_tile = reinterpret_cast<Tile*>(bars + B_COUNT + 2);   // 416 .. 464 of the 512 bytes
 
   if (tid == 0) {
     for (int s = 0; s < 4; ++s) {
@@ -286,15 +306,19 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       mbar_init(&bars[B_CB_FREE + s], 1);
       mbar_init(&bars[B_MQ + s], kGroupWarps);
       mbar_init(&bars[B_TOK_FULL + s], 1);
-      mbar_init(&bars[B_TOK_FREE + s], kEpiWarps);
+      mbar_init(&bars[B_TOK_FREE + s], kGroupWarps);
+      mbar_init(&bars[B_ACC + s], 1);
+      mbar_init(&bars[B_ACC_FREE + s], kEpiGroupWarps);
+    }
+    for (int s = 0; s < 8; ++s) {
+      mbar_init(&bars[B_ROW_FULL + s], 1);
+      mbar_init(&bars[B_ROW_FREE + s], kEpiGroupWarps);
     }
     mbar_init(&bars[B_CH_FULL], 1);
     mbar_init(&bars[B_CH_FREE], 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars[B_X_FULL + s], 1);
-      mbar_init(&bars[B_X_FREE + s], kEpiWarps);
-      mbar_init(&bars[B_ACC + s], 1);
-      mbar_init(&bars[B_ACC_FREE + s], kEpiWarps);
+      mbar_init(&bars[B_X_FREE + s], ntpu == 1 ? kEpiGroupWarps : kEpiWarps);  // the epilogues of the chunk's tiles
     }
     fence_mbar_init();
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
@@ -322,9 +346,19 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
           tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
                       (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
         mbar_wait_relaxed(&bars[B_TOK_FREE + t3], ph3 ^ 1, a.status);
+        // the scalar pack of the chunk for the mask warps
         mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4));
         bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4),
                   &bars[B_TOK_FULL + t3]);
+        // the head's per-column vectors for the epilogue (read once per 8-column piece: from global
+        // memory each read would be a long-latency load in its chain)
+        const int r8 = n & 7;
+        mbar_wait_relaxed(&bars[B_ROW_FREE + r8], ((n >> 3) & 1) ^ 1, a.status);
+        uint8_t* cols = smem + OFF_ROW + r8 * ROW_BYTES + ROW_COLS;
+        mbar_expect_tx(&bars[B_ROW_FULL + r8], (uint32_t)((CORR ? 3 : 2) * P * 4));
+        bulk_load(cols, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
+        bulk_load(cols + 256, a.s_h + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
+        if (CORR) bulk_load(cols + 512, a.corr + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
       }
     }
   } else if (warp == 2) {
@@ -345,12 +379,12 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       Tile t = *first_tile;
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
-        const int s2 = n & 1;
-        const uint32_t ph2 = (n >> 1) & 1;
-        mbar_wait_relaxed(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
-        mbar_expect_tx(&bars[B_X_FULL + s2], (uint32_t)(t.KJ * 64));
-        for (int j0 = 0; j0 < t.KJ; j0 += TM)
-          tma_load_3d(smem + OFF_X + s2 * 16384 + j0 * 64, &tm_x, &bars[B_X_FULL + s2], 0, t.h, (int)(t.tok0 + j0));
+        if (t.it != 0) continue;   // the chunk's rows were loaded with its first tile
+        const int xs = x_index(n, ntpu);
+        mbar_wait_relaxed(&bars[B_X_FREE + xs], x_phase(n, ntpu) ^ 1, a.status);
+        mbar_expect_tx(&bars[B_X_FULL + xs], (uint32_t)(Q * 64));
+        for (int j0 = 0; j0 < Q; j0 += TM)
+          tma_load_3d(smem + OFF_X + xs * 16384 + j0 * 64, &tm_x, &bars[B_X_FULL + xs], 0, t.h, (int)(t.tok0 + j0));
       }
     }
   } else if (warp == 1) {
@@ -361,11 +395,11 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
         const int it = ntpu == 1 ? 0 : (tix & 1);   // a CTA's first tile is the first of its chunk
-        const int ci = cb_index(n, it, ntpu), s2 = n & 1;
-        const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
+        const int ci = cb_index(n, it, ntpu), a4 = n & 3, xs = x_index(n, ntpu);
+        const uint32_t ph4 = (n >> 2) & 1;
         const int KJ = (it + 1) * TM;
-        const uint32_t acc = tmem + (uint32_t)s2 * 128u;
-        mbar_wait(&bars[B_ACC_FREE + s2], ph2 ^ 1, a.status);
+        const uint32_t acc = tmem + (uint32_t)a4 * 128u;
+        mbar_wait(&bars[B_ACC_FREE + a4], ph4 ^ 1, a.status);
         mbar_wait(&bars[B_CH_FULL], n & 1, a.status);
         tc_fence_after();
         // descriptors advance by a constant per 32-byte K step (their low bits are the address >> 4):
@@ -377,10 +411,10 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
         }
         mma_commit(&bars[B_CH_FREE]);
         mbar_wait(&bars[B_MQ + ci], ph4, a.status);
-        mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);
+        mbar_wait(&bars[B_X_FULL + xs], x_phase(n, ntpu), a.status);
         tc_fence_after();
         {
-          uint64_t db = tile_desc(sbase + OFF_X + s2 * 16384, 64);
+          uint64_t db = tile_desc(sbase + OFF_X + xs * 16384, 64);
           uint32_t first = 0;
 #pragma unroll 1
           for (uint32_t pn = 0; pn < (uint32_t)KJ / RBQ; ++pn) {     // panels of RBQ columns of Mq
@@ -393,81 +427,101 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
           }
         }
         mma_commit(&bars[B_CB_FREE + ci]);
-        mma_commit(&bars[B_ACC + s2]);
+        mma_commit(&bars[B_ACC + a4]);
       }
     }
   } else if (warp < kEpiWarp0) {
-    // ------------------------------------------------------------ mask warps: group g takes tiles n = g, g + 2, ...
+    // ------------------------------------------------------------ mask warps.  With two tiles per chunk, group g
+    // takes the chunks c = g, g + 2, ... of this CTA, both tiles: warp w builds the 16-row block w of the
+    // first tile and block 7 - w of the second, which is the same number of 16-column sub-blocks for every
+    // warp (the causal rows grow with the row index).  With one tile per chunk the groups alternate tiles.
     const int g = (warp - kMaskWarp0) / kGroupWarps;
-    const int gtid = tid - (kMaskWarp0 + g * kGroupWarps) * 32;
+    const int w = (warp - kMaskWarp0) % kGroupWarps;
     Tile t = *first_tile;
-    if (g) next_tile(t, a, TM, ntpu);
+    if (g) next_head(t, a, TM, ntpu);
 #pragma unroll 1
-    for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
-      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+    for (int tix = t_begin + g * ntpu, n = g * ntpu; tix < t_end; ++tix, ++n) {
+      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3, r8 = n & 7;
       const uint32_t ph4 = (n >> 2) & 1;
-      mbar_wait_relaxed(&bars[B_TOK_FULL + t3], ph4, a.status);
-      mbar_wait_relaxed(&bars[B_CB_FULL + ci], ph4, a.status);
-      mask_tile<TAPS>(smem + cb_offset(ci), reinterpret_cast<float*>(smem + OFF_TOK + t3 * TOK_BYTES), gtid, TM, RBQ, t, a);
+      const int rb = t.it ? kGroupWarps - 1 - w : w;
+      // one warp of the group polls (the scalar pack, the CBq tile, and the epilogue of the tile that
+      // used the row slot); the others wait at a hardware barrier, which costs no issue slots
+      if (w == 0 && lane < 3) {
+        const int bi = lane == 0 ? B_TOK_FULL + t3 : lane == 1 ? B_CB_FULL + ci : B_ROW_FREE + r8;
+        mbar_wait_relaxed(&bars[bi], lane == 2 ? (((n >> 3) & 1) ^ 1) : ph4, a.status);
+      }
+      named_bar_sync(1 + g, kGroupWarps * 32);
+      mask_tile<TAPS>(smem + cb_offset(ci), reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES),
+                      reinterpret_cast<float*>(smem + OFF_ROW + r8 * ROW_BYTES), rb, lane, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars[B_MQ + ci]);
-      next_tile(t, a, TM, ntpu);
-      next_tile(t, a, TM, ntpu);
+      if (lane < 2) mbar_arrive(&bars[lane == 0 ? B_MQ + ci : B_TOK_FREE + t3]);
+      if (t.it + 1 < ntpu) {   // the chunk's second tile
+        t.it = 1;
+        t.KJ = 2 * TM;
+      } else {                 // skip the other group's chunk (or tile)
+        next_head(t, a, TM, ntpu);
+        next_head(t, a, TM, ntpu);
+        tix += ntpu;
+        n += ntpu;
+      }
     }
   } else {
-    // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
+    // ------------------------------------------------------------ epilogue warps: two groups of four take
+    // alternate tiles; warp q of a group owns rows 32 q .. of the tile and all 64 columns
     const int ew = warp - kEpiWarp0;
+    const int eg = ew / kEpiGroupWarps;     // group: tiles n = eg, eg + 2, ...
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const int ch = ew >> 2;                 // column half
     const int er = q * 32 + lane;           // row of the tile
-    uint8_t* ystage = smem + OFF_YST + ew * 4096;
+    uint8_t* ystage = smem + OFF_YST + ew * 4096;   // [32][128 B], 16-byte chunks swizzled by the row
+    uint8_t* srow = ystage + lane * 128;
+    constexpr int PPR = YT ? 8 : 4;         // 8-column pieces per round (128 bytes of y per row)
     Tile t = *first_tile;
+    if (eg) next_tile(t, a, TM, ntpu);
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, a, TM, ntpu)) {
-      const int ci = cb_index(n, t.it, ntpu), s2 = n & 1, t3 = n & 3;
-      const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1, ph3 = (n >> 2) & 1;
-      const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
-      const uint8_t* sX = smem + OFF_X + s2 * 16384;
+    for (int tix = t_begin + eg, n = eg; tix < t_end; tix += 2, n += 2) {
+      const int ci = cb_index(n, t.it, ntpu), a4 = n & 3, xs = x_index(n, ntpu);
+      const uint32_t ph4 = (n >> 2) & 1;
+      const float* row = reinterpret_cast<const float*>(smem + OFF_ROW + (n & 7) * ROW_BYTES);
+      const uint8_t* sX = smem + OFF_X + xs * 16384;
       const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f, scb = a.s_cb[t.g];
-      const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
-      const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
-      const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
-      // four lanes wait side by side, one barrier each: the accumulators, the row maxima written by
-      // the mask warps, the xq rows (skip term) and the scalar pack (cs); the warp barrier passes
+      const float4* ssx = reinterpret_cast<const float4*>(row + ROW_COLS / 4);
+      const float4* ssh = ssx + 16;
+      const float4* sco = ssx + 32;
+      // four lanes wait side by side, one barrier each: the accumulators, the row scalars written by
+      // the mask warps, the xq rows (skip term) and the head's column vectors; the warp barrier passes
       // what they acquired on to the other lanes
-      if (lane < 4) {
-        const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_MQ + ci : lane == 2 ? B_X_FULL + s2 : B_TOK_FULL + t3;
-        const uint32_t bp = lane == 0 || lane == 2 ? ph2 : (lane == 1 ? ph4 : ph3);
+      if (q == 0 && lane < 4) {   // one warp of the group polls, the others wait at a hardware barrier
+        const int bi = lane == 0 ? B_ACC + a4 : lane == 1 ? B_MQ + ci : lane == 2 ? B_X_FULL + xs : B_ROW_FULL + (n & 7);
+        const uint32_t bp = lane == 2 ? x_phase(n, ntpu) : lane == 3 ? ((n >> 3) & 1) : ph4;
         mbar_wait_relaxed(&bars[bi], bp, a.status);
       }
-      __syncwarp();
+      named_bar_sync(3 + eg, kEpiGroupWarps * 32);
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
-      const float* part = tok + 1280;
-      const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
-      const float sm = ok ? scb * part[er] * (1.0f / 127.0f) : 0.f;
+      const float dec = ok ? row[128 + er] * sC : 0.f;
+      const float sm = ok ? scb * row[er] * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
-      if (lane == 3) tma_store_wait_read();  // last tile's store has finished reading the staging tile
-      __syncwarp();
-      uint8_t* srow = ystage + lane * (YT ? 64 : 128);
+      const uint32_t tbase = tmem + (uint32_t)a4 * 128u + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int pc = 0; pc < 4; ++pc) {       // 8 columns at a time (keeps the accumulators in registers)
+      for (int pc = 0; pc < 8; ++pc) {       // 8 columns at a time (keeps the accumulators in registers)
         int acc_o[8], acc_d[8];
-        const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 8);
-        tmem_ld8(taddr, acc_o);
-        tmem_ld8(taddr + 64, acc_d);
+        tmem_ld8(tbase + pc * 8, acc_o);
+        tmem_ld8(tbase + 64 + pc * 8, acc_d);
+        if ((pc & (PPR - 1)) == 0) {         // the last store has finished reading the staging tile
+          if (lane == 3) tma_store_wait_read();
+          __syncwarp();
+        }
         tmem_ld_wait();
         if (ok) {
-          const uint2 xr = *reinterpret_cast<const uint2*>(
-              sX + swz_off((uint32_t)ei, (uint32_t)(ch * 2 + (pc >> 1)), 64) + (pc & 1) * 8);
+          const uint2 xr = *reinterpret_cast<const uint2*>(sX + swz_off((uint32_t)ei, (uint32_t)(pc >> 1), 64) + (pc & 1) * 8);
           const uint32_t xw[2] = {xr.x ^ 0x80808080u, xr.y ^ 0x80808080u};
           float2 v[4];
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
-            const float4 sx4 = __ldg(gsx + pc * 2 + cc), sh4 = __ldg(gsh + pc * 2 + cc);
-            const float4 co4 = CORR ? __ldg(gco + pc * 2 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 sx4 = ssx[pc * 2 + cc], sh4 = ssh[pc * 2 + cc];
+            const float4 co4 = CORR ? sco[pc * 2 + cc] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
               const int pp = cc * 4 + e2 * 2;
@@ -481,11 +535,11 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
               r2 = __ffma2_rn(__fmul2_rn(sm2, sx2), ad, r2);
               v[cc * 2 + e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
             }
-            if (YT == 0)
-              *reinterpret_cast<float4*>(srow + (((pc * 2 + cc) ^ (lane & 7)) << 4)) =
+            if (YT == 0)   // 4 values = one 16-byte chunk
+              *reinterpret_cast<float4*>(srow + ((((pc & 3) * 2 + cc) ^ (lane & 7)) << 4)) =
                   make_float4(v[cc * 2].x, v[cc * 2].y, v[cc * 2 + 1].x, v[cc * 2 + 1].y);
           }
-          if (YT != 0) {  // 8 values = one 16-byte chunk of the [32][64 B] staging tile (64-byte swizzle)
+          if (YT != 0) {  // 8 values = one 16-byte chunk
             uint32_t h[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -497,10 +551,10 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
                 h[e] = *reinterpret_cast<const uint32_t*>(&bv);
               }
             }
-            *reinterpret_cast<uint4*>(srow + ((pc ^ ((lane >> 1) & 3)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+            *reinterpret_cast<uint4*>(srow + ((pc ^ (lane & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
           }
           if (TAPS && (a.taps.acc_off || a.taps.acc_diag)) {
-            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + ch * 32 + pc * 8;
+            const i64 o = ((t.tok0 + ei) * d.H + t.h) * P + pc * 8;
 #pragma unroll
             for (int pp = 0; pp < 8; ++pp) {
               if (a.taps.acc_off) a.taps.acc_off[o + pp] = acc_o[pp];
@@ -508,15 +562,26 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
             }
           }
         }
+        if ((pc & (PPR - 1)) == PPR - 1) {   // 128 bytes of every row are staged: store them
+          if (pc == 7) tc_fence_before();
+          fence_async_smem();
+          __syncwarp();
+          if (pc == 7 && lane < 3) {         // one release each, side by side
+            mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + a4 : lane == 1 ? B_X_FREE + xs : B_ROW_FREE + (n & 7)]);
+          } else if (lane == 3 && q * 32 < TM) {
+            tma_store_3d(&tm_y, ystage, (pc / PPR) * 32, t.h, (int)(t.tok0 + t.it * TM + q * 32));
+            tma_store_commit();
+          }
+        }
       }
-      tc_fence_before();
-      fence_async_smem();
-      __syncwarp();
-      if (lane < 3) {   // one release each, side by side
-        mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + s2 : B_TOK_FREE + t3]);
-      } else if (lane == 3 && q * 32 < TM) {
-        tma_store_3d(&tm_y, ystage, ch * 32, t.h, (int)(t.tok0 + t.it * TM + q * 32));
-        tma_store_commit();
+      if (ntpu == 2) {   // the same tile of the next head
+        const int it = t.it;
+        next_head(t, a, TM, ntpu);
+        t.it = it;
+        t.KJ = (it + 1) * TM;
+      } else {
+        next_tile(t, a, TM, ntpu);
+        next_tile(t, a, TM, ntpu);
       }
     }
     if (lane == 3) tma_store_wait_read();
@@ -568,8 +633,8 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
     const uint64_t eb = ydt ? 2 : 4;  // bytes per element of y
     uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
     uint64_t str[2] = {(uint64_t)d.P * eb, (uint64_t)d.H * d.P * eb};
-    uint32_t box[3] = {32, 1, 32};
-    if (!encode_tensor_map(&tm_y, y, (int)eb, 3, dims, str, box, ydt ? 64 : 128)) return SSDI8_ERR_CUDA;
+    uint32_t box[3] = {ydt ? 64u : 32u, 1, 32};   // 128 bytes of a row per store
+    if (!encode_tensor_map(&tm_y, y, (int)eb, 3, dims, str, box, 128)) return SSDI8_ERR_CUDA;
   }
   int dev = 0, sms = 0;
   SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
@@ -578,7 +643,7 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   const int ctas = ntiles < sms ? ntiles : sms;
   int per_cta = (ntiles + ctas - 1) / ctas;
   if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
-  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, taps, d, ntiles, per_cta, d.H / d.G};
+  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, static_cast<uint8_t*>(y), status, taps, d, ntiles, per_cta, d.H / d.G};
   const size_t smem = SMEM_BYTES + 1024;
   const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
   const bool tp = taps.acc_off || taps.rowmax || taps.Mq || taps.acc_diag;

@@ -67,6 +67,11 @@ __device__ __forceinline__ void mbar_wait_relaxed(uint64_t* bar, uint32_t parity
   if (!mbar_try_wait(bar, parity)) mbar_wait_slow(bar, parity, status, 256u);
 }
 
+// named barrier among `nthreads` threads (whole warps) of the CTA; id 0 is __syncthreads
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 // Inline forms of both waits, for kernels with few wait sites and no registers to spare around a call.
 template <uint32_t SLEEP_NS>
 __device__ __forceinline__ void mbar_wait_inline(uint64_t* bar, uint32_t parity, int32_t* status) {
@@ -122,6 +127,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* 
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// all but the most recent bulk store of this thread have finished reading shared memory
+__device__ __forceinline__ void tma_store_wait_read1() {
+  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
