@@ -311,7 +311,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       mbar_init(&bars[B_ACC_FREE + s], kEpiGroupWarps);
     }
     for (int s = 0; s < 8; ++s) {
-      mbar_init(&bars[B_ROW_FULL + s], 1);
+      mbar_init(&bars[B_ROW_FULL + s], 1 + kGroupWarps);   // the column vectors and the mask warps' row scalars
       mbar_init(&bars[B_ROW_FREE + s], kEpiGroupWarps);
     }
     mbar_init(&bars[B_CH_FULL], 1);
@@ -455,7 +455,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
                       reinterpret_cast<float*>(smem + OFF_ROW + r8 * ROW_BYTES), rb, lane, TM, RBQ, t, a);
       fence_async_smem();
       __syncwarp();
-      if (lane < 2) mbar_arrive(&bars[lane == 0 ? B_MQ + ci : B_TOK_FREE + t3]);
+      if (lane < 3) mbar_arrive(&bars[lane == 0 ? B_MQ + ci : lane == 1 ? B_TOK_FREE + t3 : B_ROW_FULL + r8]);
       if (t.it + 1 < ntpu) {   // the chunk's second tile
         t.it = 1;
         t.KJ = 2 * TM;
@@ -488,12 +488,13 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const float4* ssx = reinterpret_cast<const float4*>(row + ROW_COLS / 4);
       const float4* ssh = ssx + 16;
       const float4* sco = ssx + 32;
-      // four lanes wait side by side, one barrier each: the accumulators, the row scalars written by
-      // the mask warps, the xq rows (skip term) and the head's column vectors; the warp barrier passes
-      // what they acquired on to the other lanes
-      if (q == 0 && lane < 4) {   // one warp of the group polls, the others wait at a hardware barrier
-        const int bi = lane == 0 ? B_ACC + a4 : lane == 1 ? B_MQ + ci : lane == 2 ? B_X_FULL + xs : B_ROW_FULL + (n & 7);
-        const uint32_t bp = lane == 2 ? x_phase(n, ntpu) : lane == 3 ? ((n >> 3) & 1) : ph4;
+      // three lanes of one warp of the group poll side by side, one barrier each: the accumulators, the
+      // xq rows (skip term), and the row slot (the head's column vectors and the row scalars written by
+      // the mask warps; not the mask barrier of the CBq buffer, which may complete a second time before
+      // this group gets here); the other warps wait at a hardware barrier, which costs no issue slots
+      if (q == 0 && lane < 3) {
+        const int bi = lane == 0 ? B_ACC + a4 : lane == 1 ? B_X_FULL + xs : B_ROW_FULL + (n & 7);
+        const uint32_t bp = lane == 0 ? ph4 : lane == 1 ? x_phase(n, ntpu) : ((n >> 3) & 1);
         mbar_wait_relaxed(&bars[bi], bp, a.status);
       }
       named_bar_sync(3 + eg, kEpiGroupWarps * 32);
