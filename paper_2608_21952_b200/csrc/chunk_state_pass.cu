@@ -129,7 +129,9 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       uint8_t* sX = smem + s * STAGE + OFF_X;
       float* lut = reinterpret_cast<float*>(smem + OFF_LUT) + s * 256;
       const i64 tok0 = (i64)b * d.L + (i64)k * Q;
-      mbar_wait_inline<256>(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+      // one warp polls for the tiles; the others wait at a hardware barrier, which costs no issue slots
+      if (qt < 32) mbar_wait_inline<256>(&bars[B_FULL + s], (k >> 1) & 1, a.status);
+      named_bar(2, kQuantThreads);
       // a warp owns whole 32-token slabs (slab = one MMA): rows of a slab are split over the lanes,
       // and the warp's lane 0 issues the slab's MMA as soon as the warp has re-quantised it, so no
       // warp waits for another.  The accumulator is opened by the MMA of slab 0 (accumulate = 0);
@@ -241,6 +243,8 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
         }
       }
       fence_async_smem();
+      // one warp polls for the MMAs of this chunk; the barrier passes their completion on to the others
+      if (warp == 0) mbar_wait_inline<256>(&bars[B_MMA], k & 1, a.status);
       named_bar(1, kStateThreads);
       // ---- hq[k] leaves by TMA
       if (tid == 0) {
@@ -248,8 +252,7 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
           tma_store_2d(&tm_hq, sHQ + 16 * j * N, 0, (int)(((((i64)b * d.c + k) * d.H + h) * P) + 16 * j));
         tma_store_commit();
       }
-      // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 16 channels at a time
-      mbar_wait_inline<256>(&bars[B_MMA], k & 1, a.status);
+      // ---- epilogue of the MMA: S = fmaf(Gamma_k, S, loc), 8 channels at a time
       tc_fence_after();
       if (tid == 0 && k + 2 < d.c) issue_loads(k + 2);  // the MMA has finished reading stage s
 #pragma unroll
