@@ -127,6 +127,7 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
     tma_store_commit();
     tma_store_wait_read();
   }
+  drain_after_timeout(a.status);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 256);

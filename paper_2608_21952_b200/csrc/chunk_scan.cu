@@ -505,7 +505,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const float sm = ok ? scb * row[er] * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
       const uint32_t tbase = tmem + (uint32_t)a4 * 128u + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
+#pragma unroll 4                           // (a round of 32 columns per iteration: the piece index folds into addresses)
       for (int pc = 0; pc < 8; ++pc) {       // 8 columns at a time (keeps the accumulators in registers)
         int acc_o[8], acc_d[8];
         tmem_ld8(tbase + pc * 8, acc_o);
@@ -588,6 +588,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     if (lane == 3) tma_store_wait_read();
   }
   tc_fence_before();
+  drain_after_timeout(a.status);
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();

@@ -338,9 +338,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
       const uint32_t ph4 = (n >> 2) & 1;
-      mbar_wait(&bars[B_TOK_FULL + t3], ph4, a.status);
-      mbar_wait(&bars[B_CB_FULL + ci], ph4, a.status);
-      mbar_wait(&bars[B_AFREE + g], ((n >> 1) & 1) ^ 1, a.status);   // the MMAs of tile n - 2 have read the buffer
+      // one warp of the group polls, a barrier each on three lanes (the scalar pack, the CBq tile, and
+      // the MMAs of tile n - 2, which read the operand buffer); the others wait at a hardware barrier,
+      // which costs no issue slots
+      if (wg == 0 && lane < 3) {
+        const int bi = lane == 0 ? B_TOK_FULL + t3 : lane == 1 ? B_CB_FULL + ci : B_AFREE + g;
+        mbar_wait_relaxed(&bars[bi], lane == 2 ? (((n >> 1) & 1) ^ 1) : ph4, a.status);
+      }
+      named_bar_sync(1 + g, kGroupWarps * 32);
       tc_fence_after();
       mask_tile_f16(smem + cb_offset(ci), reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES),
                     tmem + 256u + (uint32_t)g * 128u, rq, q2, lane, TM, RBQ, t, a);
@@ -373,11 +378,11 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
       const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
       // three lanes wait side by side: the accumulators, the x rows (skip term), the scalar pack (cs)
-      if (lane < 3) {
+      if (ew == 0 && lane < 3) {   // one warp polls, the others wait at a hardware barrier
         const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_X_FULL + s2 : B_TOK_FULL + t3;
         mbar_wait_relaxed(&bars[bi], lane == 2 ? ph4 : ph2, a.status);
       }
-      __syncwarp();
+      named_bar_sync(3, kEpiWarps * 32);
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
@@ -451,6 +456,7 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     if (lane == 3) tma_store_wait_read();
   }
   tc_fence_before();
+  drain_after_timeout(a.status);
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();

@@ -148,6 +148,7 @@ chunk_state_tc(const __grid_constant__ CUtensorMap tm_B, const __grid_constant__
     }
   }
   tc_fence_before();
+  drain_after_timeout(a.status);
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();

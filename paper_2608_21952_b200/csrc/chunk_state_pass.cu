@@ -297,6 +297,7 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
     }
     if (tid == 0) tma_store_wait_read();
   }
+  drain_after_timeout(a.status);
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();

@@ -72,6 +72,14 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// At the end of a kernel whose waits are bounded: if some wait of the grid gave up (the status word is
+// set), the handshakes of this CTA may be broken and copies into its shared memory may still be in
+// flight; give them a bounded time to land before the CTA retires and its shared memory is handed on.
+__device__ __forceinline__ void drain_after_timeout(const int32_t* status) {
+  if (status && *reinterpret_cast<const volatile int32_t*>(status) != 0)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
+}
+
 // Inline forms of both waits, for kernels with few wait sites and no registers to spare around a call.
 template <uint32_t SLEEP_NS>
 __device__ __forceinline__ void mbar_wait_inline(uint64_t* bar, uint32_t parity, int32_t* status) {
