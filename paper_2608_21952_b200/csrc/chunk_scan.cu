@@ -180,28 +180,41 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
   int nv = 0;                        // chunks whose f the first pass computed
   uint2* const own_ptr = reinterpret_cast<uint2*>(chunk_ptr(I16)) + q2;
   {
-    // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
+    // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1}).  Straight-line code:
+    // a step that a row does not take multiplies by 1 (exact), a column past the diagonal is
+    // selected to 0, so the 16 rows of the warp, which all stop at different columns, do not diverge.
     const uint2 w2 = *own_ptr;
     const uint32_t ww[2] = {w2.x ^ 0x80808080u, w2.y ^ 0x80808080u};
-    const float* atc = atok_s + I16 * 16 + 1;
-    float E = 1.0f;
-    if (q2 == 0) {
-#pragma unroll
-      for (int e = 15; e >= 8; --e)
-        if (e < ri) E = __fmul_rn(E, atc[e]);
-    }
+    const float* ab = atok_s + I16 * 16;   // a_m of the sub-block at ab[m]
     const int e0 = q2 * 8;
-    const float* dtc = dt_s + I16 * 16 + e0;
-    atc += e0;
+    float E = 1.0f;
+    {
+      // the thread with the lower columns first runs the product through the upper ones: a_15 .. a_9
+      const float4 p2 = *reinterpret_cast<const float4*>(ab + 8), p3 = *reinterpret_cast<const float4*>(ab + 12);
+      const float au[7] = {p2.y, p2.z, p2.w, p3.x, p3.y, p3.z, p3.w};   // a_9 .. a_15
+      const int lim = q2 ? 0 : ri;         // steps m <= lim are taken
+#pragma unroll
+      for (int m = 15; m >= 9; --m) E = __fmul_rn(E, m <= lim ? au[m - 9] : 1.0f);
+    }
+    const float4 h0 = *reinterpret_cast<const float4*>(ab + e0), h1 = *reinterpret_cast<const float4*>(ab + e0 + 4);
+    const float hn[8] = {h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, ab[e0 + 8]};   // a_{e0+k+1}; the last one is never taken when e0 = 8
+    const float4 d0 = *reinterpret_cast<const float4*>(dt_s + I16 * 16 + e0);
+    const float4 d1 = *reinterpret_cast<const float4*>(dt_s + I16 * 16 + e0 + 4);
+    const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+    const int rr = ri - e0;                // this thread's columns k <= rr are on or below the diagonal
+    float Ev[8];
 #pragma unroll
     for (int k = 7; k >= 0; --k) {
-      float v = 0.f;
-      if (e0 + k <= ri) {
-        if (e0 + k < ri) E = __fmul_rn(E, atc[k]);
-        v = __fmul_rn(s8_to_f32(ww[k >> 2], k & 3), __fmul_rn(dtc[k], E));
-      }
-      tv[k] = v;
-      rpart = fmaxf(rpart, fabsf(v));
+      E = __fmul_rn(E, k < rr ? hn[k] : 1.0f);
+      Ev[k] = E;
+    }
+#pragma unroll
+    for (int k = 0; k < 8; k += 2) {
+      const float2 t2 = __fmul2_rn(unpack2(ww[k >> 2], k & 3),
+                                   __fmul2_rn(make_float2(dv[k], dv[k + 1]), make_float2(Ev[k], Ev[k + 1])));
+      tv[k] = k <= rr ? t2.x : 0.f;
+      tv[k + 1] = k + 1 <= rr ? t2.y : 0.f;
+      rpart = fmaxf(fmaxf(rpart, fabsf(tv[k])), fabsf(tv[k + 1]));
     }
   }
 #pragma unroll 1
