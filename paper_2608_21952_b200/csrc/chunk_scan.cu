@@ -217,17 +217,30 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
       rpart = fmaxf(fmaxf(rpart, fabsf(tv[k])), fabsf(tv[k + 1]));
     }
   }
+  // Both walks below are warp-uniform: every lane steps through the same iterations (chunk
+  // c_first - 2 it; the thread of a pair that starts one chunk farther runs out one step earlier) and
+  // the skip tests are taken by vote, so the 16 rows of the warp do not diverge; a lane whose own test
+  // says "skip" computes along with the others, which changes nothing (its values cannot raise the
+  // row maximum, or round to zero).
+  constexpr uint32_t kAll = 0xffffffffu;
+  const int nit = (I16 + 1) >> 1;
+  bool live = true;                  // this row has not reached its prefix bound yet
 #pragma unroll 1
-  for (int c = c_first; c >= 0; c -= 2) {
-    const float f = exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15]));
-    if (nv == 0) f0 = f;
-    if (nv == 1) f1 = f;
-    ++nv;
-    if (rpart >= 1e-30f && __fmul_rn(p127_s[c], f) <= rpart) break;  // nor can any farther chunk
-    if (__fmul_rn(b127_s[c], f) <= rpart) continue;
-    const uint4 w4 = *chunk_ptr(c);
+  for (int itc = 0; itc < nit; ++itc) {
+    const int c = c_first - 2 * itc;
+    live = live && c >= 0;
+    if (!__any_sync(kAll, live)) break;
+    const int cc = c < 0 ? 0 : c;
+    const float f = exp32(__fsub_rn(cs_i, cs_s[cc * 16 + 15]));
+    if (itc == 0) f0 = f;
+    if (itc == 1) f1 = f;
+    nv = itc + 1;
+    if (rpart >= 1e-30f && __fmul_rn(p127_s[cc], f) <= rpart) live = false;  // nor can any farther chunk
+    const bool need = live && !(__fmul_rn(b127_s[cc], f) <= rpart);
+    if (!__any_sync(kAll, need)) continue;
+    const uint4 w4 = *chunk_ptr(cc);
     const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-    const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
+    const float4* wo = reinterpret_cast<const float4*>(woff_s + cc * 16);
     float bmax = 0.f;
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
@@ -237,7 +250,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
       bmax = fmaxf(fmaxf(bmax, fabsf(t0.x)), fabsf(t0.y));
       bmax = fmaxf(fmaxf(bmax, fabsf(t1.x)), fabsf(t1.y));
     }
-    rpart = fmaxf(rpart, __fmul_rn(bmax, f));
+    if (need) rpart = fmaxf(rpart, __fmul_rn(bmax, f));
   }
   const float rowmax = fmaxf(rpart, __shfl_xor_sync(0xffffffffu, rpart, 1));
   const float inv = (rowmax >= 1e-30f) ? __fdiv_rn(127.0f, rowmax) : 0.f;
@@ -260,35 +273,38 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
     *own_ptr = v;
     if (TAPS && mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
   }
-  int c = c_first;
+  bool dead = false;                 // this chunk and every farther one round to zero in this row
 #pragma unroll 1
-  for (int v2 = 0; c >= 0; c -= 2, ++v2) {
-    const float f = v2 >= nv || v2 > 1 ? exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])) : (v2 ? f1 : f0);
-    const float g = __fmul_rn(f, inv);
-    if (__fmul_rn(p127_s[c], g) < 0.5f) break;  // this chunk and every farther one round to zero
-    uint4* ptr = chunk_ptr(c);
+  for (int itc = 0; itc < nit; ++itc) {
+    const int c = c_first - 2 * itc;
+    const bool valid = c >= 0;
+    const int cc = valid ? c : 0;
+    uint4* ptr = chunk_ptr(cc);
     uint4 v = zero4;
-    if (__fmul_rn(b127_s[c], g) >= 0.5f) {
-      const float2 g2 = make_float2(g, g);
-      const uint4 w4 = *ptr;
-      const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-      const float4* wo = reinterpret_cast<const float4*>(woff_s + c * 16);
-      uint32_t o[4];
+    if (__any_sync(kAll, valid && !dead)) {
+      const float f = itc >= nv || itc > 1 ? exp32(__fsub_rn(cs_i, cs_s[cc * 16 + 15])) : (itc ? f1 : f0);
+      const float g = __fmul_rn(f, inv);
+      if (__fmul_rn(p127_s[cc], g) < 0.5f) dead = true;
+      const bool need = valid && !dead && __fmul_rn(b127_s[cc], g) >= 0.5f;
+      if (__any_sync(kAll, need)) {
+        const float2 g2 = make_float2(g, g);
+        const uint4 w4 = *ptr;
+        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+        const float4* wo = reinterpret_cast<const float4*>(woff_s + cc * 16);
+        uint32_t o[4];
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const float4 fo = wo[w];
-        o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)), g2),
-                         __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2));
+        for (int w = 0; w < 4; ++w) {
+          const float4 fo = wo[w];
+          o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)), g2),
+                           __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2));
+        }
+        if (need) v = make_uint4(o[0], o[1], o[2], o[3]);
       }
-      v = make_uint4(o[0], o[1], o[2], o[3]);
     }
-    *ptr = v;
-    if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
-  }
-#pragma unroll 1
-  for (; c >= 0; c -= 2) {
-    *chunk_ptr(c) = zero4;
-    if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = zero4;
+    if (valid) {
+      *ptr = v;
+      if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
+    }
   }
 }
 
