@@ -5,21 +5,26 @@
 //   Mq[i,j]       = per-row re-quantised CBq[i,j] dt_j exp(cs_i - cs_j), j <= i   (see ssdi8.h)
 //   acc_diag[i,p] = sum_j Mq[i,j] xq[j,p]                 INT8 MMA, second TMEM accumulator
 //   y = exp(cs_i) s_C s_h acc_off + (s_cb rowmax_i / 127) s_x acc_diag + D s_x xq + corr
-// Roles (28 warps): warps 0, 2, 3 issue the TMA loads (CBq K-major and the per-token scalar pack
-// of ChunkCumsum; Cq, hq K-major; xq MN-major), each stream on its own ring; warp 1 issues the
-// MMAs; warps 4-19 build Mq in place over CBq, as two groups of 8 warps that take alternate tiles
-// (two threads per output row in adjacent lanes, so each warp owns 16 rows and runs on its own,
-// without block barriers, and two tiles are in flight); warps 20-27 read the accumulators, form y
-// and store it through a swizzled staging tile with coalesced 16-byte stores (a TMA store of rows this
-// short is slower and needs a proxy fence per tile), again as two groups (of 4 warps) on alternate
-// tiles, so one group's per-tile bookkeeping and waits run under the other's arithmetic.  Four
-// accumulator pairs and an xq buffer per chunk (shared by the chunk's two tiles) keep the MMAs of
-// the next tiles independent of the epilogue of the current ones.  Every buffer has its own "free" barrier, released by whoever reads it last
-// (tcgen05.commit for MMA operands), so loads run several tiles ahead of the mask warps.  The
-// hot loops are kept rolled: the whole kernel must stay resident in the instruction cache,
-// because every role executes different code at the same time.  No multicast; bounded waits.
+// Roles (28 warps): warps 0, 2, 3 issue the TMA loads (CBq K-major, the per-token scalar pack of
+// ChunkCumsum and the head's per-column vectors; Cq, hq K-major; xq MN-major, once per chunk), each
+// stream on its own ring; warp 1 issues the MMAs; warps 4-19 build Mq in place over CBq, as two
+// groups of 8 warps that take alternate chunks (two threads per output row in adjacent lanes, so a
+// warp owns 16 rows and needs no block barrier for the row maximum); warps 20-27 read the
+// accumulators, form y and store it through a swizzled staging tile with TMA (128-byte rows), as two
+// groups of 4 warps on alternate tiles, so one group's per-tile bookkeeping and waits run under the
+// other's arithmetic.  Four accumulator pairs, an xq buffer per chunk (shared by the chunk's two
+// tiles) and an 8-deep ring for what the mask warps hand to the epilogue keep the mask and the MMAs
+// of the next tiles independent of the epilogue of the current ones.  Every buffer has its own
+// "free" barrier, released by whoever reads it last (tcgen05.commit for MMA operands), so loads run
+// several tiles ahead.  The kernel is bound by instruction issue, so it is written to issue little:
+// in each group one warp polls the mbarriers and the others wait at a hardware barrier, the wait
+// loop is one out-of-line function, the tile walk has no divisions, and the code is kept small
+// enough for the instruction cache (every role executes different code at the same time).
+// No multicast; bounded waits.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "kernels.h"
 #include "sm100.cuh"
@@ -309,8 +314,10 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
 }
 
 // CORR: a mean-correction vector is given; TAPS: intermediate tensors are written out (tests);
-// YT: format of y (0 binary32, 1 fp16, 2 bf16: rounded to nearest even on the way to the staging tile)
-template <bool CORR, bool TAPS, int YT>
+// YT: format of y (0 binary32, 1 fp16, 2 bf16: rounded to nearest even on the way to the staging tile);
+// BIGQ: chunks of 128 tokens or more (128-row tiles with 128-byte CBq rows: the tile geometry, which
+// every role's address arithmetic depends on, is then known at compile time)
+template <bool CORR, bool TAPS, int YT, bool BIGQ>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
               const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
@@ -319,9 +326,9 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const Dims& d = a.d;
   const int Q = d.Q, N = d.N, P = d.P;
-  const int TM = Q < 128 ? Q : 128;        // valid rows of a tile
-  const int ntpu = Q / TM;                 // tiles per (batch, chunk, head)
-  const uint32_t RBN = N, RBQ = TM;        // row bytes of the N-contracted and Q-contracted tiles
+  const int TM = BIGQ ? 128 : Q;           // valid rows of a tile
+  const int ntpu = BIGQ ? Q / 128 : 1;     // tiles per (batch, chunk, head)
+  const uint32_t RBN = N, RBQ = BIGQ ? 128u : (uint32_t)Q;   // row bytes of the N-contracted and Q-contracted tiles
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t_begin = blockIdx.x * a.per_cta;
   const int t_end = min(a.ntiles, t_begin + a.per_cta);
@@ -684,15 +691,19 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
     return SSDI8_OK;
   };
   if (tp && ydt) return SSDI8_ERR_UNSUPPORTED;  // the taps come with binary32 y only
+  const bool big = d.Q >= 128;
+  auto pick = [&](auto corr_c, auto big_c) -> ssdi8_status_t {
+    constexpr bool C = decltype(corr_c)::value, B = decltype(big_c)::value;
+    if (tp) return launch(chunk_scan_tc<C, true, 0, B>);
+    if (ydt == 0) return launch(chunk_scan_tc<C, false, 0, B>);
+    if (ydt == 1) return launch(chunk_scan_tc<C, false, 1, B>);
+    return launch(chunk_scan_tc<C, false, 2, B>);
+  };
   ssdi8_status_t ls;
-  if (tp)
-    ls = corr ? launch(chunk_scan_tc<true, true, 0>) : launch(chunk_scan_tc<false, true, 0>);
-  else if (ydt == 0)
-    ls = corr ? launch(chunk_scan_tc<true, false, 0>) : launch(chunk_scan_tc<false, false, 0>);
-  else if (ydt == 1)
-    ls = corr ? launch(chunk_scan_tc<true, false, 1>) : launch(chunk_scan_tc<false, false, 1>);
+  if (corr)
+    ls = big ? pick(std::true_type{}, std::true_type{}) : pick(std::true_type{}, std::false_type{});
   else
-    ls = corr ? launch(chunk_scan_tc<true, false, 2>) : launch(chunk_scan_tc<false, false, 2>);
+    ls = big ? pick(std::false_type{}, std::true_type{}) : pick(std::false_type{}, std::false_type{});
   if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
