@@ -226,14 +226,18 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
         for (int p0 = 0; p0 < 32; p0 += 8) {
           if (p0 < npp) {
           uint32_t code[8];
+          // (cb is a multiple of 8: the eight reciprocals are two 16-byte loads)
+          const float4 i0 = *reinterpret_cast<const float4*>(col_invh + cb + p0);
+          const float4 i1 = *reinterpret_cast<const float4*>(col_invh + cb + p0 + 4);
+          const float ih[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const int pp = p0 + e;
-            code[e] = I8S ? (uint32_t)__float_as_int(S[pp])
-                          : rne_clamp_bits(__fmul_rn(S[pp], col_invh[cb + pp]));
+            code[e] = I8S ? (uint32_t)__float_as_int(S[pp]) : rne_clamp_bits(__fmul_rn(S[pp], ih[e]));
           }
+          uint8_t* hrow = sHQ + (cb + p0) * N + n;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) sHQ[(cb + p0 + e) * N + n] = (uint8_t)code[e];
+          for (int e = 0; e < 8; ++e, hrow += N) *hrow = (uint8_t)code[e];
         }
         }
         if (TAPS && !I8S && a.tap_prev) {
@@ -263,9 +267,9 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
         tmem_ld_wait();
         if (ok) {
           const i64 obase = (((((i64)b * d.c + k) * d.H + h) * P) + cb + hf * 8) * N + n;
-          float cscale[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) cscale[e] = col_scale[cb + hf * 8 + e];
+          const float4 c0v = *reinterpret_cast<const float4*>(col_scale + cb + hf * 8);
+          const float4 c1v = *reinterpret_cast<const float4*>(col_scale + cb + hf * 8 + 4);
+          const float cscale[8] = {c0v.x, c0v.y, c0v.z, c0v.w, c1v.x, c1v.y, c1v.z, c1v.w};
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const int pp = hf * 8 + e;
