@@ -47,6 +47,7 @@ constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64] fp16 (128-byte 
 constexpr uint32_t X_BYTES = 32768;
 constexpr uint32_t OFF_TOK = OFF_X + 2 * X_BYTES;   // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds)
 constexpr uint32_t TOK_BYTES = 6144;
+constexpr uint32_t TOK_COLS = 5120;   // byte offset of the head's s_x, s_h and correction vectors ([64] each) in a slot
 constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][64 B] y staging
 constexpr uint32_t OFF_BAR = OFF_YST + 16384;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
@@ -262,9 +263,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
           tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
                       (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
         mbar_wait_relaxed(&bars[B_TOK_FREE + t3], ph4 ^ 1, a.status);
-        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4));
-        bulk_load(smem + OFF_TOK + t3 * TOK_BYTES, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4),
-                  &bars[B_TOK_FULL + t3]);
+        // the scalar pack of the chunk and the head's per-column vectors (the epilogue reads them once per
+        // 8-column piece: from global memory each read would be a long-latency load in its chain)
+        uint8_t* slot = smem + OFF_TOK + t3 * TOK_BYTES;
+        mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4 + (CORR ? 3 : 2) * P * 4));
+        bulk_load(slot, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4), &bars[B_TOK_FULL + t3]);
+        bulk_load(slot + TOK_COLS, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
+        bulk_load(slot + TOK_COLS + 256, a.s_h + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
+        if (CORR) bulk_load(slot + TOK_COLS + 512, a.corr + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
       }
     }
   } else if (warp == 2) {
@@ -374,9 +380,9 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
       const uint8_t* sX = smem + OFF_X + s2 * X_BYTES;
       const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f;
-      const float4* gsx = reinterpret_cast<const float4*>(a.s_x + t.h * P) + ch * 8;
-      const float4* gsh = reinterpret_cast<const float4*>(a.s_h + t.h * P) + ch * 8;
-      const float4* gco = CORR ? reinterpret_cast<const float4*>(a.corr + t.h * P) + ch * 8 : nullptr;
+      const float4* gsx = reinterpret_cast<const float4*>(smem + OFF_TOK + t3 * TOK_BYTES + TOK_COLS) + ch * 8;
+      const float4* gsh = gsx + 16;
+      const float4* gco = gsx + 32;
       // three lanes wait side by side: the accumulators, the x rows (skip term), the scalar pack (cs)
       if (ew == 0 && lane < 3) {   // one warp polls, the others wait at a hardware barrier
         const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_X_FULL + s2 : B_TOK_FULL + t3;
@@ -406,8 +412,8 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
           float2 v[4];
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
-            const float4 sx4 = __ldg(gsx + pc * 2 + cc), sh4 = __ldg(gsh + pc * 2 + cc);
-            const float4 co4 = CORR ? __ldg(gco + pc * 2 + cc) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 sx4 = gsx[pc * 2 + cc], sh4 = gsh[pc * 2 + cc];
+            const float4 co4 = CORR ? gco[pc * 2 + cc] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
               const int pp = cc * 4 + e2 * 2;
