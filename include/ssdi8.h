@@ -199,7 +199,8 @@ typedef struct {
  * reads the intermediates a previous call left in the same workspace (per-module timing,
  * tests); any other bit set gives SSDI8_ERR_UNSUPPORTED.
  * workspace: at least ssdi8_workspace_bytes(dims, flags) bytes, 256-byte aligned; its
- * contents are scratch.  All tensor pointers 16-byte aligned. */
+ * contents are scratch.  All tensor pointers and the per-channel vectors s_x, s_xs, s_h, corr are
+ * 16-byte aligned (SSDI8_ERR_ALIGN otherwise). */
 ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* args,
                                     uint32_t flags, void* workspace, size_t workspace_bytes,
                                     void* stream);

@@ -123,7 +123,9 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
   if (!a->xq || !a->Bq || !a->Cq || !a->s_x || !a->s_B || !a->s_C || !a->dt || !a->A || !a->s_xs ||
       !a->s_cb || !a->s_h || !a->y || !workspace)
     return SSDI8_ERR_NULL;
+  // the per-channel vectors are read 16 bytes at a time (bulk copies into shared memory, float4 loads)
   const void* ptrs[] = {a->xq, a->Bq, a->Cq, a->dt, a->init_state, a->y, a->final_state,
+                        a->s_x, a->s_xs, a->s_h, a->corr,
                         a->tap_cs, a->tap_acc_cb, a->tap_CBq, a->tap_Xsq, a->tap_acc_st, a->tap_loc,
                         a->tap_prev, a->tap_hq, a->tap_acc_off, a->tap_Mq, a->tap_acc_diag};
   for (const void* p : ptrs)

@@ -81,6 +81,10 @@ def test_host_side_argument_errors():
     a.xq = 4096 + 4
     assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 0, 4096, 1 << 30, None) == bd.ERR_ALIGN
     a.xq = 4096
+    for k in ("s_x", "s_xs", "s_h", "corr"):   # per-channel vectors: read 16 bytes at a time
+        setattr(a, k, 4096 + 4)
+        assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 0, 4096, 1 << 30, None) == bd.ERR_ALIGN, k
+        setattr(a, k, 4096 if k != "corr" else None)
     assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 0, 4096 + 16, 1 << 30, None) == bd.ERR_ALIGN
     assert L.ssdi8_chunk_scan_fwd(C.byref(d), C.byref(a), 0, 4096, 16, None) == bd.ERR_WORKSPACE
     # quantiser
