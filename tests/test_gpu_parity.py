@@ -173,14 +173,22 @@ def _slice(cfg, b, h, xq, Bq, Cq, s_x, s_B, s_C, t, extra=None):
     return {k: np.ascontiguousarray(v) for k, v in d.items()}
 
 
+# chunks of 128 and of 64 tokens with about 20 tiles per CTA of the persistent scan kernel, so that its
+# rings (4, 8 deep) wrap several times in the one-tile-per-chunk geometry as well
+DEEP = {
+    "deep_q128": SSDConfig("deep_q128", 2, 4096, 48, 64, 64, 2, 128, 0.01, 50.0, 51),
+    "deep_q64": SSDConfig("deep_q64", 2, 2048, 48, 64, 128, 4, 64, 0.01, 50.0, 52),
+}
+
+
 @pytest.mark.parametrize("flags", [0, 1], ids=["int8_operand", "fp16_operand"])
-@pytest.mark.parametrize("name,npairs", [("cfg2", 4), ("cfg3", 3)])
+@pytest.mark.parametrize("name,npairs", [("cfg2", 4), ("cfg3", 3), ("deep_q128", 3), ("deep_q64", 3)])
 def test_fwd_full_size_sampled(name, npairs, flags):
     """Full-size workloads in the launch configuration the benchmark times (no taps); the
     oracle recomputes sampled (batch, head) pairs one by one.  flags = 1: the paper's FP16
     ChunkScan2 operand on both sides."""
     gh = _harness()
-    cfg = CONFIGS[name]
+    cfg = CONFIGS[name] if name in CONFIGS else DEEP[name]
     t = inputs.make_prefill(cfg)
     rng = np.random.default_rng(100 + cfg.seed)
     pairs = [(0, 0), (cfg.batch - 1, cfg.nheads - 1)]
