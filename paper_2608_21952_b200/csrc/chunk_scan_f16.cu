@@ -2,9 +2,10 @@
 // Algorithm 2, module 6): the masked operand stays in FP16 with the dequantisation scale of CB
 // fused into the look-up table,
 //   M16[i,j] = half(s_cb CBq[i,j] dt_j exp(cs_i - cs_j)), j <= i,      y_diag = s_x sum_j M16[i,j] xq[j,p],
-// instead of the per-row int8 re-quantisation of chunk_scan.cu.  Same persistent, warp-specialised
-// structure (28 warps: 3 TMA producers, 1 MMA warp, two mask groups of 8 warps on alternate
-// tiles, 8 epilogue warps), with these differences:
+// instead of the per-row int8 re-quantisation of chunk_scan.cu.  A persistent, warp-specialised
+// kernel like that one (28 warps: 2 TMA producers, 2 MMA issuers on alternate tiles, two mask groups
+// of 8 warps on alternate tiles, 8 epilogue warps; the FP16 x rows are loaded once per chunk), with
+// these differences:
 //  * the mask warps write M16 straight into tensor memory (tcgen05.st, thread = row), from where
 //    tcgen05.mma.kind::f16 takes it as its A operand: the operand never exists in shared memory,
 //    there is no row maximum, no second pass and no zero fill of shared memory;
@@ -59,8 +60,15 @@ __device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
   return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
 }
 
-enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
-       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_COUNT = 32 };
+// the x buffer of tile n and the phase of its barriers: one buffer per chunk, shared by its tiles
+__device__ __forceinline__ int x_index(int n, int ntpu) { return ntpu == 1 ? (n & 1) : ((n >> 1) & 1); }
+__device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 ? ((n >> 1) & 1) : ((n >> 2) & 1); }
+
+// The Cq/hq buffer is single, but its barriers come in pairs indexed by the parity of the tile: the two
+// MMA issuers take alternate tiles, and a barrier polled by parity must be seen phase by phase by its
+// one waiter (an issuer that skipped a phase would pass its first wait at once).
+enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_X_FULL = 14, B_X_FREE = 16,
+       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_CH_FREE = 32, B_COUNT = 34 };
 
 // two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
 __device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
@@ -229,11 +237,13 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       mbar_init(&bars[B_TOK_FULL + s], 1);
       mbar_init(&bars[B_TOK_FREE + s], kEpiWarps);
     }
-    mbar_init(&bars[B_CH_FULL], 1);
-    mbar_init(&bars[B_CH_FREE], 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bars[B_CH_FULL + s], 1);
+      mbar_init(&bars[B_CH_FREE + s], 1);
+    }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars[B_X_FULL + s], 1);
-      mbar_init(&bars[B_X_FREE + s], kEpiWarps);
+      mbar_init(&bars[B_X_FREE + s], kEpiWarps * ntpu);   // the epilogues of the chunk's tiles
       mbar_init(&bars[B_ACC + s], 1);
       mbar_init(&bars[B_ACC_FREE + s], kEpiWarps);
       mbar_init(&bars[B_AFREE + s], 1);
@@ -271,6 +281,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
         bulk_load(slot + TOK_COLS, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
         bulk_load(slot + TOK_COLS + 256, a.s_h + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
         if (CORR) bulk_load(slot + TOK_COLS + 512, a.corr + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
+        // FP16 x rows of the chunk, once, with its first tile
+        if (t.it == 0) {
+          const int xs = x_index(n, ntpu);
+          mbar_wait_relaxed(&bars[B_X_FREE + xs], x_phase(n, ntpu) ^ 1, a.status);
+          mbar_expect_tx(&bars[B_X_FULL + xs], (uint32_t)(Q * 128));
+          for (int j0 = 0; j0 < Q; j0 += TM)
+            tma_load_3d(smem + OFF_X + xs * X_BYTES + j0 * 128, &tm_x, &bars[B_X_FULL + xs], 0, t.h, (int)(t.tok0 + j0));
+        }
       }
     }
   } else if (warp == 2) {
@@ -279,51 +297,42 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       Tile t = decode_tile(t_begin, d, TM, ntpu);
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-        mbar_wait_relaxed(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
-        mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
-        tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.g, (int)(t.tok0 + t.it * TM));
-        tma_load_2d(smem + OFF_H, &tm_h, &bars[B_CH_FULL], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
+        // the MMAs of tile n - 1 (the other issuer's) have read the buffer
+        if (n > 0) mbar_wait_relaxed(&bars[B_CH_FREE + ((n - 1) & 1)], ((n - 1) >> 1) & 1, a.status);
+        uint64_t* full = &bars[B_CH_FULL + (n & 1)];
+        mbar_expect_tx(full, (uint32_t)(TM * N + 64 * N));
+        tma_load_3d(smem + OFF_C, &tm_C, full, 0, t.g, (int)(t.tok0 + t.it * TM));
+        tma_load_2d(smem + OFF_H, &tm_h, full, 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
       }
     }
-  } else if (warp == 3) {
-    // ------------------------------------------------------------ TMA producer: FP16 x rows
+  } else if (warp == 1 || warp == 3) {
+    // ------------------------------------------------------------ MMA issuers: warp 1 takes the even tiles of
+    // this CTA, warp 3 the odd ones (a tile is 12 to 20 instructions of 16 tokens each, and issuing one
+    // takes a thread about 0.1 us: one issuer alone would set the pace of the kernel)
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
-#pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-        const int s2 = n & 1;
-        const uint32_t ph2 = (n >> 1) & 1;
-        mbar_wait_relaxed(&bars[B_X_FREE + s2], ph2 ^ 1, a.status);
-        mbar_expect_tx(&bars[B_X_FULL + s2], (uint32_t)(t.KJ * 128));
-        for (int j0 = 0; j0 < t.KJ; j0 += TM)
-          tma_load_3d(smem + OFF_X + s2 * X_BYTES + j0 * 128, &tm_x, &bars[B_X_FULL + s2], 0, t.h, (int)(t.tok0 + j0));
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+      const int par = warp == 3 ? 1 : 0;
       const uint32_t idesc_off = idesc_s8(128, 64, 0, 0), idesc_diag = idesc_f16(128, 64, 1);
       const uint32_t sbase = smem_u32(smem);
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n) {
+      for (int tix = t_begin + par, n = par; tix < t_end; tix += 2, n += 2) {
         const int it = tix % ntpu;
-        const int ci = cb_index(n, it, ntpu), s2 = n & 1;
+        const int ci = cb_index(n, it, ntpu), s2 = n & 1, xs = x_index(n, ntpu);
         const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
         const int KJ = (it + 1) * TM;
         const uint32_t acc = tmem + (uint32_t)s2 * 128u;
         mbar_wait(&bars[B_ACC_FREE + s2], ph2 ^ 1, a.status);
-        mbar_wait(&bars[B_CH_FULL], n & 1, a.status);
+        mbar_wait(&bars[B_CH_FULL + par], ph2, a.status);
         tc_fence_after();
 #pragma unroll 1
         for (int q = 0; q < N / 32; ++q)
           mma_s8_ss(acc, tile_desc(sbase + OFF_C + 32 * q, RBN), tile_desc(sbase + OFF_H + 32 * q, RBN),
                     idesc_off, q > 0);
-        mma_commit(&bars[B_CH_FREE]);
+        mma_commit(&bars[B_CH_FREE + par]);
         mbar_wait(&bars[B_MQ + ci], ph4, a.status);        // the operand of this tile is in tensor memory
-        mbar_wait(&bars[B_X_FULL + s2], ph2, a.status);
+        mbar_wait(&bars[B_X_FULL + xs], x_phase(n, ntpu), a.status);
         tc_fence_after();
         // 16 tokens per instruction: 8 operand columns and 16 rows of 128 bytes of x
-        uint64_t bd = smem_desc(sbase + OFF_X + s2 * X_BYTES, 16, 1024, SWZ_128B);
+        uint64_t bd = smem_desc(sbase + OFF_X + xs * X_BYTES, 16, 1024, SWZ_128B);
         const uint32_t a_op = tmem + 256u + (uint32_t)s2 * 128u;
 #pragma unroll 1
         for (int q = 0; q < KJ / 16; ++q, bd += (16 * 128) >> 4)
@@ -375,18 +384,18 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     Tile t = decode_tile(t_begin, d, TM, ntpu);
 #pragma unroll 1
     for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
-      const int s2 = n & 1, t3 = n & 3;
+      const int s2 = n & 1, t3 = n & 3, xs = x_index(n, ntpu);
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
-      const uint8_t* sX = smem + OFF_X + s2 * X_BYTES;
+      const uint8_t* sX = smem + OFF_X + xs * X_BYTES;
       const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f;
       const float4* gsx = reinterpret_cast<const float4*>(smem + OFF_TOK + t3 * TOK_BYTES + TOK_COLS) + ch * 8;
       const float4* gsh = gsx + 16;
       const float4* gco = gsx + 32;
       // three lanes wait side by side: the accumulators, the x rows (skip term), the scalar pack (cs)
       if (ew == 0 && lane < 3) {   // one warp polls, the others wait at a hardware barrier
-        const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_X_FULL + s2 : B_TOK_FULL + t3;
-        mbar_wait_relaxed(&bars[bi], lane == 2 ? ph4 : ph2, a.status);
+        const int bi = lane == 0 ? B_ACC + s2 : lane == 1 ? B_X_FULL + xs : B_TOK_FULL + t3;
+        mbar_wait_relaxed(&bars[bi], lane == 2 ? ph4 : lane == 1 ? x_phase(n, ntpu) : ph2, a.status);
       }
       named_bar_sync(3, kEpiWarps * 32);
       tc_fence_after();
@@ -450,7 +459,7 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
           fence_async_smem();
           __syncwarp();
           if (pc == 3 && lane < 3) {
-            mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + s2 : B_TOK_FREE + t3]);
+            mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + xs : B_TOK_FREE + t3]);
           } else if (lane == 3 && q * 32 < TM) {
             tma_store_3d(&tm_y, ystage, ch * 32 + (YT != 0 ? 0 : (pc >> 1) * 16), t.h,
                          (int)(t.tok0 + t.it * TM + q * 32));
