@@ -28,9 +28,9 @@
 // against numpy int64 matmul, quantiser error bounds and idempotence, exp32
 // against libm, L2 within its quantisation error bound of L1, L3 == L0.
 //
-// Parity unpinned as exact bits: none of the paper's figures survive in the
-// text and it prints no worked example, so no stage is pinned to a value the
-// paper prints; every stage is pinned to the mathematics as listed above.
+// Every function here has such a pin; none is left unpinned.  The paper prints
+// no worked example (none of its figures survive in the text), so no pin is a
+// value the paper prints: all of them are the mathematics listed above.
 //
 // Build: g++ -O2 -fopenmp -ffp-contract=off -shared -fPIC (see oracle/build.py)
 
