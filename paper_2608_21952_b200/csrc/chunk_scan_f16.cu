@@ -342,36 +342,37 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       }
     }
   } else if (warp < kEpiWarp0) {
-    // ------------------------------------------------------------ mask warps: group g takes tiles n = g, g + 2, ...
+    // ------------------------------------------------------------ mask warps.  With two tiles per chunk, group g
+    // takes the chunks c = g, g + 2, ... of this CTA, both tiles (the second tile of a chunk has three
+    // times the sub-blocks of the first: alternating tiles would leave one group with all the large
+    // ones); with one tile per chunk the groups alternate tiles.  Tile n uses operand buffer n & 1.
     const int g = (warp - kMaskWarp0) / kGroupWarps;
     const int wg = (warp - kMaskWarp0) % kGroupWarps;
     const int rq = warp & 3;               // TMEM lane quarter of this warp = row quarter of the tile
     const int q2 = wg >> 2;                // chunk parity of this warp
     Tile t = decode_tile(t_begin, d, TM, ntpu);
-    if (g) next_tile(t, d, TM, ntpu);
 #pragma unroll 1
-    for (int tix = t_begin + g, n = g; tix < t_end; tix += 2, n += 2) {
-      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
+    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      if ((((ntpu == 1) ? n : (n >> 1)) & 1) != g) continue;
+      const int ci = cb_index(n, t.it, ntpu), t3 = n & 3, ob = n & 1;
       const uint32_t ph4 = (n >> 2) & 1;
       // one warp of the group polls, a barrier each on three lanes (the scalar pack, the CBq tile, and
       // the MMAs of tile n - 2, which read the operand buffer); the others wait at a hardware barrier,
       // which costs no issue slots
       if (wg == 0 && lane < 3) {
-        const int bi = lane == 0 ? B_TOK_FULL + t3 : lane == 1 ? B_CB_FULL + ci : B_AFREE + g;
+        const int bi = lane == 0 ? B_TOK_FULL + t3 : lane == 1 ? B_CB_FULL + ci : B_AFREE + ob;
         mbar_wait_relaxed(&bars[bi], lane == 2 ? (((n >> 1) & 1) ^ 1) : ph4, a.status);
       }
       named_bar_sync(1 + g, kGroupWarps * 32);
       tc_fence_after();
       mask_tile_f16(smem + cb_offset(ci), reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES),
-                    tmem + 256u + (uint32_t)g * 128u, rq, q2, lane, TM, RBQ, t, a);
+                    tmem + 256u + (uint32_t)ob * 128u, rq, q2, lane, TM, RBQ, t, a);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(&bars[B_MQ + ci]);
         mbar_arrive(&bars[B_CB_FREE + ci]);
       }
-      next_tile(t, d, TM, ntpu);
-      next_tile(t, d, TM, ntpu);
     }
   } else {
     // ------------------------------------------------------------ epilogue warps: rows 32 q .., columns 32 ch ..
