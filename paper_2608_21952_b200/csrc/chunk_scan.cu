@@ -61,7 +61,7 @@ constexpr uint32_t TOK_BYTES = 5120;
 // mask warps, and the head's s_x, s_h and correction vectors ([64] each, bulk-loaded).  Eight deep so
 // that the mask of a tile never waits for the epilogue of an earlier one.
 constexpr uint32_t OFF_ROW = OFF_TOK + 4 * TOK_BYTES;
-constexpr uint32_t ROW_BYTES = 2048, ROW_COLS = 1024;
+constexpr uint32_t ROW_BYTES = 2048, ROW_COLS = 1024, ROW_SCAL = 1792;   // scalars: s_C of the group, D of the head, s_cb
 constexpr uint32_t OFF_YST = OFF_ROW + 8 * ROW_BYTES;  // 8 warps x [32][128 B] y staging
 constexpr uint32_t OFF_BAR = OFF_YST + 32768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
@@ -391,7 +391,13 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
         const int r8 = n & 7;
         mbar_wait_relaxed(&bars[B_ROW_FREE + r8], ((n >> 3) & 1) ^ 1, a.status);
         uint8_t* cols = smem + OFF_ROW + r8 * ROW_BYTES + ROW_COLS;
-        mbar_expect_tx(&bars[B_ROW_FULL + r8], (uint32_t)((CORR ? 3 : 2) * P * 4));
+        {   // the tile's three scalars, fetched here so that their latency is not in the epilogue's chain
+          float* sc = reinterpret_cast<float*>(smem + OFF_ROW + r8 * ROW_BYTES + ROW_SCAL);
+          sc[0] = a.s_C[t.g];
+          sc[1] = a.D ? a.D[t.h] : 0.f;
+          sc[2] = a.s_cb[t.g];
+        }
+        mbar_expect_tx(&bars[B_ROW_FULL + r8], (uint32_t)((CORR ? 3 : 2) * P * 4));   // (an arrival: releases the stores above)
         bulk_load(cols, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
         bulk_load(cols + 256, a.s_h + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
         if (CORR) bulk_load(cols + 512, a.corr + t.h * P, (uint32_t)(P * 4), &bars[B_ROW_FULL + r8]);
@@ -520,7 +526,6 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const uint32_t ph4 = (n >> 2) & 1;
       const float* row = reinterpret_cast<const float*>(smem + OFF_ROW + (n & 7) * ROW_BYTES);
       const uint8_t* sX = smem + OFF_X + xs * 16384;
-      const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f, scb = a.s_cb[t.g];
       const float4* ssx = reinterpret_cast<const float4*>(row + ROW_COLS / 4);
       const float4* ssh = ssx + 16;
       const float4* sco = ssx + 32;
@@ -537,6 +542,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
+      const float sC = row[ROW_SCAL / 4], Dh = row[ROW_SCAL / 4 + 1], scb = row[ROW_SCAL / 4 + 2];
       const float dec = ok ? row[128 + er] * sC : 0.f;
       const float sm = ok ? scb * row[er] * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);

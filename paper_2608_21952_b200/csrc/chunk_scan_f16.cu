@@ -19,6 +19,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -211,7 +213,8 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
 }
 
 // CORR: a mean-correction vector is given; YT: format of y (0 binary32, 1 fp16, 2 bf16)
-template <bool CORR, int YT>
+// BIGQ: chunks of 128 tokens or more (128-row tiles, 128-byte CBq rows: the tile geometry is a constant)
+template <bool CORR, int YT, bool BIGQ>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtensorMap tm_h,
                   const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_cb,
@@ -220,9 +223,9 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const Dims& d = a.d;
   const int Q = d.Q, N = d.N, P = d.P;
-  const int TM = Q < 128 ? Q : 128;        // valid rows of a tile
-  const int ntpu = Q / TM;                 // tiles per (batch, chunk, head)
-  const uint32_t RBN = N, RBQ = TM;        // row bytes of the N-contracted and Q-contracted int8 tiles
+  const int TM = BIGQ ? 128 : Q;           // valid rows of a tile
+  const int ntpu = BIGQ ? Q / 128 : 1;     // tiles per (batch, chunk, head)
+  const uint32_t RBN = N, RBQ = BIGQ ? 128u : (uint32_t)Q;        // row bytes of the N-contracted and Q-contracted int8 tiles
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t_begin = blockIdx.x * a.per_cta;
   const int t_end = min(a.ntiles, t_begin + a.per_cta);
@@ -404,7 +407,7 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       const int ei = t.it * TM + er;
       const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
       const float2 dec2 = make_float2(dec, dec), Dh2 = make_float2(Dh, Dh);
-#pragma unroll 1
+#pragma unroll
       for (int pc = 0; pc < 4; ++pc) {       // 8 columns at a time
         int acc_o[8], acc_d[8];
         const uint32_t taddr = tmem + (uint32_t)s2 * 128u + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32 + pc * 8);
@@ -564,13 +567,18 @@ ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16,
     kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
     return SSDI8_OK;
   };
+  const bool big = d.Q >= 128;
+  auto pick = [&](auto corr_c, auto big_c) -> ssdi8_status_t {
+    constexpr bool C = decltype(corr_c)::value, B = decltype(big_c)::value;
+    if (ydt == 0) return launch(chunk_scan_f16_tc<C, 0, B>);
+    if (ydt == 1) return launch(chunk_scan_f16_tc<C, 1, B>);
+    return launch(chunk_scan_f16_tc<C, 2, B>);
+  };
   ssdi8_status_t ls;
-  if (ydt == 0)
-    ls = corr ? launch(chunk_scan_f16_tc<true, 0>) : launch(chunk_scan_f16_tc<false, 0>);
-  else if (ydt == 1)
-    ls = corr ? launch(chunk_scan_f16_tc<true, 1>) : launch(chunk_scan_f16_tc<false, 1>);
+  if (corr)
+    ls = big ? pick(std::true_type{}, std::true_type{}) : pick(std::true_type{}, std::false_type{});
   else
-    ls = corr ? launch(chunk_scan_f16_tc<true, 2>) : launch(chunk_scan_f16_tc<false, 2>);
+    ls = big ? pick(std::false_type{}, std::true_type{}) : pick(std::false_type{}, std::false_type{});
   if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
