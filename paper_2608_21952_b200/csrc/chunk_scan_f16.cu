@@ -50,6 +50,7 @@ constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64] fp16 (128-byte 
 constexpr uint32_t X_BYTES = 32768;
 constexpr uint32_t OFF_TOK = OFF_X + 2 * X_BYTES;   // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds)
 constexpr uint32_t TOK_BYTES = 6144;
+constexpr uint32_t TOK_SCAL = 5888;   // two scalars of the tile: s_C of the group, D of the head
 constexpr uint32_t TOK_COLS = 5120;   // byte offset of the head's s_x, s_h and correction vectors ([64] each) in a slot
 constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][64 B] y staging
 constexpr uint32_t OFF_BAR = OFF_YST + 16384;
@@ -279,6 +280,11 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
         // the scalar pack of the chunk and the head's per-column vectors (the epilogue reads them once per
         // 8-column piece: from global memory each read would be a long-latency load in its chain)
         uint8_t* slot = smem + OFF_TOK + t3 * TOK_BYTES;
+        {   // the tile's scalars, fetched here so that their latency is not in the epilogue's chain
+          float* sc = reinterpret_cast<float*>(slot + TOK_SCAL);
+          sc[0] = a.s_C[t.g];
+          sc[1] = a.D ? a.D[t.h] : 0.f;
+        }
         mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4 + (CORR ? 3 : 2) * P * 4));
         bulk_load(slot, a.pack + t.unit * kPackRows * Q, (uint32_t)(5 * Q * 4), &bars[B_TOK_FULL + t3]);
         bulk_load(slot + TOK_COLS, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
@@ -392,7 +398,6 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
       const uint8_t* sX = smem + OFF_X + xs * X_BYTES;
-      const float sC = a.s_C[t.g], Dh = a.D ? a.D[t.h] : 0.f;
       const float4* gsx = reinterpret_cast<const float4*>(smem + OFF_TOK + t3 * TOK_BYTES + TOK_COLS) + ch * 8;
       const float4* gsh = gsx + 16;
       const float4* gco = gsx + 32;
@@ -405,6 +410,7 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       tc_fence_after();
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
+      const float sC = tok[TOK_SCAL / 4], Dh = tok[TOK_SCAL / 4 + 1];
       const float dec = ok ? exp32(tok[ei]) * sC : 0.f;
       const float2 dec2 = make_float2(dec, dec), Dh2 = make_float2(Dh, Dh);
 #pragma unroll
