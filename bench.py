@@ -416,8 +416,7 @@ def run_ours(args):
         scan16 = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args16, layer.ws, flags=bd.PHASE_SCAN | bd.FLAG_Y_BF16)
         scan16(); torch.cuda.synchronize()
         kernel_ms["chunk_scan_bf16_y"] = layer.timed(scan16, max(5, min(args.steps, 20)))
-        # the paper's own ChunkScan2: FP16 masked operand (kind::f16 MMA) and FP16 y; includes the
-        # pass that writes the FP16 image of xq
+        # the paper's own ChunkScan2: FP16 masked operand (kind::f16 MMA) and FP16 y
         y_h = torch.empty(layer.y.shape, dtype=torch.float16, device="cuda")
         args_h = bd.make_fwd_args(**{**layer.args._keepalive, "y": y_h})
         fl_h = bd.PHASE_SCAN | bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16

@@ -76,8 +76,8 @@ enum {
  *                                               the exact FP16 image of its int8 codes)
  * computed with one factor per 16-token sub-block as below (own sub-block: running product of the
  * per-token decays; earlier: woff_j f), in binary32 before the rounding to FP16, so a value may
- * differ from the definition by one FP16 unit in the last place.  Needs 2 bytes per element of x
- * more workspace (ssdi8_workspace_bytes with the flag).  Not combinable with the scan taps. */
+ * differ from the definition by one FP16 unit in the last place.  The codes of x are expanded to FP16
+ * on the chip; the mode needs no workspace of its own.  Not combinable with the scan taps. */
 enum { SSDI8_FLAG_FP16_OPERAND = 1u << 0 };
 
 /* state format bit of ssdi8_chunk_scan_fwd's flags */

@@ -40,7 +40,7 @@ ssdi8_status_t check_arch() {
 }
 
 struct Workspace {
-  size_t pack, gamma, cbq, loc, hq, x16, total;
+  size_t pack, gamma, cbq, loc, hq, total;
 };
 
 Workspace layout(const Dims& d, bool fp16_operand = false) {
@@ -52,8 +52,7 @@ Workspace layout(const Dims& d, bool fp16_operand = false) {
   w.cbq = o;   o = align_up(o + (size_t)d.b * d.c * d.G * d.Q * d.Q, 256);
   w.loc = o;   o = align_up(o + sizeof(float) * nst, 256);
   w.hq = o;    o = align_up(o + nst, 256);
-  w.x16 = o;   // FP16 image of xq, only for the paper's FP16 ChunkScan2 operand
-  if (fp16_operand) o = align_up(o + 2 * (size_t)d.b * d.L * d.H * d.P, 256);
+  (void)fp16_operand;   // the FP16 operand needs no scratch of its own
   w.total = o;
   return w;
 }
@@ -168,7 +167,7 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
       return s;
   }
   if ((ph & SSDI8_PHASE_SCAN) && f16op)
-    return launch_chunk_scan_f16(d, a->xq, ws + w.x16, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack, a->D,
+    return launch_chunk_scan_f16(d, a->xq, a->Cq, cbq, hq, a->s_x, a->s_C, a->s_cb, a->s_h, pack, a->D,
                                  a->corr, a->y, ydt, a->status, st);
   if (ph & SSDI8_PHASE_SCAN) {
     ScanTaps taps = {a->tap_acc_off, a->tap_rowmax, a->tap_Mq, a->tap_acc_diag};

@@ -9,8 +9,11 @@
 //  * the mask warps write M16 straight into tensor memory (tcgen05.st, thread = row), from where
 //    tcgen05.mma.kind::f16 takes it as its A operand: the operand never exists in shared memory,
 //    there is no row maximum, no second pass and no zero fill of shared memory;
-//  * X enters as the exact FP16 image of its int8 codes (written once per call by a streaming
-//    kernel), TMA-staged MN-major with 128-byte rows; ChunkScan1 stays an int8 MMA;
+//  * X enters the MMA as the exact FP16 image of its int8 codes: the codes of a chunk arrive by TMA in
+//    the upper half of the chunk's x buffer and the mask group that takes the chunk expands them in
+//    place, a row per thread, into the MN-major tile with 128-byte swizzled rows that the MMA reads;
+//    the epilogue warps request the codes of the chunk after next when they hand a buffer back;
+//    ChunkScan1 stays an int8 MMA;
 //  * tensor memory: two accumulator pairs (INT32 C h, FP32 M16 x) and two operand buffers, 512 columns.
 // One factor per 16-column sub-block as in chunk_scan.cu: own sub-block by the running product of
 // per-token decays, earlier ones woff_j f with f = exp32(cs_i - cs_je); a sub-block whose bound
@@ -71,7 +74,7 @@ __device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 
 // MMA issuers take alternate tiles, and a barrier polled by parity must be seen phase by phase by its
 // one waiter (an issuer that skipped a phase would pass its first wait at once).
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_X_FULL = 14, B_X_FREE = 16,
-       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_CH_FREE = 32, B_COUNT = 34 };
+       B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_CH_FREE = 32, B_X_RAW = 34, B_COUNT = 36 };
 
 // two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
 __device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
@@ -214,6 +217,33 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
 }
 
 // CORR: a mean-correction vector is given; YT: format of y (0 binary32, 1 fp16, 2 bf16)
+// The xq rows of a chunk arrive as int8 codes in the upper half of the chunk's x buffer (rows of 64
+// bytes from byte 64 Q on) and are expanded in place into the MMA's FP16 operand (rows of 128 bytes,
+// 128-byte swizzle, from byte 0) by the mask group that takes the chunk: one row per thread, every
+// thread reads its codes, the group meets at its hardware barrier, every thread writes its row.  With
+// u = code ^ 0x80 the half with bits 0x6400 | u is 1024 + u exactly, and subtracting 1152 gives the
+// code (one byte permute and one packed subtraction per two codes).
+__device__ __forceinline__ void x_row_to_half(uint8_t* xb, int r, const uint4 (&w)[4]) {
+  const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+  uint8_t* row = xb + r * 128;
+#pragma unroll
+  for (int qd = 0; qd < 4; ++qd) {
+    const uint32_t ww[4] = {w[qd].x ^ 0x80808080u, w[qd].y ^ 0x80808080u, w[qd].z ^ 0x80808080u, w[qd].w ^ 0x80808080u};
+    uint32_t o[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        const uint32_t bits = __byte_perm(ww[k], 0x64646464u, p ? 0x7372u : 0x7170u);  // {0x64, b(2p+1), 0x64, b(2p)}
+        const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&bits), off);
+        o[k * 2 + p] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+    }
+    *reinterpret_cast<uint4*>(row + (((2 * qd) ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<uint4*>(row + (((2 * qd + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
 // BIGQ: chunks of 128 tokens or more (128-row tiles, 128-byte CBq rows: the tile geometry is a constant)
 template <bool CORR, int YT, bool BIGQ>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -246,7 +276,8 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       mbar_init(&bars[B_CH_FREE + s], 1);
     }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&bars[B_X_FULL + s], 1);
+      mbar_init(&bars[B_X_FULL + s], kGroupWarps);   // the warps of the mask group that expands the rows
+      mbar_init(&bars[B_X_RAW + s], 1);
       mbar_init(&bars[B_X_FREE + s], kEpiWarps * ntpu);   // the epilogues of the chunk's tiles
       mbar_init(&bars[B_ACC + s], 1);
       mbar_init(&bars[B_ACC_FREE + s], kEpiWarps);
@@ -263,9 +294,21 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
+    // ------------------------------------------------------------ TMA producer: CBq panels, scalar pack, and the
+    // int8 xq rows of each chunk (the mask group that takes the chunk expands them to FP16)
     if (lane == 0) {
       Tile t = decode_tile(t_begin, d, TM, ntpu);
+      {   // the int8 xq rows of the first two chunks (both buffers are free); later requests come from the
+          // epilogue warps, the moment they have finished with a buffer
+        Tile tn = t;
+        for (int kc = 0; kc < 2 && t_begin + kc * ntpu < t_end; ++kc) {
+          uint8_t* xb = smem + OFF_X + kc * X_BYTES;
+          mbar_expect_tx(&bars[B_X_RAW + kc], (uint32_t)(Q * 64));
+          for (int j0 = 0; j0 < Q; j0 += TM)
+            tma_load_3d(xb + Q * 64 + j0 * 64, &tm_x, &bars[B_X_RAW + kc], 0, tn.h, (int)(tn.tok0 + j0));
+          for (int i = 0; i < ntpu; ++i) next_tile(tn, d, TM, ntpu);
+        }
+      }
 #pragma unroll 1
       for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
         const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
@@ -290,14 +333,6 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
         bulk_load(slot + TOK_COLS, a.s_x + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
         bulk_load(slot + TOK_COLS + 256, a.s_h + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
         if (CORR) bulk_load(slot + TOK_COLS + 512, a.corr + t.h * P, (uint32_t)(P * 4), &bars[B_TOK_FULL + t3]);
-        // FP16 x rows of the chunk, once, with its first tile
-        if (t.it == 0) {
-          const int xs = x_index(n, ntpu);
-          mbar_wait_relaxed(&bars[B_X_FREE + xs], x_phase(n, ntpu) ^ 1, a.status);
-          mbar_expect_tx(&bars[B_X_FULL + xs], (uint32_t)(Q * 128));
-          for (int j0 = 0; j0 < Q; j0 += TM)
-            tma_load_3d(smem + OFF_X + xs * X_BYTES + j0 * 128, &tm_x, &bars[B_X_FULL + xs], 0, t.h, (int)(t.tok0 + j0));
-        }
       }
     }
   } else if (warp == 2) {
@@ -371,8 +406,24 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       if (wg == 0 && lane < 3) {
         const int bi = lane == 0 ? B_TOK_FULL + t3 : lane == 1 ? B_CB_FULL + ci : B_AFREE + ob;
         mbar_wait_relaxed(&bars[bi], lane == 2 ? (((n >> 1) & 1) ^ 1) : ph4, a.status);
+      } else if (wg == 0 && lane == 3 && t.it == 0) {
+        mbar_wait_relaxed(&bars[B_X_RAW + x_index(n, ntpu)], x_phase(n, ntpu), a.status);   // the chunk's xq codes
       }
       named_bar_sync(1 + g, kGroupWarps * 32);
+      if (t.it == 0) {   // first tile of a chunk: the group expands the chunk's xq rows to FP16, a row per thread
+        uint8_t* xb = smem + OFF_X + x_index(n, ntpu) * X_BYTES;
+        const int r = wg * 32 + lane;
+        uint4 w[4];
+        if (r < Q) {
+#pragma unroll
+          for (int qd = 0; qd < 4; ++qd) w[qd] = *reinterpret_cast<const uint4*>(xb + Q * 64 + r * 64 + qd * 16);
+        }
+        named_bar_sync(1 + g, kGroupWarps * 32);   // every code is in a register: the rows may be overwritten
+        if (r < Q) x_row_to_half(xb, r, w);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars[B_X_FULL + x_index(n, ntpu)]);
+      }
       tc_fence_after();
       mask_tile_f16(smem + cb_offset(ci), reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES),
                     tmem + 256u + (uint32_t)ob * 128u, rq, q2, lane, TM, RBQ, t, a);
@@ -470,6 +521,18 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
           __syncwarp();
           if (pc == 3 && lane < 3) {
             mbar_arrive(&bars[lane == 0 ? B_ACC_FREE + s2 : lane == 1 ? B_X_FREE + xs : B_TOK_FREE + t3]);
+            // the chunk's last tile: once every epilogue warp is through, its x buffer takes the codes of
+            // the chunk after next
+            const int n2 = n - (ntpu - 1) + 2 * ntpu;   // first tile of that chunk
+            if (ew == 0 && lane == 1 && t.it == ntpu - 1 && t_begin + n2 < t_end) {
+              mbar_wait(&bars[B_X_FREE + xs], x_phase(n, ntpu), a.status);
+              Tile tn = t;
+              for (int i = 0; i < ntpu + 1; ++i) next_tile(tn, d, TM, ntpu);
+              uint8_t* xb = smem + OFF_X + xs * X_BYTES;
+              mbar_expect_tx(&bars[B_X_RAW + xs], (uint32_t)(Q * 64));
+              for (int j0 = 0; j0 < Q; j0 += TM)
+                tma_load_3d(xb + Q * 64 + j0 * 64, &tm_x, &bars[B_X_RAW + xs], 0, tn.h, (int)(tn.tok0 + j0));
+            }
           } else if (lane == 3 && q * 32 < TM) {
             tma_store_3d(&tm_y, ystage, ch * 32 + (YT != 0 ? 0 : (pc >> 1) * 16), t.h,
                          (int)(t.tok0 + t.it * TM + q * 32));
@@ -489,43 +552,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   }
 }
 
-// FP16 image of int8 codes, 16 codes per thread.  With u = code ^ 0x80 (0..255), the half with bits
-// 0x6400 | u is 1024 + u exactly, and subtracting 1152 gives the code: one byte permute and one
-// packed subtraction per two elements, no integer-to-float conversions.
-__global__ void __launch_bounds__(256) x_to_half_kernel(const uint4* __restrict__ xq, uint4* __restrict__ x16,
-                                                        i64 n16) {
-  const i64 e = (i64)blockIdx.x * 256 + threadIdx.x;
-  if (e >= n16) return;
-  const uint4 w = __ldcs(xq + e);
-  const uint32_t ww[4] = {w.x ^ 0x80808080u, w.y ^ 0x80808080u, w.z ^ 0x80808080u, w.w ^ 0x80808080u};
-  const __half2 off = __floats2half2_rn(1152.f, 1152.f);
-  uint32_t o[8];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-#pragma unroll
-    for (int p = 0; p < 2; ++p) {
-      const uint32_t bits = __byte_perm(ww[k], 0x64646464u, p ? 0x7372u : 0x7170u);  // {0x64, b(2p+1), 0x64, b(2p)}
-      const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&bits), off);
-      o[k * 2 + p] = *reinterpret_cast<const uint32_t*>(&h);
-    }
-  }
-  __stcs(x16 + 2 * e, make_uint4(o[0], o[1], o[2], o[3]));
-  __stcs(x16 + 2 * e + 1, make_uint4(o[4], o[5], o[6], o[7]));
-}
-
 }  // namespace
 
-ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16, const int8_t* Cq,
+ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, const int8_t* Cq,
                                      const int8_t* CBq, const int8_t* hq, const float* s_x, const float* s_C,
                                      const float* s_cb, const float* s_h, const float* pack, const float* D,
                                      const float* corr, void* y, int ydt, int32_t* status, cudaStream_t st) {
   const int TM = d.Q < 128 ? d.Q : 128;
   const uint64_t T = (uint64_t)d.b * d.L;
-  // X as FP16 (exact images of the int8 codes)
-  const i64 n16 = (i64)T * d.H * d.P / 16;   // P = 64: a multiple of 16
-  x_to_half_kernel<<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint4*>(xq),
-                                                                  static_cast<uint4*>(x16), n16);
-  SSDI8_LAUNCH_CHECK();
   CUtensorMap tm_C, tm_h, tm_x, tm_cb, tm_y;
   {
     uint64_t dims[3] = {(uint64_t)d.N, (uint64_t)d.G, T};
@@ -541,9 +575,9 @@ ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16,
   }
   {
     uint64_t dims[3] = {(uint64_t)d.P, (uint64_t)d.H, T};
-    uint64_t str[2] = {(uint64_t)d.P * 2, (uint64_t)d.H * d.P * 2};
-    uint32_t box[3] = {64, 1, (uint32_t)TM};
-    if (!encode_tensor_map(&tm_x, x16, 2, 3, dims, str, box, 128)) return SSDI8_ERR_CUDA;
+    uint64_t str[2] = {(uint64_t)d.P, (uint64_t)d.H * d.P};
+    uint32_t box[3] = {64, 1, (uint32_t)TM};   // int8 codes, plain rows of 64 bytes
+    if (!encode_tensor_map(&tm_x, xq, 1, 3, dims, str, box, 0)) return SSDI8_ERR_CUDA;
   }
   {
     uint64_t dims[2] = {(uint64_t)d.Q, (uint64_t)d.b * d.c * d.G * d.Q};

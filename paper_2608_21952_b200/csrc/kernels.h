@@ -59,8 +59,8 @@ struct ScanTaps {
   int32_t* acc_off; float* rowmax; int8_t* Mq; int32_t* acc_diag;
 };
 
-// the same with the paper's FP16 ChunkScan2 operand; x16 [B,L,H,P] fp16 is scratch filled here
-ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, void* x16, const int8_t* Cq,
+// the same with the paper's FP16 ChunkScan2 operand
+ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, const int8_t* Cq,
                                      const int8_t* CBq, const int8_t* hq, const float* s_x, const float* s_C,
                                      const float* s_cb, const float* s_h, const float* pack, const float* D,
                                      const float* corr, void* y, int ydt, int32_t* status, cudaStream_t st);
