@@ -153,7 +153,7 @@ def test_host_side_argument_errors_of_the_layer_and_entry_calls():
         assert fn(C.byref(d), C.byref(a), 4096, need - 1, 0, None) == bd.ERR_WORKSPACE
         assert fn(C.byref(d), C.byref(a), 4096 + 8, need, 0, None) == bd.ERR_ALIGN
         assert fn(C.byref(d), C.byref(a), 4096, need, 1 << 13, None) == bd.ERR_UNSUPPORTED
-        assert size(C.byref(d), 1) > need                      # the FP16 operand needs the FP16 image of x
+        assert size(C.byref(d), 1) == need                     # the FP16 operand needs no scratch of its own
         bad = bd.dims_of(CONFIGS["cfg0"].replace(chunk=48))
         assert size(C.byref(bad), 0) == 0
         assert fn(C.byref(bad), C.byref(a), 4096, 1 << 40, 0, None) == bd.ERR_SHAPE
