@@ -169,30 +169,50 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
   const float kTiny = 2.9e-8f;       // below 2^-25 = 2.98e-8: rounds to zero in FP16
   const uint32_t lane_addr = a_tmem + ((uint32_t)(rq * 32) << 16);
   bool done = !row_ok;               // this row has nothing (more) to contribute
+  // The row's own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1}).  Straight-line
+  // code ahead of the walk: a step that a row does not take multiplies by 1 (exact), a column past the
+  // diagonal is selected to 0, so the 32 rows of the warp (two sub-blocks, every diagonal position) do
+  // not diverge; the walk below only picks the result up when it reaches the sub-block.
+  uint32_t own[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+  {
+    const uint4 w4 = row_ok ? *chunk_ptr(I16) : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
+    const int i0 = row_ok ? I16 * 16 : 0;
+    const float2 scb2 = make_float2(scb, scb);
+    float E = 1.0f;
+#pragma unroll
+    for (int hf = 1; hf >= 0; --hf) {   // columns 15..8, then 7..0 (the product runs on through both)
+      const float4* a4 = reinterpret_cast<const float4*>(atok_s + i0 + 8 * hf);
+      const float4* d4 = reinterpret_cast<const float4*>(dt_s + i0 + 8 * hf);
+      const float4 A0 = a4[0], A1 = a4[1];
+      const float alast = hf ? 1.0f : atok_s[i0 + 8];                      // a_{e+1} for the half's last column
+      const float an[8] = {A0.y, A0.z, A0.w, A1.x, A1.y, A1.z, A1.w, alast};
+      const float4 D0 = d4[0], D1 = d4[1];
+      const float dv[8] = {D0.x, D0.y, D0.z, D0.w, D1.x, D1.y, D1.z, D1.w};
+      const int rr = ri - 8 * hf;                                           // columns k <= rr of this half are on or below the diagonal
+      float Ev[8];
+#pragma unroll
+      for (int k = 7; k >= 0; --k) {
+        E = __fmul_rn(E, k < rr ? an[k] : 1.0f);
+        Ev[k] = E;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; k += 2) {
+        const int e = 8 * hf + k;
+        const float2 t2 = __fmul2_rn(__fmul2_rn(unpack2(ww[e >> 2], e & 3),
+                                                __fmul2_rn(make_float2(dv[k], dv[k + 1]), make_float2(Ev[k], Ev[k + 1]))), scb2);
+        own[e >> 1] = half2_bits(make_float2(k <= rr ? t2.x : 0.f, k + 1 <= rr ? t2.y : 0.f));
+      }
+    }
+  }
 #pragma unroll 1
   for (int c = ((nch - 1 - q2) & ~1) + q2; c >= 0; c -= 2) {
     uint32_t w8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-    if (!done && c <= I16) {
-      if (c == I16) {
-        // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1})
-        const uint4 w4 = *chunk_ptr(c);
-        const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-        const float* dtc = dt_s + c * 16;
-        const float* atc = atok_s + c * 16 + 1;
-        float E = 1.0f;
-        float tv[16];
+    if (!done && c == I16) {
 #pragma unroll
-        for (int e = 15; e >= 0; --e) {
-          float v = 0.f;
-          if (e <= ri) {
-            if (e < ri) E = __fmul_rn(E, atc[e]);
-            v = __fmul_rn(__fmul_rn(s8_to_f32(ww[e >> 2], e & 3), __fmul_rn(dtc[e], E)), scb);
-          }
-          tv[e] = v;
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) w8[e] = half2_bits(make_float2(tv[2 * e], tv[2 * e + 1]));
-      } else {
+      for (int e = 0; e < 8; ++e) w8[e] = own[e];
+    } else if (!done && c < I16) {
+      {
         const float g = __fmul_rn(exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])), scb);
         if (__fmul_rn(p127_s[c], g) < kTiny) {
           done = true;               // this chunk and every farther one round to zero
