@@ -183,6 +183,98 @@ def build(sim, ntiles, ntpu, speed, epilogue_waits_on_mq=False):
         sim.spawn(name, gen)
 
 
+def build_f16(sim, ntiles, ntpu, speed, one_ch_barrier=False):
+    """The FP16-operand kernel: one epilogue group of eight warps that also hands back the scalar pack,
+    two MMA issuers on alternate tiles with a barrier pair each on the single Cq/hq buffer, operand buffers
+    in tensor memory released by the MMA, and xq codes requested by the epilogue when it frees a buffer
+    and expanded to FP16 by the mask group that takes the chunk."""
+    rng = sim.rng
+    B = lambda name, count, n: [Bar(f"{name}{i}", count) for i in range(n)]
+    cb_full, cb_free, mq = B("CB_FULL", 1, 4), B("CB_FREE", 8, 4), B("MQ", 8, 4)
+    tok_full, tok_free = B("TOK_FULL", 1, 4), B("TOK_FREE", 8, 4)
+    acc, acc_free, afree = B("ACC", 1, 2), B("ACC_FREE", 8, 2), B("AFREE", 1, 2)
+    ch_full, ch_free = B("CH_FULL", 1, 2), B("CH_FREE", 1, 2)
+    x_raw, x_full, x_free = B("X_RAW", 1, 2), B("X_FULL", 8, 2), B("X_FREE", 8 * ntpu, 2)
+
+    it_of = lambda n: n % ntpu
+    cb_index = lambda n: (n & 3) if ntpu == 1 else ((0 if it_of(n) else 2) + ((n >> 1) & 1))
+    cb_use = lambda n: (n >> 2)
+    x_index = lambda n: (n & 1) if ntpu == 1 else ((n >> 1) & 1)
+    x_use = lambda n: (n >> 1) if ntpu == 1 else (n >> 2)
+    t = lambda role: rng.expovariate(1.0) * speed[role]
+    full = lambda bar, use: ("wait", bar, use & 1, use + 1)
+    free = lambda bar, use: ("wait", bar, (use & 1) ^ 1, use)
+
+    def prod_cb():
+        for kc in range(2):                                   # the codes of the first two chunks
+            if kc * ntpu < ntiles:
+                yield ("async", t("load"), [(x_raw[kc], 1)])
+        for n in range(ntiles):
+            ci, t3 = cb_index(n), n & 3
+            yield free(cb_free[ci], cb_use(n))
+            yield ("async", t("load"), [(cb_full[ci], 1)])
+            yield free(tok_free[t3], n >> 2)
+            yield ("async", t("load"), [(tok_full[t3], 1)])
+            yield ("work", t("producer"))
+
+    def prod_ch():
+        for n in range(ntiles):
+            if one_ch_barrier:
+                yield free(ch_free[0], n)
+                yield ("async", t("load"), [(ch_full[0], 1)])
+            else:
+                if n > 0:
+                    yield full(ch_free[(n - 1) & 1], (n - 1) >> 1)   # the other issuer's MMAs have read the buffer
+                yield ("async", t("load"), [(ch_full[n & 1], 1)])
+            yield ("work", t("producer"))
+
+    def issuer(par):
+        for n in range(par, ntiles, 2):
+            ci, s2, xs = cb_index(n), n & 1, x_index(n)
+            yield free(acc_free[s2], n >> 1)
+            yield full(ch_full[0], n) if one_ch_barrier else full(ch_full[par], n >> 1)
+            yield ("work", t("mma"))
+            yield ("async", t("mma"), [(ch_free[0 if one_ch_barrier else par], 1)])
+            yield full(mq[ci], cb_use(n))
+            yield full(x_full[xs], x_use(n))
+            yield ("work", t("mma"))
+            yield ("async", t("mma"), [(afree[s2], 1), (acc[s2], 1)])
+
+    def mask(g):
+        for n in range(ntiles):
+            if (((n if ntpu == 1 else n >> 1)) & 1) != g:
+                continue
+            ci, t3, ob, xs = cb_index(n), n & 3, n & 1, x_index(n)
+            yield full(tok_full[t3], n >> 2)
+            yield full(cb_full[ci], cb_use(n))
+            yield free(afree[ob], n >> 1)
+            if it_of(n) == 0:
+                yield full(x_raw[xs], x_use(n))
+                yield ("work", t("mask") * 0.2)
+                yield ("arrive", x_full[xs], 8)
+            yield ("work", t("mask") * (1 + 2 * it_of(n)))
+            yield ("arrive", mq[ci], 8)
+            yield ("arrive", cb_free[ci], 8)
+
+    def epilogue():
+        for n in range(ntiles):
+            s2, xs, t3 = n & 1, x_index(n), n & 3
+            yield full(acc[s2], n >> 1)
+            yield full(x_full[xs], x_use(n))
+            yield full(tok_full[t3], n >> 2)
+            yield ("work", t("epilogue"))
+            yield ("arrive", acc_free[s2], 8)
+            yield ("arrive", x_free[xs], 8)
+            yield ("arrive", tok_free[t3], 8)
+            if it_of(n) == ntpu - 1 and n - (ntpu - 1) + 2 * ntpu < ntiles:
+                yield full(x_free[xs], x_use(n))               # every warp is through with the chunk
+                yield ("async", t("load"), [(x_raw[xs], 1)])   # the codes of the chunk after next
+
+    for name, gen in [("prod_cb", prod_cb()), ("prod_ch", prod_ch()), ("mma0", issuer(0)), ("mma1", issuer(1)),
+                      ("mask0", mask(0)), ("mask1", mask(1)), ("epi", epilogue())]:
+        sim.spawn(name, gen)
+
+
 SPEEDS = [
     dict(load=1.0, producer=0.1, mma=0.3, mask=2.0, epilogue=2.0),     # roughly the measured ratios
     dict(load=1.0, producer=0.1, mma=0.3, mask=0.01, epilogue=5.0),    # instant mask, slow epilogue
@@ -215,3 +307,22 @@ def test_a_mask_barrier_wait_in_the_epilogue_would_be_lapped():
             assert "MQ" in str(e) or "deadlock" in str(e)
             hit += 1
     assert hit > 0
+
+
+@pytest.mark.parametrize("ntpu", [1, 2])
+@pytest.mark.parametrize("speed", range(len(SPEEDS)))
+def test_fp16_operand_kernel_protocol(ntpu, speed):
+    for seed in range(20):
+        sim = Sim(5000 + 1000 * speed + seed)
+        build_f16(sim, ntiles=36, ntpu=ntpu, speed=SPEEDS[speed])
+        sim.run()
+
+
+def test_two_issuers_on_one_barrier_pair_would_pass_a_wait_early():
+    """With a single barrier pair on the Cq/hq buffer, the issuer of the odd tiles polls the parity of
+    phase 1 before phase 0 has completed, which a fresh barrier answers with yes."""
+    with pytest.raises(AssertionError, match="CH_FULL"):
+        sim = Sim(1)
+        build_f16(sim, ntiles=36, ntpu=2, speed=SPEEDS[0], one_ch_barrier=True)
+        sim.run()
+
