@@ -9,6 +9,8 @@ role speeds, decides every wait by the parity rule alone, and checks against the
 that no wait is ever lapped, that none passes early, and that every role finishes.  It also shows
 that the tempting variant in which the epilogue takes the row scalars through the CBq buffer's mask
 barrier does get lapped when the mask is fast.
+The FP16-operand kernel's protocol (build_f16) is modelled the same way, with the variant that gave
+its two MMA issuers a single barrier pair on the Cq/hq buffer as the counter-example.
 """
 import heapq
 import random
