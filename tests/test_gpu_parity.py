@@ -550,6 +550,41 @@ def test_16_bit_y_flags_are_exclusive_and_without_taps():
     torch.cuda.synchronize()
 
 
+
+@pytest.mark.parametrize("fmt", ["float16", "bfloat16"])
+@pytest.mark.parametrize("operand", [0, 1], ids=["int8_operand", "fp16_operand"])
+def test_fwd_16_bit_y_with_correction_and_init_state(operand, fmt):
+    """The mean-correction vector (Eq. 8) and an initial state together with 16-bit y, for both operand
+    formats of ChunkScan2: the 16-bit y is the kernel's own binary32 y of the same call rounded to
+    nearest even, and that binary32 y agrees with the oracle."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SMALL[2]
+    t = inputs.make_prefill(cfg)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    corr = (0.05 * np.random.default_rng(5).standard_normal(cfg.channels)).astype(np.float32)
+    y_ref, fin_ref, _ = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"],
+                                      q["A"], q["D"], corr, q["s_xs"], q["s_cb"], q["s_h"], init, flags=operand)
+    y32, fin32, _ = gh.gpu_fwd(cfg, q, corr=corr, taps=(), flags=operand)
+    assert np.array_equal(fin32, fin_ref)
+    assert np.abs(y32 - y_ref).max() <= Y_TOL * rms(y_ref)
+    td = getattr(torch, fmt)
+    flag = operand | (bd.FLAG_Y_FP16 if fmt == "float16" else bd.FLAG_Y_BF16)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    y16 = torch.full(t["x"].shape, float("nan"), dtype=td, device="cuda")
+    fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_fwd_args(y=y16, final_state=fin, status=status, corr=gh.dev(corr), init_state=gh.dev(init), **dv)
+    bd.ssdi8_chunk_scan_fwd(dims, args, bd.alloc_workspace(dims, flags=flag), flags=flag)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(fin.cpu().numpy(), fin32)
+    want = torch.from_numpy(y32).to(td)
+    assert torch.equal(y16.cpu().view(torch.int16), want.view(torch.int16))
+
 # --------------------------------------------------------------------------- the paper's FP16 ChunkScan2 operand
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
 def test_fwd_fp16_operand_against_the_oracle_mode(cfg):
