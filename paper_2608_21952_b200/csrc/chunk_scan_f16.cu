@@ -236,7 +236,6 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
   tmem_st_wait();
 }
 
-// CORR: a mean-correction vector is given; YT: format of y (0 binary32, 1 fp16, 2 bf16)
 // The xq rows of a chunk arrive as int8 codes in the upper half of the chunk's x buffer (rows of 64
 // bytes from byte 64 Q on) and are expanded in place into the MMA's FP16 operand (rows of 128 bytes,
 // 128-byte swizzle, from byte 0) by the mask group that takes the chunk: one row per thread, every
@@ -264,6 +263,7 @@ __device__ __forceinline__ void x_row_to_half(uint8_t* xb, int r, const uint4 (&
   }
 }
 
+// CORR: a mean-correction vector is given; YT: format of y (0 binary32, 1 fp16, 2 bf16);
 // BIGQ: chunks of 128 tokens or more (128-row tiles, 128-byte CBq rows: the tile geometry is a constant)
 template <bool CORR, int YT, bool BIGQ>
 __global__ void __launch_bounds__(kThreads, 1)
