@@ -57,7 +57,7 @@ constexpr uint32_t OFF_H = 114688;      // [64][N]
 constexpr uint32_t OFF_X = 122880;      // ring of 2 x [256][64]: the xq rows of a chunk
 constexpr uint32_t OFF_TOK = 155648;    // ring of 4 x (5 Q floats: cs, dt, woff, atok, bounds), read by the mask warps
 constexpr uint32_t TOK_BYTES = 5120;
-// ring of 8 x what the epilogue needs of a tile: [128] row maxima and [128] exp(cs_i), written by the
+// ring of 8 x what the epilogue needs of a tile: [128] row maxima and [128] cs_i, written by the
 // mask warps, and the head's s_x, s_h and correction vectors ([64] each, bulk-loaded).  Eight deep so
 // that the mask of a tile never waits for the epilogue of an earlier one.
 constexpr uint32_t OFF_ROW = OFF_TOK + 4 * TOK_BYTES;
@@ -262,8 +262,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
   int8_t* mq_tap = nullptr;
   if (TAPS && a.taps.Mq) mq_tap = a.taps.Mq + ((((i64)t.b * a.d.c + t.k) * a.d.H + t.h) * Q + i) * Q;
   if (q2 == 0) {
-    rowbuf[r] = rowmax;                 // read by the epilogue warps, with the decay of the
-    rowbuf[128 + r] = exp32(cs_i);      // off-diagonal term
+    rowbuf[r] = rowmax;                 // read by the epilogue warps, with cs_i (they take its
+    rowbuf[128 + r] = cs_i;             // exponential: the mask warps set the pace of the kernel)
     if (TAPS && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
   }
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
@@ -543,7 +543,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       const bool ok = er < TM;
       const int ei = t.it * TM + er;
       const float sC = row[ROW_SCAL / 4], Dh = row[ROW_SCAL / 4 + 1], scb = row[ROW_SCAL / 4 + 2];
-      const float dec = ok ? row[128 + er] * sC : 0.f;
+      const float dec = ok ? exp32(row[128 + er]) * sC : 0.f;
       const float sm = ok ? scb * row[er] * (1.0f / 127.0f) : 0.f;
       const float2 dec2 = make_float2(dec, dec), sm2 = make_float2(sm, sm), Dh2 = make_float2(Dh, Dh);
       const uint32_t tbase = tmem + (uint32_t)a4 * 128u + ((uint32_t)(q * 32) << 16);
