@@ -2,7 +2,8 @@
 //   acc_cb[i,j] = sum_n Cq[i,n] Bq[j,n]   per (batch, chunk, group), INT32 exact in TMEM, then one
 //   INT32 -> INT8 step  CBq = rne(fmul(float(acc_cb), fdiv(fmul(s_C, s_B), s_cb))).
 // One CTA per 128-row tile of the chunk; only the columns that touch the causal half are
-// computed (row tile it needs columns j < 128 (it + 1)).  Both operands are K-major as they sit
+// computed (row tile it needs columns j < 128 (it + 1)), and within those the 16-column sub-blocks
+// after a row's own are stored as zeros.  Both operands are K-major as they sit
 // in HBM ([token][N], N contiguous): TMA stages them in the 128-byte (64-byte for N = 64)
 // swizzled layout the MMA reads.  The int8 codes leave through a swizzled staging panel and one
 // TMA store per 128-column panel.
@@ -104,8 +105,12 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
       if (a.store) {
         uint8_t* panel = smem + OFF_O + (uint32_t)(j0 / 128) * 16384u;
         const uint32_t c0 = (uint32_t)(j0 % 128) >> 4;  // first 16-byte chunk of this piece in the panel row
-        *reinterpret_cast<uint4*>(panel + swz_off((uint32_t)r, c0, RBO)) = make_uint4(o[0], o[1], o[2], o[3]);
-        *reinterpret_cast<uint4*>(panel + swz_off((uint32_t)r, c0 + 1, RBO)) = make_uint4(o[4], o[5], o[6], o[7]);
+        // 16-column sub-blocks that lie wholly above the row's own are written as zeros: the scan
+        // kernel builds its masked operand in place over this tile and then has nothing to clear there
+        const bool z0 = (j0 >> 4) > (i >> 4), z1 = (j0 >> 4) + 1 > (i >> 4);
+        const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(panel + swz_off((uint32_t)r, c0, RBO)) = z0 ? zero4 : make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(panel + swz_off((uint32_t)r, c0 + 1, RBO)) = z1 ? zero4 : make_uint4(o[4], o[5], o[6], o[7]);
       }
       if (a.tap_acc) {
 #pragma unroll

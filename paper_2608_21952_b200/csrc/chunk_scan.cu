@@ -169,7 +169,6 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
   if (r >= TM) return;               // whole warps (TM is a multiple of 16)
   const int i = t.it * TM + r;       // row within the chunk
   const int I16 = i >> 4, ri = i & 15;
-  const int nch = t.KJ >> 4;         // 16-column chunks in the contraction range
   const uint32_t cshift = RBQ == 128 ? 3u : 2u;  // log2(chunks per panel row)
   uint8_t* const rowbase = sCB + (RBQ == 128 ? (uint32_t)r * 128u : (uint32_t)r * 64u);
   const uint32_t rx = RBQ == 128 ? ((uint32_t)r & 7u) : (((uint32_t)r >> 1) & 3u);  // swizzle term of the row
@@ -267,9 +266,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
     if (TAPS && a.taps.rowmax) a.taps.rowmax[(t.tok0 + i) * a.d.H + t.h] = rowmax;
   }
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-  // chunks after the row's own contribute nothing
-#pragma unroll 1
-  for (int c = I16 + 1 + q2; c < nch; c += 2) *chunk_ptr(c) = zero4;
+  // (the chunks after the row's own arrive as zeros: ChunkBMM writes them so)
   {
     const float2 inv2 = make_float2(inv, inv);
     uint2 v;
