@@ -158,9 +158,9 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
                   make_float2(__uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7650u + e)),
                               __uint_as_float(__byte_perm(ww[w], 0x4B400000u, 0x7651u + e))),
                   make_float2(-kMagicIn, -kMagicIn));
-              const float2 v2 = __fmul2_rn(__fmul2_rn(xf, make_float2(rx[w * 4 + e], rx[w * 4 + e + 1])), l2);
-              q4[e] = rne_clamp_bits(v2.x);
-              q4[e + 1] = rne_clamp_bits(v2.y);
+              const uint2 c2 = rne_clamp_bits2(__fmul2_rn(__fmul2_rn(xf, make_float2(rx[w * 4 + e], rx[w * 4 + e + 1])), l2));
+              q4[e] = c2.x;
+              q4[e + 1] = c2.y;
             }
             o[w] = pack4_bits(q4[0], q4[1], q4[2], q4[3]);
           }
@@ -231,9 +231,16 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
           const float4 i1 = *reinterpret_cast<const float4*>(col_invh + cb + p0 + 4);
           const float ih[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
+          for (int e = 0; e < 8; e += 2) {
             const int pp = p0 + e;
-            code[e] = I8S ? (uint32_t)__float_as_int(S[pp]) : rne_clamp_bits(__fmul_rn(S[pp], ih[e]));
+            if (I8S) {
+              code[e] = (uint32_t)__float_as_int(S[pp]);
+              code[e + 1] = (uint32_t)__float_as_int(S[pp + 1]);
+            } else {
+              const uint2 c2 = rne_clamp_bits2(__fmul2_rn(make_float2(S[pp], S[pp + 1]), make_float2(ih[e], ih[e + 1])));
+              code[e] = c2.x;
+              code[e + 1] = c2.y;
+            }
           }
           uint8_t* hrow = sHQ + (cb + p0) * N + n;
 #pragma unroll
@@ -270,10 +277,24 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
           const float4 c0v = *reinterpret_cast<const float4*>(col_scale + cb + hf * 8);
           const float4 c1v = *reinterpret_cast<const float4*>(col_scale + cb + hf * 8 + 4);
           const float cscale[8] = {c0v.x, c0v.y, c0v.z, c0v.w, c1v.x, c1v.y, c1v.z, c1v.w};
+          float locv[8];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            const float2 af = __fadd2_rn(make_float2(__int_as_float(acc[e] + 0x4B400000), __int_as_float(acc[e + 1] + 0x4B400000)),
+                                         make_float2(-kMagicOut, -kMagicOut));   // exact for |acc| < 2^22
+            const float2 l2 = __fmul2_rn(af, make_float2(cscale[e], cscale[e + 1]));
+            locv[e] = l2.x;
+            locv[e + 1] = l2.y;
+            if (!I8S && !(TAPS && a.tap_loc)) {
+              const float2 s2 = __ffma2_rn(make_float2(gam, gam), make_float2(S[hf * 8 + e], S[hf * 8 + e + 1]), l2);
+              S[hf * 8 + e] = s2.x;
+              S[hf * 8 + e + 1] = s2.y;
+            }
+          }
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const int pp = hf * 8 + e;
-            const float loc = __fmul_rn(i22_to_f32(acc[e]), cscale[e]);
+            const float loc = locv[e];
             if (TAPS && a.tap_acc) a.tap_acc[obase + (i64)e * N] = acc[e];
             if (I8S) {
               const int locq = (int)(int8_t)(rne_clamp_bits(loc) & 0xffu);
@@ -281,8 +302,10 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
               const int Sn = locq + ((Gq * __float_as_int(S[pp]) + 64) >> 7);
               S[pp] = __int_as_float(max(-127, min(127, Sn)));
             } else {
-              if (TAPS && a.tap_loc) a.tap_loc[obase + (i64)e * N] = loc;
-              S[pp] = __fmaf_rn(gam, S[pp], loc);
+              if (TAPS && a.tap_loc) {
+                a.tap_loc[obase + (i64)e * N] = loc;
+                S[pp] = __fmaf_rn(gam, S[pp], loc);
+              }
             }
           }
         }

@@ -53,10 +53,22 @@ __device__ __forceinline__ float s8_to_f32(uint32_t w_xor, int k) {
 __device__ __forceinline__ float i22_to_f32(int v) {
   return __fadd_rn(__int_as_float(v + 0x4B400000), -kMagicOut);
 }
-// bits whose low byte is the int8 code rne(v) saturated to [-127, 127] (NaN -> -127): clamping
-// before rounding equals rounding before clamping, and (v + 1.5 * 2^23) rounds to nearest even
+// bits whose low byte is the int8 code rne(v) saturated to [-127, 127]: clamping before rounding
+// equals rounding before clamping, and (v + 1.5 * 2^23) rounds to nearest even.  The clamp is one
+// instruction: min(|v|, 127) with the sign of v put back.  (Used on products of finite factors; a NaN
+// would give +-127.)
 __device__ __forceinline__ uint32_t rne_clamp_bits(float v) {
-  return __float_as_uint(__fadd_rn(fminf(fmaxf(v, -127.0f), 127.0f), kMagicOut));
+  float c;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c) : "f"(v), "f"(127.0f));
+  return __float_as_uint(__fadd_rn(c, kMagicOut));
+}
+// the same for a pair (the magic addition as one packed instruction)
+__device__ __forceinline__ uint2 rne_clamp_bits2(float2 v) {
+  float2 c;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c.x) : "f"(v.x), "f"(127.0f));
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c.y) : "f"(v.y), "f"(127.0f));
+  const float2 r = __fadd2_rn(c, make_float2(kMagicOut, kMagicOut));
+  return make_uint2(__float_as_uint(r.x), __float_as_uint(r.y));
 }
 __device__ __forceinline__ uint32_t pack4_bits(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
