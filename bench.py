@@ -266,7 +266,7 @@ class Layer:
         self.quantize(0)
         return ms
 
-    LAUNCHES_PER_STEP = 7  # 3 quantiser + cumsum, BMM, fused chunk state / state passing, chunk scan
+    LAUNCHES_PER_STEP = 5  # quantisers (one launch), cumsum, BMM, fused chunk state / state passing, chunk scan
 
     def e2e_step(self):
         """The same step through the host-buffer entry point of the C-ABI: pinned fp32 x, B, C, dt in,

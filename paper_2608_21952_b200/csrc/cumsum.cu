@@ -36,9 +36,21 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
   const int h0 = blockIdx.x * CH, k = blockIdx.y, b = blockIdx.z;
   const int nh = min(CH, d.H - h0);
   const i64 t0 = (i64)b * d.L + (i64)k * Q;
-  for (int e = threadIdx.x; e < Q * CH; e += blockDim.x) {
-    int i = e / CH, hh = e % CH;
-    if (hh < nh) dts[hh * ld + i] = dt[(t0 + i) * d.H + h0 + hh];
+  // (all loads of a round of 8 before the first store: the loads are the latency of this phase)
+  for (int e0 = threadIdx.x; e0 < Q * CH; e0 += 8 * blockDim.x) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * blockDim.x;
+      const int i = e / CH, hh = e % CH;
+      v[u] = (e < Q * CH && hh < nh) ? __ldg(dt + (t0 + i) * d.H + h0 + hh) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = e0 + u * blockDim.x;
+      const int i = e / CH, hh = e % CH;
+      if (e < Q * CH && hh < nh) dts[hh * ld + i] = v[u];
+    }
   }
   __syncthreads();
   if (threadIdx.x < nh) {

@@ -59,9 +59,9 @@ Layout make_layout(const ssdi8_dims_t& d1, int full_heads, uint8_t* base, uint32
 // side streams and events, made once per device and kept for the life of the process
 struct Plumbing {
   bool ready = false;
-  cudaStream_t s_in = nullptr, s_out = nullptr, s_side = nullptr;
+  cudaStream_t s_in = nullptr, s_out = nullptr, s_side = nullptr, s_side2 = nullptr;
   cudaEvent_t start = nullptr, in_done[kStages] = {}, cmp_done[kStages] = {}, out_done[kStages] = {};
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, fork2 = nullptr, join = nullptr, join2 = nullptr;
 };
 Plumbing g_plumb[64];
 
@@ -78,9 +78,12 @@ ssdi8_status_t get_plumbing(Plumbing** out) {
     int prio_lo = 0, prio_hi = 0;
     SSDI8_CUDA_CHECK(cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
     SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side, cudaStreamNonBlocking, prio_hi));
+    SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side2, cudaStreamNonBlocking, prio_hi));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming));
+    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork2, cudaEventDisableTiming));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming));
+    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join2, cudaEventDisableTiming));
     for (int s = 0; s < kStages; ++s) {
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.in_done[s], cudaEventDisableTiming));
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.cmp_done[s], cudaEventDisableTiming));
@@ -126,20 +129,40 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
   f.init_state = init; f.y = y; f.final_state = fin; f.status = status;
   const uint32_t fl = flags & kLayerFlags;
   ssdi8_status_t s;
+  // one launch for the three quantisers needs a power-of-two N (group of a channel by a shift) and
+  // 16-byte aligned tensors (it reads four values and writes four codes at a time)
+  const bool one_launch =
+      (d.dstate & (d.dstate - 1)) == 0 &&
+      ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C) |
+        reinterpret_cast<uintptr_t>(a.s_x) | reinterpret_cast<uintptr_t>(xq) | reinterpret_cast<uintptr_t>(Bq) |
+        reinterpret_cast<uintptr_t>(Cq)) & 15) == 0;
   SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
-  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork, 0));
-  // side stream: everything that does not need xq
-  if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, p.s_side)) != SSDI8_OK) return s;
-  if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, p.s_side)) != SSDI8_OK) return s;
-  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM | SSDI8_PHASE_BMM, ws, ws_bytes, p.s_side, false)) != SSDI8_OK)
-    return s;
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side2, p.fork, 0));
+  // ChunkCumsum reads dt and A only: it runs on a side stream under the quantisers
+  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, p.s_side2, false)) != SSDI8_OK) return s;
+  SSDI8_CUDA_CHECK(cudaEventRecord(p.join2, p.s_side2));
+  // caller's stream: the three Eq. 1 quantisers
+  if (one_launch) {
+    if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
+                                 Cq, st)) != SSDI8_OK)
+      return s;
+  } else {
+    if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, st)) != SSDI8_OK) return s;
+    if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, st)) != SSDI8_OK) return s;
+    if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
+      return s;
+  }
+  // ChunkBMM needs Bq and Cq and is needed by ChunkScan only: it runs on a side stream under the
+  // state kernel
+  SSDI8_CUDA_CHECK(cudaEventRecord(p.fork2, st));
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork2, 0));
+  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM, ws, ws_bytes, p.s_side, false)) != SSDI8_OK) return s;
   SSDI8_CUDA_CHECK(cudaEventRecord(p.join, p.s_side));
-  // caller's stream: the quantiser of x, then the modules that need everything
-  if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
+  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join2, 0));
+  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING, ws, ws_bytes, st, false)) != SSDI8_OK)
     return s;
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join, 0));
-  return fwd_phases(&d, &f, fl | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING | SSDI8_PHASE_SCAN, ws,
-                    ws_bytes, st, false);
+  return fwd_phases(&d, &f, fl | SSDI8_PHASE_SCAN, ws, ws_bytes, st, false);
 }
 
 // How many equal head ranges a batch element is cut into for the host pipeline: halved while a

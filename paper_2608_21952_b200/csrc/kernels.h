@@ -7,6 +7,12 @@ namespace ssdi8 {
 ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
                                int8_t* out, cudaStream_t st);
 
+// the layer's three static quantisers as one launch: x [T][D] with D step sizes, B and C [T][G N] with G
+// step sizes each (N a power of two, D and N multiples of 4)
+ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* C, i64 T_, int D, int G, int N,
+                                   const float* s_x, const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq,
+                                   int8_t* Cq, cudaStream_t st);
+
 // Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, wmax, lut (see
 // cumsum.cu); element (u, row, i) at pack[(u * kPackRows + row) * Q + i], u = (b*H + h)*c + k.
 constexpr int kPackRows = 6;

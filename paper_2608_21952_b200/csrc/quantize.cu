@@ -39,6 +39,57 @@ __global__ void __launch_bounds__(128) quant_ch_fastest(const float4* __restrict
   }
 }
 
+// ---- the layer's three static quantisers (x per channel; B and C per group) as one launch.  Every
+// tensor is a matrix of R rows; a block covers up to 128 float4 columns and, where a row is narrower
+// than that, several rows per pass, so that a warp still reads 512 contiguous bytes.  The jobs of the
+// narrow tensors come first in the grid: they are placed at once and finish under the wide one.
+struct QuantJob {
+  const float4* in; const float* scale; uint32_t* out;
+  int ch4;          // float4 per row
+  int tpr;          // threads per row (a power of two <= 128)
+  int gx;           // column blocks per row
+  int shift;        // step size of channel c = scale[c >> shift]
+  int first_block;  // of this job in the grid
+  int rows;         // rows per block
+};
+struct QuantJobs { QuantJob job[3]; i64 R; };
+
+__global__ void __launch_bounds__(128, 8) quant_jobs(const QuantJobs a) {
+  const int jb = (int)blockIdx.x >= a.job[2].first_block ? 2 : (int)blockIdx.x >= a.job[1].first_block ? 1 : 0;
+  const QuantJob& j = a.job[jb];
+  const int rel = (int)blockIdx.x - j.first_block;
+  const int bx = rel % j.gx, by = rel / j.gx;
+  const int tr = threadIdx.x / j.tpr;          // row of this thread within a pass
+  const int rpp = 128 / j.tpr;                 // rows per pass
+  const int q = bx * j.tpr + (threadIdx.x & (j.tpr - 1));
+  if (q >= j.ch4) return;
+  float4 s;
+  if (j.shift == 0) {
+    s = __ldg(reinterpret_cast<const float4*>(j.scale) + q);
+  } else {
+    const float g = __ldg(j.scale + ((q * 4) >> j.shift));   // 4 consecutive channels share a group
+    s = make_float4(g, g, g, g);
+  }
+  const QuantStep sx = quant_step(s.x), sy = quant_step(s.y), sz = quant_step(s.z), sw = quant_step(s.w);
+  const i64 r0 = (i64)by * j.rows + tr;
+  const i64 r1 = (i64)(by + 1) * j.rows < a.R ? (i64)(by + 1) * j.rows : a.R;
+  if (r0 >= r1) return;
+  // (the launcher keeps every tensor below 2^31 float4, so 32-bit element indices do)
+  const uint32_t stride = (uint32_t)(rpp * j.ch4);   // float4 (and code words) between two passes
+  uint32_t e = (uint32_t)r0 * (uint32_t)j.ch4 + (uint32_t)q;
+  int left = (int)((r1 - r0 + rpp - 1) / rpp);       // passes this thread takes
+  const float4* __restrict__ in = j.in;
+  uint32_t* __restrict__ out = j.out;
+  for (; left >= QROWS; left -= QROWS, e += QROWS * stride) {
+    float4 v[QROWS];
+#pragma unroll
+    for (int u = 0; u < QROWS; ++u) v[u] = __ldcs(in + (e + u * stride));
+#pragma unroll
+    for (int u = 0; u < QROWS; ++u) __stcs(out + (e + u * stride), quant_code4(v[u], sx, sy, sz, sw));
+  }
+  for (; left > 0; --left, e += stride) __stcs(out + e, quant_code4(__ldcs(in + e), sx, sy, sz, sw));
+}
+
 // ---- quantise, I % 4 == 0: 4 consecutive elements share a channel
 __global__ void __launch_bounds__(QT) quant_inner(const float4* __restrict__ in,
                                                   const float* __restrict__ scale,
@@ -173,6 +224,38 @@ ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* sca
     quant_inner<<<grid, QT, 0, st>>>(reinterpret_cast<const float4*>(in), scale,
                                      reinterpret_cast<uint32_t*>(out), (uint32_t)n4, (uint32_t)(I / 4),
                                      (uint32_t)Ch);
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
+ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* C, i64 T_, int D, int G, int N,
+                                   const float* s_x, const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq,
+                                   int8_t* Cq, cudaStream_t st) {
+  if (T_ == 0) return SSDI8_OK;
+  if (T_ * D / 4 >= ((i64)1 << 31) || T_ * G * N / 4 >= ((i64)1 << 31)) return SSDI8_ERR_UNSUPPORTED;
+  QuantJobs a;
+  a.R = T_;
+  int shift = 0;
+  while ((1 << shift) < N) ++shift;   // N is a power of two here (the caller checks)
+  auto fill = [&](QuantJob& j, const float* in, const float* sc, int8_t* out, int width, int sh, int first) {
+    j.in = reinterpret_cast<const float4*>(in);
+    j.scale = sc;
+    j.out = reinterpret_cast<uint32_t*>(out);
+    j.ch4 = width / 4;
+    j.tpr = 128;
+    while (j.tpr / 2 >= j.ch4 && j.tpr > 1) j.tpr /= 2;
+    j.gx = (j.ch4 + j.tpr - 1) / j.tpr;
+    j.shift = sh;
+    j.first_block = first;
+    // short slabs: blocks that live a few microseconds each, so that the other streams' kernels find
+    // free slots all the time (a slab is at least one full round of QROWS passes)
+    j.rows = QROWS * (128 / j.tpr) < 16 ? 16 : QROWS * (128 / j.tpr);
+    return first + j.gx * (int)((T_ + j.rows - 1) / j.rows);
+  };
+  int nb = fill(a.job[0], B, s_B, Bq, G * N, shift, 0);
+  nb = fill(a.job[1], C, s_C, Cq, G * N, shift, nb);
+  nb = fill(a.job[2], x, s_x, xq, D, 0, nb);
+  quant_jobs<<<(unsigned)nb, 128, 0, st>>>(a);
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }
