@@ -42,6 +42,7 @@ PAPER_TOKENS_PER_S = {"cfg2": 16384 / 4.481e-3}
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture; see profiles/).  None until a capture of that workload exists.
 NCU_TRAFFIC_BYTES = {"cfg2": 441.9e6}  # profiles/chunk_scan_cfg2_ncu_full.md
+NCU_TRAFFIC_BYTES_DECODE = 279.6e6  # ssd_step_kernel at cfg4: profiles/ssd_step_cfg4_and_quant_jobs_cfg2_ncu.md
 
 
 def measured_peaks():
@@ -347,7 +348,8 @@ def run_decode(torch, bd, steps=64, warmup=8):
     return {"workload": "cfg4: decode step, batch 64, 80 heads x 64, d_state 128 (state 168 MB > L2)",
             "tokens_per_s": cfg.batch / (ms * 1e-3), "ms_per_step": ms, "steps": steps,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None}}
+                         "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                         "traffic": NCU_TRAFFIC_BYTES_DECODE}}
 
 
 def run_ours(args):
@@ -468,7 +470,15 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only: skip the end-to-end, per-module, decode and CPU legs (profiling runs)")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="the cfg4 decode leg alone on one GPU (profiling runs of the step kernel)")
     args = ap.parse_args()
+    if args.decode_only:
+        import torch
+        from paper_2608_21952_b200 import binding as bd
+        torch.cuda.set_device(0)
+        print(json.dumps(run_decode(torch, bd, steps=args.steps, warmup=max(args.warmup, 3))))
+        return
     if args.impl == "reference":
         if args.steps > 5:
             args.steps = 5  # each step is seconds of CPU work; keep the run within minutes
