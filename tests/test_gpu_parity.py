@@ -209,6 +209,51 @@ def test_fwd_full_size_sampled(name, npairs, flags):
         assert np.abs(y[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
 
 
+@pytest.mark.parametrize("name,npairs", [("cfg2", 3), ("cfg3", 3)])
+def test_layer_fwd_full_size_sampled(name, npairs):
+    """The call the benchmark's step makes (ssdi8_layer_fwd: fp32 x, B, C in, the three Eq. 1
+    quantisers as one launch, side streams inside) at full size; the oracle quantises the whole
+    tensors and recomputes sampled (batch, head) pairs one by one."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = CONFIGS[name]
+    t = inputs.make_prefill(cfg)
+    rng = np.random.default_rng(200 + cfg.seed)
+    pairs = [(0, 0), (cfg.batch - 1, cfg.nheads - 1)]
+    while len(pairs) < npairs:
+        pr = (int(rng.integers(cfg.batch)), int(rng.integers(cfg.nheads)))
+        if pr not in pairs:
+            pairs.append(pr)
+    q = _sampled_problem(cfg, t, pairs)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "A", "D")}
+    dv.update({k: gh.dev(t[k]) for k in ("x", "B", "C", "dt")})
+    y = torch.empty(t["x"].shape, device="cuda")
+    fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_layer_args(y=y, final_state=fin, status=status, **dv)
+    ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims, 0), dtype=torch.uint8, device="cuda")
+    y_h = fin_h = None
+    for rep in range(2):   # the second call finds the first one's contents in the workspace
+        y.fill_(float("nan")); fin.fill_(float("nan"))
+        bd.ssdi8_layer_fwd(dims, args, ws, 0)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        if rep == 0:
+            y_h, fin_h = y.cpu().numpy(), fin.cpu().numpy()
+        else:
+            assert np.array_equal(y.cpu().numpy(), y_h) and np.array_equal(fin.cpu().numpy(), fin_h)
+    assert np.all(np.isfinite(y_h)) and np.all(np.isfinite(fin_h))
+    one = cfg.replace(batch=1, nheads=1, ngroups=1)
+    for (b, h) in pairs:
+        s = _slice(cfg, b, h, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], t, extra=q)
+        y_ref, fin_ref, _ = orc.ssdi8_fwd(one, s["xq"], s["Bq"], s["Cq"], s["s_x"], s["s_B"], s["s_C"],
+                                          s["dt"], s["A"], s["D"], None, s["s_xs"], s["s_cb"], s["s_h"])
+        assert np.array_equal(fin_h[b, h], fin_ref[0, 0]), (b, h)
+        assert np.abs(y_h[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
+
+
 # --------------------------------------------------------------------------- persistent INT8 states (Eq. 4, 7)
 @pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[2]], ids=lambda c: c.name)
 def test_fwd_int8_state_mode_bit_exact(cfg):
