@@ -41,7 +41,7 @@ UNIT = "tokens/s"
 PAPER_TOKENS_PER_S = {"cfg2": 16384 / 4.481e-3}
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture; see profiles/).  None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"cfg2": 441.9e6}  # profiles/chunk_scan_cfg2_ncu_full.md
+NCU_TRAFFIC_BYTES = {"cfg2": 441.5e6}  # profiles/chunk_scan_cfg2_ncu_full.md
 NCU_TRAFFIC_BYTES_DECODE = 279.6e6  # ssd_step_kernel at cfg4: profiles/ssd_step_cfg4_and_quant_jobs_cfg2_ncu.md
 
 
