@@ -123,6 +123,19 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       const int hp = h * P + c * 16 + e;
       rx[e] = __fdiv_rn(a.s_x[hp], a.s_xs[hp]);
     }
+    // Rows that re-quantise to zero (the sparsity Eq. 3 rests on: LUT_state decays towards the start
+    // of a chunk).  fmul is monotone, so with rxm >= |rx| of every channel of this CTA's range,
+    // fmul(fmul(127, rxm), |LUT_state[i]|) < 1/2 implies |fmul(fmul(x, rx), LUT_state[i])| < 1/2 for every
+    // code x: row i of Q(X_scaled) is all zeros, exactly.  Such a row is stored as zeros without the
+    // arithmetic, and a 32-token slab of such rows is left out altogether (no MMA).
+    float rxm = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) rxm = fmaxf(rxm, fabsf(rx[e]));
+    if (ncq == 4) {
+      rxm = fmaxf(rxm, __shfl_xor_sync(0xffffffffu, rxm, 1));
+      rxm = fmaxf(rxm, __shfl_xor_sync(0xffffffffu, rxm, 2));
+    }
+    const float b127 = __fmul_rn(127.0f, rxm);
 #pragma unroll 1
     for (int k = 0; k < d.c; ++k) {
       const int s = k & 1;
@@ -134,19 +147,44 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       named_bar(2, kQuantThreads);
       // a warp owns whole 32-token slabs (slab = one MMA): rows of a slab are split over the lanes,
       // and the warp's lane 0 issues the slab's MMA as soon as the warp has re-quantised it, so no
-      // warp waits for another.  The accumulator is opened by the MMA of slab 0 (accumulate = 0);
-      // the other issuing threads order their first MMA of the chunk after it through B_OPEN.
+      // warp waits for another.  The accumulator is opened by the MMA of the first live slab
+      // (accumulate = 0); the other issuing threads order their first MMA of the chunk after it
+      // through B_OPEN.  A chunk without a live slab opens with its last slab stored as zeros.
       const int qw = qt >> 5;
+      const int nsl = Q / 32;
+      uint32_t lm = 0;   // live slabs of the chunk (every warp computes the same mask)
+      for (int sl = 0; sl < nsl; ++sl) {
+        const bool dead = __fmul_rn(b127, fabsf(lut[sl * 32 + lane])) < 0.5f;
+        if (!__all_sync(0xffffffffu, dead)) lm |= 1u << sl;
+      }
+      const bool zero_open = lm == 0;
+      if (zero_open) lm = 1u << (nsl - 1);
+      const int first = __ffs((int)lm) - 1;
       const uint32_t sBa = smem_u32(smem + s * STAGE + OFF_B), sXa = smem_u32(sX);
       const uint32_t idesc = idesc_s8(N, 64, 1, 1);
+      const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+      bool mine = false;   // this warp owns a live slab
 #pragma unroll 1
-      for (int sl = qw; sl < Q / 32; sl += kQuantThreads / 32) {
+      for (int sl = qw; sl < nsl; sl += kQuantThreads / 32) {
+        if (!((lm >> sl) & 1u)) {
+          if (TAPS && a.tap_Xsq) {
+            for (int i = sl * 32 + (lane >> lq); i < sl * 32 + 32; i += 32 >> lq)
+              *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = zero4;
+          }
+          continue;
+        }
+        mine = true;
 #pragma unroll 1
         for (int i = sl * 32 + (lane >> lq); i < sl * 32 + 32; i += 32 >> lq) {
           uint4* ptr = reinterpret_cast<uint4*>(sX + swz_off((uint32_t)i, (uint32_t)c, 64));
+          const float l = lut[i];
+          if (zero_open || __fmul_rn(b127, fabsf(l)) < 0.5f) {
+            *ptr = zero4;
+            if (TAPS && a.tap_Xsq) *reinterpret_cast<uint4*>(a.tap_Xsq + ((tok0 + i) * d.H + h) * P + c * 16) = zero4;
+            continue;
+          }
           const uint4 w4 = *ptr;
           const uint32_t ww[4] = {w4.x ^ 0x80808080u, w4.y ^ 0x80808080u, w4.z ^ 0x80808080u, w4.w ^ 0x80808080u};
-          const float l = lut[i];
           const float2 l2 = make_float2(l, l);
           uint32_t o[4];
 #pragma unroll
@@ -171,22 +209,25 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0 && qw < Q / 32) {
-        if (qw == 0) {
-          mbar_wait_inline<0>(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
-        } else {
-          mbar_wait_inline<0>(&bars[B_OPEN], k & 1, a.status);
-        }
-        tc_fence_after();
+      if (lane == 0 && qw < nsl) {
+        if (mine) {
+          if ((first & (kQuantThreads / 32 - 1)) == qw) {
+            mbar_wait_inline<0>(&bars[B_ACC_FREE], (k & 1) ^ 1, a.status);   // the state warps have read chunk k-1
+          } else {
+            mbar_wait_inline<0>(&bars[B_OPEN], k & 1, a.status);
+          }
+          tc_fence_after();
 #pragma unroll 1
-        for (int sl = qw; sl < Q / 32; sl += kQuantThreads / 32) {
-          mma_s8_ss(tmem, tile_desc(sBa + 32 * sl * N, (uint32_t)N), tile_desc(sXa + 32 * sl * 64, 64), idesc, sl > 0);
-          if (sl == 0) {
-            tc_fence_before();
-            mbar_arrive(&bars[B_OPEN]);
+          for (int sl = qw; sl < nsl; sl += kQuantThreads / 32) {
+            if (!((lm >> sl) & 1u)) continue;
+            mma_s8_ss(tmem, tile_desc(sBa + 32 * sl * N, (uint32_t)N), tile_desc(sXa + 32 * sl * 64, 64), idesc, sl != first);
+            if (sl == first) {
+              tc_fence_before();
+              mbar_arrive(&bars[B_OPEN]);
+            }
           }
         }
-        mma_commit(&bars[B_MMA]);   // arrives when this thread's MMAs are done
+        mma_commit(&bars[B_MMA]);   // arrives when this thread's MMAs are done (at once if it issued none)
       }
       __syncwarp();
     }
