@@ -133,6 +133,35 @@ def test_reciprocal_fast_path_of_the_quantiser_is_exact():
     assert 0.2 < fast.mean() < 1.0 and (~fast).sum() > 1000      # both paths exercised
 
 
+def test_zero_row_bound_of_the_fused_state_kernel_is_exact():
+    """The fused ChunkState kernel stores row i of Q(X_scaled) as zeros, without the arithmetic,
+    when fmul(fmul(127, rxm), |LUT_state[i]|) < 1/2, rxm being the largest |s_x / s_xs| of the
+    channels it covers.  Checked here in numpy binary32, every code x in [-127, 127] against
+    channel ratios up to rxm and LUT values placed on both sides of the threshold: where the bound
+    holds every code of Eq. 3, rne(fmul(fmul(x, rx), lut)), is zero; and the bound is not vacuous."""
+    import numpy as np
+    rng = np.random.default_rng(11)
+    x = np.arange(-127, 128, dtype=np.float32)
+    n_dead = n_live_nonzero = 0
+    for _ in range(100):
+        rx = (10.0 ** rng.uniform(-3, 3, 64)).astype(np.float32)
+        rxm = np.float32(np.abs(rx).max())
+        b127 = np.float32(127.0) * rxm
+        # LUT values around the threshold 0.5 / b127, of both signs, plus far smaller and larger ones
+        thr = 0.5 / float(b127)
+        lut = np.concatenate([thr * (1 + rng.uniform(-1e-3, 1e-3, 200)), thr * (1 + rng.uniform(-1e-6, 1e-6, 200)),
+                              thr * 10.0 ** rng.uniform(-6, 1, 100), [0.0, thr]]).astype(np.float32)
+        lut *= rng.choice(np.float32([1, -1]), lut.shape)
+        dead = (b127 * np.abs(lut)).astype(np.float32) < np.float32(0.5)
+        xr = (x[:, None] * rx[None, :]).astype(np.float32)                     # fmul(x, rx)
+        v = (xr[None, :, :] * lut[:, None, None]).astype(np.float32)           # fmul(., lut)
+        code = np.clip(np.rint(v), -127, 127)
+        assert not code[dead].any()
+        n_dead += int(dead.sum())
+        n_live_nonzero += int((np.abs(code[~dead]).max(axis=(1, 2)) > 0).sum())
+    assert n_dead > 10000 and n_live_nonzero > 10000
+
+
 def test_host_side_argument_errors_of_the_layer_and_entry_calls():
     """The one-call layer entries and the entry quantiser validate on the host before any CUDA
     call: these checks run without a device."""
