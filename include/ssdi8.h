@@ -180,7 +180,8 @@ typedef struct {
  *                  t = fmul(float(CBq[i,j]), w)
  *                  rowmax_i = max over sub-blocks of fmul(max_j |t|, f)
  *                  inv_i = rowmax_i >= 1e-30 ? fdiv(127, rowmax_i) : 0
- *                  Mq[i,j] = rne(fmul(t, fmul(f, inv_i)))
+ *                  Mq[i,j] = rn(t * fmul(f, inv_i)): the exact product rounded once to the nearest
+ *                            integer, ties to even (the low bits of fmaf(t, fmul(f, inv_i), 1.5 * 2^23))
  *                acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p], INT32;
  *                y_diag = (s_cb rowmax_i / 127) s_x acc_diag
  *  Output        y = y_off + y_diag + D s_x xq + corr

@@ -241,3 +241,79 @@ def prepare_quantized(cfg, t, init=None):
     s_xs, s_cb, s_h = calibrate(cfg, xq, Bq, Cq, s_x, s_B, s_C, t["dt"], t["A"], init)
     return dict(xq=xq, Bq=Bq, Cq=Cq, s_x=s_x, s_B=s_B, s_C=s_C, dt=t["dt"], A=t["A"], D=t["D"],
                 s_xs=s_xs, s_cb=s_cb, s_h=s_h, init=init)
+
+
+# ---------------------------------------------------------------------------- plain definitions
+def chunk_state_plain(cfg, xq, s_x, s_xs, dt, cs):
+    """Eq. 3 from its definition in fp64.  Returns (v = X_scaled / s_xs as float64, its code int8)."""
+    d = dims_of(cfg)
+    shp = (cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim)
+    v = np.empty(shp, np.float64)
+    code = np.empty(shp, np.int8)
+    _lib.orc_chunk_state_plain(C.byref(d), _p(_i8(xq)), _p(_f32(s_x)), _p(_f32(s_xs)), _p(_f32(dt)),
+                               _p(_f32(cs)), _p(v), _p(code))
+    return v, code
+
+
+def state_codes_plain(cfg, S, s_h):
+    """Eq. 4 from its definition in fp64: (v = State / s_h as float64, its code int8); S [b,c,H,P,N]."""
+    d = dims_of(cfg)
+    S = _f32(S)
+    v = np.empty(S.shape, np.float64)
+    code = np.empty(S.shape, np.int8)
+    _lib.orc_state_codes_plain(C.byref(d), _p(S), _p(_f32(s_h)), _p(v), _p(code))
+    return v, code
+
+
+def chunk_scan_plain(cfg, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D=None, corr=None, flags=0,
+                     want_operand=True):
+    """Algorithm 2 modules 5 and 6 from their definitions in fp64 (one libm exp per element).
+    Returns y and a dict with M (real masked operand [b,c,H,Q,Q]), sM [b,L,H] and Mq (int8 mode)."""
+    d = dims_of(cfg)
+    b, L, H, P, Q, c = cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim, cfg.chunk, cfg.nchunks
+    y = np.empty((b, L, H, P), np.float64)
+    out = {}
+    if want_operand:
+        out["M"] = np.empty((b, c, H, Q, Q), np.float64)
+        if not (flags & FLAG_FP16_OPERAND):
+            out["sM"] = np.empty((b, L, H), np.float64)
+            out["Mq"] = np.empty((b, c, H, Q, Q), np.int8)
+    _lib.orc_chunk_scan_plain(C.byref(d), _p(_i8(xq)), _p(_i8(Cq)), _p(_i8(CBq)), _p(_i8(hq)),
+                              _p(_f32(s_x)), _p(_f32(s_C)), _p(_f32(s_cb)), _p(_f32(s_h)), _p(_f32(dt)),
+                              _p(_f32(cs)), _p(_f32(D)), _p(_f32(corr)), _p(out.get("M")),
+                              _p(out.get("sM")), _p(out.get("Mq")), _p(y), C.c_uint32(flags))
+    return y, out
+
+
+def ssdi8_fwd_plain(cfg, xq, Bq, Cq, s_x, s_B, s_C, dt, A, D, corr, s_xs, s_cb, s_h, init=None, flags=0):
+    """The whole forward from the plain definitions (fp64 throughout).  Returns (y, final) float64."""
+    d = dims_of(cfg)
+    y = np.empty((cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim), np.float64)
+    fin = np.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), np.float64)
+    _lib.orc_ssdi8_fwd_plain(C.byref(d), _p(_i8(xq)), _p(_i8(Bq)), _p(_i8(Cq)), _p(_f32(s_x)),
+                             _p(_f32(s_B)), _p(_f32(s_C)), _p(_f32(dt)), _p(_f32(A)), _p(_f32(D)),
+                             _p(_f32(corr)), _p(_f32(s_xs)), _p(_f32(s_cb)), _p(_f32(s_h)),
+                             _p(_f32(init)), _p(y), _p(fin), C.c_uint32(flags))
+    return y, fin
+
+
+def prop1_mse(cfg, x, dt, cs):
+    """Proposition 1 diagnostic: (per-element MSE of Q(X_scaled), per-element MSE of Q(X) (.) LUT_state,
+    zero fraction of Q(X_scaled), the second error summed over the l axis of a chunk as in the proof)."""
+    d = dims_of(cfg)
+    out = np.empty(4, np.float64)
+    _lib.orc_prop1_mse(C.byref(d), _p(_f32(x)), _p(_f32(dt)), _p(_f32(cs)), _p(out))
+    return tuple(float(v) for v in out)
+
+
+def chunk_scan_fp16_operand(cfg, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D=None, corr=None):
+    """The binary32-defined FP16 operand of orc_chunk_scan (flags bit 0) and its y: (y, M16 [b,c,H,Q,Q])."""
+    d = dims_of(cfg)
+    b, L, H, P, Q, c = cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim, cfg.chunk, cfg.nchunks
+    y = np.empty((b, L, H, P), np.float64)
+    m16 = np.empty((b, c, H, Q, Q), np.float64)
+    _lib.orc_chunk_scan(C.byref(d), _p(_i8(xq)), _p(_i8(Cq)), _p(_i8(CBq)), _p(_i8(hq)), _p(_f32(s_x)),
+                        _p(_f32(s_C)), _p(_f32(s_cb)), _p(_f32(s_h)), _p(_f32(dt)), _p(_f32(cs)),
+                        _p(_f32(D)), _p(_f32(corr)), None, None, None, None, _p(y),
+                        C.c_uint32(FLAG_FP16_OPERAND), _p(m16))
+    return y, m16

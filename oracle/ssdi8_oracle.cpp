@@ -22,6 +22,17 @@
 // The exponential inside those values is exp32() below, a fixed sequence of
 // binary32 operations, pinned against libm's exp by the tests.
 //
+// Two forms of the internal re-quantisations.  The "plain" functions (orc_*_plain,
+// orc_ssdi8_fwd_plain) are the definitions written out: fp64, libm exp, one exponential per
+// element, no blocking of any kind; they are what a reader checks against Algorithm 2 and
+// Eq. 1, 3, 4 by eye.  The other stage functions (orc_chunk_state, orc_state_passing,
+// orc_chunk_scan) restate the operation-by-operation binary32 arithmetic that the library's
+// header fixes for every value that decides an integer code, so that a second implementation
+// can be compared bit for bit; their factorisation of the decay into 16-token sub-blocks is
+// part of that interface, not of the method.  The tests tie the two together: every code of the
+// binary32 form equals the plain form's code or is its neighbour with the fp64 value next to
+// the rounding boundary between them.
+//
 // Pins (tests/test_oracle_*.py): L1 == L0 for every chunk size (duality and
 // chunk invariance), closed form for constant inputs, A -> 0 reduces to masked
 // linear attention (numpy matmul), dt = 0 gives y = D x, integer GEMM stages
@@ -92,6 +103,14 @@ inline float exp32(float x) {
   p = std::fmaf(p, r, 1.0f);
   uint32_t u = bits_from_f(p) + ((uint32_t)((int32_t)n) << 23);
   return f_from_bits(u);
+}
+
+// round(a b) saturated, a b being the exact product (48 significant bits: exact in binary64)
+inline int8_t rne_clamp_exact_product(float a, float b) {
+  double r = std::nearbyint((double)a * (double)b);
+  if (!(r >= -127.0)) r = -127.0;
+  if (r > 127.0) r = 127.0;
+  return (int8_t)(int)r;
 }
 
 inline int sub_block(int Q) { return Q < 16 ? Q : 16; }
@@ -425,7 +444,10 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 }
 
 // ---------------------------------------------------------------------------
-// L2 stage: ChunkScan1 + ChunkScan2 + output sum (Algorithm 2 modules 5, 6).
+// L2 stage: ChunkScan1 + ChunkScan2 + output sum (Algorithm 2 modules 5, 6) in the library's
+// operation-by-operation binary32 arithmetic (the interface fixed in the library's header, so
+// that codes can be compared bit for bit).  This is NOT the definition: the definition is
+// orc_chunk_scan_plain further down, and the tests bound the distance between the two.
 //  off-diagonal:  acc_off[i,p] = sum_n Cq[i,n] hq[k][p,n]  (exact)
 //                 y_off = exp(cs_i) s_C s_h[h,p] acc_off   (decay applied after the product)
 //  diagonal: the masked operand CB o LUT_scan2 is re-quantised per output row i
@@ -438,7 +460,7 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 //     t[i,j]   = fmul(float(CBq[i,j]), w)          (w f = dt_j exp(cs_i - cs_j); every exponent <= 0)
 //     rowmax_i = max over sub-blocks J of fmul(max_{j in J, j<=i} |t[i,j]|, f)
 //     inv_i    = rowmax_i >= 1e-30 ? fdiv(127, rowmax_i) : 0
-//     Mq[i,j]  = round(fmul(t[i,j], fmul(f, inv_i)))
+//     Mq[i,j]  = round(t[i,j] * fmul(f, inv_i)), the exact product rounded once (one fused operation)
 //     acc_diag[i,p] = sum_{j<=i} Mq[i,j] xq[j,p]    (exact)
 //     y_diag   = (s_cb rowmax_i / 127) s_x[h,p] acc_diag
 //  y = y_off + y_diag + D s_x xq + corr
@@ -465,7 +487,7 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
                     const int8_t* hq, const float* s_x, const float* s_C, const float* s_cb,
                     const float* s_h, const float* dt, const float* cs, const float* D,
                     const float* corr, int32_t* acc_off, float* rowmax, int8_t* Mq,
-                    int32_t* acc_diag, double* y, uint32_t flags) {
+                    int32_t* acc_diag, double* y, uint32_t flags, double* M16) {
   const bool fp16_operand = (flags & 1u) != 0;
   const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
             G = d->ngroups, Q = d->chunk, c = L / Q, hpg = H / G;
@@ -513,6 +535,10 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
             // decision: both sides of a parity test must take it in the same precision)
             for (int j = 0; j <= i; ++j)
               m16[j] = orc_round_half((double)fmul(t[j], (j / SB == I) ? s_cb[g] : fmul(f[j / SB], s_cb[g])));
+            if (M16) {  // [b,c,H,Q,Q], zero above the diagonal
+              double* o = M16 + ((((i64)b * c + k) * H + h) * Q + i) * Q;
+              for (int j = 0; j < Q; ++j) o[j] = (j <= i) ? m16[j] : 0.0;
+            }
             const double dec = std::exp((double)csk[i]);
             for (int p = 0; p < P; ++p) {
               int32_t ao = 0;
@@ -532,7 +558,9 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
           }
           const float inv = (rmax >= 1e-30f) ? fdiv(127.0f, rmax) : 0.0f;
           for (int j = 0; j < Q; ++j) mq[j] = 0;
-          for (int j = 0; j <= i; ++j) mq[j] = rne_clamp(fmul(t[j], fmul(f[j / SB], inv)));
+          // the product t g is rounded once, to the nearest integer (ties to even): the exact product
+          // of two binary32 numbers fits a binary64
+          for (int j = 0; j <= i; ++j) mq[j] = rne_clamp_exact_product(t[j], fmul(f[j / SB], inv));
           if (rowmax) rowmax[(t0 + i) * H + h] = rmax;
           if (Mq) {
             int8_t* o = Mq + ((((i64)b * c + k) * H + h) * Q + i) * Q;
@@ -559,6 +587,234 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
         }
       }
     }
+}
+
+// ---------------------------------------------------------------------------
+// PLAIN DEFINITIONS (fp64, libm).  Nothing below is blocked, factorised or reordered.
+
+inline int8_t rne_clamp64(double v) {
+  double r = std::nearbyint(v);          // ties to even
+  if (!(r >= -127.0)) r = -127.0;
+  if (r > 127.0) r = 127.0;
+  return (int8_t)(int)r;
+}
+
+// Eq. 3, plain: X_scaled[i,p] = LUT_state[i] x[i,p] with LUT_state[i] = dt_i exp(cs_last - cs_i)
+// (Algorithm 2 module 2) and x = s_x xq; its code is round(X_scaled / s_xs).  Writes the real
+// quotient v = X_scaled / s_xs [b,L,H,P] (may be NULL) and the code (may be NULL).
+void orc_chunk_state_plain(const Dims* d, const int8_t* xq, const float* s_x, const float* s_xs,
+                           const float* dt, const float* cs, double* v_out, int8_t* Xsq) {
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, Q = d->chunk, c = L / Q;
+#pragma omp parallel for collapse(2)
+  for (int b = 0; b < b_; ++b)
+    for (int h = 0; h < H; ++h)
+      for (int k = 0; k < c; ++k) {
+        const float* csk = cs + (((i64)b * H + h) * c + k) * Q;
+        for (int i = 0; i < Q; ++i) {
+          const i64 t = (i64)b * L + (i64)k * Q + i;
+          const double lut = (double)dt[t * H + h] * std::exp((double)csk[Q - 1] - (double)csk[i]);
+          for (int p = 0; p < P; ++p) {
+            const i64 o = (t * H + h) * P + p;
+            const double v = (double)xq[o] * (double)s_x[h * P + p] * lut / (double)s_xs[h * P + p];
+            if (v_out) v_out[o] = v;
+            if (Xsq) Xsq[o] = rne_clamp64(v);
+          }
+        }
+      }
+}
+
+// Eq. 4, plain: the code of a state element is round(State / s_h), per-(H,P) step size.
+// S [b,c,H,P,N] (the state entering each chunk) -> v = S / s_h and its code.
+void orc_state_codes_plain(const Dims* d, const float* S, const float* s_h, double* v_out,
+                           int8_t* hq) {
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
+            Q = d->chunk, c = L / Q;
+  for (i64 u = 0; u < (i64)b_ * c; ++u)
+    for (int h = 0; h < H; ++h)
+      for (int p = 0; p < P; ++p)
+        for (int n = 0; n < N; ++n) {
+          const i64 o = ((u * H + h) * P + p) * N + n;
+          const double v = (double)S[o] / (double)s_h[h * P + p];
+          if (v_out) v_out[o] = v;
+          if (hq) hq[o] = rne_clamp64(v);
+        }
+}
+
+// Algorithm 2 modules 5 and 6 and the output sum, plain.
+//   ChunkScan1  y_off[i,p]  = exp(cs_i) sum_n C[i,n] State[p,n],  C = s_C Cq, State = s_h hq
+//   ChunkScan2  LUT_scan2[i,j] = dt_j exp(cs_i - cs_j), j <= i (0 above the diagonal)
+//               M[i,j]      = CB[i,j] LUT_scan2[i,j],  CB = s_cb CBq
+//     int8 operand (flags bit 0 clear): Eq. 1 applied to each row of M,
+//               s_M[i] = max_j |M[i,j]| / 127 (1 if the row is zero), Mq = round(M / s_M),
+//               y_diag[i,p] = s_M[i] s_x[p] sum_j Mq[i,j] xq[j,p]
+//     FP16 operand (flags bit 0 set; Section 4.2): M16 = half(M),
+//               y_diag[i,p] = s_x[p] sum_j M16[i,j] xq[j,p]
+//   y = y_off + y_diag + D s_x xq + corr
+// Optional outputs: M [b,c,H,Q,Q] (the real operand, zero above the diagonal), sM [b,L,H]
+// (int8 mode), Mq [b,c,H,Q,Q] (int8 mode).
+void orc_chunk_scan_plain(const Dims* d, const int8_t* xq, const int8_t* Cq, const int8_t* CBq,
+                          const int8_t* hq, const float* s_x, const float* s_C, const float* s_cb,
+                          const float* s_h, const float* dt, const float* cs, const float* D,
+                          const float* corr, double* M_out, double* sM_out, int8_t* Mq_out,
+                          double* y, uint32_t flags) {
+  const bool fp16_operand = (flags & 1u) != 0;
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
+            G = d->ngroups, Q = d->chunk, c = L / Q, hpg = H / G;
+#pragma omp parallel for collapse(2)
+  for (int b = 0; b < b_; ++b)
+    for (int h = 0; h < H; ++h) {
+      const int g = h / hpg;
+      std::vector<double> M(Q), W(Q);
+      for (int k = 0; k < c; ++k) {
+        const i64 t0 = (i64)b * L + (i64)k * Q;
+        const float* csk = cs + (((i64)b * H + h) * c + k) * Q;
+        const int8_t* cbk = CBq + (((i64)b * c + k) * G + g) * Q * Q;
+        const int8_t* hqk = hq + (((i64)b * c + k) * H + h) * P * N;
+        for (int i = 0; i < Q; ++i) {
+          double amax = 0.0;
+          for (int j = 0; j < Q; ++j) {
+            M[j] = 0.0;
+            if (j <= i) {
+              const double lut = (double)dt[(t0 + j) * H + h] * std::exp((double)csk[i] - (double)csk[j]);
+              M[j] = (double)s_cb[g] * (double)cbk[(size_t)i * Q + j] * lut;
+            }
+            amax = std::fmax(amax, std::fabs(M[j]));
+          }
+          const i64 row = ((((i64)b * c + k) * H + h) * Q + i) * Q;
+          if (M_out) for (int j = 0; j < Q; ++j) M_out[row + j] = M[j];
+          double sM = 1.0;
+          if (fp16_operand) {
+            for (int j = 0; j < Q; ++j) W[j] = orc_round_half(M[j]);
+          } else {
+            sM = (amax == 0.0) ? 1.0 : amax / 127.0;
+            for (int j = 0; j < Q; ++j) {
+              const int8_t q = rne_clamp64(M[j] / sM);
+              W[j] = (double)q;
+              if (Mq_out) Mq_out[row + j] = q;
+            }
+            if (sM_out) sM_out[(t0 + i) * H + h] = sM;
+          }
+          const double dec = std::exp((double)csk[i]);
+          for (int p = 0; p < P; ++p) {
+            double off = 0.0;
+            for (int n = 0; n < N; ++n)
+              off += (double)Cq[((t0 + i) * G + g) * N + n] * (double)hqk[(size_t)p * N + n];
+            double diag = 0.0;
+            for (int j = 0; j <= i; ++j) diag += W[j] * (double)xq[((t0 + j) * H + h) * P + p];
+            const i64 o = ((t0 + i) * H + h) * P + p;
+            double v = dec * (double)s_C[g] * (double)s_h[h * P + p] * off +
+                       sM * (double)s_x[h * P + p] * diag;
+            if (D) v += (double)D[h] * (double)s_x[h * P + p] * (double)xq[o];
+            if (corr) v += (double)corr[h * P + p];
+            y[o] = v;
+          }
+        }
+      }
+    }
+}
+
+// The whole SSDi8 forward from the plain definitions alone (Algorithm 2 with Eq. 1, 3, 4; fp32
+// inter-chunk states replaced by fp64 ones), every rounding decided on fp64 values.  It shares
+// only the exact integer stages and the cumulative sum with orc_ssdi8_fwd.  y fp64, final fp64.
+void orc_ssdi8_fwd_plain(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8_t* Cq,
+                         const float* s_x, const float* s_B, const float* s_C, const float* dt,
+                         const float* A, const float* D, const float* corr, const float* s_xs,
+                         const float* s_cb, const float* s_h, const float* init, double* y,
+                         double* final_state, uint32_t flags) {
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, N = d->dstate,
+            G = d->ngroups, Q = d->chunk, c = L / Q, hpg = H / G;
+  std::vector<float> cs((size_t)b_ * H * L);
+  orc_chunk_cumsum(d, dt, A, cs.data());                       // module 1
+  // module 4: ChunkBMM, one INT32 -> INT8 step (Section 4.2)
+  std::vector<int32_t> acc_cb((size_t)b_ * c * G * Q * Q);
+  std::vector<int8_t> CBq(acc_cb.size());
+  orc_chunk_bmm(d, Cq, Bq, s_C, s_B, nullptr, acc_cb.data(), nullptr);
+  for (i64 u = 0; u < (i64)b_ * c; ++u)
+    for (int g = 0; g < G; ++g)
+      for (i64 e = 0; e < (i64)Q * Q; ++e) {
+        const i64 o = (u * G + g) * Q * Q + e;
+        CBq[o] = rne_clamp64((double)acc_cb[o] * (double)s_C[g] * (double)s_B[g] / (double)s_cb[g]);
+      }
+  // module 2: ChunkState (Eq. 3), exact integer product, Eq. 4 rescale to a real-valued state
+  std::vector<int8_t> Xsq((size_t)b_ * L * H * P);
+  orc_chunk_state_plain(d, xq, s_x, s_xs, dt, cs.data(), nullptr, Xsq.data());
+  const size_t nst = (size_t)b_ * c * H * P * N;
+  std::vector<int8_t> hq(nst);
+#pragma omp parallel for collapse(2)
+  for (int b = 0; b < b_; ++b)
+    for (int h = 0; h < H; ++h) {
+      const int g = h / hpg;
+      std::vector<double> S((size_t)P * N, 0.0);
+      if (init) for (int e = 0; e < P * N; ++e) S[e] = (double)init[((i64)b * H + h) * P * N + e];
+      for (int k = 0; k < c; ++k) {
+        const i64 t0 = (i64)b * L + (i64)k * Q;
+        const double gam = std::exp((double)cs[(((i64)b * H + h) * c + k) * Q + Q - 1]);  // Eq. 5
+        for (int p = 0; p < P; ++p)
+          for (int n = 0; n < N; ++n) {
+            const i64 o = ((((i64)b * c + k) * H + h) * P + p) * N + n;
+            hq[o] = rne_clamp64(S[(size_t)p * N + n] / (double)s_h[h * P + p]);   // Eq. 4
+            i64 a = 0;
+            for (int i = 0; i < Q; ++i)
+              a += (i64)Xsq[((t0 + i) * H + h) * P + p] * (i64)Bq[((t0 + i) * G + g) * N + n];
+            const double loc = (double)a * (double)s_xs[h * P + p] * (double)s_B[g];
+            S[(size_t)p * N + n] = loc + gam * S[(size_t)p * N + n];               // Eq. 6
+          }
+      }
+      if (final_state)
+        for (int e = 0; e < P * N; ++e) final_state[((i64)b * H + h) * P * N + e] = S[e];
+    }
+  orc_chunk_scan_plain(d, xq, Cq, CBq.data(), hq.data(), s_x, s_C, s_cb, s_h, dt, cs.data(), D,
+                       corr, nullptr, nullptr, nullptr, y, flags);
+}
+
+// ---------------------------------------------------------------------------
+// Diagnostic of Proposition 1 (Appendix A): mean squared error of the two ways of putting
+// y = x (.) lut on an 8-bit grid, on real-valued x [b,L,H,P]:
+//   out[0] = error of deq(Q(x (.) LUT_state))   (the reformulation, Eq. 3: quantise X_scaled),
+//            mean over all elements (the proof's MSE_x_scaled: an expectation per element)
+//   out[1] = error of deq(Q(x)) (.) LUT_state   (quantise X, scale afterwards), mean over all elements
+//   out[2] = fraction of Q(X_scaled) codes that are zero (the proof's 1 - rho)
+//   out[3] = the proof's MSE_x: the squared norm of the second error over the l axis of one chunk
+//            (its Step 3 sums over l), mean over chunks, heads and channels; equals out[1] * Q.
+// The proposition as printed compares out[0] with out[3], i.e. a per-element mean with a per-vector
+// sum; both normalisations are returned.  Each Q is Eq. 1 with one step size per channel (h,p)
+// calibrated on the tensor it is applied to (absmax / 127), LUT_state[i] = dt_i exp(cs_last - cs_i).
+void orc_prop1_mse(const Dims* d, const float* x, const float* dt, const float* cs, double* out) {
+  const int b_ = d->batch, L = d->seqlen, H = d->nheads, P = d->headdim, Q = d->chunk, c = L / Q;
+  const i64 T = (i64)b_ * L;
+  std::vector<double> lut((size_t)T * H), ax((size_t)H * P, 0.0), ay((size_t)H * P, 0.0);
+  for (int b = 0; b < b_; ++b)
+    for (int h = 0; h < H; ++h)
+      for (int k = 0; k < c; ++k) {
+        const float* csk = cs + (((i64)b * H + h) * c + k) * Q;
+        for (int i = 0; i < Q; ++i) {
+          const i64 t = (i64)b * L + (i64)k * Q + i;
+          lut[t * H + h] = (double)dt[t * H + h] * std::exp((double)csk[Q - 1] - (double)csk[i]);
+        }
+      }
+  for (i64 t = 0; t < T; ++t)
+    for (int ch = 0; ch < H * P; ++ch) {
+      const double xv = (double)x[t * H * P + ch], yv = xv * lut[t * H + ch / P];
+      ax[ch] = std::fmax(ax[ch], std::fabs(xv));
+      ay[ch] = std::fmax(ay[ch], std::fabs(yv));
+    }
+  double e_scaled = 0.0, e_x = 0.0;
+  i64 zeros = 0;
+  for (i64 t = 0; t < T; ++t)
+    for (int ch = 0; ch < H * P; ++ch) {
+      const double l = lut[t * H + ch / P], xv = (double)x[t * H * P + ch], yv = xv * l;
+      const double sx = ax[ch] == 0.0 ? 1.0 : ax[ch] / 127.0, sy = ay[ch] == 0.0 ? 1.0 : ay[ch] / 127.0;
+      const int qy = (int)rne_clamp64(yv / sy), qx = (int)rne_clamp64(xv / sx);
+      zeros += (qy == 0);
+      const double ea = sy * qy - yv, eb = sx * qx * l - yv;
+      e_scaled += ea * ea;
+      e_x += eb * eb;
+    }
+  const double n = (double)T * H * P;
+  out[0] = e_scaled / n;
+  out[1] = e_x / n;
+  out[2] = (double)zeros / n;
+  out[3] = out[1] * (double)Q;
 }
 
 // ---------------------------------------------------------------------------
@@ -677,7 +933,7 @@ void orc_ssdi8_fwd(const Dims* d, const int8_t* xq, const int8_t* Bq, const int8
     orc_state_passing(d, loc, gamma.data(), init, s_h, prev, final_state, hq);
   }
   orc_chunk_scan(d, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D, corr, tp->acc_off,
-                 tp->rowmax, tp->Mq, tp->acc_diag, y, flags);
+                 tp->rowmax, tp->Mq, tp->acc_diag, y, flags, nullptr);
 }
 
 // ---------------------------------------------------------------------------

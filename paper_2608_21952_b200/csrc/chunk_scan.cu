@@ -90,10 +90,14 @@ __device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
                                __uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7651u + k)));
   return __fadd2_rn(m, make_float2(-kMagicIn, -kMagicIn));
 }
-// rne(v) for |v| < 2^22 sits in the low bits of (v + 1.5 * 2^23); callers guarantee |v| < 127.5
-__device__ __forceinline__ uint32_t pack4_rne(float2 a, float2 b) {
-  const float2 ra = __fadd2_rn(a, make_float2(kMagicOut, kMagicOut));
-  const float2 rb = __fadd2_rn(b, make_float2(kMagicOut, kMagicOut));
+// four codes rn(a g), the exact product rounded once to the nearest integer (ties to even): for
+// |a g| < 2^22 that integer sits in the low bits of fma(a, g, 1.5 * 2^23); callers guarantee
+// |a g| < 127.5.  (One fused operation by definition: a packed multiply followed by a packed add of
+// the rounding constant is not an alternative, the assembler contracts that pair into this very
+// fused operation, which differs from the two-step result wherever the rounded product is a tie.)
+__device__ __forceinline__ uint32_t pack4_rn_product(float2 a, float2 b, float2 g) {
+  const float2 ra = __ffma2_rn(a, g, make_float2(kMagicOut, kMagicOut));
+  const float2 rb = __ffma2_rn(b, g, make_float2(kMagicOut, kMagicOut));
   return __byte_perm(__byte_perm(__float_as_uint(ra.x), __float_as_uint(ra.y), 0x0040u),
                      __byte_perm(__float_as_uint(rb.x), __float_as_uint(rb.y), 0x0040u), 0x5410u);
 }
@@ -270,8 +274,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
   {
     const float2 inv2 = make_float2(inv, inv);
     uint2 v;
-    v.x = pack4_rne(__fmul2_rn(make_float2(tv[0], tv[1]), inv2), __fmul2_rn(make_float2(tv[2], tv[3]), inv2));
-    v.y = pack4_rne(__fmul2_rn(make_float2(tv[4], tv[5]), inv2), __fmul2_rn(make_float2(tv[6], tv[7]), inv2));
+    v.x = pack4_rn_product(make_float2(tv[0], tv[1]), make_float2(tv[2], tv[3]), inv2);
+    v.y = pack4_rn_product(make_float2(tv[4], tv[5]), make_float2(tv[6], tv[7]), inv2);
     *own_ptr = v;
     if (TAPS && mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
   }
@@ -297,8 +301,8 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           const float4 fo = wo[w];
-          o[w] = pack4_rne(__fmul2_rn(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)), g2),
-                           __fmul2_rn(__fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2));
+          o[w] = pack4_rn_product(__fmul2_rn(unpack2(ww[w], 0), make_float2(fo.x, fo.y)),
+                                  __fmul2_rn(unpack2(ww[w], 2), make_float2(fo.z, fo.w)), g2);
         }
         if (need) v = make_uint4(o[0], o[1], o[2], o[3]);
       }

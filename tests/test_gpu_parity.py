@@ -10,7 +10,7 @@ import pytest
 from oracle import oracle as orc
 from paper_2608_21952_b200 import inputs
 from paper_2608_21952_b200.inputs import CONFIGS, SSDConfig
-from helpers import rms
+from helpers import census, half_neighbours, rms
 
 pytestmark = pytest.mark.gpu
 
@@ -254,6 +254,128 @@ def test_layer_fwd_full_size_sampled(name, npairs):
         assert np.abs(y_h[b, :, h] - y_ref[0, :, 0]).max() <= Y_TOL * rms(y_ref), (b, h)
 
 
+
+# --------------------------------------------------------------------------- against the plain definitions
+PLAIN_CASES = {
+    "cfg0": (CONFIGS["cfg0"], None), "cfg1": (CONFIGS["cfg1"], None),
+    "slow": (SMALL[1], _scale_A(0.01)), "fast": (SMALL[2], _scale_A(8.0)), "very_fast": (SMALL[1], _scale_A(200.0)),
+}
+
+
+@pytest.mark.parametrize("case", list(PLAIN_CASES))
+def test_fwd_boundary_aware_against_the_plain_definitions(case, capsys):
+    """The GPU's integer tensors against the fp64 definitions (libm exp, no sub-blocks): a code
+    equals round(v) of the fp64 value v, or is its neighbour with v inside the derived window around
+    the rounding boundary between the two; the row maxima within 1e-5; y against the y of the plain
+    definitions on the same integer inputs as a relative L2 distance."""
+    gh = _harness()
+    cfg, mutate = PLAIN_CASES[case]
+    t = inputs.make_prefill(cfg)
+    if mutate is not None:
+        mutate(t)
+    init = inputs.make_init_state(cfg, 0.3)
+    q = orc.prepare_quantized(cfg, t, init)
+    y, fin, got = gh.gpu_fwd(cfg, q)
+    rep = {}
+    v, _ = orc.chunk_state_plain(cfg, q["xq"], q["s_x"], q["s_xs"], q["dt"], got["cs"])
+    rep["Xsq"], worst, outside = census(got["Xsq"], v, 4e-6)
+    assert worst <= 1 and outside == 0
+    v, _ = orc.state_codes_plain(cfg, got["prev"], q["s_h"])
+    rep["hq"], worst, outside = census(got["hq"], v, 4e-6)
+    assert worst <= 1 and outside == 0
+    y_plain, out = orc.chunk_scan_plain(cfg, q["xq"], q["Cq"], got["CBq"] * _causal(cfg), got["hq"], q["s_x"], q["s_C"],
+                                        q["s_cb"], q["s_h"], q["dt"], got["cs"], q["D"], None)
+    b, c, Q, H = cfg.batch, cfg.nchunks, cfg.chunk, cfg.nheads
+    sM = out["sM"].reshape(b, c, Q, H).transpose(0, 1, 3, 2)[..., None]
+    # the library treats a row whose largest |CBq dt_j exp(cs_i - cs_j)| is below 1e-30 as a zero row
+    # (and exponentials below e^-80 as zero); Eq. 1 taken literally would still spread such a row over
+    # the 8-bit range.  Those rows (they contribute less than 1e-30 to y) must be all-zero codes.
+    rm = got["rowmax"].reshape(b, c, Q, H).transpose(0, 1, 3, 2)                 # [b,c,H,Q]
+    flushed = rm < 1e-30
+    assert np.all(got["Mq"][flushed] == 0)
+    rep["flushed_rows"] = float(flushed.mean())
+    keep = ~flushed
+    rep["Mq"], worst, outside = census(got["Mq"][keep], (out["M"] / sM)[keep], 1e-5)
+    assert worst <= 1 and outside == 0
+    hg = np.arange(H) // (H // cfg.ngroups)
+    rowmax = got["rowmax"].astype(np.float64) * q["s_cb"].astype(np.float64)[hg][None, None, :]
+    amax = np.abs(out["M"]).max(-1).transpose(0, 1, 3, 2).reshape(b, c * Q, H)
+    live = got["rowmax"] >= 1e-30
+    assert np.allclose(rowmax[live], amax[live], rtol=1e-5, atol=0) and np.all(amax[~live] < 4e-30)
+    rep["y_rel_l2"] = float(np.sqrt(((y - y_plain) ** 2).sum() / (y_plain ** 2).sum()))
+    assert rep["y_rel_l2"] < 1e-3
+    # the whole forward from the plain definitions alone (no tensor of the GPU run enters it)
+    y_ind, fin_ind = orc.ssdi8_fwd_plain(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"], q["A"],
+                                         q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], init)
+    rep["y_rel_l2_independent"] = float(np.sqrt(((y - y_ind) ** 2).sum() / (y_ind ** 2).sum()))
+    rep["final_rel_l2_independent"] = float(np.sqrt(((fin - fin_ind) ** 2).sum() / (fin_ind ** 2).sum()))
+    assert rep["y_rel_l2_independent"] < 5e-3 and rep["final_rel_l2_independent"] < 5e-3
+    with capsys.disabled():
+        print(f"\n[GPU vs plain, {case}] " + ", ".join(f"{k} {v:.2e}" for k, v in rep.items()))
+
+
+# --------------------------------------------------------------------------- the benchmark's own problem, every pair
+@pytest.mark.parametrize("name,flags", [("cfg2", 0), ("cfg2", 2), ("cfg2", 1), ("cfg3", 0)],
+                         ids=["cfg2", "cfg2_int8_state", "cfg2_fp16_operand", "cfg3"])
+def test_fwd_full_size_all_pairs(name, flags):
+    """Exactly what the benchmark runs: Eq. 1 on the whole tensors, internal step sizes from
+    ssdi8_calibrate on the whole tensors (compared bit for bit with the oracle's calibration), then
+    ssdi8_layer_fwd without taps; the oracle recomputes EVERY (batch, head) pair, one batch element
+    at a time.  Final state bit for bit, y within the tolerance per pair."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = CONFIGS[name]
+    t = inputs.make_prefill(cfg)
+    T = cfg.tokens
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(t[k]) for k in ("x", "B", "C", "dt", "A", "D")}
+    i8 = lambda k: torch.empty(t[k].shape, dtype=torch.int8, device="cuda")
+    xq, Bq, Cq = i8("x"), i8("B"), i8("C")
+    z = lambda n: torch.empty(n, device="cuda")
+    s_x, s_B, s_C = z(cfg.channels), z(cfg.ngroups), z(cfg.ngroups)
+    s_xs, s_cb, s_h = z(cfg.channels), z(cfg.ngroups), z(cfg.channels)
+    bd.ssdi8_quantize_act(dv["x"], T, cfg.channels, 1, s_x, 1, xq)
+    bd.ssdi8_quantize_act(dv["B"], T, cfg.ngroups, cfg.dstate, s_B, 1, Bq)
+    bd.ssdi8_quantize_act(dv["C"], T, cfg.ngroups, cfg.dstate, s_C, 1, Cq)
+    ws = bd.alloc_workspace(dims)
+    cal = bd.make_fwd_args(xq=xq, Bq=Bq, Cq=Cq, s_x=s_x, s_B=s_B, s_C=s_C, dt=dv["dt"], A=dv["A"])
+    bd.ssdi8_calibrate(dims, cal, s_xs, s_cb, s_h, ws)
+    torch.cuda.synchronize()
+    q = orc.prepare_quantized(cfg, t)
+    for k, g in (("xq", xq), ("Bq", Bq), ("Cq", Cq), ("s_x", s_x), ("s_B", s_B), ("s_C", s_C), ("s_xs", s_xs),
+                 ("s_cb", s_cb), ("s_h", s_h)):
+        assert np.array_equal(g.cpu().numpy(), q[k]), k
+    del ws, xq, Bq, Cq
+    td = torch.float16 if flags & 1 else torch.float32
+    yflag = bd.FLAG_Y_FP16 if flags & 1 else 0     # the paper's operand with the paper's output format
+    y = torch.full(t["x"].shape, float("nan"), dtype=td, device="cuda")
+    fin = torch.full((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), float("nan"), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_layer_args(x=dv["x"], B=dv["B"], C=dv["C"], dt=dv["dt"], A=dv["A"], D=dv["D"], s_x=s_x, s_B=s_B,
+                              s_C=s_C, s_xs=s_xs, s_cb=s_cb, s_h=s_h, y=y, final_state=fin, status=status)
+    lws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims, flags | yflag), dtype=torch.uint8, device="cuda")
+    bd.ssdi8_layer_fwd(dims, args, lws, flags | yflag)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    y_h, fin_h = y.float().cpu().numpy(), fin.cpu().numpy()
+    del y, lws
+    one = cfg.replace(batch=1)
+    worst = 0.0
+    for b in range(cfg.batch):
+        sl = lambda a: np.ascontiguousarray(a[b:b + 1])
+        y_ref, fin_ref, _ = orc.ssdi8_fwd(one, sl(q["xq"]), sl(q["Bq"]), sl(q["Cq"]), q["s_x"], q["s_B"], q["s_C"],
+                                          sl(q["dt"]), q["A"], q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], flags=flags)
+        assert np.array_equal(fin_h[b], fin_ref[0]), b
+        pair_rms = np.sqrt((y_ref[0] ** 2).mean(axis=(0, 2)))                       # [H]
+        err = np.abs(y_h[b] - y_ref[0])
+        if flags & 1:   # fp16 y: half a unit in the last place of each element on top
+            err = np.maximum(err - 1.01 * 2.0 ** -11 * np.abs(y_ref[0]), 0.0)
+        pair_err = err.max(axis=(0, 2))
+        assert np.all(pair_err <= Y_TOL * pair_rms), (b, int(np.argmax(pair_err / pair_rms)))
+        worst = max(worst, float((pair_err / pair_rms).max()))
+    print(f"{name} flags={flags}: worst pair max|dy|/rms = {worst:.2e} over {cfg.batch * cfg.nheads} pairs")
+
 # --------------------------------------------------------------------------- persistent INT8 states (Eq. 4, 7)
 @pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[2]], ids=lambda c: c.name)
 def test_fwd_int8_state_mode_bit_exact(cfg):
@@ -459,6 +581,11 @@ def test_step_n64_groups():
 
 def test_step_full_size_batch():
     _decode_case(CONFIGS["cfg4"], 8)
+
+
+def test_step_full_size_batch_all_256_steps():
+    """cfg4 as specified: batch 64, 256 steps; y of every step and the state after the last one."""
+    _decode_case(CONFIGS["cfg4"], 256)
 
 
 # --------------------------------------------------------------------------- host-buffer entry point
