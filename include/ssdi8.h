@@ -311,6 +311,23 @@ ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const 
                               const float* s_C, const float* dt, const float* A, const float* D,
                               const float* corr, float* state, float* y, void* stream);
 
+/* Measurement aid (the paper has no counterpart): what tcgen05.mma.kind::i8 sustains on the current
+ * device, for the "fraction of the int8 tensor-pipe peak" a benchmark reports.  One CTA per SM issues
+ * `mma_per_sm` (rounded down to a multiple of 128, at least 128) dense MMAs of M 128 x N 256 x K 32
+ * back to back on operands resident in shared memory, accumulating into tensor memory.  *ops (HOST)
+ * receives the number of integer operations the launch performs (2 per multiply-accumulate); divide
+ * by the device time of the call, measured by the caller with events on `stream`.  status: 1 word on
+ * the DEVICE or NULL, written only if a bounded wait ran out. */
+ssdi8_status_t ssdi8_int8_mma_peak(int64_t mma_per_sm, double* ops, int32_t* status, void* stream);
+
+/* Self-test of the time-out path every kernel of this library shares (Section references: none, the
+ * paper has no counterpart).  Launches one thread that waits, through the library's bounded mbarrier
+ * wait with a cap of 48 polls, on a barrier nothing ever arrives on: no copy is in flight and no
+ * tensor memory is held, so nothing can fault or hang.  After about a millisecond the wait gives up,
+ * writes SSDI8_ERR_DEVICE_TIMEOUT to *status (DEVICE, 1 word, required) and the kernel returns
+ * normally; the context stays usable. */
+ssdi8_status_t ssdi8_selftest_bounded_wait(int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

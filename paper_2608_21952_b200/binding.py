@@ -35,7 +35,8 @@ EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
            "ssdi8_state_passing", "ssdi8_ssd_step", "ssdi8_mean_correction",
            "ssdi8_mean_correction_workspace_bytes", "ssdi8_quantize_entry",
            "ssdi8_layer_fwd", "ssdi8_layer_fwd_workspace_bytes",
-           "ssdi8_layer_fwd_host", "ssdi8_layer_fwd_host_scratch_bytes")
+           "ssdi8_layer_fwd_host", "ssdi8_layer_fwd_host_scratch_bytes",
+           "ssdi8_int8_mma_peak", "ssdi8_selftest_bounded_wait")
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 
@@ -248,6 +249,24 @@ def ssdi8_ssd_step(dims: Dims, xq, s_x, Bq, s_B, Cq, s_C, dt, A, D, corr, state,
     _check(_lib.ssdi8_ssd_step(C.byref(dims), _ptr(xq), _ptr(s_x), _ptr(Bq), _ptr(s_B), _ptr(Cq),
                                _ptr(s_C), _ptr(dt), _ptr(A), _ptr(D), _ptr(corr), _ptr(state), _ptr(y),
                                _stream(stream)), "ssdi8_ssd_step")
+
+
+_lib.ssdi8_int8_mma_peak.restype = C.c_int32
+_lib.ssdi8_int8_mma_peak.argtypes = [C.c_int64, C.POINTER(C.c_double), C.c_void_p, C.c_void_p]
+_lib.ssdi8_selftest_bounded_wait.restype = C.c_int32
+_lib.ssdi8_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_void_p]
+
+
+def ssdi8_int8_mma_peak(mma_per_sm: int, status=None, stream=None) -> float:
+    """Launches the dense INT8 MMA loop; returns the number of integer operations of the launch."""
+    ops = C.c_double(0.0)
+    _check(_lib.ssdi8_int8_mma_peak(mma_per_sm, C.byref(ops), _ptr(status), _stream(stream)),
+           "ssdi8_int8_mma_peak")
+    return float(ops.value)
+
+
+def ssdi8_selftest_bounded_wait(status, stream=None) -> None:
+    _check(_lib.ssdi8_selftest_bounded_wait(_ptr(status), _stream(stream)), "ssdi8_selftest_bounded_wait")
 
 
 def alloc_workspace(dims: Dims, device="cuda", flags: int = 0):

@@ -1,5 +1,6 @@
 // C-ABI entry points of libssdi8: argument validation, workspace layout, kernel sequencing.
 #include <cstring>
+#include <mutex>
 
 #include "kernels.h"
 
@@ -24,11 +25,14 @@ bool dims_supported(const ssdi8_dims_t* d, bool need_chunks) {
 }
 
 // The kernels are built for sm_100a only (tensor-memory MMA does not exist elsewhere).
+// (First use on a device fills the cache under a lock: two threads may make their first call at once.)
 ssdi8_status_t check_arch() {
   static int ok_device[64];  // 0 unknown, 1 ok, -1 wrong
+  static std::mutex mu;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SSDI8_ERR_CUDA;
   if (dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
   if (ok_device[dev] == 0) {
     int major = 0, minor = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -286,6 +290,26 @@ ssdi8_status_t ssdi8_mean_correction(const float* y_ref, const float* y_q, int64
                                 static_cast<cudaStream_t>(stream));
 }
 
+ssdi8_status_t ssdi8_int8_mma_peak(int64_t mma_per_sm, double* ops, int32_t* status, void* stream) {
+  if (!ops) return SSDI8_ERR_NULL;
+  const int per_batch = int8_mma_peak_batch();
+  if (mma_per_sm < per_batch || mma_per_sm > ((int64_t)1 << 24)) return SSDI8_ERR_SHAPE;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  const int nbatch = (int)(mma_per_sm / per_batch);
+  int ctas = 0;
+  if ((s = launch_int8_mma_peak(nbatch, status, &ctas, static_cast<cudaStream_t>(stream))) != SSDI8_OK) return s;
+  *ops = 2.0 * 128.0 * 256.0 * 32.0 * (double)per_batch * (double)nbatch * (double)ctas;
+  return SSDI8_OK;
+}
+
+ssdi8_status_t ssdi8_selftest_bounded_wait(int32_t* status, void* stream) {
+  if (!status) return SSDI8_ERR_NULL;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_bounded_wait_expires(status, static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------
 // Forward pass with library-owned scratch (no allocation by anyone).
 //
@@ -307,9 +331,15 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
   if (need == 0)
     return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
   if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
+  // (before the symbol lookup: on a device of another architecture the lookup itself fails, and the
+  // caller should learn that the device is the wrong one)
+  const ssdi8_status_t arch = check_arch();
+  if (arch != SSDI8_OK) return arch;
   static void* ws_of_device[64];  // resolved address of g_static_ws, per device
+  static std::mutex ws_mu;        // two threads may make their first call on a device at once
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(ws_mu);
   if (!ws_of_device[dev]) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) {

@@ -9,6 +9,8 @@
 // caller's stream: the PCIe link is busy in both directions for the whole call instead of
 // idle during the kernels and one-directional during the copies.  Only stream and event
 // plumbing lives here; every arithmetic step is a kernel of this library.
+#include <mutex>
+
 #include "kernels.h"
 
 namespace ssdi8 {
@@ -64,12 +66,14 @@ struct Plumbing {
   cudaEvent_t fork = nullptr, fork2 = nullptr, join = nullptr, join2 = nullptr;
 };
 Plumbing g_plumb[64];
+std::mutex g_plumb_mu;   // two threads may make their first call on a device at once
 
 ssdi8_status_t get_plumbing(Plumbing** out) {
   int dev = 0;
   SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SSDI8_ERR_CUDA;
   Plumbing& p = g_plumb[dev];
+  std::lock_guard<std::mutex> lock(g_plumb_mu);
   if (!p.ready) {
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));

@@ -89,6 +89,12 @@ int mean_correction_slabs(i64 R);
 ssdi8_status_t launch_mean_correction(const float* y, const float* yq, i64 R, i64 Ch, float eta, float* corr,
                                       double* partial, cudaStream_t st);
 
+// measurement aid and self-test (selftest.cu): `nbatch` batches of int8_mma_peak_batch() MMAs of
+// M 128 x N 256 x K 32 on every SM (ctas = number of CTAs launched); a bounded wait that runs out
+ssdi8_status_t launch_int8_mma_peak(int nbatch, int32_t* status, int* ctas, cudaStream_t st);
+int int8_mma_peak_batch();
+ssdi8_status_t launch_bounded_wait_expires(int32_t* status, cudaStream_t st);
+
 // scale[k] = bits[k] == 0 ? 1 : fdiv(as_float(bits[k]) [* mul], 127)   (in place)
 ssdi8_status_t launch_finalize_scales(float* scale_bits, i64 n, const float* mul_a,
                                       const float* mul_b, int bits_are_int, cudaStream_t st);

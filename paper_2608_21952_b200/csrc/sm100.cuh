@@ -59,9 +59,12 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 // The polling loop is one out-of-line function: a call site is the first attempt and a branch, so
 // the many waits of a warp-specialised kernel do not bloat its instruction footprint.
 constexpr uint32_t kWaitCap = 1u << 17;
+// (CAP is a template parameter only so that the library's self-test can run this very loop with a
+// cap of a few dozen polls on a barrier nobody arrives on; every kernel of the layer uses kWaitCap.)
+template <uint32_t CAP = kWaitCap>
 static __device__ __noinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, int32_t* status,
                                                    uint32_t sleep_ns) {
-  for (uint32_t it = 0; it < kWaitCap; ++it) {
+  for (uint32_t it = 0; it < CAP; ++it) {
     if (mbar_try_wait(bar, parity)) return;
     if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 255u) == 255u && status && *reinterpret_cast<volatile int32_t*>(status) != 0) return;
