@@ -2,15 +2,22 @@
 """Benchmark of the B200 INT8 SSD layer (SSDi8 hot path).
 
 One step = one pass of the whole hot path over one batch of seeded synthetic input:
-Eq. 1 quantisation of fp32 x, B, C with static step sizes (3 launches), then the
+Eq. 1 quantisation of fp32 x, B, C with static step sizes (one launch), then the
 layer forward (ChunkCumsum, ChunkBMM, fused ChunkState+StatePassing, ChunkScan)
 from int8 x, B, C to the fp32 output y and the final state.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
 
-N > 1: launched by torch.distributed.run, one rank per GPU.  The layer shards over
+N > 1: one rank per GPU under torch.distributed.run (started by the caller, or by this
+script itself when WORLD_SIZE is not in the environment).  The layer shards over
 (batch, head) with no exchange, so every rank runs the same workload on its own
 GPU (weak scaling, no data-path collective); the time is the maximum over ranks.
+
+The K timed steps are repeated as rounds (each bracketed by a barrier and a device
+synchronisation) until at least half a second has been timed; `ms_per_step` is the median
+round, so that the clock record covers hundreds of samples.  Every timed call carries a
+status word that must read 0 after its round, and after the timed loop the output and final
+state of the last step are compared with the CPU oracle (`parity`); a failure exits non-zero.
 
 Prints ONE JSON line.  `--impl reference` times the CPU oracle (as it stands) on
 the host cores on a bounded sample of the same workload.
@@ -20,7 +27,9 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -39,10 +48,15 @@ UNIT = "tokens/s"
 # (SSD module of block 55, Mamba-2 2.7B, batch 8, L = 2048: 4.481 ms on an RTX A5000):
 # 16384 tokens / 4.481 ms.  Another machine's number: context, not the target.
 PAPER_TOKENS_PER_S = {"cfg2": 16384 / 4.481e-3}
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum
-# of one ncu capture; see profiles/).  None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"cfg2": 441.5e6}  # profiles/chunk_scan_cfg2_ncu_full.md
+# Figures read from ncu captures (a number taken under a profiler is never a bench value; these are
+# byte counts and a pipe utilisation, which do not depend on the clock): DRAM bytes per launch
+# (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel and of the decode step kernel,
+# and the tensor-pipe active share of the scan kernel, each with the summary file it comes from.
+NCU_SCAN = {"cfg2": {"traffic": 441.5e6, "tensor_active_pct": 8.3,
+                     "source": "profiles/chunk_scan_cfg2_ncu_full.md"}}
 NCU_TRAFFIC_BYTES_DECODE = 279.6e6  # ssd_step_kernel at cfg4: profiles/ssd_step_cfg4_and_quant_jobs_cfg2_ncu.md
+INT8_NOMINAL_TOPS = 4500.0          # dense INT8 figure of the B200 data sheet
+MIN_TIMED_SECONDS = 0.5
 
 
 def measured_peaks():
@@ -62,6 +76,23 @@ def scan_algorithmic_bytes(cfg) -> int:
     state = cfg.batch * c * H * P * N
     group = T * G * N + cfg.batch * c * G * (Q * (Q + 1) // 2)
     return T * H * per_token_head + state + group
+
+
+def layer_ideal_bytes(cfg) -> int:
+    """Bytes Algorithm 2 must move from the int8 tensors to y if nothing were written and read back:
+    int8 x, B, C and fp32 dt in, fp32 y and the final state out."""
+    T = cfg.tokens
+    return (T * cfg.channels + 2 * T * cfg.ngroups * cfg.dstate + T * cfg.nheads * 4 +
+            T * cfg.channels * 4 + cfg.batch * cfg.channels * cfg.dstate * 4)
+
+
+def scan_mma_ops(cfg) -> float:
+    """Integer operations (2 per multiply-accumulate) of the MMAs the scan kernel issues: per 128-row
+    tile C h over N and the masked operand times x over the columns up to the tile's last row."""
+    TM = min(cfg.chunk, 128)
+    ntpu = cfg.chunk // TM
+    per_unit = sum(2.0 * TM * cfg.headdim * (cfg.dstate + (it + 1) * TM) for it in range(ntpu))
+    return per_unit * cfg.batch * cfg.nchunks * cfg.nheads
 
 
 def step_algorithmic_bytes(cfg) -> int:
@@ -202,7 +233,7 @@ class Layer:
     def __init__(self, cfg, torch, bd):
         self.cfg, self.torch, self.bd = cfg, torch, bd
         self.dims = bd.dims_of(cfg)
-        t = inputs.make_prefill(cfg)
+        t = self.t = inputs.make_prefill(cfg)
         self.host = {k: torch.from_numpy(t[k]).pin_memory() for k in ("x", "B", "C", "dt")}
         self.f = {k: v.cuda(non_blocking=True) for k, v in self.host.items()}
         self.A = torch.from_numpy(t["A"]).cuda(); self.D = torch.from_numpy(t["D"]).cuda()
@@ -214,10 +245,12 @@ class Layer:
         self.y = torch.empty(t["x"].shape, device="cuda")
         self.fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
         self.y_host = torch.empty(t["x"].shape).pin_memory()
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")   # written by a kernel whose wait ran out
         self.ws = bd.alloc_workspace(self.dims)
         self.args = bd.make_fwd_args(xq=self.xq, Bq=self.Bq, Cq=self.Cq, s_x=self.s_x, s_B=self.s_B,
                                      s_C=self.s_C, dt=self.f["dt"], A=self.A, D=self.D, s_xs=self.s_xs,
-                                     s_cb=self.s_cb, s_h=self.s_h, y=self.y, final_state=self.fin)
+                                     s_cb=self.s_cb, s_h=self.s_h, y=self.y, final_state=self.fin,
+                                     status=self.status)
         # static calibration (untimed)
         self.quantize(mode=1)
         bd.ssdi8_calibrate(self.dims, self.args, self.s_xs, self.s_cb, self.s_h, self.ws)
@@ -247,7 +280,7 @@ class Layer:
             self.layer_args = bd.make_layer_args(
                 x=self.f["x"], B=self.f["B"], C=self.f["C"], dt=self.f["dt"], A=self.A, D=self.D,
                 s_x=self.s_x, s_B=self.s_B, s_C=self.s_C, s_xs=self.s_xs, s_cb=self.s_cb, s_h=self.s_h,
-                y=self.y, final_state=self.fin)
+                y=self.y, final_state=self.fin, status=self.status)
         self.bd.ssdi8_layer_fwd(self.dims, self.layer_args, self.layer_ws)
 
     def step_separate(self):
@@ -289,6 +322,16 @@ class Layer:
     def d2h_bytes(self):
         return self.y_host.numel() * self.y_host.element_size()
 
+    def check_status(self, where):
+        """The status word of the timed calls: non-zero means a bounded wait of a kernel ran out and
+        the launch finished with undefined results, which must never be timed as a success."""
+        self.torch.cuda.synchronize()
+        code = int(self.status.item())
+        if self.host_args is not None:
+            code = code or int(self.host_status[0])
+        if code != 0:
+            raise RuntimeError(f"{where}: device status word = {code} ({self.bd.ssdi8_status_string(code)})")
+
     def timed(self, fn, iters):
         """Average device time of fn in ms (CUDA events on the current stream); the L2 flush
         of small workloads sits outside the event pairs."""
@@ -313,9 +356,63 @@ class Layer:
             tot += e0.elapsed_time(e1)
         return tot / iters
 
+    def timed_rounds(self, fn, iters, min_seconds, where, barrier=None, reduce=None, max_rounds=4000):
+        """Rounds of `iters` calls, each bracketed by a barrier and a device synchronisation, until
+        `min_seconds` have been timed (at least 3 rounds).  Returns (median, min, max, rounds) of the
+        per-call time in ms; with several ranks every round's time is the slowest rank's, so all
+        ranks take the same decisions."""
+        per_call, total = [], 0.0
+        while (total < min_seconds * 1e3 or len(per_call) < 3) and len(per_call) < max_rounds:
+            if barrier is not None:
+                barrier()
+            ms = self.timed(fn, iters)
+            if reduce is not None:
+                ms = reduce(ms)
+            self.check_status(where)
+            per_call.append(ms)
+            total += ms * iters
+        return float(statistics.median(per_call)), float(min(per_call)), float(max(per_call)), len(per_call)
 
-def run_decode(torch, bd, steps=64, warmup=8):
-    """Recurrent-mode decode at 2.7B shapes (batch 64): tokens/s and HBM fraction of the step kernel."""
+
+def parity_check(layer, npairs=8):
+    """The output and final state the GPU holds after its last step against the CPU oracle, which
+    quantises and calibrates the whole tensors itself (nothing of the GPU run enters the oracle):
+    step sizes bit for bit, then `npairs` random (batch, head) pairs (all pairs of small workloads)
+    recomputed one by one, final state bit for bit and y within 1e-3 of the pair's RMS."""
+    from oracle import oracle as orc
+    cfg, t = layer.cfg, layer.t
+    layer.torch.cuda.synchronize()
+    q = orc.prepare_quantized(cfg, t)
+    g = lambda v: v.cpu().numpy()
+    scales_ok = all(np.array_equal(g(getattr(layer, k)), q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h"))
+    y, fin = g(layer.y), g(layer.fin)
+    total = cfg.batch * cfg.nheads
+    rng = np.random.default_rng(1000 + cfg.seed)
+    if total <= 32:
+        pairs = [(b, h) for b in range(cfg.batch) for h in range(cfg.nheads)]
+    else:
+        pairs = [(int(v) // cfg.nheads, int(v) % cfg.nheads) for v in rng.choice(total, size=npairs, replace=False)]
+    one = cfg.replace(batch=1, nheads=1, ngroups=1)
+    P, hpg = cfg.headdim, cfg.nheads // cfg.ngroups
+    worst, fin_ok = 0.0, True
+    for (b, h) in pairs:
+        gi = h // hpg
+        c_ = np.ascontiguousarray
+        y_ref, fin_ref, _ = orc.ssdi8_fwd(
+            one, c_(q["xq"][b:b + 1, :, h:h + 1]), c_(q["Bq"][b:b + 1, :, gi:gi + 1]), c_(q["Cq"][b:b + 1, :, gi:gi + 1]),
+            q["s_x"][h * P:(h + 1) * P], q["s_B"][gi:gi + 1], q["s_C"][gi:gi + 1], c_(t["dt"][b:b + 1, :, h:h + 1]),
+            t["A"][h:h + 1], t["D"][h:h + 1], None, q["s_xs"][h * P:(h + 1) * P], q["s_cb"][gi:gi + 1],
+            q["s_h"][h * P:(h + 1) * P])
+        fin_ok = fin_ok and np.array_equal(fin[b, h], fin_ref[0, 0])
+        rms = float(np.sqrt((y_ref ** 2).mean()))
+        worst = max(worst, float(np.abs(y[b, :, h] - y_ref[0, :, 0]).max()) / max(rms, 1e-30))
+    ok = bool(scales_ok and fin_ok and worst <= 1e-3)
+    return {"pairs": len(pairs), "of": total, "max_err_over_rms": worst, "final_state_bit_exact": bool(fin_ok),
+            "step_sizes_bit_exact": bool(scales_ok), "status": 0, "ok": ok}
+
+
+def run_decode(torch, bd, steps=256, warmup=8):
+    """Recurrent-mode decode at 2.7B shapes (batch 64, 256 steps): tokens/s and HBM fractions of the step kernel."""
     cfg = inputs.CONFIGS["cfg4"]
     dims = bd.dims_of(cfg)
     prm = inputs.make_decode_params(cfg)
@@ -334,22 +431,102 @@ def run_decode(torch, bd, steps=64, warmup=8):
     call = lambda: bd.ssdi8_ssd_step(dims, xq, s_x, Bq, s_B, Cq, s_C, dt, A, D, None, state, y)
     for _ in range(warmup):
         call()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(steps):
-        call()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
+    per = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        per.append(e0.elapsed_time(e1) / steps)
+    ms = float(statistics.median(per))
     nbytes = 2 * state.numel() * 4 + xq.numel() + Bq.numel() + Cq.numel() + dt.numel() * 4 + y.numel() * 4
     peaks = measured_peaks()
     gbs = nbytes / (ms * 1e-3) / 1e9
+    dram_gbs = NCU_TRAFFIC_BYTES_DECODE / (ms * 1e-3) / 1e9
     return {"workload": "cfg4: decode step, batch 64, 80 heads x 64, d_state 128 (state 168 MB > L2)",
-            "tokens_per_s": cfg.batch / (ms * 1e-3), "ms_per_step": ms, "steps": steps,
+            "tokens_per_s": cfg.batch / (ms * 1e-3), "ms_per_step": ms, "steps": steps, "rounds": len(per),
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                         "traffic": NCU_TRAFFIC_BYTES_DECODE}}
+                         "algorithmic_bytes": nbytes, "traffic": NCU_TRAFFIC_BYTES_DECODE,
+                         "dram_frac": dram_gbs / peaks["hbm_gbs"],
+                         "note": "frac counts the algorithmic bytes (state read and written once per step); "
+                                 "dram_frac the DRAM bytes of an ncu capture (part of the state written by one "
+                                 "step is still in L2 when the next step reads it)"}}
+
+
+def measure_int8_peak(torch, bd):
+    """Dense tcgen05.mma.kind::i8 throughput of this device: best single launch (about 1 ms) and a
+    back-to-back loop of about 0.3 s, CUDA events on the launching stream."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bd.ssdi8_int8_mma_peak(2048, status)
+    torch.cuda.synchronize()
+    best = 0.0
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); ops = bd.ssdi8_int8_mma_peak(16384, status); e1.record()
+        torch.cuda.synchronize()
+        best = max(best, ops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 256
+    e0.record()
+    for _ in range(n):
+        ops = bd.ssdi8_int8_mma_peak(16384, status)
+    e1.record()
+    torch.cuda.synchronize()
+    sustained = n * ops / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    if int(status.item()) != 0:
+        raise RuntimeError("int8 MMA loop: a bounded wait ran out")
+    return {"burst_tops": best, "sustained_tops": sustained,
+            "how": "ssdi8_int8_mma_peak: one CTA per SM, M 128 x N 256 x K 32 MMAs on operands resident in shared memory"}
+
+
+def measure_workload(cfg, torch, bd, steps, warmup, min_seconds, peaks, int8_peak, full, barrier=None, reduce=None,
+                     clock_index=0):
+    """Times one workload.  full = the headline workload (every leg); otherwise the short record of the
+    `workloads` list.  Returns (record, layer)."""
+    layer = Layer(cfg, torch, bd)
+    for _ in range(warmup):
+        if layer.flush is not None:
+            layer.flush.fill_(1)
+        layer.step()
+    layer.check_status("warm-up")
+    with ClockSampler(clock_index) as clk:
+        ms, ms_min, ms_max, rounds = layer.timed_rounds(layer.step, steps, min_seconds, "timed steps", barrier, reduce)
+    it = max(5, min(steps, 20))
+    rec = {"workload": cfg.name, "tokens_per_step": cfg.tokens, "ms_per_step": ms, "ms_per_step_min": ms_min,
+           "ms_per_step_max": ms_max, "rounds": rounds, "steps_per_round": steps,
+           "tokens_per_s": cfg.tokens / (ms * 1e-3), "clocks": clk.summary()}
+    if reduce is not None and not full:
+        return rec, layer
+    sec = min_seconds / 5
+    layer_only, _, _, _ = layer.timed_rounds(lambda: layer.fwd(0), it, sec, "layer only")
+    scan_ms, _, _, _ = layer.timed_rounds(lambda: layer.fwd(bd.PHASE_SCAN), it, sec, "chunk scan")
+    alg = scan_algorithmic_bytes(cfg)
+    scan_gbs = alg / (scan_ms * 1e-3) / 1e9
+    ideal = layer_ideal_bytes(cfg)
+    tops = scan_mma_ops(cfg) / (scan_ms * 1e-3) / 1e12
+    rec.update({
+        "layer_only_ms": layer_only, "layer_only_tokens_per_s": cfg.tokens / (layer_only * 1e-3),
+        "layer_only_hbm": {"ideal_bytes": ideal, "achieved_gbs": ideal / (layer_only * 1e-3) / 1e9,
+                           "frac": ideal / (layer_only * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "chunk_scan_ms": scan_ms,
+        "chunk_scan_hbm": {"algorithmic_bytes": alg, "achieved_gbs": scan_gbs, "frac": scan_gbs / peaks["hbm_gbs"]},
+        "chunk_scan_int8": {"mma_ops": scan_mma_ops(cfg), "achieved_tops": tops,
+                            "frac_of_measured": tops / int8_peak["sustained_tops"] if int8_peak else None,
+                            "frac_of_4.5POPS": tops / INT8_NOMINAL_TOPS},
+        "launch_bound": bool(8 * cfg.tokens * cfg.channels <= 126e6)})
+    return rec, layer
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher: start N ranks under torch.distributed.run."""
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def run_ours(args):
@@ -363,119 +540,169 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     cfg = inputs.CONFIGS[args.workload]
-    layer = Layer(cfg, torch, bd)
+    peaks = measured_peaks()
+    int8_peak = measure_int8_peak(torch, bd) if (rank == 0 and not args.quick) else None
 
     def barrier():
         ranks.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        if layer.flush is not None:
-            layer.flush.fill_(1)
-        layer.step()
-    barrier()
-    with ClockSampler(local) as clk:
-        ms = layer.timed(layer.step, args.steps)
-        torch.cuda.synchronize()
-    barrier()
-    ms = ranks.max_over_ranks(ms, "cuda")
+    reduce = (lambda v: ranks.max_over_ranks(v, "cuda")) if world > 1 else None
+    head, layer = measure_workload(cfg, torch, bd, args.steps, args.warmup,
+                                   0.0 if args.quick else MIN_TIMED_SECONDS, peaks, int8_peak,
+                                   full=not args.quick, barrier=barrier, reduce=reduce, clock_index=local)
+    ms = head["ms_per_step"]
     value = ranks.whole_job_tokens_per_s(cfg.tokens, world, ms)
 
     if args.quick:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
                               "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "quick": True,
-                              "config": workload_config(cfg, world), "clocks": clk.summary()}))
+                              "config": workload_config(cfg, world), "clocks": head["clocks"]}))
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
         return
 
+    # parity of what was just timed: y and the final state of the last step against the CPU oracle
+    layer.step()
+    parity = parity_check(layer) if rank == 0 else None
+
     # end to end: pinned host fp32 inputs -> device, the step, fp32 y -> pinned host
     for _ in range(2):
         layer.e2e_step()
-    barrier()
-    ms_e2e = layer.timed(layer.e2e_step, max(3, min(args.steps, 10)))
-    barrier()
-    ms_e2e = ranks.max_over_ranks(ms_e2e, "cuda")
+    ms_e2e, _, _, e2e_rounds = layer.timed_rounds(layer.e2e_step, max(3, min(args.steps, 10)), 0.3, "end to end",
+                                                  barrier, reduce)
 
     line = None
     if rank == 0:
-        peaks = measured_peaks()
+        it = max(5, min(args.steps, 20))
+        sec = MIN_TIMED_SECONDS / 5
+        t_of = lambda fn, where: layer.timed_rounds(fn, it, sec, where)[0]
         # per-module device time (CUDA events around partial runs of the same call)
         phases = {"quantize": lambda: layer.quantize(0), "cumsum": lambda: layer.fwd(bd.PHASE_CUMSUM),
                   "bmm": lambda: layer.fwd(bd.PHASE_BMM),
                   "chunk_state_passing": lambda: layer.fwd(bd.PHASE_CHUNK_STATE | bd.PHASE_STATE_PASSING),
-                  "chunk_scan": lambda: layer.fwd(bd.PHASE_SCAN)}
+                  "chunk_state_passing_int8_state":
+                      lambda: layer.fwd(bd.PHASE_CHUNK_STATE | bd.PHASE_STATE_PASSING | bd.FLAG_INT8_STATE)}
         layer.step(); torch.cuda.synchronize()
-        kernel_ms = {k: layer.timed(fn, max(5, min(args.steps, 20))) for k, fn in phases.items()}
-        dom = max((k for k in kernel_ms if k != "quantize"), key=lambda k: kernel_ms[k])
-        # Algorithm 2 alone, from the int8 tensors to y and the final state (one ssdi8_chunk_scan_fwd call)
-        layer_only_ms = layer.timed(lambda: layer.fwd(0), max(5, min(args.steps, 20)))
-        entry_ms = layer.entry_fused_ms(max(5, min(args.steps, 20)))
-        ms_separate = layer.timed(layer.step_separate, max(5, min(args.steps, 20)))
+        kernel_ms = {k: t_of(fn, k) for k, fn in phases.items()}
+        layer.fwd(bd.PHASE_CHUNK_STATE | bd.PHASE_STATE_PASSING); torch.cuda.synchronize()   # fp32-state hq back in the workspace
+        kernel_ms["chunk_scan"] = head["chunk_scan_ms"]
+        dom = max((k for k in kernel_ms if k not in ("quantize", "chunk_state_passing_int8_state")), key=lambda k: kernel_ms[k])
+        entry_ms = layer.entry_fused_ms(it)
+        ms_separate = t_of(layer.step_separate, "separate calls")
         # the scan kernel with the paper's 16-bit output format (beside the step, which keeps fp32 y)
         y16 = torch.empty(layer.y.shape, dtype=torch.bfloat16, device="cuda")
         args16 = bd.make_fwd_args(**{**layer.args._keepalive, "y": y16})
         scan16 = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args16, layer.ws, flags=bd.PHASE_SCAN | bd.FLAG_Y_BF16)
         scan16(); torch.cuda.synchronize()
-        kernel_ms["chunk_scan_bf16_y"] = layer.timed(scan16, max(5, min(args.steps, 20)))
+        kernel_ms["chunk_scan_bf16_y"] = t_of(scan16, "chunk scan, bf16 y")
         # the paper's own ChunkScan2: FP16 masked operand (kind::f16 MMA) and FP16 y
         y_h = torch.empty(layer.y.shape, dtype=torch.float16, device="cuda")
         args_h = bd.make_fwd_args(**{**layer.args._keepalive, "y": y_h})
         fl_h = bd.PHASE_SCAN | bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16
         ws_h = bd.alloc_workspace(layer.dims, flags=bd.FLAG_FP16_OPERAND)
-        layer.fwd_into = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args_h, ws_h, flags=bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16)
-        layer.fwd_into(); torch.cuda.synchronize()
+        bd.ssdi8_chunk_scan_fwd(layer.dims, args_h, ws_h, flags=bd.FLAG_FP16_OPERAND | bd.FLAG_Y_FP16)
+        torch.cuda.synchronize()
         scan_h = lambda: bd.ssdi8_chunk_scan_fwd(layer.dims, args_h, ws_h, flags=fl_h)
-        kernel_ms["chunk_scan_fp16_operand_fp16_y"] = layer.timed(scan_h, max(5, min(args.steps, 20)))
-        alg = scan_algorithmic_bytes(cfg)
-        scan_gbs = alg / (kernel_ms["chunk_scan"] * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "chunk_scan", "achieved": scan_gbs, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": scan_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "algorithmic_bytes": alg, "launch_ms": kernel_ms["chunk_scan"],
-                    "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "slowest_module": dom}
+        kernel_ms["chunk_scan_fp16_operand_fp16_y"] = t_of(scan_h, "chunk scan, FP16 operand")
+        del y16, y_h, ws_h
+        ncu = NCU_SCAN.get(cfg.name, {})
+        roofline = {"bound": "hbm", "kernel": "chunk_scan", "achieved": head["chunk_scan_hbm"]["achieved_gbs"],
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": head["chunk_scan_hbm"]["frac"],
+                    "peak_source": peaks["source"], "algorithmic_bytes": head["chunk_scan_hbm"]["algorithmic_bytes"],
+                    "launch_ms": kernel_ms["chunk_scan"], "traffic": ncu.get("traffic"),
+                    "traffic_source": ncu.get("source"), "slowest_module": dom,
+                    "limiter": "instruction issue of the CUDA cores that build the int8 masked operand and the "
+                               "fp32 output around the MMAs (neither DRAM nor the tensor pipe is saturated); "
+                               "HBM is the roof the bytes of this kernel set"}
+        roofline_tensor = dict(head["chunk_scan_int8"])
+        roofline_tensor.update({"int8_tops_measured": int8_peak, "tensor_active_pct": ncu.get("tensor_active_pct"),
+                                "tensor_active_source": ncu.get("source")})
         step_gbs = step_algorithmic_bytes(cfg) / (ms * 1e-3) / 1e9
+        layer_h2d, layer_d2h = layer.h2d_bytes(), layer.d2h_bytes()
         decode = run_decode(torch, bd) if world == 1 else None
         cpu_baseline, _ = oracle_sample(cfg, 20.0) if world == 1 else (None, 0)
+        # the other workloads, one after the other on this GPU (single-GPU runs only)
+        workloads = [{k: v for k, v in head.items()}]
+        if world == 1 and not args.no_workloads:
+            del layer
+            torch.cuda.empty_cache()
+            for name in ("cfg0", "cfg1", "cfg2", "cfg3"):
+                if name == cfg.name:
+                    continue
+                rec, lay = measure_workload(inputs.CONFIGS[name], torch, bd, args.steps, args.warmup,
+                                            MIN_TIMED_SECONDS / 2, peaks, int8_peak, full=True)
+                lay.step()
+                rec["parity"] = parity_check(lay)
+                workloads.append(rec)
+                del lay
+                torch.cuda.empty_cache()
+            workloads.sort(key=lambda r: r["workload"])
         paper = PAPER_TOKENS_PER_S.get(cfg.name)
+        config = workload_config(cfg, world)
+        config["value_is"] = ("tokens/s of the whole step: the Eq. 1 quantisers of fp32 x, B, C (one launch) plus "
+                              "Algorithm 2; layer_only_* is Algorithm 2 alone from the int8 tensors")
+        config["timing"] = (f"median of {head['rounds']} rounds of {args.steps} steps, each round bracketed by a "
+                            f"barrier and a device synchronisation, at least {MIN_TIMED_SECONDS} s timed in all")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": (value / paper) if (paper and world == 1) else None, "dtype": "s8",
-                "data": "synthetic", "config": workload_config(cfg, world),
-                "clocks": clk.summary(),
+                "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_min": head["ms_per_step_min"],
+                "ms_per_step_max": head["ms_per_step_max"], "rounds": head["rounds"],
+                "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "s8",
+                "data": "synthetic", "config": config,
+                "clocks": head["clocks"],
                 "e2e": {"value": ranks.whole_job_tokens_per_s(cfg.tokens, world, ms_e2e), "unit": UNIT,
-                        "h2d_bytes_per_step": layer.h2d_bytes(), "d2h_bytes_per_step": layer.d2h_bytes(),
-                        "ms_per_step": ms_e2e, "api": "ssdi8_layer_fwd_host (pinned host buffers; copies pipelined per batch element)"},
-                "gpu_launches": Layer.LAUNCHES_PER_STEP * args.steps,
+                        "h2d_bytes_per_step": layer_h2d, "d2h_bytes_per_step": layer_d2h,
+                        "ms_per_step": ms_e2e, "rounds": e2e_rounds,
+                        "api": "ssdi8_layer_fwd_host (pinned host buffers; copies pipelined per batch element)"},
+                "gpu_launches": Layer.LAUNCHES_PER_STEP * args.steps * head["rounds"],
+                "gpu_launches_per_step": Layer.LAUNCHES_PER_STEP,
+                "parity": parity,
                 "roofline": roofline,
+                "roofline_tensor": roofline_tensor,
+                "int8_tops_measured": int8_peak["sustained_tops"] if int8_peak else None,
                 "step_hbm": {"algorithmic_bytes": step_algorithmic_bytes(cfg), "achieved_gbs": step_gbs,
                              "frac_of_peak": step_gbs / peaks["hbm_gbs"]},
                 "kernel_ms": kernel_ms,
                 "ms_per_step_separate_calls_one_stream": ms_separate,
                 "entry_quantizer_bf16_xBC_one_launch_ms": entry_ms,
-                "layer_only_ms": layer_only_ms,
-                "layer_only_tokens_per_s": world * cfg.tokens / (layer_only_ms * 1e-3),
-                "decode": decode, "cpu_baseline": cpu_baseline}
+                "layer_only_ms": head["layer_only_ms"],
+                "layer_only_tokens_per_s": world * cfg.tokens / (head["layer_only_ms"] * 1e-3),
+                "layer_only_hbm": head["layer_only_hbm"],
+                "workloads": workloads,
+                "decode": decode, "cpu_baseline": cpu_baseline,
+                "paper_context": ({"tokens_per_s": paper, "hardware": "RTX A5000",
+                                   "source": "the paper's block-latency table: SSD module of block 55, Mamba-2 2.7B, "
+                                             "batch 8, L = 2048, 4.481 ms; another machine, context only"}
+                                  if paper else None)}
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     if line is not None:
         print(json.dumps(line))
+        bad = [w["workload"] for w in line["workloads"] if w.get("parity") and not w["parity"]["ok"]]
+        if not line["parity"]["ok"] or bad:
+            sys.stderr.write(f"parity failed: headline {line['parity']}, workloads {bad}\n")
+            sys.exit(1)
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only: skip the end-to-end, per-module, decode and CPU legs (profiling runs)")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the list of the other workloads")
     ap.add_argument("--decode-only", action="store_true",
                     help="the cfg4 decode leg alone on one GPU (profiling runs of the step kernel)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus))
     if args.decode_only:
         import torch
         from paper_2608_21952_b200 import binding as bd
