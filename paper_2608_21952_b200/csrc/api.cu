@@ -108,6 +108,12 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
 }  // extern "C"
 
 namespace ssdi8 {
+void workspace_pack_gamma(const Dims& d, void* workspace, float** pack, float** gamma) {
+  const Workspace w = layout(d);
+  *pack = reinterpret_cast<float*>(static_cast<char*>(workspace) + w.pack);
+  *gamma = reinterpret_cast<float*>(static_cast<char*>(workspace) + w.gamma);
+}
+
 ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
                           size_t workspace_bytes, void* stream, bool clear_status) {
   if (!dims || !a) return SSDI8_ERR_NULL;

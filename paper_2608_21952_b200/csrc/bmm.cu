@@ -22,7 +22,7 @@ struct BmmArgs {
   int store;  // 0: calibration pass (no CBq written)
 };
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 512;   // 16 warps: warp w reads TMEM lane quarter w % 4 (rows) and every fourth 32-column piece from w / 4
 constexpr uint32_t OFF_A = 0;        // [128][N]  Cq rows of the tile
 constexpr uint32_t OFF_B = 16384;    // [256][N]  Bq rows 0 .. KJ-1
 constexpr uint32_t OFF_O = 49152;    // 2 x [128][128] int8 staging panels
@@ -54,11 +54,13 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
     fence_mbar_init();
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_B); tma_prefetch_desc(&tm_o);
   }
+  pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, 256);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();
 
   if (tid == 0) {
     mbar_expect_tx(&bars[0], (uint32_t)(TM * N + KJ * N));
@@ -76,18 +78,20 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
   mbar_wait(&bars[1], 0, a.status);
   tc_fence_after();
 
-  // ---- epilogue: thread = row i of the tile, 32 columns at a time
+  // ---- epilogue: thread = row i of the tile, 32 columns at a time; the four warps that share a
+  // lane quarter take alternate 32-column pieces
   const float r_cb = a.s_cb ? __fdiv_rn(__fmul_rn(a.s_C[g], a.s_B[g]), a.s_cb[g]) : 0.f;
-  const int r = warp * 32 + lane;
+  const int wq = warp & 3, wc = warp >> 2;
+  const int r = wq * 32 + lane;
   const int i = it * TM + r;
   const bool ok = r < TM;
   const uint32_t RBO = (uint32_t)TM;  // row bytes of a staging panel (128, or 64 when Q = 64)
   int amax = 0;
   const i64 obase = (((i64)bk * d.G + g) * Q + i) * Q;
 #pragma unroll 1
-  for (int j0 = 0; j0 < KJ; j0 += 32) {
+  for (int j0 = wc * 32; j0 < KJ; j0 += 32 * (kThreads / 128)) {
     int acc[32];
-    tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, acc);
+    tmem_ld32(tmem + ((uint32_t)(wq * 32) << 16) + (uint32_t)j0, acc);
     tmem_ld_wait();
     if (ok) {
       uint32_t o[8];
@@ -165,7 +169,7 @@ ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, con
   const size_t smem = SMEM_BYTES + 1024;
   SSDI8_CUDA_CHECK(cudaFuncSetAttribute(bmm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const unsigned grid = (unsigned)((i64)d.b * d.c * d.G * (d.Q / TM));
-  bmm_tc<<<grid, kThreads, smem, st>>>(tm_C, tm_B, tm_o, a);
+  if (launch_pdl(bmm_tc, dim3(grid), dim3(kThreads), smem, st, tm_C, tm_B, tm_o, a) != cudaSuccess) return SSDI8_ERR_CUDA;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

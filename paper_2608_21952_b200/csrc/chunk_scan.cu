@@ -362,11 +362,13 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     tma_prefetch_desc(&tm_cb); tma_prefetch_desc(&tm_y);
     *first_tile = decode_tile(t_begin, a, TM, ntpu);
   }
+  pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();   // every role below reads or writes global memory
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer: CBq panels + scalar pack
@@ -694,8 +696,7 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   const bool tp = taps.acc_off || taps.rowmax || taps.Mq || taps.acc_diag;
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
-    return SSDI8_OK;
+    return launch_pdl(kernel, dim3(grid), dim3(kThreads), smem, st, tm_C, tm_h, tm_x, tm_cb, tm_y, a) == cudaSuccess ? SSDI8_OK : SSDI8_ERR_CUDA;
   };
   if (tp && ydt) return SSDI8_ERR_UNSUPPORTED;  // the taps come with binary32 y only
   const bool big = d.Q >= 128;

@@ -307,11 +307,13 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_cb); tma_prefetch_desc(&tm_y);
   }
+  pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();   // every role below reads or writes global memory
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer: CBq panels, scalar pack, and the
@@ -624,8 +626,7 @@ ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, const int8
   const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<grid, kThreads, smem, st>>>(tm_C, tm_h, tm_x, tm_cb, tm_y, a);
-    return SSDI8_OK;
+    return launch_pdl(kernel, dim3(grid), dim3(kThreads), smem, st, tm_C, tm_h, tm_x, tm_cb, tm_y, a) == cudaSuccess ? SSDI8_OK : SSDI8_ERR_CUDA;
   };
   const bool big = d.Q >= 128;
   auto pick = [&](auto corr_c, auto big_c) -> ssdi8_status_t {

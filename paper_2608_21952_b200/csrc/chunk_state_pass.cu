@@ -85,7 +85,9 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
     tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_hq);
   }
+  pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, 64);
+  pdl_wait();   // everything below reads global memory
   if (tid < 64) {
     const float sxb = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]), sh = a.s_h[h * P + tid];
     col_scale[tid] = I8S ? __fdiv_rn(sxb, sh) : sxb;
@@ -436,8 +438,7 @@ ssdi8_status_t launch_chunk_state_passing(const Dims& d, const int8_t* xq, const
   const bool taps = tap_loc || tap_prev || tap_Xsq || tap_acc;
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<grid, kThreads, smem, st>>>(tm_B, tm_x, tm_hq, a);
-    return SSDI8_OK;
+    return launch_pdl(kernel, dim3(grid), dim3(kThreads), smem, st, tm_B, tm_x, tm_hq, a) == cudaSuccess ? SSDI8_OK : SSDI8_ERR_CUDA;
   };
   ssdi8_status_t ls;
   if (int8_state)

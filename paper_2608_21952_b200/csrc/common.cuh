@@ -110,6 +110,14 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
 
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xff); }
 
+// Programmatic dependent launch.  Every kernel of the layer lets its successor in the stream be
+// scheduled early (launch_dependents at its start) and itself waits for its predecessor's completion
+// and memory flush (pdl_wait) before its first access to global memory, so only work that touches no
+// global memory (barrier and tensor-memory set-up, descriptor prefetch) runs under the predecessor's
+// tail.  Both are no-ops in a kernel that was launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct Dims {
   int b, L, H, P, N, G, Q, c;
 };

@@ -140,21 +140,34 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
       ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C) |
         reinterpret_cast<uintptr_t>(a.s_x) | reinterpret_cast<uintptr_t>(xq) | reinterpret_cast<uintptr_t>(Bq) |
         reinterpret_cast<uintptr_t>(Cq)) & 15) == 0;
-  SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
-  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side2, p.fork, 0));
-  // ChunkCumsum reads dt and A only: it runs on a side stream under the quantisers
-  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, p.s_side2, false)) != SSDI8_OK) return s;
-  SSDI8_CUDA_CHECK(cudaEventRecord(p.join2, p.s_side2));
-  // caller's stream: the three Eq. 1 quantisers
-  if (one_launch) {
+  // Small workloads (every kernel is a few microseconds: the step is bound by launches and stream joins)
+  // take ChunkCumsum, which reads dt and A only, into the quantisers' launch.  Large ones run it on a side
+  // stream under the quantisers instead: inside one grid its long-lived blocks cost the bandwidth-bound
+  // quantiser of x more slots than the launch saves (measured at batch 8 x 2048 x 80 heads: 0.327 ms per
+  // step merged against 0.315 ms on the side stream; at 2048 x 24 heads: 0.059 against 0.070 ms).
+  const bool merged = one_launch && (int64_t)T * d.nheads * d.headdim <= ((int64_t)1 << 23);
+  if (merged) {
+    const Dims dd = make_dims(&d);
+    float *pack = nullptr, *gamma = nullptr;
+    workspace_pack_gamma(dd, ws, &pack, &gamma);
     if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
-                                 Cq, st)) != SSDI8_OK)
+                                 Cq, &dd, dt, a.A, pack, gamma, st)) != SSDI8_OK)
       return s;
   } else {
-    if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, st)) != SSDI8_OK) return s;
-    if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, st)) != SSDI8_OK) return s;
-    if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
-      return s;
+    SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
+    SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side2, p.fork, 0));
+    if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, p.s_side2, false)) != SSDI8_OK) return s;
+    SSDI8_CUDA_CHECK(cudaEventRecord(p.join2, p.s_side2));
+    if (one_launch) {
+      if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
+                                   Cq, nullptr, nullptr, nullptr, nullptr, nullptr, st)) != SSDI8_OK)
+        return s;
+    } else {
+      if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, st)) != SSDI8_OK) return s;
+      if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, st)) != SSDI8_OK) return s;
+      if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
+        return s;
+    }
   }
   // ChunkBMM needs Bq and Cq and is needed by ChunkScan only: it runs on a side stream under the
   // state kernel
@@ -162,7 +175,7 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork2, 0));
   if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM, ws, ws_bytes, p.s_side, false)) != SSDI8_OK) return s;
   SSDI8_CUDA_CHECK(cudaEventRecord(p.join, p.s_side));
-  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join2, 0));
+  if (!merged) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join2, 0));
   if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING, ws, ws_bytes, st, false)) != SSDI8_OK)
     return s;
   SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join, 0));

@@ -2,16 +2,38 @@
 #pragma once
 #include "common.cuh"
 
+#include <utility>
+
 namespace ssdi8 {
+
+// kernel<<<grid, block, smem, st>>>(args...) with programmatic stream serialization allowed: the
+// kernel may be scheduled while its predecessor in the stream drains (see pdl_wait in common.cuh)
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* scale, int mode,
                                int8_t* out, cudaStream_t st);
 
 // the layer's three static quantisers as one launch: x [T][D] with D step sizes, B and C [T][G N] with G
-// step sizes each (N a power of two, D and N multiples of 4)
+// step sizes each (N a power of two, D and N multiples of 4).  With cs_dims non-NULL the blocks of
+// ChunkCumsum for those dimensions (dt, A -> pack, gamma; see launch_cumsum) lead the same grid.
 ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* C, i64 T_, int D, int G, int N,
                                    const float* s_x, const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq,
-                                   int8_t* Cq, cudaStream_t st);
+                                   int8_t* Cq, const Dims* cs_dims, const float* dt, const float* A, float* pack,
+                                   float* gamma, cudaStream_t st);
 
 // Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, wmax, lut (see
 // cumsum.cu); element (u, row, i) at pack[(u * kPackRows + row) * Q + i], u = (b*H + h)*c + k.
@@ -27,6 +49,9 @@ ssdi8_status_t launch_quantize_entry(const void* xBC, int dtype, i64 T_, int D, 
 // the modules as several calls clear it once themselves)
 ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
                           size_t workspace_bytes, void* stream, bool clear_status);
+
+// where ChunkCumsum's outputs live inside a workspace of ssdi8_workspace_bytes
+void workspace_pack_gamma(const Dims& d, void* workspace, float** pack, float** gamma);
 
 // pack [b,H,c,6,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
