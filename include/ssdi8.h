@@ -83,6 +83,18 @@ enum { SSDI8_FLAG_FP16_OPERAND = 1u << 0 };
 /* state format bit of ssdi8_chunk_scan_fwd's flags */
 enum { SSDI8_FLAG_INT8_STATE = 1u << 1 };
 
+/* time-step bit of ssdi8_chunk_scan_fwd's flags: `dt` holds the raw time step and ChunkCumsum starts, as
+ * Algorithm 2 module 1 does, from dt = softplus(dt_raw + dt_bias[h]) (dt_bias = NULL: no bias).  The
+ * value is formed in binary64, each step one correctly rounded operation, and rounded to binary32 once:
+ *   v = (double) fadd(dt_raw, dt_bias);  a = |v|
+ *   u = exp(-a): n = rint(-a LOG2E), r = fma(n, -LN2_HI, -a), r = fma(n, -LN2_LO, r) with
+ *       LOG2E = 0x1.71547652b82fep+0, LN2_HI = 0x1.62e42fee00000p-1, LN2_LO = 0x1.a39ef35793c76p-33,
+ *       degree-13 Taylor polynomial in r by Horner with fma, times 2^n through the exponent field; 0 if a > 700
+ *   s = u / (2 + u), z = s s, q = 1 + z/3 + ... + z^13/27 by Horner with fma, lp = (2 s) q   (= log(1 + u))
+ *   dt = (float)(max(v, 0) + lp)
+ * which equals the correctly rounded softplus in all but about one value in ten million. */
+enum { SSDI8_FLAG_DT_SOFTPLUS = 1u << 4 };
+
 /* output format bits (at most one): y is written as 16-bit elements, the paper's own output
  * format being FP16 (Algorithm 2 keeps Y in half precision); default is binary32 */
 enum { SSDI8_FLAG_Y_FP16 = 1u << 2, SSDI8_FLAG_Y_BF16 = 1u << 3 };
@@ -127,7 +139,7 @@ typedef struct {
   const float* s_x;        /* [H*P] step sizes of xq                                    */
   const float* s_B;        /* [G]                                                       */
   const float* s_C;        /* [G]                                                       */
-  const float* dt;         /* [B,L,H] time step, already positive (after softplus)      */
+  const float* dt;         /* [B,L,H] time step, already positive (after softplus), or raw with SSDI8_FLAG_DT_SOFTPLUS */
   const float* A;          /* [H] decay rate, negative                                  */
   const float* D;          /* [H] skip weight, or NULL                                  */
   const float* corr;       /* [H*P] per-channel mean correction (Eq. 8), or NULL        */
@@ -153,10 +165,13 @@ typedef struct {
   float* tap_rowmax;       /* [B,L,H]     absmax of each row of the masked operand      */
   int8_t* tap_Mq;          /* [B,c,H,Q,Q] int8 masked operand, zero above the diagonal  */
   int32_t* tap_acc_diag;   /* [B,L,H,P]   INT32 Mq x                                    */
+  /* with SSDI8_FLAG_DT_SOFTPLUS: bias added to the raw time step before the softplus, or NULL */
+  const float* dt_bias;    /* [H]                                                        */
 } ssdi8_fwd_args_t;
 
 /* SSD layer forward (Algorithm 2) from int8 x, B, C to fp32 y and final state.
- *  ChunkCumsum   cs[k,i] = (float) sum_{i'<=i} (double)dt * (double)A, in token order;
+ *  ChunkCumsum   (with SSDI8_FLAG_DT_SOFTPLUS first dt = softplus(dt + dt_bias), see the flag)
+ *                cs[k,i] = (float) sum_{i'<=i} (double)dt * (double)A, in token order;
  *                Gamma_k = exp32(cs[k,Q-1])                         (Decay_pass, Eq. 5)
  *  ChunkBMM      acc_cb[i,j] = sum_n Cq[i,n] Bq[j,n]  per (b, chunk, group), INT32;
  *                CBq = rne(fmul(float(acc_cb), fdiv(fmul(s_C, s_B), s_cb)))
@@ -310,6 +325,13 @@ ssdi8_status_t ssdi8_ssd_step(const ssdi8_dims_t* dims, const int8_t* xq, const 
                               const int8_t* Bq, const float* s_B, const int8_t* Cq,
                               const float* s_C, const float* dt, const float* A, const float* D,
                               const float* corr, float* state, float* y, void* stream);
+
+/* dt = softplus(dt_raw + dt_bias[h]) alone (Algorithm 2 module 1, first line), the arithmetic of
+ * SSDI8_FLAG_DT_SOFTPLUS: for callers that calibrate step sizes (ssdi8_calibrate takes the positive time
+ * step) or run the recurrent step on raw time steps.  dt_raw, dt [rows][H]; dt_bias [H] or NULL; dt may
+ * alias dt_raw. */
+ssdi8_status_t ssdi8_softplus_dt(const float* dt_raw, const float* dt_bias, int64_t rows, int32_t H, float* dt,
+                                 void* stream);
 
 /* Measurement aid (the paper has no counterpart): what tcgen05.mma.kind::i8 sustains on the current
  * device, for the "fraction of the int8 tensor-pipe peak" a benchmark reports.  One CTA per SM issues

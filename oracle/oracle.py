@@ -317,3 +317,14 @@ def chunk_scan_fp16_operand(cfg, xq, Cq, CBq, hq, s_x, s_C, s_cb, s_h, dt, cs, D
                         _p(_f32(D)), _p(_f32(corr)), None, None, None, None, _p(y),
                         C.c_uint32(FLAG_FP16_OPERAND), _p(m16))
     return y, m16
+
+
+def softplus_dt(dt_raw, bias=None, plain=False):
+    """dt = softplus(dt_raw + bias[h]) (Algorithm 2 module 1), dt_raw [..., H] -> float32.  plain=True:
+    the libm definition in fp64; otherwise the library's operation-by-operation binary64 sequence."""
+    x = _f32(dt_raw)
+    H = x.shape[-1]
+    out = np.empty_like(x)
+    fn = _lib.orc_softplus_dt_plain if plain else _lib.orc_softplus_dt
+    fn(_p(x), _p(_f32(bias)), C.c_int64(x.size // H), C.c_int64(H), _p(out))
+    return out

@@ -280,6 +280,60 @@ void orc_ssd_chunked(const Dims* d, const double* x, const double* B, const doub
 }
 
 // ---------------------------------------------------------------------------
+// Algorithm 2 module 1, first line: dt = softplus(dt_raw + dt_bias).
+// Plain definition: log(1 + exp(v)) with libm in binary64, rounded to binary32 once; v = dt_raw + bias is
+// the sum of two binary32 tensors as a binary32 tensor (the reading taken: the bias is added in the
+// tensors' own precision, as a framework would, before the softplus is evaluated).
+void orc_softplus_dt_plain(const float* dt_raw, const float* bias, i64 rows, i64 H, float* out) {
+  for (i64 r = 0; r < rows; ++r)
+    for (i64 h = 0; h < H; ++h) {
+      const float v32 = bias ? dt_raw[r * H + h] + bias[h] : dt_raw[r * H + h];
+      const double v = (double)v32;
+      out[r * H + h] = (float)(std::fmax(v, 0.0) + std::log1p(std::exp(-std::fabs(v))));
+    }
+}
+
+// The library's operation-by-operation softplus (binary64, every operation a single correctly rounded
+// add, multiply, divide or fused multiply-add), so that dt is defined bit for bit:
+//   v  = (double) fadd(dt_raw, bias)            (binary32 sum, then widened)
+//   a  = |v|;  u = exp(-a):  n = rint(-a LOG2E), r = fma(n, -LN2_HI, -a), r = fma(n, -LN2_LO, r),
+//        degree-13 Taylor polynomial in r (Horner, fma), scaled by 2^n; u = 0 for a > 700
+//   lp = log(1 + u) = 2 atanh(s), s = u / (2 + u): 2 s (1 + z/3 + z^2/5 + ... + z^13/27), z = s s (Horner, fma)
+//   dt = (float)(max(v, 0) + lp)
+inline double softplus64(double v) {
+  const double a = std::fabs(v);
+  double u = 0.0;
+  if (a <= 700.0) {
+    const double LOG2E = 0x1.71547652b82fep+0, LN2_HI = 0x1.62e42fee00000p-1, LN2_LO = 0x1.a39ef35793c76p-33;
+    const double n = std::nearbyint(-a * LOG2E);
+    double r = std::fma(n, -LN2_HI, -a);
+    r = std::fma(n, -LN2_LO, r);
+    double p = 1.0 / 6227020800.0;                    // 1/13!
+    const double inv_fact[13] = {1.0 / 479001600.0, 1.0 / 39916800.0, 1.0 / 3628800.0, 1.0 / 362880.0,
+                                 1.0 / 40320.0, 1.0 / 5040.0, 1.0 / 720.0, 1.0 / 120.0, 1.0 / 24.0,
+                                 1.0 / 6.0, 0.5, 1.0, 1.0};
+    for (int k = 0; k < 13; ++k) p = std::fma(p, r, inv_fact[k]);
+    uint64_t bits;
+    std::memcpy(&bits, &p, 8);
+    bits += (uint64_t)((int64_t)n) << 52;             // p 2^n: n >= -1010, p in [0.7, 1.42], so the result is normal
+    std::memcpy(&u, &bits, 8);
+  }
+  const double s = u / (2.0 + u), z = s * s;
+  double q = 1.0 / 27.0;
+  for (int k = 12; k >= 0; --k) q = std::fma(q, z, 1.0 / (double)(2 * k + 1));
+  const double lp = 2.0 * s * q;
+  return (v > 0.0 ? v : 0.0) + lp;
+}
+
+void orc_softplus_dt(const float* dt_raw, const float* bias, i64 rows, i64 H, float* out) {
+  for (i64 r = 0; r < rows; ++r)
+    for (i64 h = 0; h < H; ++h) {
+      const float v32 = bias ? dt_raw[r * H + h] + bias[h] : dt_raw[r * H + h];
+      out[r * H + h] = (float)softplus64((double)v32);
+    }
+}
+
+// ---------------------------------------------------------------------------
 // L2 stage: ChunkCumsum (Algorithm 2, module 1).  dt is already positive
 // (post-softplus).  The running sum is carried in fp64 in token order (each
 // product dt*A of two binary32 numbers is exact in fp64) and stored as

@@ -28,6 +28,7 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TI
 FLAG_FP16_OPERAND = 1 << 0
 FLAG_INT8_STATE = 1 << 1
 FLAG_Y_FP16, FLAG_Y_BF16 = 1 << 2, 1 << 3
+FLAG_DT_SOFTPLUS = 1 << 4
 PHASE_CUMSUM, PHASE_BMM, PHASE_CHUNK_STATE, PHASE_STATE_PASSING, PHASE_SCAN = (1 << k for k in range(8, 13))
 
 EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
@@ -36,7 +37,7 @@ EXPORTS = ("ssdi8_status_string", "ssdi8_workspace_bytes", "ssdi8_quantize_act",
            "ssdi8_mean_correction_workspace_bytes", "ssdi8_quantize_entry",
            "ssdi8_layer_fwd", "ssdi8_layer_fwd_workspace_bytes",
            "ssdi8_layer_fwd_host", "ssdi8_layer_fwd_host_scratch_bytes",
-           "ssdi8_int8_mma_peak", "ssdi8_selftest_bounded_wait")
+           "ssdi8_int8_mma_peak", "ssdi8_selftest_bounded_wait", "ssdi8_softplus_dt")
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 
@@ -48,7 +49,7 @@ class Dims(C.Structure):
 _FWD_FIELDS = ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "corr", "s_xs", "s_cb", "s_h",
                "init_state", "y", "final_state", "status",
                "tap_cs", "tap_acc_cb", "tap_CBq", "tap_Xsq", "tap_acc_st", "tap_loc", "tap_prev",
-               "tap_hq", "tap_acc_off", "tap_rowmax", "tap_Mq", "tap_acc_diag")
+               "tap_hq", "tap_acc_off", "tap_rowmax", "tap_Mq", "tap_acc_diag", "dt_bias")
 
 
 class FwdArgs(C.Structure):
@@ -255,6 +256,15 @@ _lib.ssdi8_int8_mma_peak.restype = C.c_int32
 _lib.ssdi8_int8_mma_peak.argtypes = [C.c_int64, C.POINTER(C.c_double), C.c_void_p, C.c_void_p]
 _lib.ssdi8_selftest_bounded_wait.restype = C.c_int32
 _lib.ssdi8_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_void_p]
+
+
+_lib.ssdi8_softplus_dt.restype = C.c_int32
+_lib.ssdi8_softplus_dt.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
+
+
+def ssdi8_softplus_dt(dt_raw, dt_bias, rows: int, H: int, dt, stream=None) -> None:
+    _check(_lib.ssdi8_softplus_dt(_ptr(dt_raw), _ptr(dt_bias), rows, H, _ptr(dt), _stream(stream)),
+           "ssdi8_softplus_dt")
 
 
 def ssdi8_int8_mma_peak(mma_per_sm: int, status=None, stream=None) -> float:

@@ -8,6 +8,9 @@ using namespace ssdi8;
 
 namespace {
 
+constexpr uint32_t kFwdFlags = SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 |
+                               SSDI8_FLAG_Y_BF16 | SSDI8_FLAG_DT_SOFTPLUS;
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -81,7 +84,7 @@ const char* ssdi8_status_string(ssdi8_status_t s) {
 }
 
 size_t ssdi8_workspace_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0 || !dims_supported(dims, true)) return 0;
+  if ((flags & ~kFwdFlags) != 0 || !dims_supported(dims, true)) return 0;
   return layout(make_dims(dims), (flags & SSDI8_FLAG_FP16_OPERAND) != 0).total;
 }
 
@@ -117,7 +120,7 @@ void workspace_pack_gamma(const Dims& d, void* workspace, float** pack, float** 
 ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, uint32_t flags, void* workspace,
                           size_t workspace_bytes, void* stream, bool clear_status) {
   if (!dims || !a) return SSDI8_ERR_NULL;
-  if ((flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) != 0) return SSDI8_ERR_UNSUPPORTED;
+  if ((flags & ~kFwdFlags) != 0) return SSDI8_ERR_UNSUPPORTED;
   const bool i8s = (flags & SSDI8_FLAG_INT8_STATE) != 0;
   if ((flags & SSDI8_FLAG_Y_FP16) && (flags & SSDI8_FLAG_Y_BF16)) return SSDI8_ERR_UNSUPPORTED;
   const int ydt = (flags & SSDI8_FLAG_Y_FP16) ? 1 : (flags & SSDI8_FLAG_Y_BF16) ? 2 : 0;
@@ -154,7 +157,8 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
   int8_t* hq = a->tap_hq ? a->tap_hq : reinterpret_cast<int8_t*>(ws + w.hq);
   if (a->status && clear_status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
 
-  if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st)) != SSDI8_OK)
+  if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st, a->dt_bias,
+                                                     (flags & SSDI8_FLAG_DT_SOFTPLUS) != 0)) != SSDI8_OK)
     return s;
   if ((ph & SSDI8_PHASE_BMM) &&
       (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, a->status, st)) !=
@@ -296,6 +300,15 @@ ssdi8_status_t ssdi8_mean_correction(const float* y_ref, const float* y_q, int64
                                 static_cast<cudaStream_t>(stream));
 }
 
+ssdi8_status_t ssdi8_softplus_dt(const float* dt_raw, const float* dt_bias, int64_t rows, int32_t H, float* dt,
+                                 void* stream) {
+  if (!dt_raw || !dt) return SSDI8_ERR_NULL;
+  if (rows < 0 || H <= 0) return SSDI8_ERR_SHAPE;
+  ssdi8_status_t s = check_arch();
+  if (s != SSDI8_OK) return s;
+  return launch_softplus_dt(dt_raw, dt_bias, dt, rows, H, static_cast<cudaStream_t>(stream));
+}
+
 ssdi8_status_t ssdi8_int8_mma_peak(int64_t mma_per_sm, double* ops, int32_t* status, void* stream) {
   if (!ops) return SSDI8_ERR_NULL;
   const int per_batch = int8_mma_peak_batch();
@@ -335,7 +348,7 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
   if (!dims || !args) return SSDI8_ERR_NULL;
   const size_t need = ssdi8_workspace_bytes(dims, flags);
   if (need == 0)
-    return (flags & ~(uint32_t)(SSDI8_PHASE_ALL | SSDI8_FLAG_FP16_OPERAND | SSDI8_FLAG_INT8_STATE | SSDI8_FLAG_Y_FP16 | SSDI8_FLAG_Y_BF16)) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
+    return (flags & ~kFwdFlags) ? SSDI8_ERR_UNSUPPORTED : SSDI8_ERR_SHAPE;
   if (need > (size_t)SSDI8_STATIC_WORKSPACE_BYTES) return SSDI8_ERR_WORKSPACE;  // beyond the built-in scratch
   // (before the symbol lookup: on a device of another architecture the lookup itself fails, and the
   // caller should learn that the device is the wrong one)

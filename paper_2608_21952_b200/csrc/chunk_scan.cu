@@ -577,9 +577,10 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
               const float2 xv = unpack2(xw[cc], e2 * 2);
               const float2 ao = make_float2((float)acc_o[pp], (float)acc_o[pp + 1]);
               const float2 ad = make_float2((float)acc_d[pp], (float)acc_d[pp + 1]);
-              float2 r2 = __ffma2_rn(__fmul2_rn(Dh2, sx2), xv, co2);
-              r2 = __ffma2_rn(__fmul2_rn(sm2, sx2), ad, r2);
-              v[cc * 2 + e2] = __ffma2_rn(__fmul2_rn(dec2, sh2), ao, r2);
+              // y = s_x (s_M acc_diag + D x) + s_h (dec acc_off) + corr: five packed operations
+              const float2 u2 = __ffma2_rn(sm2, ad, __fmul2_rn(Dh2, xv));
+              const float2 r2 = __ffma2_rn(sx2, u2, co2);
+              v[cc * 2 + e2] = __ffma2_rn(sh2, __fmul2_rn(dec2, ao), r2);
             }
             if (YT == 0)   // 4 values = one 16-byte chunk
               *reinterpret_cast<float4*>(srow + ((((pc & 3) * 2 + cc) ^ (lane & 7)) << 4)) =

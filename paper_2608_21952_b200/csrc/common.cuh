@@ -110,6 +110,44 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
 
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xff); }
 
+// softplus of the raw time step (Algorithm 2 module 1) in binary64, every operation a single correctly
+// rounded add, multiply, divide or fused multiply-add in the order written in ssdi8.h, so that the
+// binary32 result is defined bit for bit: v = (double)fadd(dt_raw, bias); u = exp(-|v|) by Cody-Waite
+// reduction and a degree-13 Taylor polynomial; log(1 + u) = 2 atanh(u / (2 + u)) by its odd series up
+// to the 27th power; dt = (float)(max(v, 0) + log(1 + u)).
+__device__ __forceinline__ float softplus_dt(float dt_raw, float bias) {
+  const double v = (double)__fadd_rn(dt_raw, bias);
+  const double a = fabs(v);
+  double u = 0.0;
+  if (a <= 700.0) {
+    const double LOG2E = 0x1.71547652b82fep+0, LN2_HI = 0x1.62e42fee00000p-1, LN2_LO = 0x1.a39ef35793c76p-33;
+    const double n = rint(__dmul_rn(-a, LOG2E));
+    double r = __fma_rn(n, -LN2_HI, -a);
+    r = __fma_rn(n, -LN2_LO, r);
+    double p = 1.0 / 6227020800.0;
+    p = __fma_rn(p, r, 1.0 / 479001600.0);
+    p = __fma_rn(p, r, 1.0 / 39916800.0);
+    p = __fma_rn(p, r, 1.0 / 3628800.0);
+    p = __fma_rn(p, r, 1.0 / 362880.0);
+    p = __fma_rn(p, r, 1.0 / 40320.0);
+    p = __fma_rn(p, r, 1.0 / 5040.0);
+    p = __fma_rn(p, r, 1.0 / 720.0);
+    p = __fma_rn(p, r, 1.0 / 120.0);
+    p = __fma_rn(p, r, 1.0 / 24.0);
+    p = __fma_rn(p, r, 1.0 / 6.0);
+    p = __fma_rn(p, r, 0.5);
+    p = __fma_rn(p, r, 1.0);
+    p = __fma_rn(p, r, 1.0);
+    u = __longlong_as_double(__double_as_longlong(p) + ((long long)__double2int_rn(n) << 52));
+  }
+  const double s = __ddiv_rn(u, __dadd_rn(2.0, u)), z = __dmul_rn(s, s);
+  double q = 1.0 / 27.0;
+#pragma unroll
+  for (int k = 12; k >= 0; --k) q = __fma_rn(q, z, 1.0 / (double)(2 * k + 1));
+  const double lp = __dmul_rn(__dmul_rn(2.0, s), q);
+  return (float)__dadd_rn(v > 0.0 ? v : 0.0, lp);
+}
+
 // Programmatic dependent launch.  Every kernel of the layer lets its successor in the stream be
 // scheduled early (launch_dependents at its start) and itself waits for its predecessor's completion
 // and memory flush (pdl_wait) before its first access to global memory, so only work that touches no

@@ -15,21 +15,42 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
                                                      const float* __restrict__ A,
                                                      float* __restrict__ pack,
                                                      float* __restrict__ gamma,
-                                                     float* __restrict__ tap_cs, Dims d) {
+                                                     float* __restrict__ tap_cs, Dims d,
+                                                     const float* __restrict__ dt_bias, int softplus) {
   extern __shared__ float tile[];
   pdl_launch_dependents();
   pdl_wait();
-  cumsum_body<kChunksPerBlock>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile);
+  cumsum_body<kChunksPerBlock>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias, softplus);
+}
+
+// dt = softplus(dt_raw + dt_bias[h]) alone (for callers that calibrate on the positive time step)
+__global__ void softplus_dt_kernel(const float* __restrict__ dt_raw, const float* __restrict__ dt_bias,
+                                   float* __restrict__ out, i64 n, int H) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e < n) out[e] = softplus_dt(dt_raw[e], dt_bias ? __ldg(dt_bias + (int)(e % H)) : 0.f);
 }
 
 }  // namespace
 
+ssdi8_status_t launch_softplus_dt(const float* dt_raw, const float* dt_bias, float* out, i64 rows, int H,
+                                  cudaStream_t st) {
+  const i64 n = rows * H;
+  if (n == 0) return SSDI8_OK;
+  if (launch_pdl(softplus_dt_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, dt_raw, dt_bias, out, n, H) !=
+      cudaSuccess)
+    return SSDI8_ERR_CUDA;
+  SSDI8_LAUNCH_CHECK();
+  return SSDI8_OK;
+}
+
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
-                             float* gamma, float* tap_cs, cudaStream_t st) {
+                             float* gamma, float* tap_cs, cudaStream_t st, const float* dt_bias, bool softplus) {
   dim3 grid((d.H + kCumsumHeads - 1) / kCumsumHeads, (d.c + kChunksPerBlock - 1) / kChunksPerBlock, d.b);
   const size_t smem = cumsum_smem_bytes(d.Q, kChunksPerBlock);
   SSDI8_CUDA_CHECK(cudaFuncSetAttribute(cumsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  if (launch_pdl(cumsum_kernel, grid, dim3(256), smem, st, dt, A, pack, gamma, tap_cs, d) != cudaSuccess)
+  if (launch_pdl(cumsum_kernel, grid, dim3(256), smem, st, dt, A, pack, gamma, tap_cs, d, dt_bias, softplus ? 1 : 0) != cudaSuccess)
     return SSDI8_ERR_CUDA;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;

@@ -30,11 +30,14 @@ __host__ __device__ inline size_t cumsum_smem_bytes(int Q, int KC) {
 
 // One block's work: heads 8 bx .. and chunks KC kx .. of batch element b.  Any whole number of warps
 // may run it (every loop strides by the block size); `tile` is cumsum_smem_bytes(Q, KC) of shared memory.
+// softplus != 0: dt holds the raw time step and dt = softplus(dt + dt_bias[h]) (dt_bias may be NULL)
+// is applied as the values are staged (Algorithm 2 module 1 starts there).
 template <int KC>
 __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const float* __restrict__ A,
                                             float* __restrict__ pack, float* __restrict__ gamma,
                                             float* __restrict__ tap_cs, const Dims& d, int bx, int kx, int b,
-                                            float* tile) {
+                                            float* tile, const float* __restrict__ dt_bias = nullptr,
+                                            int softplus = 0) {
   constexpr int CH = kCumsumHeads, NU = CH * KC;   // unit u = hh * KC + kk
   const int Q = d.Q, ld = Q + 1;
   const int lq = 31 - __clz(Q);  // Q is a power of two
@@ -58,7 +61,9 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + u * blockDim.x;
       const int t = e / CH, hh = e % CH;
-      if (e < ntok * CH && hh < nh) dts[(hh * KC + (t >> lq)) * ld + (t & (Q - 1))] = v[u];
+      if (e < ntok * CH && hh < nh)
+        dts[(hh * KC + (t >> lq)) * ld + (t & (Q - 1))] =
+            softplus ? softplus_dt(v[u], dt_bias ? __ldg(dt_bias + h0 + hh) : 0.f) : v[u];
     }
   }
   __syncthreads();

@@ -54,8 +54,12 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
 void workspace_pack_gamma(const Dims& d, void* workspace, float** pack, float** gamma);
 
 // pack [b,H,c,6,Q], gamma [b,H,c], tap_cs [b,H,c,Q] or NULL
+// softplus: dt is the raw time step, dt = softplus(dt + dt_bias[h]) is applied first (dt_bias may be NULL)
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
-                             float* gamma, float* tap_cs, cudaStream_t st);
+                             float* gamma, float* tap_cs, cudaStream_t st, const float* dt_bias = nullptr,
+                             bool softplus = false);
+ssdi8_status_t launch_softplus_dt(const float* dt_raw, const float* dt_bias, float* out, i64 rows, int H,
+                                  cudaStream_t st);
 
 // acc_cb (tap, may be NULL), CBq (may be NULL when s_cb is NULL), absmax_acc: per-group
 // running max of |acc_cb| over the causal half (calibration; may be NULL)

@@ -26,12 +26,14 @@ def tap_shapes(cfg):
     }
 
 
-def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use", flags=0):
+def gpu_fwd(cfg, q, corr=None, taps=TAP_NAMES, D="use", flags=0, dt_bias=None):
     """q: dict with xq,Bq,Cq,s_x,s_B,s_C,dt,A,D,s_xs,s_cb,s_h,init (numpy).  Returns y, final, taps."""
     dims = bd.dims_of(cfg)
     t = {k: dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "s_xs", "s_cb", "s_h")}
     t["D"] = dev(q["D"]) if D == "use" else None
     t["corr"] = dev(corr)
+    if dt_bias is not None:
+        t["dt_bias"] = dev(dt_bias)
     t["init_state"] = dev(q.get("init"))
     y = torch.full((cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim), float("nan"), device="cuda")
     fin = torch.full((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), float("nan"), device="cuda")

@@ -376,6 +376,55 @@ def test_fwd_full_size_all_pairs(name, flags):
         worst = max(worst, float((pair_err / pair_rms).max()))
     print(f"{name} flags={flags}: worst pair max|dy|/rms = {worst:.2e} over {cfg.batch * cfg.nheads} pairs")
 
+# --------------------------------------------------------------------------- softplus of the raw time step
+@pytest.mark.parametrize("with_bias", [True, False])
+def test_fwd_from_the_raw_time_step(with_bias):
+    """SSDI8_FLAG_DT_SOFTPLUS: ChunkCumsum starts from dt = softplus(dt_raw + dt_bias) (Algorithm 2 module 1).
+    The oracle applies its own softplus and runs the forward on the positive time step; every tap,
+    the final state and y must agree as in the default mode."""
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SMALL[1]
+    t = inputs.make_prefill(cfg)
+    rng = np.random.default_rng(77)
+    raw = rng.normal(-3.0, 1.0, t["dt"].shape).astype(np.float32)
+    raw[0, :4, 0] = [60.0, -60.0, 0.0, -100.0]              # both tails and the middle of the softplus
+    bias = rng.normal(0.0, 0.3, cfg.nheads).astype(np.float32) if with_bias else None
+    t["dt"] = orc.softplus_dt(raw, bias)
+    q = orc.prepare_quantized(cfg, t)
+    y_ref, fin_ref, ref = orc.ssdi8_fwd(cfg, q["xq"], q["Bq"], q["Cq"], q["s_x"], q["s_B"], q["s_C"], q["dt"], q["A"],
+                                        q["D"], None, q["s_xs"], q["s_cb"], q["s_h"], None, taps=gh.TAP_NAMES)
+    qg = dict(q)
+    qg["dt"] = raw
+    y, fin, got = gh.gpu_fwd(cfg, qg, flags=bd.FLAG_DT_SOFTPLUS, dt_bias=bias)
+    tril = _causal(cfg)
+    for name in ("cs", "Xsq", "acc_st", "loc", "prev", "hq", "acc_off", "rowmax", "Mq", "acc_diag"):
+        assert np.array_equal(got[name], ref[name]), name
+    assert np.array_equal(got["CBq"][..., tril], ref["CBq"][..., tril])
+    assert np.array_equal(fin, fin_ref)
+    assert np.abs(y - y_ref).max() <= Y_TOL * rms(y_ref)
+
+
+def test_softplus_dt_entry_point_bit_exact():
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    rng = np.random.default_rng(78)
+    H = 80
+    raw = np.concatenate([rng.normal(-3, 1.5, (30000, H)), rng.uniform(-95, 95, (3000, H))]).astype(np.float32)
+    bias = rng.normal(0, 0.5, H).astype(np.float32)
+    for b in (bias, None):
+        want = orc.softplus_dt(raw, b)
+        d_raw = gh.dev(raw)
+        out = torch.empty_like(d_raw)
+        bd.ssdi8_softplus_dt(d_raw, gh.dev(b), raw.shape[0], H, out)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy(), want)
+        # and against the libm definition: the same binary32 value in all but a handful of elements
+        plain = orc.softplus_dt(raw, b, plain=True)
+        assert np.mean(out.cpu().numpy() != plain) < 1e-5
+
+
 # --------------------------------------------------------------------------- persistent INT8 states (Eq. 4, 7)
 @pytest.mark.parametrize("cfg", [SMALL[0], SMALL[1], SMALL[2]], ids=lambda c: c.name)
 def test_fwd_int8_state_mode_bit_exact(cfg):

@@ -240,3 +240,31 @@ def test_prop1_mse_against_numpy():
     e2 = (sx * qx * lut - yv) ** 2
     want = (((sy * qy - yv) ** 2).mean(), e2.mean(), (qy == 0).mean(), e2.sum(2).mean())
     assert np.allclose(got, want, rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- softplus of the raw time step
+def test_softplus_dt_against_numpy_and_its_limits():
+    """Algorithm 2 module 1 starts from dt = softplus(dt_raw + bias).  The plain function is libm's; the
+    operation-by-operation binary64 sequence agrees with numpy.logaddexp(0, v) to a few 1e-16 before the
+    rounding to binary32, so that the two binary32 results differ (by one unit) in fewer than one element
+    in a million; large |v| reduce to v and to exp(v)."""
+    rng = np.random.default_rng(31)
+    H = 6
+    raw = np.concatenate([rng.normal(-3, 1.5, (40000, H)), rng.uniform(-90, 90, (20000, H)),
+                          np.array([[0, -0.0, 1e-30, -1e-30, 50, -50]] * 2)]).astype(np.float32)
+    bias = rng.normal(0, 0.5, H).astype(np.float32)
+    v = (raw + bias).astype(np.float64)                       # binary32 sum, widened
+    want64 = np.logaddexp(0.0, v)
+    plain = orc.softplus_dt(raw, bias, plain=True)
+    spec = orc.softplus_dt(raw, bias)
+    assert np.mean(plain != want64.astype(np.float32)) < 1e-6
+    assert np.mean(plain != spec) < 1e-6
+    assert np.mean(spec != want64.astype(np.float32)) < 1e-6
+    normal = want64 > 1.2e-38                                  # (binary32 subnormals round more coarsely)
+    assert np.all(np.abs(spec.astype(np.float64) - want64)[normal] <= 6.0e-8 * want64[normal])
+    assert np.all(spec[normal] > 0)
+    big = orc.softplus_dt(np.array([[60.0, -60.0]], np.float32))
+    assert big[0, 0] == np.float32(60.0) and abs(float(big[0, 1]) / np.exp(-60.0) - 1) < 1e-6
+    assert orc.softplus_dt(np.zeros((1, 1), np.float32))[0, 0] == np.float32(np.log(2.0))
+    # without a bias the raw value is used as it is
+    assert np.array_equal(orc.softplus_dt(raw, None), orc.softplus_dt(raw, np.zeros(H, np.float32)))
