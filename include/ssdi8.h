@@ -232,7 +232,9 @@ ssdi8_status_t ssdi8_chunk_scan_fwd(const ssdi8_dims_t* dims, const ssdi8_fwd_ar
  *    SSDI8_ERR_WORKSPACE; use ssdi8_chunk_scan_fwd with your own workspace for those.
  *  - The call allocates nothing and frees nothing, on the host or on the device.
  *  - The first call on each device looks up the array's device address (with that device
- *    current); make that first call before any stream capture begins.
+ *    current) and keeps it for the life of the process; make that first call before any stream
+ *    capture begins, and do not reset the device (cudaDeviceReset) afterwards: the kept address
+ *    would then be stale.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.
  *    Nothing in it has to start at zero (every region is written before it is read), but two
  *    calls that overlap on the GPU (different streams, no dependency) race on it: order them.

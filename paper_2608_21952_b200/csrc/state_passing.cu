@@ -11,7 +11,7 @@ namespace {
 constexpr int SP_T = 256;
 
 __global__ void __launch_bounds__(SP_T) state_passing_kernel(
-    const float4* __restrict__ loc, const float* __restrict__ gamma, const float4* __restrict__ init,
+    const float4* loc /* may alias prev: no __restrict__ */, const float* __restrict__ gamma, const float4* __restrict__ init,
     const float* __restrict__ s_h, float4* prev, float4* __restrict__ final_state,
     uint32_t* __restrict__ hq, uint32_t* __restrict__ absmax_h, Dims d) {
   const int N4 = d.N / 4;

@@ -70,6 +70,27 @@ def test_static_entry_matches_workspace_entry_twice_in_a_row():
         results.append(y_st)
     assert all(np.all(np.isfinite(r)) for r in results)
 
+    # one flagged mode through the same scratch: the paper's persistent INT8 states (Eq. 4, 7)
+    cfg = CONFIGS["cfg0"]
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    dims = bd.dims_of(cfg)
+    dv = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    outs = []
+    for static in (False, True):
+        y = torch.full((cfg.batch, cfg.seqlen, cfg.nheads, cfg.headdim), float("nan"), device="cuda")
+        fin = torch.full((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), float("nan"), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        args = bd.make_fwd_args(y=y, final_state=fin, status=status, **dv)
+        if static:
+            bd.ssdi8_chunk_scan_fwd_static(dims, args, flags=bd.FLAG_INT8_STATE)
+        else:
+            bd.ssdi8_chunk_scan_fwd(dims, args, bd.alloc_workspace(dims), flags=bd.FLAG_INT8_STATE)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        outs.append((y.cpu().numpy(), fin.cpu().numpy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
     with pytest.raises(bd.SSDi8Error) as e:
         big = CONFIGS["cfg2"]
         bd.ssdi8_chunk_scan_fwd_static(bd.dims_of(big), bd.FwdArgs())
