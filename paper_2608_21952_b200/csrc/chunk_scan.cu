@@ -280,14 +280,17 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
     if (TAPS && mq_tap) *reinterpret_cast<uint2*>(mq_tap + I16 * 16 + q2 * 8) = v;
   }
   bool dead = false;                 // this chunk and every farther one round to zero in this row
+  int itc = 0;
 #pragma unroll 1
-  for (int itc = 0; itc < nit; ++itc) {
+  for (; itc < nit; ++itc) {
     const int c = c_first - 2 * itc;
     const bool valid = c >= 0;
     const int cc = valid ? c : 0;
+    // once no row of the warp has a chunk left that does not round to zero, what remains is zero fill
+    if (!__any_sync(kAll, valid && !dead)) break;
     uint4* ptr = chunk_ptr(cc);
     uint4 v = zero4;
-    if (__any_sync(kAll, valid && !dead)) {
+    {
       const float f = itc >= nv || itc > 1 ? exp32(__fsub_rn(cs_i, cs_s[cc * 16 + 15])) : (itc ? f1 : f0);
       const float g = __fmul_rn(f, inv);
       if (__fmul_rn(p127_s[cc], g) < 0.5f) dead = true;
@@ -311,6 +314,12 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
       *ptr = v;
       if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = v;
     }
+  }
+  // the chunks farther left are zeros in every row of the warp
+#pragma unroll 1
+  for (int c = c_first - 2 * itc; c >= 0; c -= 2) {
+    *chunk_ptr(c) = zero4;
+    if (TAPS && mq_tap) *reinterpret_cast<uint4*>(mq_tap + c * 16) = zero4;
   }
 }
 
