@@ -11,16 +11,17 @@ namespace {
 // leave fewer of them to overlap.)
 constexpr int kChunksPerBlock = 1;
 
+template <bool SOFTPLUS>
 __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ dt,
                                                      const float* __restrict__ A,
                                                      float* __restrict__ pack,
                                                      float* __restrict__ gamma,
                                                      float* __restrict__ tap_cs, Dims d,
-                                                     const float* __restrict__ dt_bias, int softplus) {
+                                                     const float* __restrict__ dt_bias) {
   extern __shared__ float tile[];
   pdl_launch_dependents();
   pdl_wait();
-  cumsum_body<kChunksPerBlock>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias, softplus);
+  cumsum_body<kChunksPerBlock, SOFTPLUS>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias);
 }
 
 // dt = softplus(dt_raw + dt_bias[h]) alone (for callers that calibrate on the positive time step)
@@ -49,9 +50,13 @@ ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, flo
                              float* gamma, float* tap_cs, cudaStream_t st, const float* dt_bias, bool softplus) {
   dim3 grid((d.H + kCumsumHeads - 1) / kCumsumHeads, (d.c + kChunksPerBlock - 1) / kChunksPerBlock, d.b);
   const size_t smem = cumsum_smem_bytes(d.Q, kChunksPerBlock);
-  SSDI8_CUDA_CHECK(cudaFuncSetAttribute(cumsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  if (launch_pdl(cumsum_kernel, grid, dim3(256), smem, st, dt, A, pack, gamma, tap_cs, d, dt_bias, softplus ? 1 : 0) != cudaSuccess)
-    return SSDI8_ERR_CUDA;
+  auto launch = [&](auto kernel) -> ssdi8_status_t {
+    SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    return launch_pdl(kernel, grid, dim3(256), smem, st, dt, A, pack, gamma, tap_cs, d, dt_bias) == cudaSuccess
+               ? SSDI8_OK : SSDI8_ERR_CUDA;
+  };
+  const ssdi8_status_t ls = softplus ? launch(cumsum_kernel<true>) : launch(cumsum_kernel<false>);
+  if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }

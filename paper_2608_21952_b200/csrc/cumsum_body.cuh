@@ -30,14 +30,14 @@ __host__ __device__ inline size_t cumsum_smem_bytes(int Q, int KC) {
 
 // One block's work: heads 8 bx .. and chunks KC kx .. of batch element b.  Any whole number of warps
 // may run it (every loop strides by the block size); `tile` is cumsum_smem_bytes(Q, KC) of shared memory.
-// softplus != 0: dt holds the raw time step and dt = softplus(dt + dt_bias[h]) (dt_bias may be NULL)
+// SOFTPLUS: dt holds the raw time step and dt = softplus(dt + dt_bias[h]) (dt_bias may be NULL)
 // is applied as the values are staged (Algorithm 2 module 1 starts there).
-template <int KC>
+// (a template parameter: the binary64 softplus costs registers, and the plain instance must keep its occupancy)
+template <int KC, bool SOFTPLUS = false>
 __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const float* __restrict__ A,
                                             float* __restrict__ pack, float* __restrict__ gamma,
                                             float* __restrict__ tap_cs, const Dims& d, int bx, int kx, int b,
-                                            float* tile, const float* __restrict__ dt_bias = nullptr,
-                                            int softplus = 0) {
+                                            float* tile, const float* __restrict__ dt_bias = nullptr) {
   constexpr int CH = kCumsumHeads, NU = CH * KC;   // unit u = hh * KC + kk
   const int Q = d.Q, ld = Q + 1;
   const int lq = 31 - __clz(Q);  // Q is a power of two
@@ -63,7 +63,7 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
       const int t = e / CH, hh = e % CH;
       if (e < ntok * CH && hh < nh)
         dts[(hh * KC + (t >> lq)) * ld + (t & (Q - 1))] =
-            softplus ? softplus_dt(v[u], dt_bias ? __ldg(dt_bias + h0 + hh) : 0.f) : v[u];
+            SOFTPLUS ? softplus_dt(v[u], dt_bias ? __ldg(dt_bias + h0 + hh) : 0.f) : v[u];
     }
   }
   __syncthreads();
