@@ -250,9 +250,9 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  *
  * ssdi8_layer_fwd: every pointer is a DEVICE pointer.  The three quantisers are one launch on
  *   `stream` (separate launches when d_state is not a power of two or a tensor is not 16-byte
- *   aligned); ChunkCumsum (reads dt and A only) runs on a side stream under them and ChunkBMM
- *   (needed by ChunkScan only) on a second side stream under the state kernel; the side streams
- *   join `stream` before ChunkState and before ChunkScan.  workspace: 256-byte aligned,
+ *   aligned); ChunkCumsum (reads dt and A only) runs inside that launch for small workloads and on a
+ *   side stream under it, joined before the state kernel, for large ones; the state kernel, ChunkBMM
+ *   and ChunkScan follow on `stream`.  workspace: 256-byte aligned,
  *   ssdi8_layer_fwd_workspace_bytes(dims, flags) bytes (the int8 tensors plus ssdi8_workspace_bytes).
  * ssdi8_layer_fwd_host: x, B, C, dt, y, final_state, status are HOST pointers (page-locked memory, or
  *   the copies neither overlap nor run asynchronously), the rest DEVICE pointers.  One slice at a

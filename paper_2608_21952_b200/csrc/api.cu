@@ -160,7 +160,11 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
   if ((ph & SSDI8_PHASE_CUMSUM) && (s = launch_cumsum(d, a->dt, a->A, pack, gamma, a->tap_cs, st, a->dt_bias,
                                                      (flags & SSDI8_FLAG_DT_SOFTPLUS) != 0)) != SSDI8_OK)
     return s;
-  if ((ph & SSDI8_PHASE_BMM) &&
+  // ChunkBMM depends on neither ChunkCumsum nor the state kernel and is needed by ChunkScan only.  When the
+  // fused state kernel runs in this call, ChunkBMM is launched after it and works beside its last wave.
+  const bool fused_state = (ph & SSDI8_PHASE_CHUNK_STATE) && (ph & SSDI8_PHASE_STATE_PASSING);
+  const bool bmm_late = (ph & SSDI8_PHASE_BMM) && fused_state;
+  if ((ph & SSDI8_PHASE_BMM) && !bmm_late &&
       (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, a->status, st)) !=
           SSDI8_OK)
     return s;
@@ -169,6 +173,9 @@ ssdi8_status_t fwd_phases(const ssdi8_dims_t* dims, const ssdi8_fwd_args_t* a, u
     if ((s = launch_chunk_state_passing(d, a->xq, a->Bq, a->s_x, a->s_xs, a->s_B, a->s_h, pack, gamma,
                                         a->init_state, hq, a->final_state, a->tap_loc, a->tap_prev,
                                         a->tap_Xsq, a->tap_acc_st, a->status, i8s, st)) != SSDI8_OK)
+      return s;
+    if (bmm_late && (s = launch_bmm(d, a->Cq, a->Bq, a->s_C, a->s_B, a->s_cb, cbq, a->tap_acc_cb, nullptr, a->status,
+                                    st, true)) != SSDI8_OK)
       return s;
   } else {
     if ((ph & SSDI8_PHASE_CHUNK_STATE) &&

@@ -20,6 +20,7 @@ struct BmmArgs {
   int32_t* tap_acc; uint32_t* absmax_acc; int32_t* status;
   Dims d;
   int store;  // 0: calibration pass (no CBq written)
+  int late_wait;  // 1: launched right after the fused state kernel, which it does not depend on (see below)
 };
 
 constexpr int kThreads = 512;   // 16 warps: warp w reads TMEM lane quarter w % 4 (rows) and every fourth 32-column piece from w / 4
@@ -60,7 +61,12 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  pdl_wait();
+  // Programmatic dependent launch.  Normally: wait for the predecessor before the first global access.
+  // Launched right after the fused state kernel (which waits for ITS predecessor before it lets this
+  // kernel be scheduled), the work below runs beside that kernel's last wave, and the wait moves to
+  // the end, where it only keeps "this kernel complete" implying "the state kernel complete" for the
+  // scan kernel that follows.
+  if (!a.late_wait) pdl_wait();
 
   if (tid == 0) {
     mbar_expect_tx(&bars[0], (uint32_t)(TM * N + KJ * N));
@@ -141,13 +147,14 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
     tc_fence_after();
     tmem_dealloc(tmem, 256);
   }
+  if (a.late_wait) pdl_wait();
 }
 
 }  // namespace
 
 ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, const float* s_C,
                           const float* s_B, const float* s_cb, int8_t* CBq, int32_t* tap_acc,
-                          uint32_t* absmax_acc, int32_t* status, cudaStream_t st) {
+                          uint32_t* absmax_acc, int32_t* status, cudaStream_t st, bool after_state_kernel) {
   const int TM = d.Q < 128 ? d.Q : 128;
   const uint64_t T = (uint64_t)d.b * d.L;
   CUtensorMap tm_C, tm_B, tm_o;
@@ -165,7 +172,7 @@ ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, con
     uint32_t obox[2] = {(uint32_t)TM, (uint32_t)TM};
     if (!encode_tensor_map(&tm_o, base, 1, 2, odims, ostr, obox, TM)) return SSDI8_ERR_CUDA;
   }
-  BmmArgs a = {s_C, s_B, s_cb, tap_acc, absmax_acc, status, d, store ? 1 : 0};
+  BmmArgs a = {s_C, s_B, s_cb, tap_acc, absmax_acc, status, d, store ? 1 : 0, after_state_kernel ? 1 : 0};
   const size_t smem = SMEM_BYTES + 1024;
   SSDI8_CUDA_CHECK(cudaFuncSetAttribute(bmm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const unsigned grid = (unsigned)((i64)d.b * d.c * d.G * (d.Q / TM));

@@ -100,9 +100,11 @@ __device__ __forceinline__ void fused_body(const CUtensorMap& tm_B, const CUtens
     tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_hq);
   }
-  pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
   pdl_wait();   // everything below reads global memory
+  // (after the wait, not before it: ChunkBMM, launched next, reads and writes global memory without waiting
+  // for this kernel, so it must not be scheduled before this kernel's predecessors have completed)
+  pdl_launch_dependents();
   if (tid < 64) {
     const float sxb = __fmul_rn(a.s_xs[h * P + tid], a.s_B[g]), sh = a.s_h[h * P + tid];
     col_scale[tid] = I8S ? __fdiv_rn(sxb, sh) : sxb;

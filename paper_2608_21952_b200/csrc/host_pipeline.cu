@@ -1,8 +1,9 @@
 // The layer step as one call: Eq. 1 quantisation of fp32 x, B, C with static step sizes and the SSD
 // layer forward (Algorithm 2).
-// ssdi8_layer_fwd (device buffers): the modules that do not depend on xq (the quantisers of B and C,
-// ChunkCumsum, ChunkBMM; all latency-bound) run on a side stream under the HBM-bound quantiser of
-// x, then the two streams join for ChunkState/StatePassing and ChunkScan.
+// ssdi8_layer_fwd (device buffers): ChunkCumsum reads dt and A only, so it runs beside the quantisers
+// (inside their launch for small workloads, on a side stream under the bandwidth-bound quantiser of x
+// for large ones); the state kernel, ChunkBMM and ChunkScan follow on the caller's stream, chained by
+// programmatic dependent launch.
 // ssdi8_layer_fwd_host (host buffers): the same, one batch element at a time.  Batch elements are
 // independent, so the host->device copies of element b+1 and the device->host copy of the
 // output of element b-1 run on two side streams while the kernels of element b run on the
@@ -61,9 +62,9 @@ Layout make_layout(const ssdi8_dims_t& d1, int full_heads, uint8_t* base, uint32
 // side streams and events, made once per device and kept for the life of the process
 struct Plumbing {
   bool ready = false;
-  cudaStream_t s_in = nullptr, s_out = nullptr, s_side = nullptr, s_side2 = nullptr;
+  cudaStream_t s_in = nullptr, s_out = nullptr, s_side2 = nullptr;
   cudaEvent_t start = nullptr, in_done[kStages] = {}, cmp_done[kStages] = {}, out_done[kStages] = {};
-  cudaEvent_t fork = nullptr, fork2 = nullptr, join = nullptr, join2 = nullptr;
+  cudaEvent_t fork = nullptr, join2 = nullptr;
 };
 Plumbing g_plumb[64];
 std::mutex g_plumb_mu;   // two threads may make their first call on a device at once
@@ -81,12 +82,9 @@ ssdi8_status_t get_plumbing(Plumbing** out) {
     // placed as soon as the bandwidth-bound quantiser of x frees a slot instead of behind its whole grid
     int prio_lo = 0, prio_hi = 0;
     SSDI8_CUDA_CHECK(cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
-    SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side, cudaStreamNonBlocking, prio_hi));
     SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side2, cudaStreamNonBlocking, prio_hi));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming));
-    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork2, cudaEventDisableTiming));
-    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join2, cudaEventDisableTiming));
     for (int s = 0; s < kStages; ++s) {
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.in_done[s], cudaEventDisableTiming));
@@ -169,17 +167,12 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
         return s;
     }
   }
-  // ChunkBMM needs Bq and Cq and is needed by ChunkScan only: it runs on a side stream under the
-  // state kernel
-  SSDI8_CUDA_CHECK(cudaEventRecord(p.fork2, st));
-  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side, p.fork2, 0));
-  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM, ws, ws_bytes, p.s_side, false)) != SSDI8_OK) return s;
-  SSDI8_CUDA_CHECK(cudaEventRecord(p.join, p.s_side));
+  // the rest on the caller's stream, chained by programmatic dependent launch: the fused state kernel,
+  // ChunkBMM (needed by ChunkScan only: launched behind the state kernel, it works beside that kernel's
+  // last wave), ChunkScan
   if (!merged) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join2, 0));
-  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING, ws, ws_bytes, st, false)) != SSDI8_OK)
-    return s;
-  SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join, 0));
-  return fwd_phases(&d, &f, fl | SSDI8_PHASE_SCAN, ws, ws_bytes, st, false);
+  return fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING | SSDI8_PHASE_SCAN,
+                    ws, ws_bytes, st, false);
 }
 
 // How many equal head ranges a batch element is cut into for the host pipeline: halved while a

@@ -62,10 +62,11 @@ ssdi8_status_t launch_softplus_dt(const float* dt_raw, const float* dt_bias, flo
                                   cudaStream_t st);
 
 // acc_cb (tap, may be NULL), CBq (may be NULL when s_cb is NULL), absmax_acc: per-group
-// running max of |acc_cb| over the causal half (calibration; may be NULL)
+// running max of |acc_cb| over the causal half (calibration; may be NULL).  after_state_kernel: the launch
+// directly follows launch_chunk_state_passing in the same stream and may run beside it (see bmm.cu)
 ssdi8_status_t launch_bmm(const Dims& d, const int8_t* Cq, const int8_t* Bq, const float* s_C,
                           const float* s_B, const float* s_cb, int8_t* CBq, int32_t* tap_acc,
-                          uint32_t* absmax_acc, int32_t* status, cudaStream_t st);
+                          uint32_t* absmax_acc, int32_t* status, cudaStream_t st, bool after_state_kernel = false);
 
 // absmax_xs: per-channel running max (as binary32 bits) of |x_scaled| (calibration; may be
 // NULL).  When absmax_xs is non-NULL only that is computed.
