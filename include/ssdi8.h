@@ -8,8 +8,13 @@
  *
  * Conventions for every entry point
  *  - All pointers are DEVICE pointers unless the comment says "host".  The
- *    caller owns every buffer; except where stated the library allocates no
- *    device memory and keeps no mutable global state.
+ *    caller owns every buffer and the library allocates no device memory.  It keeps
+ *    no mutable state between calls, with three exceptions, each stated again at its
+ *    entry point: per device, the result of the architecture check (every call);
+ *    the address of the built-in scratch (ssdi8_chunk_scan_fwd_static); one side
+ *    stream and its events (ssdi8_layer_fwd, ssdi8_layer_fwd_host, created at the
+ *    first call on a device and kept for the life of the process).  All three are
+ *    filled under a lock, so first calls may come from several threads at once.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *    Calls are asynchronous on that stream.
  *  - The return value reports everything that can be checked on the host
