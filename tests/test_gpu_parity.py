@@ -701,6 +701,54 @@ def test_layer_fwd_matches_the_separate_calls_bit_for_bit(cfg, flags):
         assert np.array_equal(y.cpu().numpy(), y_dev) and np.array_equal(fin.cpu().numpy(), fin_dev)
 
 
+def test_layer_fwd_back_to_back_on_one_workspace_with_alternating_inputs():
+    """The kernels of consecutive calls overlap at their edges (programmatic dependent launch: a kernel may be
+    scheduled while its predecessor drains, and ChunkBMM runs beside the state kernel), and all calls share
+    one workspace.  Forty calls without a synchronisation in between, alternating between two inputs and two
+    outputs: every call must still produce what the same call produces alone."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SSDConfig("b2b", 2, 1024, 24, 64, 128, 2, 256, 0.02, 20.0, 61)
+    dims = bd.dims_of(cfg)
+    sets = []
+    for seed in (61, 62):
+        t = inputs.make_prefill(cfg.replace(seed=seed))
+        q = orc.prepare_quantized(cfg, t)
+        dv = {k: gh.dev(q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "A", "D")}
+        dv.update({k: gh.dev(t[k]) for k in ("x", "B", "C", "dt")})
+        y = torch.empty(t["x"].shape, device="cuda")
+        fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        sets.append(dict(args=bd.make_layer_args(y=y, final_state=fin, status=status, **dv), y=y, fin=fin, status=status))
+    ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims), dtype=torch.uint8, device="cuda")
+    ref = []
+    for s_ in sets:   # each call alone
+        bd.ssdi8_layer_fwd(dims, s_["args"], ws)
+        torch.cuda.synchronize()
+        ref.append((s_["y"].clone(), s_["fin"].clone()))
+        s_["y"].fill_(float("nan")); s_["fin"].fill_(float("nan"))
+    for i in range(40):
+        bd.ssdi8_layer_fwd(dims, sets[i & 1]["args"], ws)
+    torch.cuda.synchronize()
+    for s_, (y0, f0) in zip(sets, ref):
+        assert int(s_["status"].item()) == 0
+        assert torch.equal(s_["y"], y0) and torch.equal(s_["fin"], f0)
+    # and Algorithm 2 alone (ssdi8_chunk_scan_fwd) the same way, on the int8 tensors of the first input
+    t = inputs.make_prefill(cfg.replace(seed=61))
+    q = orc.prepare_quantized(cfg, t)
+    y_a, fin_a, _ = gh.gpu_fwd(cfg, q, taps=())
+    dq = {k: gh.dev(q[k]) for k in ("xq", "Bq", "Cq", "s_x", "s_B", "s_C", "dt", "A", "D", "s_xs", "s_cb", "s_h")}
+    y = torch.empty(t["x"].shape, device="cuda")
+    fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+    args = bd.make_fwd_args(y=y, final_state=fin, **dq)
+    ws2 = bd.alloc_workspace(dims)
+    for i in range(40):
+        bd.ssdi8_chunk_scan_fwd(dims, args, ws2)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), y_a) and np.array_equal(fin.cpu().numpy(), fin_a)
+
+
 def test_layer_fwd_host_rejects_a_short_scratch():
     import torch
     from paper_2608_21952_b200 import binding as bd
