@@ -196,7 +196,10 @@ typedef struct {
  *                  same sub-block : running product of the per-token decays
  *                                   a_m = exp32(fsub(cs_m, cs_{m-1})): E[i,i] = 1,
  *                                   E[i,j] = fmul(E[i,j+1], a_{j+1}); w = fmul(dt_j, E[i,j]), f = 1
- *                  earlier block  : w = fmul(dt_j, exp32(fsub(cs_je, cs_j))), f = exp32(fsub(cs_i, cs_je))
+ *                  earlier block  : w = fmul(dt_j, exp32(fsub(cs_je, cs_j))),
+ *                                   f = fmul(exp32(fsub(cs_i, cs_pe)), exp32(fsub(cs_pe, cs_je))), pe the last
+ *                                   token of the sub-block before the row's own (the second factor
+ *                                   depends on the two sub-blocks only: ChunkCumsum tabulates it)
  *                  t = fmul(float(CBq[i,j]), w)
  *                  rowmax_i = max over sub-blocks of fmul(max_j |t|, f)
  *                  inv_i = rowmax_i >= 1e-30 ? fdiv(127, rowmax_i) : 0

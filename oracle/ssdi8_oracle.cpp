@@ -510,7 +510,9 @@ void orc_chunk_decay(const Dims* d, const float* cs, float* gamma) {
 //     same sub-block:  the decay is the running product of the per-token decays
 //                      a_m = exp32(fsub(cs_m, cs_{m-1})):  E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1});
 //                      w = fmul(dt_j, E[i,j]),  f = 1
-//     earlier block :  w = fmul(dt_j, exp32(fsub(cs_je, cs_j))), f = exp32(fsub(cs_i, cs_je))
+//     earlier block :  w = fmul(dt_j, exp32(fsub(cs_je, cs_j))),
+//                      f = fmul(exp32(fsub(cs_i, cs_pe)), exp32(fsub(cs_pe, cs_je))), pe = last token of the
+//                      sub-block before the row's own
 //     t[i,j]   = fmul(float(CBq[i,j]), w)          (w f = dt_j exp(cs_i - cs_j); every exponent <= 0)
 //     rowmax_i = max over sub-blocks J of fmul(max_{j in J, j<=i} |t[i,j]|, f)
 //     inv_i    = rowmax_i >= 1e-30 ? fdiv(127, rowmax_i) : 0
@@ -565,7 +567,11 @@ void orc_chunk_scan(const Dims* d, const int8_t* xq, const int8_t* Cq, const int
           float rmax = 0.0f;
           for (int J = 0; J <= I; ++J) {
             const int je = J * SB + SB - 1;
-            f[J] = (J == I) ? 1.0f : exp32(fsub(csk[i], csk[je]));
+            // earlier block: the decay from the block's last token to row i as the product of the row's
+            // decay to the end of the block before its own (pe) and the block-to-block decay from there
+            // (1 for the block next to the row's own: pe = je)
+            const int pe = I * SB - 1;
+            f[J] = (J == I) ? 1.0f : fmul(exp32(fsub(csk[i], csk[pe])), exp32(fsub(csk[pe], csk[je])));
             float bmax = 0.0f;
             float E = 1.0f;
             for (int j = (J == I ? i : je); j >= J * SB; --j) {

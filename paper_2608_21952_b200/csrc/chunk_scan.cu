@@ -191,8 +191,10 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
   const int c_first = I16 - 1 - q2;  // nearest earlier chunk of this thread (may be < 0)
   float tv[8];                       // t of this thread's half of the row's own sub-block
   float rpart = 0.f;
-  float f0 = 0.f, f1 = 0.f;          // f of the first two chunks visited
-  int nv = 0;                        // chunks whose f the first pass computed
+  // f of an earlier chunk c: the row's decay to the end of the chunk before its own, times the tabulated
+  // decay from there to the end of chunk c (gtab[c]; 1 for c = I16 - 1)
+  const float ri_dec = I16 > 0 ? exp32(__fsub_rn(cs_i, cs_s[I16 * 16 - 1])) : 0.f;
+  const float* const gtab = b127_s + 32 + ((I16 * (I16 - 1)) >> 1);
   uint2* const own_ptr = reinterpret_cast<uint2*>(chunk_ptr(I16)) + q2;
   {
     // own sub-block, right to left: E[i,i] = 1, E[i,j] = fmul(E[i,j+1], a_{j+1}).  Straight-line code:
@@ -246,10 +248,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
     live = live && c >= 0;
     if (!__any_sync(kAll, live)) break;
     const int cc = c < 0 ? 0 : c;
-    const float f = exp32(__fsub_rn(cs_i, cs_s[cc * 16 + 15]));
-    if (itc == 0) f0 = f;
-    if (itc == 1) f1 = f;
-    nv = itc + 1;
+    const float f = __fmul_rn(ri_dec, gtab[cc]);
     if (rpart >= 1e-30f && __fmul_rn(p127_s[cc], f) <= rpart) live = false;  // nor can any farther chunk
     const bool need = live && !(__fmul_rn(b127_s[cc], f) <= rpart);
     if (!__any_sync(kAll, need)) continue;
@@ -298,7 +297,7 @@ __device__ __forceinline__ void mask_tile(uint8_t* sCB, const float* tokbuf, flo
     uint4* ptr = chunk_ptr(cc);
     uint4 v = zero4;
     {
-      const float f = itc >= nv || itc > 1 ? exp32(__fsub_rn(cs_i, cs_s[cc * 16 + 15])) : (itc ? f1 : f0);
+      const float f = __fmul_rn(ri_dec, gtab[cc]);
       const float g = __fmul_rn(f, inv);
       if (__fmul_rn(p127_s[cc], g) < 0.5f) dead = true;
       const bool need = valid && !dead && __fmul_rn(b127_s[cc], g) >= 0.5f;

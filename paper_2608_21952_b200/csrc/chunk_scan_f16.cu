@@ -166,6 +166,10 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
   };
   const float cs_i = row_ok ? cs_s[i] : 0.f;
   const float scb = a.s_cb[t.g];
+  // decay to an earlier chunk c: the row's decay to the end of the chunk before its own, times the
+  // tabulated decay from there to the end of chunk c (1 for c = I16 - 1)
+  const float ri_dec = I16 > 0 ? exp32(__fsub_rn(cs_i, cs_s[I16 * 16 - 1])) : 0.f;
+  const float* const gtab = b127_s + 32 + ((I16 * (I16 - 1)) >> 1);
   const float kTiny = 2.9e-8f;       // below 2^-25 = 2.98e-8: rounds to zero in FP16
   const uint32_t lane_addr = a_tmem + ((uint32_t)(rq * 32) << 16);
   bool done = !row_ok;               // this row has nothing (more) to contribute
@@ -213,7 +217,7 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
       for (int e = 0; e < 8; ++e) w8[e] = own[e];
     } else if (!done && c < I16) {
       {
-        const float g = __fmul_rn(exp32(__fsub_rn(cs_i, cs_s[c * 16 + 15])), scb);
+        const float g = __fmul_rn(__fmul_rn(ri_dec, gtab[c]), scb);
         if (__fmul_rn(p127_s[c], g) < kTiny) {
           done = true;               // this chunk and every farther one round to zero
         } else if (__fmul_rn(b127_s[c], g) >= kTiny) {

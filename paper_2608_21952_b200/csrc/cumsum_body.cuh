@@ -8,7 +8,10 @@
 //          output bit): [c] = fmul(127, wmax_c), wmax_c the maximum of |woff| over the 16-token
 //          sub-block c; [16 + c] = the maximum of the former over sub-blocks 0..c, times
 //          1.00001, or +inf when cs is not non-increasing over the chunk (some dt A > 0), which
-//          switches the early exits of the scan kernel off; entries from 32 on are not written
+//          switches the early exits of the scan kernel off; [32 + I (I - 1) / 2 + c], c < I: the decay
+//          between the ends of sub-blocks c and I - 1, exp32(fsub(cs[16 I - 1], cs[16 c + 15])), which
+//          the scan kernel multiplies by a row's own decay to the end of sub-block I - 1; the rest of
+//          the row is not written
 //   row 5  lut[i]   = fmul(dt_i, exp32(fsub(cs_last, cs_i)))                       (LUT_state)
 // and Gamma[b,h,k] = exp32(cs[Q-1]) (Decay_pass, Eq. 5).  The sum order is part of the definition
 // (it decides rounding downstream), so each (b, chunk, head) is scanned sequentially by one
@@ -124,6 +127,20 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (live && (i & 15) == 0) wmx[u * 16 + (i >> 4)] = __fmul_rn(127.0f, m);
+  }
+  // block-to-block decays G[I][c], c < I (triangular: 120 entries for 16 sub-blocks); they need cs only,
+  // so they go out ahead of the barrier that the bounds wait for
+  const int nsb = Q >> 4, ntri = nsb * (nsb - 1) / 2;
+  for (int e = threadIdx.x; e < NU * 128; e += blockDim.x) {
+    const int u = e >> 7, idx = e & 127;
+    const int hh = u / KC, kk = u % KC;
+    if (hh >= nh || kk >= nk || idx >= ntri) continue;
+    // I (I - 1) / 2 <= idx < (I + 1) I / 2; 1 + 8 idx is (2 I - 1)^2 at the lower end, so the root is exact there
+    const int I = (int)((1.0f + sqrtf((float)(1 + 8 * idx))) * 0.5f);
+    const int c = idx - I * (I - 1) / 2;
+    const float* cc = css + u * ld;
+    const i64 un = ((i64)b * d.H + h0 + hh) * d.c + k0 + kk;
+    pack[((un * kPackRows + PACK_WMAX) << lq) + 32 + idx] = exp32(__fsub_rn(cc[16 * I - 1], cc[16 * c + 15]));
   }
   __syncthreads();
   for (int e = threadIdx.x; e < 32 * NU; e += blockDim.x) {   // the first 32 entries of the bounds row
