@@ -110,9 +110,9 @@ __global__ void __launch_bounds__(128, 8) quant_jobs(const QuantJobs a) {
 #pragma unroll
     for (int u = 0; u < QROWS; ++u) v[u] = __ldcs(in + (e + u * stride));
 #pragma unroll
-    for (int u = 0; u < QROWS; ++u) __stcs(out + (e + u * stride), quant_code4(v[u], sx, sy, sz, sw));
+    for (int u = 0; u < QROWS; ++u) out[e + u * stride] = quant_code4(v[u], sx, sy, sz, sw);
   }
-  for (; left > 0; --left, e += stride) __stcs(out + e, quant_code4(__ldcs(in + e), sx, sy, sz, sw));
+  for (; left > 0; --left, e += stride) out[e] = quant_code4(__ldcs(in + e), sx, sy, sz, sw);
 }
 
 // ---- quantise, I % 4 == 0: 4 consecutive elements share a channel
