@@ -97,10 +97,31 @@ __device__ __forceinline__ uint32_t quant_code_bits(float v, const QuantStep& s)
   if (fabsf(e) > s.thr) return rne_clamp_bits(__fdiv_rn(v, s.alpha));
   return __float_as_uint(m);
 }
+// Four codes as one word.  The common path is packed arithmetic and one branch for the four elements:
+// products, clamp (min(|t|, 127) with the sign of t), the magic addition, the rounded value and the distance
+// of the product from it; only a word with an element near a rounding boundary (or an abnormal step size)
+// goes through the divisions, element by element.
 __device__ __forceinline__ uint32_t quant_code4(const float4& v, const QuantStep& a, const QuantStep& b,
                                                 const QuantStep& c, const QuantStep& d) {
-  return pack4_bits(quant_code_bits(v.x, a), quant_code_bits(v.y, b), quant_code_bits(v.z, c),
-                    quant_code_bits(v.w, d));
+  const float2 t01 = __fmul2_rn(make_float2(v.x, v.y), make_float2(a.rcp, b.rcp));
+  const float2 t23 = __fmul2_rn(make_float2(v.z, v.w), make_float2(c.rcp, d.rcp));
+  float2 c01, c23;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c01.x) : "f"(t01.x), "f"(127.0f));
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c01.y) : "f"(t01.y), "f"(127.0f));
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c23.x) : "f"(t23.x), "f"(127.0f));
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c23.y) : "f"(t23.y), "f"(127.0f));
+  const float2 mg = make_float2(kMagicOut, kMagicOut), ng = make_float2(-kMagicOut, -kMagicOut);
+  const float2 m01 = __fadd2_rn(c01, mg), m23 = __fadd2_rn(c23, mg);
+  const float2 m1 = make_float2(-1.0f, -1.0f);   // e = c - (m - magic): both differences are exact
+  const float2 e01 = __ffma2_rn(__fadd2_rn(m01, ng), m1, c01), e23 = __ffma2_rn(__fadd2_rn(m23, ng), m1, c23);
+  uint32_t b0 = __float_as_uint(m01.x), b1 = __float_as_uint(m01.y), b2 = __float_as_uint(m23.x), b3 = __float_as_uint(m23.y);
+  if (fabsf(e01.x) > a.thr || fabsf(e01.y) > b.thr || fabsf(e23.x) > c.thr || fabsf(e23.y) > d.thr) {
+    if (fabsf(e01.x) > a.thr) b0 = rne_clamp_bits(__fdiv_rn(v.x, a.alpha));
+    if (fabsf(e01.y) > b.thr) b1 = rne_clamp_bits(__fdiv_rn(v.y, b.alpha));
+    if (fabsf(e23.x) > c.thr) b2 = rne_clamp_bits(__fdiv_rn(v.z, c.alpha));
+    if (fabsf(e23.y) > d.thr) b3 = rne_clamp_bits(__fdiv_rn(v.w, d.alpha));
+  }
+  return pack4_bits(b0, b1, b2, b3);
 }
 
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {

@@ -19,8 +19,11 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
                                                      float* __restrict__ tap_cs, Dims d,
                                                      const float* __restrict__ dt_bias) {
   extern __shared__ float tile[];
-  pdl_launch_dependents();
+  // The wait comes first: a successor that needs nothing of this kernel (the layer step's quantiser of x, B
+  // and C) is launched without a wait of its own at its start, so by the time it may be scheduled everything
+  // that precedes this kernel in the stream must have completed.
   pdl_wait();
+  pdl_launch_dependents();
   cumsum_body<kChunksPerBlock, SOFTPLUS>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias);
 }
 

@@ -62,9 +62,8 @@ Layout make_layout(const ssdi8_dims_t& d1, int full_heads, uint8_t* base, uint32
 // side streams and events, made once per device and kept for the life of the process
 struct Plumbing {
   bool ready = false;
-  cudaStream_t s_in = nullptr, s_out = nullptr, s_side2 = nullptr;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
   cudaEvent_t start = nullptr, in_done[kStages] = {}, cmp_done[kStages] = {}, out_done[kStages] = {};
-  cudaEvent_t fork = nullptr, join2 = nullptr;
 };
 Plumbing g_plumb[64];
 std::mutex g_plumb_mu;   // two threads may make their first call on a device at once
@@ -78,14 +77,7 @@ ssdi8_status_t get_plumbing(Plumbing** out) {
   if (!p.ready) {
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
     SSDI8_CUDA_CHECK(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
-    // the side stream carries short latency-bound kernels: highest priority, so that their blocks are
-    // placed as soon as the bandwidth-bound quantiser of x frees a slot instead of behind its whole grid
-    int prio_lo = 0, prio_hi = 0;
-    SSDI8_CUDA_CHECK(cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
-    SSDI8_CUDA_CHECK(cudaStreamCreateWithPriority(&p.s_side2, cudaStreamNonBlocking, prio_hi));
     SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
-    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming));
-    SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.join2, cudaEventDisableTiming));
     for (int s = 0; s < kStages; ++s) {
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.in_done[s], cudaEventDisableTiming));
       SSDI8_CUDA_CHECK(cudaEventCreateWithFlags(&p.cmp_done[s], cudaEventDisableTiming));
@@ -121,7 +113,7 @@ LayerWs layer_ws(const ssdi8_dims_t& d, uint8_t* base, uint32_t flags) {
 ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, const float* x, const float* B,
                           const float* C, const float* dt, const float* init, float* y, float* fin,
                           int32_t* status, int8_t* xq, int8_t* Bq, int8_t* Cq, void* ws, size_t ws_bytes,
-                          uint32_t flags, Plumbing& p, cudaStream_t st) {
+                          uint32_t flags, cudaStream_t st) {
   const int64_t T = (int64_t)d.batch * d.seqlen;
   ssdi8_fwd_args_t f = {};
   f.xq = xq; f.Bq = Bq; f.Cq = Cq;
@@ -138,27 +130,18 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
       ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C) |
         reinterpret_cast<uintptr_t>(a.s_x) | reinterpret_cast<uintptr_t>(xq) | reinterpret_cast<uintptr_t>(Bq) |
         reinterpret_cast<uintptr_t>(Cq)) & 15) == 0;
-  // Small workloads (every kernel is a few microseconds: the step is bound by launches and stream joins)
-  // take ChunkCumsum, which reads dt and A only, into the quantisers' launch.  Large ones run it on a side
-  // stream under the quantisers instead: inside one grid its long-lived blocks cost the bandwidth-bound
-  // quantiser of x more slots than the launch saves (measured at batch 8 x 2048 x 80 heads: 0.327 ms per
-  // step merged against 0.315 ms on the side stream; at 2048 x 24 heads: 0.059 against 0.070 ms).
-  const bool merged = one_launch && (int64_t)T * d.nheads * d.headdim <= ((int64_t)1 << 23);
-  if (merged) {
-    const Dims dd = make_dims(&d);
-    float *pack = nullptr, *gamma = nullptr;
-    workspace_pack_gamma(dd, ws, &pack, &gamma);
-    if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
-                                 Cq, &dd, dt, a.A, pack, gamma, st)) != SSDI8_OK)
-      return s;
-  } else {
-    SSDI8_CUDA_CHECK(cudaEventRecord(p.fork, st));
-    SSDI8_CUDA_CHECK(cudaStreamWaitEvent(p.s_side2, p.fork, 0));
-    if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, p.s_side2, false)) != SSDI8_OK) return s;
-    SSDI8_CUDA_CHECK(cudaEventRecord(p.join2, p.s_side2));
+  // ChunkCumsum (it reads dt and A only) and the quantisers need nothing of each other.  ChunkCumsum goes
+  // first and lets its successor be scheduled once its own wait for the work ahead of the layer is over;
+  // the quantisers' launch then starts without a wait and runs beside it, with the wait at the end of its
+  // last block (see quant_jobs), so that the state kernel, which waits for the quantisers' launch, has
+  // ChunkCumsum complete as well.  One stream, no events.  Measured per step, this chain / ChunkCumsum on a
+  // side stream / ChunkCumsum's blocks inside the quantisers' grid: 0.286 / 0.293 / 0.287 ms at batch
+  // 8 x 2048 x 80 heads, 0.056 / 0.062 / 0.062 ms at 2048 x 24 heads.
+  {
+    if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, st, false)) != SSDI8_OK) return s;
     if (one_launch) {
       if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
-                                   Cq, nullptr, nullptr, nullptr, nullptr, nullptr, st)) != SSDI8_OK)
+                                   Cq, st, true)) != SSDI8_OK)
         return s;
     } else {
       if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, st)) != SSDI8_OK) return s;
@@ -167,10 +150,8 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
         return s;
     }
   }
-  // the rest on the caller's stream, chained by programmatic dependent launch: the fused state kernel,
-  // ChunkBMM (needed by ChunkScan only: launched behind the state kernel, it works beside that kernel's
-  // last wave), ChunkScan
-  if (!merged) SSDI8_CUDA_CHECK(cudaStreamWaitEvent(st, p.join2, 0));
+  // the rest, chained by programmatic dependent launch: the fused state kernel, ChunkBMM (needed by ChunkScan
+  // only: launched behind the state kernel, it works beside that kernel's last wave), ChunkScan
   return fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING | SSDI8_PHASE_SCAN,
                     ws, ws_bytes, st, false);
 }
@@ -233,13 +214,10 @@ ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_
   if (workspace_bytes < need) return SSDI8_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return SSDI8_ERR_ALIGN;
   const LayerWs w = layer_ws(*dims, static_cast<uint8_t*>(workspace), flags);
-  Plumbing* p = nullptr;
-  ssdi8_status_t s = get_plumbing(&p);
-  if (s != SSDI8_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));
   return layer_step(*dims, *a, a->x, a->B, a->C, a->dt, a->init_state, a->y, a->final_state, a->status, w.xq, w.Bq,
-                    w.Cq, w.ws, w.ws_bytes, flags, *p, st);
+                    w.Cq, w.ws, w.ws_bytes, flags, st);
 }
 
 size_t ssdi8_layer_fwd_host_scratch_bytes(const ssdi8_dims_t* dims, uint32_t flags) {
@@ -315,8 +293,7 @@ ssdi8_status_t ssdi8_layer_fwd_host(const ssdi8_dims_t* dims, const ssdi8_layer_
     as.s_B = a->s_B + g0; as.s_C = a->s_C + g0; as.s_cb = a->s_cb + g0;
     const size_t fin_off = (b * H + h0) * P * N;
     s = layer_step(d1, as, sb.x, sb.B, sb.C, sb.dt, a->init_state ? a->init_state + fin_off : nullptr, sb.y,
-                   a->final_state ? sb.fin : nullptr, lo.status, sb.xq, sb.Bq, sb.Cq, lo.ws, lo.ws_bytes, flags, *p,
-                   s_cmp);
+                   a->final_state ? sb.fin : nullptr, lo.status, sb.xq, sb.Bq, sb.Cq, lo.ws, lo.ws_bytes, flags, s_cmp);
     if (s != SSDI8_OK) return s;
     SSDI8_CUDA_CHECK(cudaEventRecord(p->cmp_done[st], s_cmp));
     // outputs of the slice

@@ -28,12 +28,12 @@ ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* sca
                                int8_t* out, cudaStream_t st);
 
 // the layer's three static quantisers as one launch: x [T][D] with D step sizes, B and C [T][G N] with G
-// step sizes each (N a power of two, D and N multiples of 4).  With cs_dims non-NULL the blocks of
-// ChunkCumsum for those dimensions (dt, A -> pack, gamma; see launch_cumsum) lead the same grid.
+// step sizes each (N a power of two, D and N multiples of 4).
+// after_cumsum: the launch directly follows launch_cumsum of the same layer in the same stream and runs beside
+// it (see quant_jobs).
 ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* C, i64 T_, int D, int G, int N,
                                    const float* s_x, const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq,
-                                   int8_t* Cq, const Dims* cs_dims, const float* dt, const float* A, float* pack,
-                                   float* gamma, cudaStream_t st);
+                                   int8_t* Cq, cudaStream_t st, bool after_cumsum = false);
 
 // Per-(batch, head, chunk) pack of kPackRows rows of Q floats: cs, dt, woff, atok, wmax, lut (see
 // cumsum.cu); element (u, row, i) at pack[(u * kPackRows + row) * Q + i], u = (b*H + h)*c + k.

@@ -2,7 +2,7 @@
 // of the view in[R][Ch][I].  HBM-bound: 16-byte loads, 4-byte packed stores, every warp
 // instruction fully coalesced; absmax by per-thread running maxima, warp shuffles and
 // one order-independent atomicMax on the (non-negative) binary32 bit pattern.
-#include "cumsum_body.cuh"
+#include "kernels.h"
 
 namespace ssdi8 {
 namespace {
@@ -52,34 +52,26 @@ struct QuantJob {
   int first_block;  // of this job in the grid
   int rows;         // rows per block
 };
-// Optionally the blocks of ChunkCumsum (Algorithm 2 module 1: it reads dt and A only, so it depends on
-// nothing the quantisers write) lead the grid: they are compute-heavy and short, the quantisers are
-// bandwidth-bound, so the two share the SMs well and the layer step saves a launch.
-struct CumsumJob {
-  const float* dt; const float* A; float* pack; float* gamma;
-  Dims d;
-  int nblocks, gx;   // blocks of the job (0: none), head blocks per (batch, chunk)
-  int stride;        // grid positions 0, stride, 2 stride, ... are this job's
+struct QuantJobs {
+  QuantJob job[3]; i64 R;
+  int late_wait;   // 1: launched right behind ChunkCumsum of the same layer, which it does not depend on (see the kernel)
 };
-struct QuantJobs { QuantJob job[3]; i64 R; CumsumJob cs; };
 
 __global__ void __launch_bounds__(128, 8) quant_jobs(const QuantJobs a) {
-  extern __shared__ float cs_tile[];
   pdl_launch_dependents();
-  pdl_wait();
-  // every cs.stride-th block of the grid is a ChunkCumsum block until they are used up (they live
-  // several times longer than a quantiser block, so they are spread over the first half of the grid
-  // instead of taking all the slots at the start)
-  int blk = (int)blockIdx.x;
-  if (a.cs.nblocks > 0) {
-    const int slot = blk / a.cs.stride;
-    if (slot < a.cs.nblocks && blk - slot * a.cs.stride == 0) {
-      const int bx = slot % a.cs.gx, bk = slot / a.cs.gx;
-      cumsum_body<1>(a.cs.dt, a.cs.A, a.cs.pack, a.cs.gamma, nullptr, a.cs.d, bx, bk % a.cs.d.c, bk / a.cs.d.c, cs_tile);
-      return;
-    }
-    blk -= min(a.cs.nblocks, slot + 1);
-  }
+  // Programmatic dependent launch.  Normally: wait for the predecessor before the first global access.
+  // Launched right behind ChunkCumsum (which waits for ITS predecessor before it lets this kernel be
+  // scheduled, and whose outputs this kernel does not touch), the blocks start at once and work beside
+  // that kernel.  The wait moves to the end of the grid's last block (one waiting block is enough, and a
+  // wait in every block would keep the early ones resident until ChunkCumsum has finished): it keeps
+  // "this kernel complete" implying "ChunkCumsum complete" for the state kernel that follows, and by then
+  // it returns at once.
+  if (!a.late_wait) pdl_wait();
+  struct LateWait {
+    bool on;
+    __device__ ~LateWait() { if (on) pdl_wait(); }
+  } late_wait_at_exit{a.late_wait != 0 && blockIdx.x == gridDim.x - 1};
+  const int blk = (int)blockIdx.x;
   const int jb = blk >= a.job[2].first_block ? 2 : blk >= a.job[1].first_block ? 1 : 0;
   const QuantJob& j = a.job[jb];
   const int rel = blk - j.first_block;
@@ -255,8 +247,7 @@ ssdi8_status_t launch_quantize(const float* in, i64 R, i64 Ch, i64 I, float* sca
 
 ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* C, i64 T_, int D, int G, int N,
                                    const float* s_x, const float* s_B, const float* s_C, int8_t* xq, int8_t* Bq,
-                                   int8_t* Cq, const Dims* cs_dims, const float* dt, const float* A, float* pack,
-                                   float* gamma, cudaStream_t st) {
+                                   int8_t* Cq, cudaStream_t st, bool after_cumsum) {
   if (T_ == 0) return SSDI8_OK;
   if (T_ * D / 4 >= ((i64)1 << 31) || T_ * G * N / 4 >= ((i64)1 << 31)) return SSDI8_ERR_UNSUPPORTED;
   QuantJobs a;
@@ -273,7 +264,7 @@ ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* 
     j.gx = (j.ch4 + j.tpr - 1) / j.tpr;
     j.shift = sh;
     j.first_block = first;
-    // short slabs: blocks that live a few microseconds each, so that the other streams' kernels find
+    // short slabs: blocks that live a few microseconds each, so that a kernel running beside this one finds
     // free slots all the time (a slab is at least one full round of QROWS passes)
     j.rows = QROWS * (128 / j.tpr) < 16 ? 16 : QROWS * (128 / j.tpr);
     return first + j.gx * (int)((T_ + j.rows - 1) / j.rows);
@@ -281,17 +272,8 @@ ssdi8_status_t launch_quantize_xbc(const float* x, const float* B, const float* 
   int nb = fill(a.job[0], B, s_B, Bq, G * N, shift, 0);
   nb = fill(a.job[1], C, s_C, Cq, G * N, shift, nb);
   nb = fill(a.job[2], x, s_x, xq, D, 0, nb);
-  a.cs = CumsumJob{};
-  size_t smem = 0;
-  if (cs_dims) {   // ChunkCumsum of the same layer in the same launch, its blocks first
-    a.cs.dt = dt; a.cs.A = A; a.cs.pack = pack; a.cs.gamma = gamma; a.cs.d = *cs_dims;
-    a.cs.gx = (cs_dims->H + kCumsumHeads - 1) / kCumsumHeads;
-    a.cs.nblocks = a.cs.gx * cs_dims->c * cs_dims->b;
-    smem = cumsum_smem_bytes(cs_dims->Q, 1);
-    a.cs.stride = (nb + a.cs.nblocks) / (2 * a.cs.nblocks);
-    if (a.cs.stride < 1) a.cs.stride = 1;
-  }
-  if (launch_pdl(quant_jobs, dim3((unsigned)(nb + a.cs.nblocks)), dim3(128), smem, st, a) != cudaSuccess) return SSDI8_ERR_CUDA;
+  a.late_wait = after_cumsum ? 1 : 0;
+  if (launch_pdl(quant_jobs, dim3((unsigned)nb), dim3(128), 0, st, a) != cudaSuccess) return SSDI8_ERR_CUDA;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;
 }
