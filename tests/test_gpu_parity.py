@@ -749,6 +749,113 @@ def test_layer_fwd_back_to_back_on_one_workspace_with_alternating_inputs():
     assert np.array_equal(y.cpu().numpy(), y_a) and np.array_equal(fin.cpu().numpy(), fin_a)
 
 
+def test_layer_fwd_and_decode_steps_replay_from_a_cuda_graph():
+    """The library's calls are stream work only (no allocation, no synchronisation, no host read of a device
+    value), so a caller can capture them into a CUDA graph and replay it: the layer forward (five kernels
+    chained by programmatic dependent launch) and a run of decode steps, each replayed on new input values
+    written into the captured buffers, must equal the same calls made directly."""
+    import torch
+    from paper_2608_21952_b200 import binding as bd
+    gh = _harness()
+    cfg = SSDConfig("graph", 2, 512, 6, 64, 128, 2, 128, 0.02, 20.0, 71)
+    dims = bd.dims_of(cfg)
+    data = []
+    for seed in (71, 72):
+        t = inputs.make_prefill(cfg.replace(seed=seed))
+        data.append({k: gh.dev(t[k]) for k in ("x", "B", "C", "dt")})
+    t = inputs.make_prefill(cfg)
+    q = orc.prepare_quantized(cfg, t)
+    dv = {k: gh.dev(q[k]) for k in ("s_x", "s_B", "s_C", "s_xs", "s_cb", "s_h", "A", "D")}
+    buf = {k: torch.empty_like(v) for k, v in data[0].items()}       # the captured input buffers
+    y = torch.empty(t["x"].shape, device="cuda")
+    fin = torch.empty((cfg.batch, cfg.nheads, cfg.headdim, cfg.dstate), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = bd.make_layer_args(y=y, final_state=fin, status=status, **dv, **buf)
+    ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(dims), dtype=torch.uint8, device="cuda")
+    ref = []
+    for dset in data:   # direct calls
+        for k in buf:
+            buf[k].copy_(dset[k])
+        bd.ssdi8_layer_fwd(dims, args, ws)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref.append((y.clone(), fin.clone()))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):   # (torch asks for a warm-up on a side stream before a capture)
+        bd.ssdi8_layer_fwd(dims, args, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        bd.ssdi8_layer_fwd(dims, args, ws)
+    for rep in range(3):
+        for dset, (y0, f0) in zip(data, ref):
+            for k in buf:
+                buf[k].copy_(dset[k])
+            y.fill_(float("nan")); fin.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            assert torch.equal(y, y0) and torch.equal(fin, f0)
+
+    # decode: four steps per graph, the state carried in place from replay to replay
+    dc = CONFIGS["cfg4"].replace(batch=4, nheads=8)
+    ddims = bd.dims_of(dc)
+    prm = inputs.make_decode_params(dc)
+    nsteps = 12
+    raw = [inputs.make_decode_step(dc, s_) for s_ in range(nsteps)]
+    s_x = np.zeros(dc.channels, np.float32); s_B = np.zeros(dc.ngroups, np.float32); s_C = np.zeros(dc.ngroups, np.float32)
+    for r in raw:
+        _, s_x = orc.quantize(r["x"], dc.batch, dc.channels, 1, scale=s_x, mode=2, want_out=False)
+        _, s_B = orc.quantize(r["B"], dc.batch, dc.ngroups, dc.dstate, scale=s_B, mode=2, want_out=False)
+        _, s_C = orc.quantize(r["C"], dc.batch, dc.ngroups, dc.dstate, scale=s_C, mode=2, want_out=False)
+    codes = []
+    for r in raw:
+        codes.append(dict(xq=gh.dev(orc.quantize(r["x"], dc.batch, dc.channels, 1, scale=s_x, mode=0)[0]),
+                          Bq=gh.dev(orc.quantize(r["B"], dc.batch, dc.ngroups, dc.dstate, scale=s_B, mode=0)[0]),
+                          Cq=gh.dev(orc.quantize(r["C"], dc.batch, dc.ngroups, dc.dstate, scale=s_C, mode=0)[0]),
+                          dt=gh.dev(r["dt"])))
+    d = {k: gh.dev(v) for k, v in dict(s_x=s_x, s_B=s_B, s_C=s_C, A=prm["A"], D=prm["D"]).items()}
+    shape_state = (dc.batch, dc.nheads, dc.headdim, dc.dstate)
+
+    def step(c, state, yy):
+        bd.ssdi8_ssd_step(ddims, c["xq"], d["s_x"], c["Bq"], d["s_B"], c["Cq"], d["s_C"], c["dt"], d["A"], d["D"], None,
+                          state, yy)
+
+    state_ref = torch.zeros(shape_state, device="cuda")
+    y_ref = [torch.empty((dc.batch, dc.nheads, dc.headdim), device="cuda") for _ in range(nsteps)]
+    for i in range(nsteps):
+        step(codes[i], state_ref, y_ref[i])
+    torch.cuda.synchronize()
+    slots = [{k: torch.empty_like(v) for k, v in codes[0].items()} for _ in range(4)]
+    ys = [torch.empty_like(y_ref[0]) for _ in range(4)]
+    state = torch.zeros(shape_state, device="cuda")
+    with torch.cuda.stream(side):
+        side.wait_stream(torch.cuda.current_stream())
+        warm = torch.zeros(shape_state, device="cuda")
+        for j in range(4):
+            for k in slots[j]:
+                slots[j][k].copy_(codes[j][k])
+            step(slots[j], warm, ys[j])
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g2):
+        for j in range(4):
+            step(slots[j], state, ys[j])
+    state.zero_()
+    for i0 in range(0, nsteps, 4):
+        for j in range(4):
+            for k in slots[j]:
+                slots[j][k].copy_(codes[i0 + j][k])
+        g2.replay()
+        torch.cuda.synchronize()
+        for j in range(4):
+            assert torch.equal(ys[j], y_ref[i0 + j])
+    assert torch.equal(state, state_ref)
+
+
 def test_layer_fwd_host_rejects_a_short_scratch():
     import torch
     from paper_2608_21952_b200 import binding as bd
