@@ -27,7 +27,11 @@ __device__ __forceinline__ float exp32(float x) {
   const float LOG2E = __uint_as_float(0x3FB8AA3Bu);
   const float LN2_HI = __uint_as_float(0x3F317200u);
   const float LN2_LO = __uint_as_float(0x35BFBE8Eu);
-  float n = rintf(__fmul_rn(x, LOG2E));
+  // n = rint(fmul(x, LOG2E)): |x LOG2E| < 2^22, so adding and subtracting 1.5 * 2^23 rounds to the nearest
+  // integer, ties to even, exactly as rint does, and leaves n in the low mantissa bits of the sum (both
+  // conversions stay off the conversion pipe)
+  const float nm = __fadd_rn(__fmul_rn(x, LOG2E), 12582912.0f);
+  const float n = __fadd_rn(nm, -12582912.0f);
   float r = __fmaf_rn(n, -LN2_HI, x);
   r = __fmaf_rn(n, -LN2_LO, r);
   float p = __uint_as_float(0x39500D01u);                 // 1/5040
@@ -38,7 +42,7 @@ __device__ __forceinline__ float exp32(float x) {
   p = __fmaf_rn(p, r, 0.5f);
   p = __fmaf_rn(p, r, 1.0f);
   p = __fmaf_rn(p, r, 1.0f);
-  return __uint_as_float(__float_as_uint(p) + ((uint32_t)__float2int_rn(n) << 23));
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(nm) << 23));   // bits(nm) = 0x4B400000 + n: the shift keeps n
 }
 
 // ---- conversions that stay off the quarter-rate conversion pipe (all exact)

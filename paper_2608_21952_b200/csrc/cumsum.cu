@@ -11,7 +11,7 @@ namespace {
 // leave fewer of them to overlap.)
 constexpr int kChunksPerBlock = 1;
 
-template <bool SOFTPLUS>
+template <bool SOFTPLUS, bool PRE>
 __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ dt,
                                                      const float* __restrict__ A,
                                                      float* __restrict__ pack,
@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(256) cumsum_kernel(const float* __restrict__ d
   // that precedes this kernel in the stream must have completed.
   pdl_wait();
   pdl_launch_dependents();
-  cumsum_body<kChunksPerBlock, SOFTPLUS>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias);
+  cumsum_body<kChunksPerBlock, SOFTPLUS, PRE>(dt, A, pack, gamma, tap_cs, d, blockIdx.x, blockIdx.y, blockIdx.z, tile, dt_bias);
 }
 
 // dt = softplus(dt_raw + dt_bias[h]) alone (for callers that calibrate on the positive time step)
@@ -52,13 +52,19 @@ ssdi8_status_t launch_softplus_dt(const float* dt_raw, const float* dt_bias, flo
 ssdi8_status_t launch_cumsum(const Dims& d, const float* dt, const float* A, float* pack,
                              float* gamma, float* tap_cs, cudaStream_t st, const float* dt_bias, bool softplus) {
   dim3 grid((d.H + kCumsumHeads - 1) / kCumsumHeads, (d.c + kChunksPerBlock - 1) / kChunksPerBlock, d.b);
-  const size_t smem = cumsum_smem_bytes(d.Q, kChunksPerBlock);
+  // a grid that leaves SMs empty is waited for block by block: the variant with the shorter chain
+  int dev = 0, sms = 0;
+  SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
+  SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const bool pre = (long long)grid.x * grid.y * grid.z <= sms;
+  const size_t smem = cumsum_smem_bytes(d.Q, kChunksPerBlock, pre);
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     return launch_pdl(kernel, grid, dim3(256), smem, st, dt, A, pack, gamma, tap_cs, d, dt_bias) == cudaSuccess
                ? SSDI8_OK : SSDI8_ERR_CUDA;
   };
-  const ssdi8_status_t ls = softplus ? launch(cumsum_kernel<true>) : launch(cumsum_kernel<false>);
+  const ssdi8_status_t ls = softplus ? (pre ? launch(cumsum_kernel<true, true>) : launch(cumsum_kernel<true, false>))
+                                     : (pre ? launch(cumsum_kernel<false, true>) : launch(cumsum_kernel<false, false>));
   if (ls != SSDI8_OK) return ls;
   SSDI8_LAUNCH_CHECK();
   return SSDI8_OK;

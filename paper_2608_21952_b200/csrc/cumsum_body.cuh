@@ -26,9 +26,10 @@ namespace ssdi8 {
 
 constexpr int kCumsumHeads = 8;  // heads per block
 
-// shared memory of a block: dt and cs rows of its 8 KC (head, chunk) units, their flags and bounds
-__host__ __device__ inline size_t cumsum_smem_bytes(int Q, int KC) {
-  return sizeof(float) * (size_t)(kCumsumHeads * KC) * (2 * (size_t)(Q + 1) + 16);
+// shared memory of a block: dt and cs rows of its 8 KC (head, chunk) units, their flags and bounds, and the
+// binary64 increments dt A of the scan
+__host__ __device__ inline size_t cumsum_smem_bytes(int Q, int KC, bool pre = false) {
+  return sizeof(float) * (size_t)(kCumsumHeads * KC) * (2 * (size_t)(Q + 1) + 16 + (pre ? 2 * (size_t)Q + 2 : 0));
 }
 
 // One block's work: heads 8 bx .. and chunks KC kx .. of batch element b.  Any whole number of warps
@@ -36,7 +37,12 @@ __host__ __device__ inline size_t cumsum_smem_bytes(int Q, int KC) {
 // SOFTPLUS: dt holds the raw time step and dt = softplus(dt + dt_bias[h]) (dt_bias may be NULL)
 // is applied as the values are staged (Algorithm 2 module 1 starts there).
 // (a template parameter: the binary64 softplus costs registers, and the plain instance must keep its occupancy)
-template <int KC, bool SOFTPLUS = false>
+// PRE: the scan's binary64 increments dt A are formed by all threads while dt is staged and kept in shared
+// memory, which leaves the sequential part one addition per token.  That shortens a block's chain (what a
+// small grid waits for: 0.0164 against 0.0184 ms at 2048 x 24 heads) and costs shared memory and binary64 work
+// that a full device has no room for (0.027 against 0.025 ms at batch 8 x 2048 x 80 heads), so the launcher
+// takes it for grids that leave SMs empty only; `tile` is then cumsum_smem_bytes(Q, KC, true).
+template <int KC, bool SOFTPLUS = false, bool PRE = false>
 __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const float* __restrict__ A,
                                             float* __restrict__ pack, float* __restrict__ gamma,
                                             float* __restrict__ tap_cs, const Dims& d, int bx, int kx, int b,
@@ -47,10 +53,17 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
   float* dts = tile;                   // [NU][Q + 1]; entry Q of a row: 1 if cs is non-increasing over the chunk
   float* css = tile + NU * ld;         // [NU][Q + 1]
   float* wmx = tile + 2 * NU * ld;     // [NU][16]: 127 max|woff| per 16-token sub-block
+  // [NU][Q] binary64 increments (double)dt (double)A, exact; 8-byte aligned: 2 NU (Q + 1) + 16 NU floats precede it
+  double* inc = reinterpret_cast<double*>(tile + 2 * NU * ld + 16 * NU);
   const int h0 = bx * CH, k0 = kx * KC;
   const int nh = min(CH, d.H - h0), nk = min(KC, d.c - k0);
   const i64 t0 = (i64)b * d.L + (i64)k0 * Q;
   const int ntok = nk * Q;             // tokens of the block's chunks (contiguous in time)
+  // entry Q of a dt row: 1 until a token is met whose increment dt A is positive
+  if (PRE) {
+    if (threadIdx.x < NU) dts[threadIdx.x * ld + Q] = 1.0f;
+    __syncthreads();
+  }
   // (all loads of a round of 8 before the first store: the loads are the latency of this phase)
   for (int e0 = threadIdx.x; e0 < ntok * CH; e0 += 8 * blockDim.x) {
     float v[8];
@@ -64,40 +77,63 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + u * blockDim.x;
       const int t = e / CH, hh = e % CH;
-      if (e < ntok * CH && hh < nh)
-        dts[(hh * KC + (t >> lq)) * ld + (t & (Q - 1))] =
-            SOFTPLUS ? softplus_dt(v[u], dt_bias ? __ldg(dt_bias + h0 + hh) : 0.f) : v[u];
+      if (e < ntok * CH && hh < nh) {
+        const float dv = SOFTPLUS ? softplus_dt(v[u], dt_bias ? __ldg(dt_bias + h0 + hh) : 0.f) : v[u];
+        const float af = PRE ? __ldg(A + h0 + hh) : 0.f;
+        const int un = hh * KC + (t >> lq), i = t & (Q - 1);
+        dts[un * ld + i] = dv;
+        // the scan's increment, formed here by all threads: the product of two binary32 numbers is exact in
+        // binary64, so only the additions are left to the sequential part
+        if (PRE) {
+          inc[un * Q + i] = (double)dv * (double)af;
+          if ((af > 0.f && dv > 0.f) || (af < 0.f && dv < 0.f)) dts[un * ld + Q] = 0.0f;
+        }
+      }
     }
   }
   __syncthreads();
   if (threadIdx.x < NU) {
     const int u = threadIdx.x, hh = u / KC, kk = u % KC;
     if (hh < nh && kk < nk) {
-      const double a = (double)A[h0 + hh];
       double acc = 0.0;
       float last = 0.f;
-      float dmin = 0.f, dmax = 0.f;  // every increment dt A <= 0  <=>  no dt has the sign of A
-      // Q is a multiple of 8: loads and products (exact in binary64) of 8 tokens are independent,
-      // only the additions form the chain
-      for (int i0 = 0; i0 < Q; i0 += 8) {
-        float dv[8];
-        double pr[8];
+      if (PRE) {
+        // Q is a multiple of 8: the loads of 8 increments are independent, only the additions form the chain
+        for (int i0 = 0; i0 < Q; i0 += 8) {
+          double pr[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          dv[j] = dts[u * ld + i0 + j];
-          pr[j] = (double)dv[j] * a;
-          dmin = fminf(dmin, dv[j]);
-          dmax = fmaxf(dmax, dv[j]);
-        }
+          for (int j = 0; j < 8; ++j) pr[j] = inc[u * Q + i0 + j];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          acc += pr[j];
-          last = (float)acc;
-          css[u * ld + i0 + j] = last;
+          for (int j = 0; j < 8; ++j) {
+            acc += pr[j];
+            last = (float)acc;
+            css[u * ld + i0 + j] = last;
+          }
         }
+      } else {
+        const double a = (double)A[h0 + hh];
+        float dmin = 0.f, dmax = 0.f;  // every increment dt A <= 0  <=>  no dt has the sign of A
+        // loads and products (exact in binary64) of 8 tokens are independent, only the additions form the chain
+        for (int i0 = 0; i0 < Q; i0 += 8) {
+          float dv[8];
+          double pr[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            dv[j] = dts[u * ld + i0 + j];
+            pr[j] = (double)dv[j] * a;
+            dmin = fminf(dmin, dv[j]);
+            dmax = fmaxf(dmax, dv[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            acc += pr[j];
+            last = (float)acc;
+            css[u * ld + i0 + j] = last;
+          }
+        }
+        const bool mono = a > 0.0 ? dmax <= 0.f : (a < 0.0 ? dmin >= 0.f : true);
+        dts[u * ld + Q] = mono ? 1.0f : 0.0f;
       }
-      const bool mono = a > 0.0 ? dmax <= 0.f : (a < 0.0 ? dmin >= 0.f : true);
-      dts[u * ld + Q] = mono ? 1.0f : 0.0f;
       gamma[((i64)b * d.H + h0 + hh) * d.c + k0 + kk] = exp32(last);
     }
   }
