@@ -272,7 +272,7 @@ class Layer:
 
     def step(self):
         """One pass of the hot path through the one-call entry point: the three Eq. 1 quantisers and
-        the layer forward (inside, the modules that do not need xq run under the quantiser of x)."""
+        the layer forward (inside, ChunkCumsum runs beside the quantisers and ChunkBMM beside the state kernel)."""
         if self.layer_args is None:
             bd, torch = self.bd, self.torch
             self.layer_ws = torch.empty(bd.ssdi8_layer_fwd_workspace_bytes(self.dims), dtype=torch.uint8,
