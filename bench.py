@@ -52,7 +52,7 @@ PAPER_TOKENS_PER_S = {"cfg2": 16384 / 4.481e-3}
 # byte counts and a pipe utilisation, which do not depend on the clock): DRAM bytes per launch
 # (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel and of the decode step kernel,
 # and the tensor-pipe active share of the scan kernel, each with the summary file it comes from.
-NCU_SCAN = {"cfg2": {"traffic": 441.0e6, "tensor_active_pct": 8.5,
+NCU_SCAN = {"cfg2": {"traffic": 435.5e6, "tensor_active_pct": 8.8,
                      "source": "profiles/chunk_scan_cfg2_ncu_full.md"}}
 NCU_TRAFFIC_BYTES_DECODE = 276.6e6  # ssd_step_kernel at cfg4: profiles/launch_list_bench_cfg2.md
 INT8_NOMINAL_TOPS = 4500.0          # dense INT8 figure of the B200 data sheet
