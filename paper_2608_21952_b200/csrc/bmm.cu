@@ -147,7 +147,10 @@ bmm_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ CUtenso
     tc_fence_after();
     tmem_dealloc(tmem, 256);
   }
-  if (a.late_wait) pdl_wait();
+  // (in the grid's last block only: one waiting block is enough for "this kernel complete" to imply "the state
+  // kernel complete", and a wait in every block would keep the blocks of the first wave resident, and the rest
+  // of a larger grid unscheduled, until the state kernel has finished)
+  if (a.late_wait && blockIdx.x == gridDim.x - 1) pdl_wait();
 }
 
 }  // namespace
