@@ -27,12 +27,14 @@
 #include <type_traits>
 
 #include "kernels.h"
+#include "scan_common.cuh"
 #include "sm100.cuh"
 
 namespace ssdi8 {
 namespace {
 
 using namespace sm100;
+using namespace scan;
 
 struct ScanArgs {
   const float* s_x; const float* s_C; const float* s_cb; const float* s_h;
@@ -41,16 +43,13 @@ struct ScanArgs {
   int32_t* status;
   ScanTaps taps;
   Dims d;
-  int units;        // (batch, chunk, head) units of the launch; CTA j takes units j, j + grid, j + 2 grid, ...
-  int dh, dk, db;   // the grid size as a step (db, dk, dh) in (batch, chunk, head) mixed radix
-  int hpg;          // heads per group
+  UnitWalk w;       // CTA j takes units j, j + grid, j + 2 grid, ...
 };
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
 constexpr int kMaskWarp0 = 4, kGroupWarps = 8;
 constexpr int kEpiWarp0 = 20, kEpiWarps = 8, kEpiGroupWarps = 4;
 constexpr uint32_t kTmemCols = 512;  // four accumulator pairs: acc_off at 128 a, acc_diag at 128 a + 64
-constexpr uint32_t PANEL = 16384;    // [128][128] int8
 // shared memory (bytes, from a 1024-byte aligned base)
 constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1-panel buffers
 constexpr uint32_t OFF_C = 98304;       // [128][N]
@@ -67,30 +66,13 @@ constexpr uint32_t OFF_YST = OFF_ROW + 8 * ROW_BYTES;  // 8 warps x [32][128 B] 
 constexpr uint32_t OFF_BAR = OFF_YST + 32768;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
-__device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
-  return OFF_CB + (idx < 2 ? (uint32_t)idx * 32768u : 65536u + (uint32_t)(idx - 2) * 16384u);
-}
-// which CBq buffer tile n of this CTA uses: with two tiles per chunk the second (two panels)
-// alternates between buffers 0,1 and the first (one panel) between 2,3; otherwise all four rotate
-__device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
-  return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
-}
-
-// the xq buffer of tile n and the phase of its barriers: one buffer per chunk
-__device__ __forceinline__ int x_index(int n, int ntpu) { return ntpu == 1 ? (n & 1) : ((n >> 1) & 1); }
-__device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 ? ((n >> 1) & 1) : ((n >> 2) & 1); }
+__device__ __forceinline__ uint32_t cb_offset(int idx) { return scan::cb_offset(OFF_CB, idx); }
 
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_CH_FREE = 13, B_X_FULL = 14, B_X_FREE = 16,
        B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 30, B_ROW_FULL = 34, B_ROW_FREE = 42,
        B_COUNT = 50 };
 
 
-// two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
-__device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
-  const float2 m = make_float2(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)),
-                               __uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7651u + k)));
-  return __fadd2_rn(m, make_float2(-kMagicIn, -kMagicIn));
-}
 // four codes rn(a g), the exact product rounded once to the nearest integer (ties to even): for
 // |a g| < 2^22 that integer sits in the low bits of fma(a, g, 1.5 * 2^23); callers guarantee
 // |a g| < 127.5.  (One fused operation by definition: a packed multiply followed by a packed add of
@@ -101,54 +83,6 @@ __device__ __forceinline__ uint32_t pack4_rn_product(float2 a, float2 b, float2 
   const float2 rb = __ffma2_rn(b, g, make_float2(kMagicOut, kMagicOut));
   return __byte_perm(__byte_perm(__float_as_uint(ra.x), __float_as_uint(ra.y), 0x0040u),
                      __byte_perm(__float_as_uint(rb.x), __float_as_uint(rb.y), 0x0040u), 0x5410u);
-}
-
-struct Tile {
-  int b, k, h, it, KJ;
-  i64 tok0, unit;              // tok0 = b L + k Q, unit = (b*H + h)*c + k
-};
-// A CTA walks the units u = blockIdx.x + i gridDim.x (head fastest, then chunk, then batch), both tiles of
-// a unit in turn.  The CTAs of the grid therefore work on neighbouring heads of the same tokens at the same
-// time: the rows of x they read and the rows of y they write (256 bytes per token and head, the heads of a
-// token adjacent in memory) fill whole DRAM pages while they are in L2, and the Cq / CBq tiles of a group
-// are fetched once for all its heads.  (With consecutive units per CTA instead, a token's heads were
-// written minutes of kernel time apart and the writes reached DRAM in 256-byte pieces: measured on a copy
-// of the kernel with its arithmetic compiled out, 0.125 against 0.115 ms.)
-// The step to the CTA's next unit, without divisions (every role walks the tiles, so this is inlined many
-// times and runs once per tile on each role's critical path).
-__device__ __forceinline__ void next_unit(Tile& x, const ScanArgs& a) {
-  x.h += a.dh;
-  x.k += a.dk;
-  x.b += a.db;
-  if (x.h >= a.d.H) { x.h -= a.d.H; ++x.k; }
-  if (x.k >= a.d.c) { x.k -= a.d.c; ++x.b; }
-  x.tok0 = ((i64)x.b * a.d.c + x.k) * a.d.Q;      // L = c Q
-  x.unit = ((i64)x.b * a.d.H + x.h) * a.d.c + x.k;
-}
-__device__ __forceinline__ void next_tile(Tile& x, const ScanArgs& a, int TM, int ntpu) {
-  if (++x.it == ntpu) {
-    x.it = 0;
-    next_unit(x, a);
-  }
-  x.KJ = (x.it + 1) * TM;
-}
-// the first tile of the CTA's next unit
-__device__ __forceinline__ void next_head(Tile& x, const ScanArgs& a, int TM, int ntpu) {
-  x.it = ntpu - 1;
-  next_tile(x, a, TM, ntpu);
-}
-// first tile of a CTA (unit u): computed once, by one thread, and handed to the roles through shared memory
-__device__ __forceinline__ Tile decode_unit(int u, const ScanArgs& a, int TM) {
-  const Dims& d = a.d;
-  Tile x;
-  x.it = 0;
-  x.h = u % d.H; u /= d.H;
-  x.k = u % d.c;
-  x.b = u / d.c;
-  x.KJ = TM;
-  x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
-  x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
-  return x;
 }
 
 // ---- the masked operand of one tile, in place over CBq.  Two threads per output row, in
@@ -347,7 +281,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
   const uint32_t RBN = N, RBQ = BIGQ ? 128u : (uint32_t)Q;   // row bytes of the N-contracted and Q-contracted tiles
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // tiles of this CTA: its units blockIdx.x, blockIdx.x + gridDim.x, ..., ntpu tiles each
-  const int n_end = (((a.units - 1 - (int)blockIdx.x) / (int)gridDim.x) + 1) * ntpu;
+  const int n_end = tiles_of_cta(a.w, (int)blockIdx.x, (int)gridDim.x, ntpu);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   Tile* first_tile = reinterpret_cast<Tile*>(bars + B_COUNT + 2);   // 416 .. 464 of the 512 bytes
@@ -375,7 +309,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     fence_mbar_init();
     tma_prefetch_desc(&tm_C); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_x);
     tma_prefetch_desc(&tm_cb); tma_prefetch_desc(&tm_y);
-    *first_tile = decode_unit((int)blockIdx.x, a, TM);
+    *first_tile = decode_unit((int)blockIdx.x, d, TM);
   }
   pdl_launch_dependents();
   if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
@@ -390,8 +324,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     if (lane == 0) {
       Tile t = *first_tile;
 #pragma unroll 1
-      for (int n = 0; n < n_end; ++n, next_tile(t, a, TM, ntpu)) {
-        const int tg = t.h / a.hpg;   // group of the head (one division per tile in this one thread)
+      for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
+        const int tg = t.h / a.w.hpg;   // group of the head (one division per tile in this one thread)
         const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
         const uint32_t ph4 = (n >> 2) & 1, ph3 = (n >> 2) & 1;
         mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
@@ -427,10 +361,10 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     if (lane == 0) {
       Tile t = *first_tile;
 #pragma unroll 1
-      for (int n = 0; n < n_end; ++n, next_tile(t, a, TM, ntpu)) {
+      for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
         mbar_wait_relaxed(&bars[B_CH_FREE], (n & 1) ^ 1, a.status);
         mbar_expect_tx(&bars[B_CH_FULL], (uint32_t)(TM * N + 64 * N));
-        tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.h / a.hpg, (int)(t.tok0 + t.it * TM));
+        tma_load_3d(smem + OFF_C, &tm_C, &bars[B_CH_FULL], 0, t.h / a.w.hpg, (int)(t.tok0 + t.it * TM));
         tma_load_2d(smem + OFF_H, &tm_h, &bars[B_CH_FULL], 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
       }
     }
@@ -439,7 +373,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     if (lane == 0) {
       Tile t = *first_tile;
 #pragma unroll 1
-      for (int n = 0; n < n_end; ++n, next_tile(t, a, TM, ntpu)) {
+      for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
         if (t.it != 0) continue;   // the chunk's rows were loaded with its first tile
         const int xs = x_index(n, ntpu);
         mbar_wait_relaxed(&bars[B_X_FREE + xs], x_phase(n, ntpu) ^ 1, a.status);
@@ -499,7 +433,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     const int g = (warp - kMaskWarp0) / kGroupWarps;
     const int w = (warp - kMaskWarp0) % kGroupWarps;
     Tile t = *first_tile;
-    if (g) next_head(t, a, TM, ntpu);
+    if (g) next_head(t, d, a.w, TM, ntpu);
 #pragma unroll 1
     for (int n = g * ntpu; n < n_end; ++n) {
       const int ci = cb_index(n, t.it, ntpu), t3 = n & 3, r8 = n & 7;
@@ -521,8 +455,8 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
         t.it = 1;
         t.KJ = 2 * TM;
       } else {                 // skip the other group's chunk (or tile)
-        next_head(t, a, TM, ntpu);
-        next_head(t, a, TM, ntpu);
+        next_head(t, d, a.w, TM, ntpu);
+        next_head(t, d, a.w, TM, ntpu);
         n += ntpu;
       }
     }
@@ -537,7 +471,7 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
     uint8_t* srow = ystage + lane * 128;
     constexpr int PPR = YT ? 8 : 4;         // 8-column pieces per round (128 bytes of y per row)
     Tile t = *first_tile;
-    if (eg) next_tile(t, a, TM, ntpu);
+    if (eg) next_tile(t, d, a.w, TM, ntpu);
 #pragma unroll 1
     for (int n = eg; n < n_end; n += 2) {
       const int ci = cb_index(n, t.it, ntpu), a4 = n & 3, xs = x_index(n, ntpu);
@@ -638,12 +572,12 @@ chunk_scan_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constant__ 
       }
       if (ntpu == 2) {   // the same tile of the next head
         const int it = t.it;
-        next_head(t, a, TM, ntpu);
+        next_head(t, d, a.w, TM, ntpu);
         t.it = it;
         t.KJ = (it + 1) * TM;
       } else {
-        next_tile(t, a, TM, ntpu);
-        next_tile(t, a, TM, ntpu);
+        next_tile(t, d, a.w, TM, ntpu);
+        next_tile(t, d, a.w, TM, ntpu);
       }
     }
     if (lane == 3) tma_store_wait_read();
@@ -702,22 +636,10 @@ ssdi8_status_t launch_chunk_scan(const Dims& d, const int8_t* xq, const int8_t* 
   int dev = 0, sms = 0;
   SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
   SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const i64 units64 = (i64)d.b * d.c * d.H;
-  if (units64 * (d.Q / TM) >= ((i64)1 << 30)) return SSDI8_ERR_SHAPE;
-  const int units = (int)units64;
-  // One CTA per SM; when there are more units than SMs, the grid size is taken coprime with the number of
-  // heads (a few CTAs fewer at most), so that the heads a CTA meets, h0 + i * grid mod H, run through all
-  // heads instead of a fraction of them: the mask's work differs from head to head with the decay rate, and
-  // the kernel ends with its slowest CTA.
-  int grid_i = units < sms ? units : sms;
-  if (units > sms) {
-    auto gcd = [](int x, int y) { while (y) { const int t = x % y; x = y; y = t; } return x; };
-    for (int gtry = grid_i; gtry > grid_i - 8 && gtry > 1; --gtry)
-      if (gcd(gtry, d.H) == 1) { grid_i = gtry; break; }
-  }
-  // the grid size as a step in (batch, chunk, head) mixed radix, head fastest
-  const int dh = grid_i % d.H, dk = (grid_i / d.H) % d.c, db = grid_i / d.H / d.c;
-  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, static_cast<uint8_t*>(y), status, taps, d, units, dh, dk, db, d.H / d.G};
+  UnitWalk walk;
+  int grid_i = 0;
+  if (!make_unit_walk(d, TM, sms, &walk, &grid_i)) return SSDI8_ERR_SHAPE;
+  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, static_cast<uint8_t*>(y), status, taps, d, walk};
   const size_t smem = SMEM_BYTES + 1024;
   const unsigned grid = (unsigned)grid_i;
   const bool tp = taps.acc_off || taps.rowmax || taps.Mq || taps.acc_diag;

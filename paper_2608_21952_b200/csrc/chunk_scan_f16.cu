@@ -16,7 +16,8 @@
 //    ChunkScan1 stays an int8 MMA;
 //  * tensor memory: two accumulator pairs (INT32 C h, FP32 M16 x) and two operand buffers, 512 columns.
 // One factor per 16-column sub-block as in chunk_scan.cu: own sub-block by the running product of
-// per-token decays, earlier ones woff_j f with f = exp32(cs_i - cs_je); a sub-block whose bound
+// per-token decays, earlier ones woff_j f with f the row's decay to the end of the sub-block before its own
+// times ChunkCumsum's tabulated block-to-block decay; a sub-block whose bound
 // says every |value| < 2^-25 (half of the smallest FP16 subnormal) is zero, and so is every
 // farther one where cs does not increase (p127, see cumsum.cu).  No multicast; bounded waits.
 #include <cuda_bf16.h>
@@ -25,26 +26,27 @@
 #include <type_traits>
 
 #include "kernels.h"
+#include "scan_common.cuh"
 #include "sm100.cuh"
 
 namespace ssdi8 {
 namespace {
 
 using namespace sm100;
+using namespace scan;
 
 struct ScanArgs {
   const float* s_x; const float* s_C; const float* s_cb; const float* s_h;
   const float* pack; const float* D; const float* corr;
   int32_t* status;
   Dims d;
-  int ntiles, per_cta;
+  UnitWalk w;       // CTA j takes units j, j + grid, j + 2 grid, ...
 };
 
 constexpr int kWarps = 28, kThreads = kWarps * 32;
 constexpr int kMaskWarp0 = 4, kGroupWarps = 8;
 constexpr int kEpiWarp0 = 20, kEpiWarps = 8;
 constexpr uint32_t kTmemCols = 512;  // accumulator pair a at 128 a (+0 INT32 C h, +64 FP32 M16 x); operand buffer g at 256 + 128 g
-constexpr uint32_t PANEL = 16384;    // [128][128] int8
 // shared memory (bytes, from a 1024-byte aligned base)
 constexpr uint32_t OFF_CB = 0;          // ring of 4: two 2-panel buffers, two 1-panel buffers
 constexpr uint32_t OFF_C = 98304;       // [128][N]
@@ -59,16 +61,7 @@ constexpr uint32_t OFF_YST = OFF_TOK + 4 * TOK_BYTES;  // 8 warps x [32][64 B] y
 constexpr uint32_t OFF_BAR = OFF_YST + 16384;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 512;
 
-__device__ __forceinline__ uint32_t cb_offset(int idx) {  // buffers 0,1: 32 KB; buffers 2,3: 16 KB
-  return OFF_CB + (idx < 2 ? (uint32_t)idx * 32768u : 65536u + (uint32_t)(idx - 2) * 16384u);
-}
-__device__ __forceinline__ int cb_index(int n, int it, int ntpu) {
-  return ntpu == 1 ? (n & 3) : ((it ? 0 : 2) + ((n >> 1) & 1));
-}
-
-// the x buffer of tile n and the phase of its barriers: one buffer per chunk, shared by its tiles
-__device__ __forceinline__ int x_index(int n, int ntpu) { return ntpu == 1 ? (n & 1) : ((n >> 1) & 1); }
-__device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 ? ((n >> 1) & 1) : ((n >> 2) & 1); }
+__device__ __forceinline__ uint32_t cb_offset(int idx) { return scan::cb_offset(OFF_CB, idx); }
 
 // The Cq/hq buffer is single, but its barriers come in pairs indexed by the parity of the tile: the two
 // MMA issuers take alternate tiles, and a barrier polled by parity must be seen phase by phase by its
@@ -76,12 +69,6 @@ __device__ __forceinline__ uint32_t x_phase(int n, int ntpu) { return ntpu == 1 
 enum { B_CB_FULL = 0, B_CB_FREE = 4, B_MQ = 8, B_CH_FULL = 12, B_X_FULL = 14, B_X_FREE = 16,
        B_TOK_FULL = 18, B_TOK_FREE = 22, B_ACC = 26, B_ACC_FREE = 28, B_AFREE = 30, B_CH_FREE = 32, B_X_RAW = 34, B_COUNT = 36 };
 
-// two int8 of w_xor (= word ^ 0x80808080), bytes k and k+1, as exact floats
-__device__ __forceinline__ float2 unpack2(uint32_t w_xor, int k) {
-  const float2 m = make_float2(__uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7650u + k)),
-                               __uint_as_float(__byte_perm(w_xor, 0x4B400000u, 0x7651u + k)));
-  return __fadd2_rn(m, make_float2(-kMagicIn, -kMagicIn));
-}
 __device__ __forceinline__ uint32_t half2_bits(float2 v) {
   const __half2 h = __floats2half2_rn(v.x, v.y);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -105,37 +92,6 @@ __device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uin
 // instruction descriptor for kind::f16: FP16 A (K-major, in tensor memory) and B, FP32 accumulator
 __host__ __device__ constexpr uint32_t idesc_f16(int M, int N, int b_mn_major) {
   return (1u << 4) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-struct Tile {
-  int b, k, h, g, it, KJ;
-  i64 tok0, unit;  // unit = (b*H + h)*c + k
-};
-__device__ __forceinline__ void next_tile(Tile& x, const Dims& d, int TM, int ntpu) {
-  if (++x.it == ntpu) {
-    x.it = 0;
-    if (++x.h == d.H) {
-      x.h = 0;
-      if (++x.k == d.c) { x.k = 0; ++x.b; }
-    }
-    x.g = x.h / (d.H / d.G);
-    x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
-    x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
-  }
-  x.KJ = (x.it + 1) * TM;
-}
-__device__ __forceinline__ Tile decode_tile(int t, const Dims& d, int TM, int ntpu) {
-  Tile x;
-  x.it = t % ntpu;
-  int u = t / ntpu;
-  x.h = u % d.H; u /= d.H;
-  x.k = u % d.c;
-  x.b = u / d.c;
-  x.g = x.h / (d.H / d.G);
-  x.KJ = (x.it + 1) * TM;
-  x.tok0 = (i64)x.b * d.L + (i64)x.k * d.Q;
-  x.unit = ((i64)x.b * d.H + x.h) * d.c + x.k;
-  return x;
 }
 
 // ---- the FP16 operand of one tile, written to tensor memory.  A warp owns 32 rows (lane = row =
@@ -165,7 +121,7 @@ __device__ __forceinline__ void mask_tile_f16(const uint8_t* sCB, const float* t
     return reinterpret_cast<const uint4*>(rowbase + pn * PANEL + ((cc ^ rx) << 4));
   };
   const float cs_i = row_ok ? cs_s[i] : 0.f;
-  const float scb = a.s_cb[t.g];
+  const float scb = a.s_cb[t.h / a.w.hpg];
   // decay to an earlier chunk c: the row's decay to the end of the chunk before its own, times the
   // tabulated decay from there to the end of chunk c (1 for c = I16 - 1)
   const float ri_dec = I16 > 0 ? exp32(__fsub_rn(cs_i, cs_s[I16 * 16 - 1])) : 0.f;
@@ -282,8 +238,8 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   const int ntpu = BIGQ ? Q / 128 : 1;     // tiles per (batch, chunk, head)
   const uint32_t RBN = N, RBQ = BIGQ ? 128u : (uint32_t)Q;        // row bytes of the N-contracted and Q-contracted int8 tiles
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int t_begin = blockIdx.x * a.per_cta;
-  const int t_end = min(a.ntiles, t_begin + a.per_cta);
+  // tiles of this CTA: its units blockIdx.x, blockIdx.x + gridDim.x, ..., ntpu tiles each
+  const int n_end = tiles_of_cta(a.w, (int)blockIdx.x, (int)gridDim.x, ntpu);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
 
@@ -323,20 +279,21 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     // ------------------------------------------------------------ TMA producer: CBq panels, scalar pack, and the
     // int8 xq rows of each chunk (the mask group that takes the chunk expands them to FP16)
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      Tile t = decode_unit((int)blockIdx.x, d, TM);
       {   // the int8 xq rows of the first two chunks (both buffers are free); later requests come from the
           // epilogue warps, the moment they have finished with a buffer
         Tile tn = t;
-        for (int kc = 0; kc < 2 && t_begin + kc * ntpu < t_end; ++kc) {
+        for (int kc = 0; kc < 2 && kc * ntpu < n_end; ++kc) {
           uint8_t* xb = smem + OFF_X + kc * X_BYTES;
           mbar_expect_tx(&bars[B_X_RAW + kc], (uint32_t)(Q * 64));
           for (int j0 = 0; j0 < Q; j0 += TM)
             tma_load_3d(xb + Q * 64 + j0 * 64, &tm_x, &bars[B_X_RAW + kc], 0, tn.h, (int)(tn.tok0 + j0));
-          for (int i = 0; i < ntpu; ++i) next_tile(tn, d, TM, ntpu);
+          next_head(tn, d, a.w, TM, ntpu);
         }
       }
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
+        const int tg = t.h / a.w.hpg;   // group of the head
         const int ci = cb_index(n, t.it, ntpu), t3 = n & 3;
         const uint32_t ph4 = (n >> 2) & 1;
         mbar_wait_relaxed(&bars[B_CB_FREE + ci], ph4 ^ 1, a.status);
@@ -344,14 +301,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
         mbar_expect_tx(&bars[B_CB_FULL + ci], (uint32_t)(npanel * TM * RBQ));
         for (int pn = 0; pn < npanel; ++pn)
           tma_load_2d(smem + cb_offset(ci) + pn * PANEL, &tm_cb, &bars[B_CB_FULL + ci], pn * (int)RBQ,
-                      (int)((((i64)t.b * d.c + t.k) * d.G + t.g) * Q + t.it * TM));
+                      (int)((((i64)t.b * d.c + t.k) * d.G + tg) * Q + t.it * TM));
         mbar_wait_relaxed(&bars[B_TOK_FREE + t3], ph4 ^ 1, a.status);
         // the scalar pack of the chunk and the head's per-column vectors (the epilogue reads them once per
         // 8-column piece: from global memory each read would be a long-latency load in its chain)
         uint8_t* slot = smem + OFF_TOK + t3 * TOK_BYTES;
         {   // the tile's scalars, fetched here so that their latency is not in the epilogue's chain
           float* sc = reinterpret_cast<float*>(slot + TOK_SCAL);
-          sc[0] = a.s_C[t.g];
+          sc[0] = a.s_C[tg];
           sc[1] = a.D ? a.D[t.h] : 0.f;
         }
         mbar_expect_tx(&bars[B_TOK_FULL + t3], (uint32_t)(5 * Q * 4 + (CORR ? 3 : 2) * P * 4));
@@ -364,14 +321,14 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
   } else if (warp == 2) {
     // ------------------------------------------------------------ TMA producer: Cq, hq
     if (lane == 0) {
-      Tile t = decode_tile(t_begin, d, TM, ntpu);
+      Tile t = decode_unit((int)blockIdx.x, d, TM);
 #pragma unroll 1
-      for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+      for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
         // the MMAs of tile n - 1 (the other issuer's) have read the buffer
         if (n > 0) mbar_wait_relaxed(&bars[B_CH_FREE + ((n - 1) & 1)], ((n - 1) >> 1) & 1, a.status);
         uint64_t* full = &bars[B_CH_FULL + (n & 1)];
         mbar_expect_tx(full, (uint32_t)(TM * N + 64 * N));
-        tma_load_3d(smem + OFF_C, &tm_C, full, 0, t.g, (int)(t.tok0 + t.it * TM));
+        tma_load_3d(smem + OFF_C, &tm_C, full, 0, t.h / a.w.hpg, (int)(t.tok0 + t.it * TM));
         tma_load_2d(smem + OFF_H, &tm_h, full, 0, (int)((((i64)t.b * d.c + t.k) * d.H + t.h) * P));
       }
     }
@@ -384,8 +341,8 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
       const uint32_t idesc_off = idesc_s8(128, 64, 0, 0), idesc_diag = idesc_f16(128, 64, 1);
       const uint32_t sbase = smem_u32(smem);
 #pragma unroll 1
-      for (int tix = t_begin + par, n = par; tix < t_end; tix += 2, n += 2) {
-        const int it = tix % ntpu;
+      for (int n = par; n < n_end; n += 2) {
+        const int it = ntpu == 1 ? 0 : (n & 1);   // a CTA's first tile is the first of its unit
         const int ci = cb_index(n, it, ntpu), s2 = n & 1, xs = x_index(n, ntpu);
         const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
         const int KJ = (it + 1) * TM;
@@ -420,9 +377,9 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     const int wg = (warp - kMaskWarp0) % kGroupWarps;
     const int rq = warp & 3;               // TMEM lane quarter of this warp = row quarter of the tile
     const int q2 = wg >> 2;                // chunk parity of this warp
-    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    Tile t = decode_unit((int)blockIdx.x, d, TM);
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+    for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
       if ((((ntpu == 1) ? n : (n >> 1)) & 1) != g) continue;
       const int ci = cb_index(n, t.it, ntpu), t3 = n & 3, ob = n & 1;
       const uint32_t ph4 = (n >> 2) & 1;
@@ -468,9 +425,9 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
     const int er = q * 32 + lane;           // row of the tile
     uint8_t* ystage = smem + OFF_YST + ew * 2048;   // [32][64 B], 64-byte swizzle
     uint8_t* srow = ystage + lane * 64;
-    Tile t = decode_tile(t_begin, d, TM, ntpu);
+    Tile t = decode_unit((int)blockIdx.x, d, TM);
 #pragma unroll 1
-    for (int tix = t_begin, n = 0; tix < t_end; ++tix, ++n, next_tile(t, d, TM, ntpu)) {
+    for (int n = 0; n < n_end; ++n, next_tile(t, d, a.w, TM, ntpu)) {
       const int s2 = n & 1, t3 = n & 3, xs = x_index(n, ntpu);
       const uint32_t ph4 = (n >> 2) & 1, ph2 = (n >> 1) & 1;
       const float* tok = reinterpret_cast<const float*>(smem + OFF_TOK + t3 * TOK_BYTES);
@@ -550,10 +507,11 @@ chunk_scan_f16_tc(const __grid_constant__ CUtensorMap tm_C, const __grid_constan
             // the chunk's last tile: once every epilogue warp is through, its x buffer takes the codes of
             // the chunk after next
             const int n2 = n - (ntpu - 1) + 2 * ntpu;   // first tile of that chunk
-            if (ew == 0 && lane == 1 && t.it == ntpu - 1 && t_begin + n2 < t_end) {
+            if (ew == 0 && lane == 1 && t.it == ntpu - 1 && n2 < n_end) {
               mbar_wait(&bars[B_X_FREE + xs], x_phase(n, ntpu), a.status);
               Tile tn = t;
-              for (int i = 0; i < ntpu + 1; ++i) next_tile(tn, d, TM, ntpu);
+              next_unit(tn, d, a.w);
+              next_unit(tn, d, a.w);
               uint8_t* xb = smem + OFF_X + xs * X_BYTES;
               mbar_expect_tx(&bars[B_X_RAW + xs], (uint32_t)(Q * 64));
               for (int j0 = 0; j0 < Q; j0 += TM)
@@ -621,13 +579,12 @@ ssdi8_status_t launch_chunk_scan_f16(const Dims& d, const int8_t* xq, const int8
   int dev = 0, sms = 0;
   SSDI8_CUDA_CHECK(cudaGetDevice(&dev));
   SSDI8_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const int ntiles = (int)((i64)d.b * d.c * d.H * (d.Q / TM));
-  const int ctas = ntiles < sms ? ntiles : sms;
-  int per_cta = (ntiles + ctas - 1) / ctas;
-  if (d.Q > 128 && (per_cta & 1)) ++per_cta;  // keep both tiles of a chunk in one CTA (buffer rings assume it)
-  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, d, ntiles, per_cta};
+  UnitWalk walk;
+  int grid_i = 0;
+  if (!make_unit_walk(d, TM, sms, &walk, &grid_i)) return SSDI8_ERR_SHAPE;
+  ScanArgs a = {s_x, s_C, s_cb, s_h, pack, D, corr, status, d, walk};
   const size_t smem = SMEM_BYTES + 1024;
-  const unsigned grid = (unsigned)((ntiles + per_cta - 1) / per_cta);
+  const unsigned grid = (unsigned)grid_i;
   auto launch = [&](auto kernel) -> ssdi8_status_t {
     SSDI8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     return launch_pdl(kernel, dim3(grid), dim3(kThreads), smem, st, tm_C, tm_h, tm_x, tm_cb, tm_y, a) == cudaSuccess ? SSDI8_OK : SSDI8_ERR_CUDA;
