@@ -178,6 +178,17 @@ __device__ __forceinline__ float softplus_dt(float dt_raw, float bias) {
 // and memory flush (pdl_wait) before its first access to global memory, so only work that touches no
 // global memory (barrier and tensor-memory set-up, descriptor prefetch) runs under the predecessor's
 // tail.  Both are no-ops in a kernel that was launched without the attribute.
+// A store whose line is to stay in L2 ahead of ordinary ones (for data a later kernel of the same layer reads
+// after other kernels have streamed more than an L2 of traffic in between).
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void st_global_hint(float* a, float v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(a), "f"(v), "l"(pol) : "memory");
+}
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -138,6 +138,7 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
     }
   }
   __syncthreads();
+  const uint64_t pol = l2_policy_evict_last();
   // per-token rows of the pack.  Consecutive threads take consecutive tokens of one unit, so a row's
   // stores coalesce and the 16 tokens of a sub-block sit in 16 adjacent lanes (Q is a multiple of 32)
   for (int e = threadIdx.x; e < NU * Q; e += blockDim.x) {
@@ -150,12 +151,14 @@ __device__ __forceinline__ void cumsum_body(const float* __restrict__ dt, const 
       const float ci = c[i], di = dts[u * ld + i];
       const i64 un = ((i64)b * d.H + h0 + hh) * d.c + k0 + kk;
       float* p = pack + ((un * kPackRows) << lq) + i;
-      p[0] = ci;
-      p[Q] = di;
+      // (the pack is read by the state kernel and by ChunkScan after the quantisers and the state kernel have
+      // streamed several times the size of L2: its lines are kept ahead of theirs)
+      st_global_hint(p, ci, pol);
+      st_global_hint(p + Q, di, pol);
       wo = __fmul_rn(di, exp32(__fsub_rn(c[i | 15], ci)));
-      p[PACK_WOFF * Q] = wo;
-      p[PACK_ATOK * Q] = i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f;
-      p[PACK_LUT * Q] = __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci)));
+      st_global_hint(p + PACK_WOFF * Q, wo, pol);
+      st_global_hint(p + PACK_ATOK * Q, i > 0 ? exp32(__fsub_rn(ci, c[i - 1])) : 1.0f, pol);
+      st_global_hint(p + PACK_LUT * Q, __fmul_rn(di, exp32(__fsub_rn(c[Q - 1], ci))), pol);
       if (tap_cs) tap_cs[(un << lq) + i] = ci;
     }
     // sub-block maxima of |woff|, times 127
