@@ -11,9 +11,9 @@
  *    caller owns every buffer and the library allocates no device memory.  It keeps
  *    no mutable state between calls, with three exceptions, each stated again at its
  *    entry point: per device, the result of the architecture check (every call);
- *    the address of the built-in scratch (ssdi8_chunk_scan_fwd_static); one side
- *    stream and its events (ssdi8_layer_fwd, ssdi8_layer_fwd_host, created at the
- *    first call on a device and kept for the life of the process).  All three are
+ *    the address of the built-in scratch (ssdi8_chunk_scan_fwd_static); two copy
+ *    streams and their events (ssdi8_layer_fwd_host, created at the first call on
+ *    a device and kept for the life of the process).  All three are
  *    filled under a lock, so first calls may come from several threads at once.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *    Calls are asynchronous on that stream.
@@ -258,23 +258,24 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  *
  * ssdi8_layer_fwd: every pointer is a DEVICE pointer.  The three quantisers are one launch on
  *   `stream` (separate launches when d_state is not a power of two or a tensor is not 16-byte
- *   aligned); ChunkCumsum (reads dt and A only) runs inside that launch for small workloads and on a
- *   side stream under it, joined before the state kernel, for large ones; the state kernel, ChunkBMM
- *   and ChunkScan follow on `stream`.  workspace: 256-byte aligned,
+ *   aligned); all kernels run on `stream`, chained by programmatic dependent launch: ChunkCumsum (reads
+ *   dt and A only) first, the quantisers' launch beside it, then the state kernel, ChunkBMM beside the
+ *   state kernel's last wave, and ChunkScan; no other stream, no event.  The call may be captured into a
+ *   CUDA graph.  workspace: 256-byte aligned,
  *   ssdi8_layer_fwd_workspace_bytes(dims, flags) bytes (the int8 tensors plus ssdi8_workspace_bytes).
  * ssdi8_layer_fwd_host: x, B, C, dt, y, final_state, status are HOST pointers (page-locked memory, or
  *   the copies neither overlap nor run asynchronously), the rest DEVICE pointers.  One slice at a
  *   time, a slice being a batch element or, when an element's x exceeds 96 MB, an equal range of its
  *   heads (Algorithm 2 has no term across batch elements or heads): the host->device copies of slice
- *   i+1 and the device->host copy of y of slice i-1 run on two more side streams while the kernels
+ *   i+1 and the device->host copy of y of slice i-1 run on two copy streams while the kernels
  *   of slice i run, so both directions of the host link stay busy.  scratch: DEVICE, 256-byte
  *   aligned, ssdi8_layer_fwd_host_scratch_bytes(dims, flags) bytes (two stages of one slice's tensors).
  * Layouts as in ssdi8_fwd_args_t; D, corr, init_state, final_state, status may be NULL.  Both calls
  * return once everything is enqueued and leave `stream` waiting for the last piece of work, so
  * synchronising `stream` completes them.  flags: any of SSDI8_FLAG_INT8_STATE, SSDI8_FLAG_Y_FP16,
- * SSDI8_FLAG_Y_BF16 (`y` then points to 16-bit elements), SSDI8_FLAG_FP16_OPERAND.  The side streams and
- * events are created at the first call on each device and shared by later calls: calls on one
- * device must not overlap in time.  Errors: as ssdi8_quantize_act / ssdi8_chunk_scan_fwd, plus
+ * SSDI8_FLAG_Y_BF16 (`y` then points to 16-bit elements), SSDI8_FLAG_FP16_OPERAND.  The copy streams and
+ * events of ssdi8_layer_fwd_host are created at the first call on each device and shared by later calls:
+ * calls of ssdi8_layer_fwd_host on one device must not overlap in time.  Errors: as ssdi8_quantize_act / ssdi8_chunk_scan_fwd, plus
  * SSDI8_ERR_WORKSPACE for a short workspace or scratch. */
 typedef struct {
   const float* x; const float* B; const float* C; const float* dt;   /* [B,L,H,P], [B,L,G,N] x2, [B,L,H] */
