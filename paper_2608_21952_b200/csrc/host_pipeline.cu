@@ -1,12 +1,11 @@
 // The layer step as one call: Eq. 1 quantisation of fp32 x, B, C with static step sizes and the SSD
 // layer forward (Algorithm 2).
-// ssdi8_layer_fwd (device buffers): ChunkCumsum reads dt and A only, so it runs beside the quantisers
-// (inside their launch for small workloads, on a side stream under the bandwidth-bound quantiser of x
-// for large ones); the state kernel, ChunkBMM and ChunkScan follow on the caller's stream, chained by
-// programmatic dependent launch.
+// ssdi8_layer_fwd (device buffers): one chain on the caller's stream, linked by programmatic dependent
+// launch.  ChunkCumsum reads dt and A only, so the quantisers' launch behind it starts without waiting
+// for it and works beside it; the state kernel, ChunkBMM and ChunkScan follow.
 // ssdi8_layer_fwd_host (host buffers): the same, one batch element at a time.  Batch elements are
 // independent, so the host->device copies of element b+1 and the device->host copy of the
-// output of element b-1 run on two side streams while the kernels of element b run on the
+// output of element b-1 run on two copy streams while the kernels of element b run on the
 // caller's stream: the PCIe link is busy in both directions for the whole call instead of
 // idle during the kernels and one-directional during the copies.  Only stream and event
 // plumbing lives here; every arithmetic step is a kernel of this library.
@@ -59,7 +58,7 @@ Layout make_layout(const ssdi8_dims_t& d1, int full_heads, uint8_t* base, uint32
   return lo;
 }
 
-// side streams and events, made once per device and kept for the life of the process
+// copy streams and events of the host-buffer entry point, made once per device and kept for the life of the process
 struct Plumbing {
   bool ready = false;
   cudaStream_t s_in = nullptr, s_out = nullptr;
