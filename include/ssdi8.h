@@ -256,9 +256,9 @@ ssdi8_status_t ssdi8_chunk_scan_fwd_static(const ssdi8_dims_t* dims, const ssdi8
  * modules are separate kernels on device-resident tensors); the arithmetic is exactly that of
  * the two calls it replaces, and so is the result.
  *
- * ssdi8_layer_fwd: every pointer is a DEVICE pointer.  The three quantisers are one launch on
- *   `stream` (separate launches when d_state is not a power of two or a tensor is not 16-byte
- *   aligned); all kernels run on `stream`, chained by programmatic dependent launch: ChunkCumsum (reads
+ * ssdi8_layer_fwd: every pointer is a DEVICE pointer.  The three quantisers are one launch (x, B and C
+ *   must be 16-byte aligned like every other tensor: SSDI8_ERR_ALIGN otherwise, before anything is
+ *   enqueued); all kernels run on `stream`, chained by programmatic dependent launch: ChunkCumsum (reads
  *   dt and A only) first, the quantisers' launch beside it, then the state kernel, ChunkBMM beside the
  *   state kernel's last wave, and ChunkScan; no other stream, no event.  The call may be captured into a
  *   CUDA graph.  workspace: 256-byte aligned,

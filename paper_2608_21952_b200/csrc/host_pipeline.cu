@@ -122,13 +122,9 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
   f.init_state = init; f.y = y; f.final_state = fin; f.status = status;
   const uint32_t fl = flags & kLayerFlags;
   ssdi8_status_t s;
-  // one launch for the three quantisers needs a power-of-two N (group of a channel by a shift) and
-  // 16-byte aligned tensors (it reads four values and writes four codes at a time)
-  const bool one_launch =
-      (d.dstate & (d.dstate - 1)) == 0 &&
-      ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C) |
-        reinterpret_cast<uintptr_t>(a.s_x) | reinterpret_cast<uintptr_t>(xq) | reinterpret_cast<uintptr_t>(Bq) |
-        reinterpret_cast<uintptr_t>(Cq)) & 15) == 0;
+  // (the three quantisers are one launch: it needs a power-of-two N, which every supported N is, and 16-byte
+  // aligned tensors, which the entry points have checked or provide themselves)
+  if ((d.dstate & (d.dstate - 1)) != 0) return SSDI8_ERR_UNSUPPORTED;
   // ChunkCumsum (it reads dt and A only) and the quantisers need nothing of each other.  ChunkCumsum goes
   // first and lets its successor be scheduled once its own wait for the work ahead of the layer is over;
   // the quantisers' launch then starts without a wait and runs beside it, with the wait at the end of its
@@ -136,19 +132,10 @@ ssdi8_status_t layer_step(const ssdi8_dims_t& d, const ssdi8_layer_args_t& a, co
   // ChunkCumsum complete as well.  One stream, no events.  Measured per step, this chain / ChunkCumsum on a
   // side stream / ChunkCumsum's blocks inside the quantisers' grid: 0.286 / 0.293 / 0.287 ms at batch
   // 8 x 2048 x 80 heads, 0.056 / 0.062 / 0.062 ms at 2048 x 24 heads.
-  {
-    if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, st, false)) != SSDI8_OK) return s;
-    if (one_launch) {
-      if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq,
-                                   Cq, st, true)) != SSDI8_OK)
-        return s;
-    } else {
-      if ((s = ssdi8_quantize_act(B, T, d.ngroups, d.dstate, const_cast<float*>(a.s_B), 0, Bq, st)) != SSDI8_OK) return s;
-      if ((s = ssdi8_quantize_act(C, T, d.ngroups, d.dstate, const_cast<float*>(a.s_C), 0, Cq, st)) != SSDI8_OK) return s;
-      if ((s = ssdi8_quantize_act(x, T, (int64_t)d.nheads * d.headdim, 1, const_cast<float*>(a.s_x), 0, xq, st)) != SSDI8_OK)
-        return s;
-    }
-  }
+  if ((s = fwd_phases(&d, &f, fl | SSDI8_PHASE_CUMSUM, ws, ws_bytes, st, false)) != SSDI8_OK) return s;
+  if ((s = launch_quantize_xbc(x, B, C, T, d.nheads * d.headdim, d.ngroups, d.dstate, a.s_x, a.s_B, a.s_C, xq, Bq, Cq, st,
+                               true)) != SSDI8_OK)
+    return s;
   // the rest, chained by programmatic dependent launch: the fused state kernel, ChunkBMM (needed by ChunkScan
   // only: launched behind the state kernel, it works beside that kernel's last wave), ChunkScan
   return fwd_phases(&d, &f, fl | SSDI8_PHASE_BMM | SSDI8_PHASE_CHUNK_STATE | SSDI8_PHASE_STATE_PASSING | SSDI8_PHASE_SCAN,
@@ -212,6 +199,10 @@ ssdi8_status_t ssdi8_layer_fwd(const ssdi8_dims_t* dims, const ssdi8_layer_args_
   if (need == 0) return SSDI8_ERR_SHAPE;
   if (workspace_bytes < need) return SSDI8_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return SSDI8_ERR_ALIGN;
+  // the quantisers read x, B and C sixteen bytes at a time (the other tensors are checked by the forward pass,
+  // also before anything is enqueued)
+  if ((reinterpret_cast<uintptr_t>(a->x) | reinterpret_cast<uintptr_t>(a->B) | reinterpret_cast<uintptr_t>(a->C)) & 15)
+    return SSDI8_ERR_ALIGN;
   const LayerWs w = layer_ws(*dims, static_cast<uint8_t*>(workspace), flags);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (a->status) SSDI8_CUDA_CHECK(cudaMemsetAsync(a->status, 0, sizeof(int32_t), st));

@@ -182,6 +182,11 @@ def test_host_side_argument_errors_of_the_layer_and_entry_calls():
         assert fn(C.byref(d), C.byref(a), 4096, need - 1, 0, None) == bd.ERR_WORKSPACE
         assert fn(C.byref(d), C.byref(a), 4096 + 8, need, 0, None) == bd.ERR_ALIGN
         assert fn(C.byref(d), C.byref(a), 4096, need, 1 << 13, None) == bd.ERR_UNSUPPORTED
+        if fn is L.ssdi8_layer_fwd:   # device tensors are read 16 bytes at a time: refused before anything is enqueued
+            for k in ("x", "B", "C"):
+                setattr(a, k, 4096 + 4)
+                assert fn(C.byref(d), C.byref(a), 4096, need, 0, None) == bd.ERR_ALIGN
+                setattr(a, k, 4096)
         assert size(C.byref(d), 1) == need                     # the FP16 operand needs no scratch of its own
         bad = bd.dims_of(CONFIGS["cfg0"].replace(chunk=48))
         assert size(C.byref(bad), 0) == 0
